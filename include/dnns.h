@@ -1,0 +1,248 @@
+/*
+ * dnns.h - C ABI of the sparse-to-pruned conversion path of DNNShifter on one GPU.
+ *
+ * The path turns a dense CNN into a portfolio of smaller model variants:
+ *
+ *   dnns_magnitude_threshold  rank the prunable weights by magnitude and find, for every
+ *                             requested prune count k, the k-th smallest magnitude
+ *                             (Phase 1's "unstructured ranking", Section III-C; a compression
+ *                             ratio C leaves C-1 of every C weights zero, Section IV-B-1);
+ *   dnns_apply_mask           set the k weights of least magnitude to zero - the sparse model,
+ *                             which is not yet smaller (Section III-C);
+ *   dnns_zero_structures      Module 2, Sparsity Analyser: all-zero 2-D kernels, then the
+ *                             channels all of whose kernels are zero (Section III-D, Figure 2);
+ *   dnns_propagate_keep       Module 3, Prune Planner (Algorithm 1): which channels every layer
+ *                             drops, planned for all layers at once;
+ *   dnns_compact              Module 4, Model Pruner (Algorithm 2): rebuild every layer without
+ *                             its prunable in/out channels, biases and BatchNorm entries, all
+ *                             layers in one batch.
+ *
+ * General rules
+ *   - Every function returns a dnns_status; nothing throws, aborts or traps.  Argument and
+ *     graph errors are found on the host before anything is launched.
+ *   - "device" pointers are CUDA device memory of the current device, owned by the caller.
+ *     The library allocates no device memory: tables and scratch live in the caller's
+ *     workspace (dnns_workspace_bytes).  Host pointers are only read during the call.
+ *   - Every compute call enqueues its kernels on `stream` (a cudaStream_t passed as void*,
+ *     NULL = the default stream) and returns without synchronising.  Only
+ *     dnns_last_device_status and dnns_plan_destroy synchronise.
+ *   - Calls on one plan must be issued in stream order on one stream at a time: the plan's
+ *     workspace is shared state.
+ *
+ * Layouts
+ *   - Weights are OIHW, contiguous, row-major: filter o is I*KH*KW consecutive elements, the
+ *     2-D kernel (o,i) is KH*KW consecutive elements.  A fully-connected layer is [O][I] with
+ *     KH = KW = 1 and I = C_in*in_spatial; the columns of input channel c are
+ *     c*in_spatial .. (c+1)*in_spatial-1.  Tensor data pointers must be 16-byte aligned.
+ *   - A magnitude is compared as the stored word with its sign bit cleared (31-bit keys for
+ *     fp32, 15-bit keys for bf16), as an unsigned integer: -0 equals +0, denormals order
+ *     numerically, infinities lie above all finite values, NaNs above those.  A weight is
+ *     "zero" when that key is 0.
+ *   - Bit sets are uint32 words, bit b in word b/32 at position b%32.  Per-tensor and
+ *     per-group bit sets and index lists are packed one after another into ONE device array
+ *     each, at the word/element offsets dnns_plan_layout reports (each set starts on a word).
+ *   - A "masked arena" holds a copy of every weight tensor of the model at the byte offsets
+ *     dnns_plan_layout reports (256-byte aligned, descriptor order).
+ */
+#ifndef DNNS_H
+#define DNNS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DNNS_OK = 0,
+    DNNS_ERR_INVALID_ARG = 1, /* null pointer, non-positive extent, misaligned data, k above its segment */
+    DNNS_ERR_BAD_GRAPH = 2,   /* tensor / BN / group extents that do not agree                             */
+    DNNS_ERR_WORKSPACE = 3,   /* workspace or destination arena too small                                   */
+    DNNS_ERR_UNSUPPORTED = 4, /* mixed dtypes, unknown dtype, extents beyond the documented limits          */
+    DNNS_ERR_CUDA = 5,        /* a CUDA runtime call failed                                                 */
+    DNNS_ERR_TIMEOUT = 6      /* reserved for bounded device-side waits (the current kernels have none)     */
+} dnns_status;
+
+typedef enum { DNNS_F32 = 0, DNNS_BF16 = 1 } dnns_dtype;
+typedef enum { DNNS_SCOPE_GLOBAL = 0, DNNS_SCOPE_PER_TENSOR = 1 } dnns_scope;
+
+/* policy bits of dnns_propagate_keep */
+enum { DNNS_RULE_PRODUCER = 1, DNNS_RULE_CONSUMER = 2, DNNS_SHIFT_STRICT = 4 };
+/* group flags */
+enum { DNNS_GROUP_FROZEN = 1 };
+
+/* One weight tensor.  out_group / in_group name the channel groups of its two axes. */
+typedef struct {
+    void* data;         /* device, 16-byte aligned, O*I*KH*KW elements of `dtype`            */
+    int32_t dtype;      /* dnns_dtype; all tensors of a model share one dtype                 */
+    int32_t O, I, KH, KW;
+    int32_t in_spatial; /* S: columns per input channel (1 for convs and after global pooling)*/
+    int32_t prunable;   /* takes part in ranking and masking                                  */
+    int32_t out_group;  /* group of the O axis; O == groups[out_group].C                      */
+    int32_t in_group;   /* group of the I axis; I == groups[in_group].C * in_spatial          */
+    float* bias;        /* device, fp32, length O; NULL when the layer has none               */
+} dnns_tensor;
+
+/* BatchNorm following conv `tensor`; its vectors follow that tensor's out-axis. */
+typedef struct {
+    float *gamma, *beta, *mean, *var; /* device, fp32, length C */
+    int32_t C;
+    int32_t tensor;
+    float eps;
+} dnns_bn;
+
+/* A set of channels shared by the out-axes that write it (producers) and the in-axes that
+ * read it (consumers): one layer boundary in a chain, a whole residual stream in a ResNet. */
+typedef struct {
+    int32_t C;
+    uint32_t flags; /* DNNS_GROUP_FROZEN: never pruned (network input, class axis) */
+} dnns_group;
+
+typedef struct {
+    int32_t n_tensors;
+    const dnns_tensor* tensors;
+    int32_t n_bn;
+    const dnns_bn* bns;
+    int32_t n_groups;
+    const dnns_group* groups;
+} dnns_model;
+
+/* Result of the ranking for one (variant, segment). */
+typedef struct {
+    uint32_t tau_bits; /* magnitude key of the k-th smallest weight                  */
+    uint32_t pad;
+    uint64_t n_below;  /* weights whose key is below tau                             */
+    uint64_t n_tie;    /* k - n_below: weights equal to tau that are masked (>= 1)   */
+    uint64_t n_equal;  /* weights whose key equals tau                               */
+} dnns_threshold;     /* k == 0 gives the all-zero record                           */
+
+/* Sizes and offsets of the packed buffers, all host memory owned by the plan. */
+typedef struct {
+    int32_t n_tensors, n_bn, n_groups, n_segments, n_bias;
+    int32_t elem_bytes;            /* 4 or 2                                                        */
+    uint64_t n_prunable;           /* prunable weights in the model                                 */
+    uint64_t masked_arena_bytes;   /* size of a masked arena                                        */
+    uint64_t mask_words;           /* uint32 words of the packed mask bits (numel bits per tensor)  */
+    uint64_t nz_map_words;         /* packed kernel maps (O*I bits per tensor)                      */
+    uint64_t out_nz_words;         /* packed out flags (O bits per tensor)                          */
+    uint64_t in_nz_words;          /* packed in flags (I bits per tensor)                           */
+    uint64_t keep_words;           /* packed keep bits (C bits per group)                           */
+    uint64_t keep_idx_len;         /* packed keep index lists (C entries per group)                 */
+    uint64_t compact_arena_bytes;  /* worst-case size of a destination arena for dnns_compact       */
+    int32_t n_compact_items;       /* n_tensors + 4*n_bn + n_bias                                   */
+    const uint64_t* arena_offset;  /* [n_tensors] byte offset of tensor t in a masked arena         */
+    const uint64_t* mask_offset;   /* [n_tensors] word offsets into the packed arrays ...           */
+    const uint64_t* nz_map_offset; /* [n_tensors]                                                   */
+    const uint64_t* out_nz_offset; /* [n_tensors]                                                   */
+    const uint64_t* in_nz_offset;  /* [n_tensors]                                                   */
+    const uint64_t* keep_offset;   /* [n_groups] word offset of the group's keep bits               */
+    const uint64_t* keep_idx_offset; /* [n_groups] element offset of the group's index list         */
+    const uint64_t* segment_size;  /* [n_segments] prunable weights per ranking segment             */
+    const int32_t* segment_of_tensor; /* [n_tensors] segment index, -1 when not prunable            */
+} dnns_layout;
+
+typedef struct dnns_plan dnns_plan; /* opaque; host object */
+
+/* Device bytes a plan needs for `max_variants` prune counts per segment.  0 on invalid input. */
+size_t dnns_workspace_bytes(const dnns_model* model, dnns_scope scope, int32_t max_variants);
+
+/*
+ * Validate the model (host descriptors holding device pointers), build the tile, segment and
+ * group tables and upload them into the workspace.  scope fixes the ranking segments
+ * (Section III-C leaves global or per-layer ranking open: GLOBAL = one segment of all prunable
+ * weights in descriptor order, PER_TENSOR = one segment per prunable tensor).
+ * ws_dev must be 256-byte aligned and stay valid and untouched until the plan is destroyed.
+ * Errors: INVALID_ARG, BAD_GRAPH (an out-axis whose O differs from its group's C, an in-axis
+ * whose I differs from C*in_spatial, a BN whose C differs from its tensor's O, two BNs on one
+ * tensor), UNSUPPORTED (mixed or unknown dtype, a tensor of 2^31 or more elements, a segment
+ * of 2^32 or more weights, a group above 65536 channels, max_variants outside 1..64),
+ * WORKSPACE, CUDA.
+ */
+dnns_status dnns_plan_create(const dnns_model* model, dnns_scope scope, int32_t max_variants, void* ws_dev,
+                             size_t ws_bytes, void* stream, dnns_plan** plan_out);
+/* Synchronises the device, then frees the host object.  The workspace stays the caller's. */
+void dnns_plan_destroy(dnns_plan* plan);
+dnns_status dnns_plan_layout(const dnns_plan* plan, dnns_layout* out);
+/* Kernels this plan has launched so far (memsets and copies not counted). */
+uint64_t dnns_plan_launch_count(const dnns_plan* plan);
+
+/*
+ * Step 1 - exact k-th-magnitude threshold by radix select over the magnitude keys.
+ * k (host): k[v*n_segments + s] = how many weights of segment s variant v masks, 0 <= k <= the
+ * segment's size, 1 <= n_k <= max_variants.  thr_dev (device, n_k*n_segments records, same
+ * indexing) receives the records.  One call serves the whole portfolio: the sweeps over the
+ * weights are shared by all n_k counts.  The call also leaves, in the workspace, the per-tile
+ * tie tables that dnns_apply_mask needs to mask exactly k weights when several weights equal
+ * tau; they belong to this call's thr_dev.
+ * Errors: INVALID_ARG (null, n_k out of range, a k above its segment), CUDA.
+ */
+dnns_status dnns_magnitude_threshold(dnns_plan* plan, const uint64_t* k, int32_t n_k, dnns_threshold* thr_dev,
+                                     void* stream);
+
+/*
+ * Step 2 - mask variant `variant` of the latest dnns_magnitude_threshold call on this plan
+ * (thr_dev is that call's output array).  A weight is masked when its key is below tau, or
+ * equals tau and fewer than n_tie equal weights precede it in the segment (tensors in
+ * descriptor order, row-major inside): exactly k weights per segment.  Masked weights become
+ * +0, the others are copied bit for bit; tensors that are not prunable are copied.
+ * masked_arena (device): destination in arena layout, or NULL to mask the model's tensors in
+ * place (only meaningful for the weights the thresholds were computed on).
+ * mask_bits (device, nullable): packed mask bits, 1 = kept; padding bits are written as 0.
+ */
+dnns_status dnns_apply_mask(dnns_plan* plan, const dnns_threshold* thr_dev, int32_t variant, void* masked_arena,
+                            uint32_t* mask_bits, void* stream);
+
+/*
+ * Step 3 - zero structures of a sparse model.  masked_arena (device): the weights to analyse in
+ * arena layout, or NULL for the model's own tensors (a sparse model that arrived from training).
+ * Per tensor: nz_map (nullable) bit o*I+i = kernel (o,i) has a non-zero element; out_nz bit o =
+ * filter o has one; in_nz bit i = some filter reads input column i.  All three are packed device
+ * arrays (see dnns_layout) and are fully overwritten.
+ */
+dnns_status dnns_zero_structures(dnns_plan* plan, const void* masked_arena, uint32_t* nz_map, uint32_t* out_nz,
+                                 uint32_t* in_nz, void* stream);
+
+/*
+ * Step 4 - keep sets per channel group (Algorithm 1 generalised from a chain to groups).
+ * Channel j of a group is removed when
+ *   (policy & RULE_PRODUCER) and every producer's filter j is all zero [the paper's rule], and,
+ *       under SHIFT_STRICT, the constant each of those zero filters still emits through its
+ *       BatchNorm / bias is structurally zero (beta == 0 and (gamma == 0 or mean == bias); no BN:
+ *       bias == 0); or
+ *   (policy & RULE_CONSUMER) and no consumer has a non-zero weight in the columns of channel j.
+ * Frozen groups keep everything.  If fewer than min(min_keep, C) channels stay, removed channels
+ * are taken back in ascending order.  Single pass, nothing is re-evaluated after removal.
+ * Outputs (device, packed per group): keep_bits, keep_idx (kept channels ascending; entries past
+ * keep_count are left untouched), keep_count [n_groups].  stats (device, nullable, 4 words):
+ * [0] removed (producer, channel) pairs whose non-zero constant is dropped while some consumer
+ * still reads the channel, [1] channels removed, [2] channels taken back by min_keep, [3] 0.
+ */
+dnns_status dnns_propagate_keep(dnns_plan* plan, const uint32_t* out_nz, const uint32_t* in_nz, uint32_t policy,
+                                int32_t min_keep, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count,
+                                uint64_t* stats, void* stream);
+
+/*
+ * Step 5 - rebuild every tensor with its kept channels only (Algorithm 2):
+ *   W'[a][c][s][y][x] = W[keep_out[a]][keep_in[c]][s][y][x],  v'[a] = v[keep_out[a]] for every
+ * BatchNorm vector and bias.  masked_arena as in step 3.  The destination arena receives, at
+ * 256-byte aligned offsets computed on the device from keep_count, first the n_tensors weight
+ * tensors in descriptor order, then gamma, beta, mean, var of every BN in order, then the biases
+ * of the tensors that have one.  dst_offsets_dev [n_compact_items] receives those byte offsets,
+ * dst_shapes_dev [n_tensors][2] the new (O', I').  dst_bytes >= layout.compact_arena_bytes always
+ * suffices; if the arena is too small for this variant nothing is copied and the device status
+ * becomes DNNS_ERR_WORKSPACE.
+ */
+dnns_status dnns_compact(dnns_plan* plan, const void* masked_arena, const int32_t* keep_idx,
+                         const int32_t* keep_count, void* dst_arena, size_t dst_bytes, uint64_t* dst_offsets_dev,
+                         int32_t* dst_shapes_dev, void* stream);
+
+/* Synchronises `stream`, then returns (and clears) the status recorded by the plan's kernels. */
+dnns_status dnns_last_device_status(dnns_plan* plan, void* stream);
+
+const char* dnns_status_string(dnns_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DNNS_H */

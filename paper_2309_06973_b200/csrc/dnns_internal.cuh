@@ -1,0 +1,233 @@
+// Internal declarations shared by the kernels of libdnns: device-side descriptor tables, the
+// workspace map and the launch wrappers.  Nothing here is part of the public ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dnns.h"
+
+namespace dnns {
+
+// A tile is 16 KB of one tensor: the unit of work of every sweep and the granularity of the
+// tie tables.  Tiles never straddle tensors; the last tile of a tensor may be ragged.
+constexpr uint32_t kTileBytes = 16384;
+constexpr int kTileThreads = 256;
+constexpr int kVecPerThread = kTileBytes / 16 / kTileThreads;  // 4 x 16-byte vectors per thread
+
+constexpr uint32_t kHistBins = 32768;    // first radix digit: the top 15 bits of a key
+constexpr uint32_t kLowBins = 65536;     // second digit of a 31-bit key
+constexpr uint32_t kBitmapWords = kHistBins / 32;
+constexpr int kMaxVariants = 64;
+constexpr uint32_t kInSmemBits = 32768;  // input-column flags accumulate in shared memory up to this many columns
+
+struct TensorDesc {
+    const void* src;        // the model's tensor
+    const float* bias;      // nullable
+    uint64_t arena_off;     // byte offset in a masked arena
+    uint32_t numel;
+    int32_t O, I, KK, S;    // KK = KH*KW, S = in_spatial
+    int32_t out_group, in_group;
+    int32_t seg;            // ranking segment, -1 when not prunable
+    int32_t bn;             // BatchNorm that follows it, -1 when none
+    uint32_t tile0, n_tiles;
+    uint32_t off_mask, off_nzmap, off_outnz, off_innz;  // word offsets into the packed bit arrays
+};
+
+struct GroupDesc {
+    int32_t C;
+    uint32_t flags;
+    uint32_t off_bits;      // word offset of the keep bits
+    uint32_t off_idx;       // element offset of the keep index list
+    int32_t prod_begin, prod_end;  // range in prod_list (tensor ids writing this group)
+    int32_t cons_begin, cons_end;  // range in cons_list (tensor ids reading this group)
+};
+
+struct BnDesc {
+    const float *gamma, *beta, *mean, *var;
+    int32_t C, tensor;
+};
+
+struct SegDesc {
+    uint32_t tile_begin, tile_end;  // tiles [begin, end) cover the segment (tiles of other tensors in between count 0)
+    uint64_t size;
+};
+
+// One gather job of the rebuild: a weight tensor, a BatchNorm vector or a bias.
+struct ItemDesc {
+    const void* src;        // absolute source, or NULL when the source is tensor `tensor` of the arena/model
+    int32_t tensor;         // tensor index for weight items, -1 otherwise
+    int32_t O, Cin, blk;    // rows, input channels, elements per (row, input channel)
+    int32_t out_group, in_group;  // in_group -1: columns are kept as they are
+    int32_t elem_bytes;
+};
+
+// Per (variant, segment) state of the radix select between its two passes.
+struct SelectState {
+    uint64_t k;
+    uint64_t below;   // keys whose first digit is below `digit`
+    uint32_t digit;   // first digit of the k-th key
+    uint32_t slot;    // which second-pass histogram of the segment serves this digit
+    uint32_t count;   // keys in that first-digit bucket
+    uint32_t pad;
+};
+
+struct Tables {
+    const TensorDesc* tensors;
+    const GroupDesc* groups;
+    const BnDesc* bns;
+    const SegDesc* segs;
+    const ItemDesc* items;
+    const uint32_t* tile_tensor;
+    const int32_t* prod_list;
+    const int32_t* cons_list;
+    uint32_t* status;       // device status word (a dnns_status, 0 = ok)
+    uint32_t n_tensors, n_groups, n_bn, n_segs, n_items, n_tiles;
+    uint32_t tile_elems;    // 4096 (fp32) or 8192 (bf16)
+    int32_t dtype;
+};
+
+struct ThresholdWs {
+    uint64_t* k_dev;        // [n_k][S]
+    uint32_t* hist1;        // [S][kHistBins]
+    uint32_t* hist2;        // [S][n_k][kLowBins] (fp32 only)
+    uint32_t* bitmap;       // [S][kBitmapWords]: first digits that some variant selected
+    SelectState* sel;       // [n_k][S]
+    uint32_t* need;         // [n_k][S]: the variant masks only part of the weights equal to tau
+    uint32_t* any_need;     // [1]
+    uint32_t* tile_ties;    // [max_variants][n_tiles]: weights equal to tau_v in the tile
+    uint32_t* tie_prefix;   // [max_variants][n_tiles]: those in earlier tiles of the segment
+};
+
+struct CompactWs {
+    uint32_t* unit_prefix;  // [n_items + 1] gather units before each item
+    uint64_t* item_off;     // [n_items] byte offset in the destination arena
+    int32_t* item_dims;     // [n_items][2] rows', input channels' of the rebuilt item
+};
+
+// ---- launch wrappers (each returns the number of kernels it launched, or -1 on a CUDA error) ----
+int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, int n_k_stride, dnns_threshold* thr_dev,
+                     int n_sm, cudaStream_t st);
+int launch_tile_sweep(const Tables& tb, const ThresholdWs& ws, bool do_mask, bool do_struct,
+                      const dnns_threshold* thr_dev, int variant, const void* src_arena, void* dst_arena,
+                      uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz, int n_sm,
+                      cudaStream_t st);
+int launch_propagate(const Tables& tb, const uint32_t* out_nz, const uint32_t* in_nz, uint32_t policy,
+                     int32_t min_keep, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count, uint64_t* stats,
+                     cudaStream_t st);
+int launch_compact(const Tables& tb, const CompactWs& ws, const void* src_arena, const int32_t* keep_idx,
+                   const int32_t* keep_count, void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets,
+                   int32_t* dst_shapes, int n_sm, cudaStream_t st);
+cudaError_t init_kernel_attributes();
+
+// ---- small device helpers ----
+template <int DT>
+struct Elem;
+template <>
+struct Elem<DNNS_F32> {
+    static constexpr int kPerVec = 4;
+    static constexpr int kBytes = 4;
+};
+template <>
+struct Elem<DNNS_BF16> {
+    static constexpr int kPerVec = 8;
+    static constexpr int kBytes = 2;
+};
+
+// Magnitude keys of the elements of one 16-byte vector, in element order.
+template <int DT>
+__device__ __forceinline__ void vec_keys(const uint4& v, uint32_t (&key)[Elem<DT>::kPerVec]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    if (DT == DNNS_F32) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) key[j] = w[j] & 0x7FFFFFFFu;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            key[2 * j] = w[j] & 0x7FFFu;
+            key[2 * j + 1] = (w[j] >> 16) & 0x7FFFu;
+        }
+    }
+}
+
+// First radix digit (top 15 bits) of a key.
+template <int DT>
+__device__ __forceinline__ uint32_t digit_of(uint32_t key) {
+    return DT == DNNS_F32 ? key >> 16 : key;
+}
+
+// Load the vector holding elements [e, e + kPerVec) of a tensor of `numel` elements; elements
+// past the end read as zero.  Returns how many elements are valid.
+template <int DT, bool READ_ONLY = true>
+__device__ __forceinline__ int load_vec(const void* base, uint32_t e, uint32_t numel, uint4& v) {
+    constexpr int P = Elem<DT>::kPerVec;
+    if (e + P <= numel) {
+        const uint4* p = reinterpret_cast<const uint4*>(static_cast<const char*>(base) + (size_t)e * Elem<DT>::kBytes);
+        v = READ_ONLY ? __ldg(p) : *p;   // READ_ONLY = false when the kernel may overwrite the tensor in place
+        return P;
+    }
+    v = make_uint4(0, 0, 0, 0);
+    if (e >= numel) return 0;
+    const int n = (int)(numel - e);
+    uint32_t w[4] = {0, 0, 0, 0};
+    if (DT == DNNS_F32) {
+        const uint32_t* p = static_cast<const uint32_t*>(base) + e;
+        for (int j = 0; j < n; ++j) w[j] = p[j];
+    } else {
+        const uint16_t* p = static_cast<const uint16_t*>(base) + e;
+        for (int j = 0; j < n; ++j) w[j >> 1] |= (uint32_t)p[j] << (16 * (j & 1));
+    }
+    v = make_uint4(w[0], w[1], w[2], w[3]);
+    return n;
+}
+
+template <int DT>
+__device__ __forceinline__ void store_vec(void* base, uint32_t e, uint32_t numel, const uint4& v) {
+    constexpr int P = Elem<DT>::kPerVec;
+    if (e + P <= numel) {
+        *reinterpret_cast<uint4*>(static_cast<char*>(base) + (size_t)e * Elem<DT>::kBytes) = v;
+        return;
+    }
+    if (e >= numel) return;
+    const int n = (int)(numel - e);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    if (DT == DNNS_F32) {
+        uint32_t* p = static_cast<uint32_t*>(base) + e;
+        for (int j = 0; j < n; ++j) p[j] = w[j];
+    } else {
+        uint16_t* p = static_cast<uint16_t*>(base) + e;
+        for (int j = 0; j < n; ++j) p[j] = (uint16_t)(w[j >> 1] >> (16 * (j & 1)));
+    }
+}
+
+// Exclusive prefix sum over the threads of a block (blockDim.x a multiple of 32, at most 1024).
+// `scratch` holds 33 words of shared memory.  Returns the exclusive prefix; *total gets the sum.
+template <typename T>
+__device__ __forceinline__ T block_exclusive_scan(T x, T* scratch, T* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    T incl = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        T y = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += y;
+    }
+    __syncthreads();
+    if (lane == 31) scratch[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        T w = lane < nwarp ? scratch[lane] : T(0);
+        T wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            T y = __shfl_up_sync(0xffffffffu, wi, d);
+            if (lane >= d) wi += y;
+        }
+        scratch[lane] = wi - w;
+        if (lane == 31) scratch[32] = wi;
+    }
+    __syncthreads();
+    *total = scratch[32];
+    return scratch[warp] + incl - x;
+}
+
+}  // namespace dnns

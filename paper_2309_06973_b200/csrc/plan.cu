@@ -1,0 +1,438 @@
+// Host side of libdnns: model validation, table construction, workspace map and the C entry
+// points.  Every entry point checks its arguments on the host, enqueues kernels and returns.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "dnns_internal.cuh"
+
+using namespace dnns;
+
+namespace {
+
+constexpr uint64_t kAlign = 256;
+inline uint64_t align_up(uint64_t x, uint64_t a = kAlign) { return (x + a - 1) / a * a; }
+
+// Byte offsets of every section of the workspace.
+struct WsMap {
+    uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, status;
+    uint64_t tables_end;  // everything before this is uploaded once at plan creation
+    uint64_t k_dev, bitmap, sel, tie_prefix, unit_prefix, item_off, item_dims;
+    uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
+    uint64_t any_need, need, tile_ties, hist1, hist2;
+    uint64_t total;
+};
+
+struct Counts {
+    uint32_t T = 0, G = 0, B = 0, S = 0, items = 0, tiles = 0, n_bias = 0;
+    int dtype = 0, elem_bytes = 4;
+};
+
+bool tensor_extents_ok(const dnns_tensor& t) {
+    return t.O > 0 && t.I > 0 && t.KH > 0 && t.KW > 0 && t.in_spatial > 0;
+}
+
+// Shape-level validation and counting; no device access.
+dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts* c) {
+    if (!m || !m->tensors || !m->groups || m->n_tensors <= 0 || m->n_groups <= 0 || m->n_bn < 0) return DNNS_ERR_INVALID_ARG;
+    if (m->n_bn > 0 && !m->bns) return DNNS_ERR_INVALID_ARG;
+    if (scope != DNNS_SCOPE_GLOBAL && scope != DNNS_SCOPE_PER_TENSOR) return DNNS_ERR_INVALID_ARG;
+    if (maxv < 1 || maxv > kMaxVariants) return DNNS_ERR_UNSUPPORTED;
+    c->T = m->n_tensors, c->G = m->n_groups, c->B = m->n_bn;
+    c->dtype = m->tensors[0].dtype;
+    if (c->dtype != DNNS_F32 && c->dtype != DNNS_BF16) return DNNS_ERR_UNSUPPORTED;
+    c->elem_bytes = c->dtype == DNNS_F32 ? 4 : 2;
+    for (int g = 0; g < m->n_groups; ++g) {
+        if (m->groups[g].C <= 0) return DNNS_ERR_INVALID_ARG;
+        if (m->groups[g].C > 65536) return DNNS_ERR_UNSUPPORTED;
+    }
+    uint64_t n_prunable = 0, seg_count = 0;
+    for (int i = 0; i < m->n_tensors; ++i) {
+        const dnns_tensor& t = m->tensors[i];
+        if (!t.data || !tensor_extents_ok(t)) return DNNS_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(t.data) & 15) return DNNS_ERR_INVALID_ARG;
+        if (t.dtype != c->dtype) return DNNS_ERR_UNSUPPORTED;
+        if (t.out_group < 0 || t.out_group >= m->n_groups || t.in_group < 0 || t.in_group >= m->n_groups)
+            return DNNS_ERR_BAD_GRAPH;
+        if (t.O != m->groups[t.out_group].C) return DNNS_ERR_BAD_GRAPH;
+        if ((int64_t)t.I != (int64_t)m->groups[t.in_group].C * t.in_spatial) return DNNS_ERR_BAD_GRAPH;
+        const uint64_t numel = (uint64_t)t.O * t.I * t.KH * t.KW;
+        if (numel >= (1ull << 31)) return DNNS_ERR_UNSUPPORTED;
+        c->tiles += (uint32_t)((numel * c->elem_bytes + kTileBytes - 1) / kTileBytes);
+        if (t.bias) ++c->n_bias;
+        if (t.prunable) {
+            n_prunable += numel;
+            ++seg_count;
+        }
+    }
+    if (scope == DNNS_SCOPE_GLOBAL) {
+        if (n_prunable >= (1ull << 32)) return DNNS_ERR_UNSUPPORTED;
+        c->S = n_prunable ? 1 : 0;
+    } else {
+        c->S = (uint32_t)seg_count;
+    }
+    std::vector<char> has_bn(m->n_tensors, 0);
+    for (int b = 0; b < m->n_bn; ++b) {
+        const dnns_bn& bn = m->bns[b];
+        if (!bn.gamma || !bn.beta || !bn.mean || !bn.var) return DNNS_ERR_INVALID_ARG;
+        if (bn.tensor < 0 || bn.tensor >= m->n_tensors) return DNNS_ERR_BAD_GRAPH;
+        if (bn.C != m->tensors[bn.tensor].O) return DNNS_ERR_BAD_GRAPH;
+        if (has_bn[bn.tensor]) return DNNS_ERR_BAD_GRAPH;
+        has_bn[bn.tensor] = 1;
+    }
+    c->items = c->T + 4 * c->B + c->n_bias;
+    return DNNS_OK;
+}
+
+WsMap map_workspace(const Counts& c, int32_t maxv) {
+    WsMap w{};
+    uint64_t o = 0;
+    auto take = [&](uint64_t bytes) {
+        const uint64_t at = o;
+        o = align_up(o + bytes);
+        return at;
+    };
+    w.tensors = take(sizeof(TensorDesc) * c.T);
+    w.groups = take(sizeof(GroupDesc) * c.G);
+    w.bns = take(sizeof(BnDesc) * (c.B ? c.B : 1));
+    w.segs = take(sizeof(SegDesc) * (c.S ? c.S : 1));
+    w.items = take(sizeof(ItemDesc) * c.items);
+    w.tile_tensor = take(4ull * c.tiles);
+    w.prod_list = take(4ull * c.T);
+    w.cons_list = take(4ull * c.T);
+    w.status = take(4);
+    w.tables_end = o;
+    const uint64_t vs = (uint64_t)maxv * (c.S ? c.S : 1);
+    w.k_dev = take(8 * vs);
+    w.bitmap = take(4ull * kBitmapWords * (c.S ? c.S : 1));
+    w.sel = take(sizeof(SelectState) * vs);
+    w.tie_prefix = take(4ull * maxv * c.tiles);
+    w.unit_prefix = take(4ull * (c.items + 1));
+    w.item_off = take(8ull * c.items);
+    w.item_dims = take(8ull * c.items);
+    w.clear_begin = o;
+    w.any_need = take(4);
+    w.need = take(4 * vs);
+    w.tile_ties = take(4ull * maxv * c.tiles);
+    w.hist1 = take(4ull * kHistBins * (c.S ? c.S : 1));
+    w.hist2 = take(c.dtype == DNNS_F32 ? 4ull * kLowBins * vs : 0);
+    w.total = o;
+    return w;
+}
+
+}  // namespace
+
+struct dnns_plan {
+    Counts c;
+    WsMap map;
+    dnns_scope scope;
+    int32_t maxv;
+    int n_sm;
+    char* ws;
+    Tables tb;
+    ThresholdWs tws;
+    CompactWs cws;
+    uint64_t launches;
+    int last_n_k;
+    // host-side layout, handed out by dnns_plan_layout
+    std::vector<uint64_t> arena_off, mask_off, nzmap_off, outnz_off, innz_off, keep_off, keepidx_off, seg_size;
+    std::vector<int32_t> seg_of_tensor;
+    dnns_layout layout;
+};
+
+extern "C" {
+
+const char* dnns_status_string(dnns_status s) {
+    switch (s) {
+        case DNNS_OK: return "ok";
+        case DNNS_ERR_INVALID_ARG: return "invalid argument";
+        case DNNS_ERR_BAD_GRAPH: return "inconsistent model graph";
+        case DNNS_ERR_WORKSPACE: return "workspace or destination arena too small";
+        case DNNS_ERR_UNSUPPORTED: return "unsupported dtype or extent";
+        case DNNS_ERR_CUDA: return "CUDA runtime error";
+        case DNNS_ERR_TIMEOUT: return "device-side wait expired";
+    }
+    return "unknown status";
+}
+
+size_t dnns_workspace_bytes(const dnns_model* model, dnns_scope scope, int32_t max_variants) {
+    Counts c;
+    if (inspect(model, scope, max_variants, &c) != DNNS_OK) return 0;
+    return (size_t)map_workspace(c, max_variants).total;
+}
+
+dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv, void* ws_dev, size_t ws_bytes,
+                             void* stream, dnns_plan** plan_out) {
+    if (!plan_out) return DNNS_ERR_INVALID_ARG;
+    *plan_out = nullptr;
+    Counts c;
+    dnns_status s = inspect(m, scope, maxv, &c);
+    if (s != DNNS_OK) return s;
+    if (!ws_dev || (reinterpret_cast<uintptr_t>(ws_dev) & (kAlign - 1))) return DNNS_ERR_INVALID_ARG;
+    const WsMap map = map_workspace(c, maxv);
+    if (ws_bytes < map.total) return DNNS_ERR_WORKSPACE;
+
+    dnns_plan* p = new (std::nothrow) dnns_plan();
+    if (!p) return DNNS_ERR_INVALID_ARG;
+    p->c = c, p->map = map, p->scope = scope, p->maxv = maxv, p->ws = static_cast<char*>(ws_dev);
+    p->launches = 0, p->last_n_k = 0;
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&p->n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        init_kernel_attributes() != cudaSuccess) {
+        delete p;
+        return DNNS_ERR_CUDA;
+    }
+
+    // ---- build the tables on the host
+    std::vector<char> host(map.tables_end, 0);
+    auto* td = reinterpret_cast<TensorDesc*>(host.data() + map.tensors);
+    auto* gd = reinterpret_cast<GroupDesc*>(host.data() + map.groups);
+    auto* bd = reinterpret_cast<BnDesc*>(host.data() + map.bns);
+    auto* sd = reinterpret_cast<SegDesc*>(host.data() + map.segs);
+    auto* id = reinterpret_cast<ItemDesc*>(host.data() + map.items);
+    auto* tile_tensor = reinterpret_cast<uint32_t*>(host.data() + map.tile_tensor);
+    auto* prod_list = reinterpret_cast<int32_t*>(host.data() + map.prod_list);
+    auto* cons_list = reinterpret_cast<int32_t*>(host.data() + map.cons_list);
+
+    p->arena_off.resize(c.T), p->mask_off.resize(c.T), p->nzmap_off.resize(c.T), p->outnz_off.resize(c.T);
+    p->innz_off.resize(c.T), p->seg_of_tensor.assign(c.T, -1), p->keep_off.resize(c.G), p->keepidx_off.resize(c.G);
+    p->seg_size.assign(c.S ? c.S : 1, 0);
+    uint64_t arena = 0, mask_w = 0, map_w = 0, out_w = 0, in_w = 0, compact_bytes = 0, n_prunable = 0;
+    uint32_t tile = 0, seg = 0;
+    for (uint32_t S = 0; S < c.S; ++S) sd[S] = SegDesc{0xFFFFFFFFu, 0, 0};
+    for (uint32_t i = 0; i < c.T; ++i) {
+        const dnns_tensor& t = m->tensors[i];
+        TensorDesc& d = td[i];
+        d.src = t.data, d.bias = t.bias;
+        d.numel = (uint32_t)((uint64_t)t.O * t.I * t.KH * t.KW);
+        d.O = t.O, d.I = t.I, d.KK = t.KH * t.KW, d.S = t.in_spatial;
+        d.out_group = t.out_group, d.in_group = t.in_group;
+        d.bn = -1;
+        d.arena_off = arena, p->arena_off[i] = arena;
+        arena = align_up(arena + (uint64_t)d.numel * c.elem_bytes);
+        d.tile0 = tile;
+        d.n_tiles = (uint32_t)(((uint64_t)d.numel * c.elem_bytes + kTileBytes - 1) / kTileBytes);
+        for (uint32_t k = 0; k < d.n_tiles; ++k) tile_tensor[tile + k] = i;
+        d.off_mask = (uint32_t)mask_w, p->mask_off[i] = mask_w, mask_w += ((uint64_t)d.numel + 31) / 32;
+        d.off_nzmap = (uint32_t)map_w, p->nzmap_off[i] = map_w, map_w += ((uint64_t)t.O * t.I + 31) / 32;
+        d.off_outnz = (uint32_t)out_w, p->outnz_off[i] = out_w, out_w += ((uint64_t)t.O + 31) / 32;
+        d.off_innz = (uint32_t)in_w, p->innz_off[i] = in_w, in_w += ((uint64_t)t.I + 31) / 32;
+        d.seg = -1;
+        if (t.prunable) {
+            const uint32_t sgi = scope == DNNS_SCOPE_GLOBAL ? 0 : seg++;
+            d.seg = (int32_t)sgi;
+            p->seg_of_tensor[i] = (int32_t)sgi;
+            if (sd[sgi].tile_begin == 0xFFFFFFFFu) sd[sgi].tile_begin = tile;
+            sd[sgi].tile_end = tile + d.n_tiles;
+            sd[sgi].size += d.numel;
+            p->seg_size[sgi] += d.numel;
+            n_prunable += d.numel;
+        }
+        tile += d.n_tiles;
+    }
+    if (mask_w >= (1ull << 32) || map_w >= (1ull << 32)) {
+        delete p;
+        return DNNS_ERR_UNSUPPORTED;
+    }
+    for (uint32_t S = 0; S < c.S; ++S)
+        if (p->seg_size[S] >= (1ull << 32)) {
+            delete p;
+            return DNNS_ERR_UNSUPPORTED;
+        }
+    uint64_t keep_w = 0, keep_i = 0;
+    int np = 0, nc = 0;
+    for (uint32_t g = 0; g < c.G; ++g) {
+        GroupDesc& G = gd[g];
+        G.C = m->groups[g].C, G.flags = m->groups[g].flags;
+        G.off_bits = (uint32_t)keep_w, p->keep_off[g] = keep_w, keep_w += ((uint64_t)G.C + 31) / 32;
+        G.off_idx = (uint32_t)keep_i, p->keepidx_off[g] = keep_i, keep_i += G.C;
+        G.prod_begin = np;
+        for (uint32_t i = 0; i < c.T; ++i)
+            if (m->tensors[i].out_group == (int)g) prod_list[np++] = (int32_t)i;
+        G.prod_end = np;
+        G.cons_begin = nc;
+        for (uint32_t i = 0; i < c.T; ++i)
+            if (m->tensors[i].in_group == (int)g) cons_list[nc++] = (int32_t)i;
+        G.cons_end = nc;
+    }
+    for (uint32_t b = 0; b < c.B; ++b) {
+        const dnns_bn& bn = m->bns[b];
+        bd[b] = BnDesc{bn.gamma, bn.beta, bn.mean, bn.var, bn.C, bn.tensor};
+        td[bn.tensor].bn = (int32_t)b;
+    }
+    // gather items: weights, then BN vectors, then biases
+    uint32_t n_it = 0;
+    for (uint32_t i = 0; i < c.T; ++i) {
+        const dnns_tensor& t = m->tensors[i];
+        id[n_it++] = ItemDesc{nullptr, (int32_t)i, t.O, t.I / t.in_spatial, t.KH * t.KW * t.in_spatial,
+                              t.out_group, t.in_group, c.elem_bytes};
+        compact_bytes += align_up((uint64_t)td[i].numel * c.elem_bytes);
+    }
+    for (uint32_t b = 0; b < c.B; ++b) {
+        const dnns_bn& bn = m->bns[b];
+        const float* vec[4] = {bn.gamma, bn.beta, bn.mean, bn.var};
+        for (int k = 0; k < 4; ++k) {
+            id[n_it++] = ItemDesc{vec[k], -1, bn.C, 1, 1, m->tensors[bn.tensor].out_group, -1, 4};
+            compact_bytes += align_up(4ull * bn.C);
+        }
+    }
+    for (uint32_t i = 0; i < c.T; ++i)
+        if (m->tensors[i].bias) {
+            id[n_it++] = ItemDesc{m->tensors[i].bias, -1, m->tensors[i].O, 1, 1, m->tensors[i].out_group, -1, 4};
+            compact_bytes += align_up(4ull * m->tensors[i].O);
+        }
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(p->ws, host.data(), map.tables_end, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        delete p;
+        return DNNS_ERR_CUDA;
+    }
+
+    char* w = p->ws;
+    Tables& tb = p->tb;
+    tb.tensors = reinterpret_cast<TensorDesc*>(w + map.tensors);
+    tb.groups = reinterpret_cast<GroupDesc*>(w + map.groups);
+    tb.bns = reinterpret_cast<BnDesc*>(w + map.bns);
+    tb.segs = reinterpret_cast<SegDesc*>(w + map.segs);
+    tb.items = reinterpret_cast<ItemDesc*>(w + map.items);
+    tb.tile_tensor = reinterpret_cast<uint32_t*>(w + map.tile_tensor);
+    tb.prod_list = reinterpret_cast<int32_t*>(w + map.prod_list);
+    tb.cons_list = reinterpret_cast<int32_t*>(w + map.cons_list);
+    tb.status = reinterpret_cast<uint32_t*>(w + map.status);
+    tb.n_tensors = c.T, tb.n_groups = c.G, tb.n_bn = c.B, tb.n_segs = c.S, tb.n_items = c.items, tb.n_tiles = c.tiles;
+    tb.tile_elems = kTileBytes / c.elem_bytes;
+    tb.dtype = c.dtype;
+    ThresholdWs& t = p->tws;
+    t.k_dev = reinterpret_cast<uint64_t*>(w + map.k_dev);
+    t.hist1 = reinterpret_cast<uint32_t*>(w + map.hist1);
+    t.hist2 = reinterpret_cast<uint32_t*>(w + map.hist2);
+    t.bitmap = reinterpret_cast<uint32_t*>(w + map.bitmap);
+    t.sel = reinterpret_cast<SelectState*>(w + map.sel);
+    t.need = reinterpret_cast<uint32_t*>(w + map.need);
+    t.any_need = reinterpret_cast<uint32_t*>(w + map.any_need);
+    t.tile_ties = reinterpret_cast<uint32_t*>(w + map.tile_ties);
+    t.tie_prefix = reinterpret_cast<uint32_t*>(w + map.tie_prefix);
+    p->cws.unit_prefix = reinterpret_cast<uint32_t*>(w + map.unit_prefix);
+    p->cws.item_off = reinterpret_cast<uint64_t*>(w + map.item_off);
+    p->cws.item_dims = reinterpret_cast<int32_t*>(w + map.item_dims);
+
+    dnns_layout& L = p->layout;
+    L.n_tensors = c.T, L.n_bn = c.B, L.n_groups = c.G, L.n_segments = c.S, L.n_bias = c.n_bias;
+    L.elem_bytes = c.elem_bytes;
+    L.n_prunable = n_prunable;
+    L.masked_arena_bytes = arena;
+    L.mask_words = mask_w, L.nz_map_words = map_w, L.out_nz_words = out_w, L.in_nz_words = in_w;
+    L.keep_words = keep_w, L.keep_idx_len = keep_i;
+    L.compact_arena_bytes = compact_bytes;
+    L.n_compact_items = (int32_t)c.items;
+    L.arena_offset = p->arena_off.data(), L.mask_offset = p->mask_off.data(), L.nz_map_offset = p->nzmap_off.data();
+    L.out_nz_offset = p->outnz_off.data(), L.in_nz_offset = p->innz_off.data();
+    L.keep_offset = p->keep_off.data(), L.keep_idx_offset = p->keepidx_off.data();
+    L.segment_size = p->seg_size.data(), L.segment_of_tensor = p->seg_of_tensor.data();
+    *plan_out = p;
+    return DNNS_OK;
+}
+
+void dnns_plan_destroy(dnns_plan* plan) {
+    if (!plan) return;
+    cudaDeviceSynchronize();
+    delete plan;
+}
+
+dnns_status dnns_plan_layout(const dnns_plan* plan, dnns_layout* out) {
+    if (!plan || !out) return DNNS_ERR_INVALID_ARG;
+    *out = plan->layout;
+    return DNNS_OK;
+}
+
+uint64_t dnns_plan_launch_count(const dnns_plan* plan) { return plan ? plan->launches : 0; }
+
+dnns_status dnns_magnitude_threshold(dnns_plan* p, const uint64_t* k, int32_t n_k, dnns_threshold* thr_dev,
+                                     void* stream) {
+    if (!p || !k || !thr_dev || n_k < 1 || n_k > p->maxv) return DNNS_ERR_INVALID_ARG;
+    const uint32_t S = p->c.S;
+    if (S == 0) return DNNS_OK;
+    for (int v = 0; v < n_k; ++v)
+        for (uint32_t s = 0; s < S; ++s)
+            if (k[(size_t)v * S + s] > p->seg_size[s]) return DNNS_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint64_t clear_end = p->map.hist2 + (p->c.dtype == DNNS_F32 ? 4ull * kLowBins * S * n_k : 0);
+    if (cudaMemsetAsync(p->ws + p->map.clear_begin, 0, clear_end - p->map.clear_begin, st) != cudaSuccess)
+        return DNNS_ERR_CUDA;
+    if (cudaMemcpyAsync(p->tws.k_dev, k, 8ull * n_k * S, cudaMemcpyHostToDevice, st) != cudaSuccess) return DNNS_ERR_CUDA;
+    const int n = launch_threshold(p->tb, p->tws, n_k, n_k, thr_dev, p->n_sm, st);
+    if (n < 0) return DNNS_ERR_CUDA;
+    p->launches += n;
+    p->last_n_k = n_k;
+    return DNNS_OK;
+}
+
+dnns_status dnns_apply_mask(dnns_plan* p, const dnns_threshold* thr_dev, int32_t variant, void* masked_arena,
+                            uint32_t* mask_bits, void* stream) {
+    if (!p || !thr_dev || variant < 0 || variant >= p->maxv) return DNNS_ERR_INVALID_ARG;
+    if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
+    const int n = launch_tile_sweep(p->tb, p->tws, true, false, thr_dev, variant, nullptr, masked_arena, mask_bits,
+                                    nullptr, nullptr, nullptr, p->n_sm, static_cast<cudaStream_t>(stream));
+    if (n < 0) return DNNS_ERR_CUDA;
+    p->launches += n;
+    return DNNS_OK;
+}
+
+dnns_status dnns_zero_structures(dnns_plan* p, const void* masked_arena, uint32_t* nz_map, uint32_t* out_nz,
+                                 uint32_t* in_nz, void* stream) {
+    if (!p || !out_nz || !in_nz) return DNNS_ERR_INVALID_ARG;
+    if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dnns_layout& L = p->layout;
+    if (cudaMemsetAsync(out_nz, 0, 4 * L.out_nz_words, st) != cudaSuccess ||
+        cudaMemsetAsync(in_nz, 0, 4 * L.in_nz_words, st) != cudaSuccess ||
+        (nz_map && cudaMemsetAsync(nz_map, 0, 4 * L.nz_map_words, st) != cudaSuccess))
+        return DNNS_ERR_CUDA;
+    const int n = launch_tile_sweep(p->tb, p->tws, false, true, nullptr, 0, masked_arena, nullptr, nullptr, nz_map,
+                                    out_nz, in_nz, p->n_sm, st);
+    if (n < 0) return DNNS_ERR_CUDA;
+    p->launches += n;
+    return DNNS_OK;
+}
+
+dnns_status dnns_propagate_keep(dnns_plan* p, const uint32_t* out_nz, const uint32_t* in_nz, uint32_t policy,
+                                int32_t min_keep, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count,
+                                uint64_t* stats, void* stream) {
+    if (!p || !out_nz || !in_nz || !keep_bits || !keep_idx || !keep_count) return DNNS_ERR_INVALID_ARG;
+    if (policy & ~(uint32_t)(DNNS_RULE_PRODUCER | DNNS_RULE_CONSUMER | DNNS_SHIFT_STRICT)) return DNNS_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (stats && cudaMemsetAsync(stats, 0, 32, st) != cudaSuccess) return DNNS_ERR_CUDA;
+    const int n = launch_propagate(p->tb, out_nz, in_nz, policy, min_keep, keep_bits, keep_idx, keep_count, stats, st);
+    if (n < 0) return DNNS_ERR_CUDA;
+    p->launches += n;
+    return DNNS_OK;
+}
+
+dnns_status dnns_compact(dnns_plan* p, const void* masked_arena, const int32_t* keep_idx, const int32_t* keep_count,
+                         void* dst_arena, size_t dst_bytes, uint64_t* dst_offsets_dev, int32_t* dst_shapes_dev,
+                         void* stream) {
+    if (!p || !keep_idx || !keep_count || !dst_arena || !dst_offsets_dev || !dst_shapes_dev) return DNNS_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) ||
+        (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)))
+        return DNNS_ERR_INVALID_ARG;
+    const int n = launch_compact(p->tb, p->cws, masked_arena, keep_idx, keep_count, dst_arena, dst_bytes,
+                                 dst_offsets_dev, dst_shapes_dev, p->n_sm, static_cast<cudaStream_t>(stream));
+    if (n < 0) return DNNS_ERR_CUDA;
+    p->launches += n;
+    return DNNS_OK;
+}
+
+dnns_status dnns_last_device_status(dnns_plan* p, void* stream) {
+    if (!p) return DNNS_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t s = 0;
+    if (cudaMemcpyAsync(&s, p->tb.status, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemsetAsync(p->tb.status, 0, 4, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+        return DNNS_ERR_CUDA;
+    return static_cast<dnns_status>(s);
+}
+
+}  // extern "C"

@@ -1,0 +1,234 @@
+"""Device-side plumbing around the C ABI: torch is used for device memory and streams only.
+
+``DeviceModel`` puts a workload's arrays on the GPU and fills the ``dnns_model`` descriptors;
+``Session`` owns a plan, its workspace and one set of output buffers, and exposes the five
+steps plus read-back helpers.  No step of the method is computed here.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+REC_DTYPE = np.dtype([("tau_bits", "<u4"), ("pad", "<u4"), ("n_below", "<u8"), ("n_tie", "<u8"), ("n_equal", "<u8")])
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _to_dev(a: np.ndarray, device) -> torch.Tensor:
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.uint16:
+        a = a.view(np.int16)
+    elif a.dtype == np.uint32:
+        a = a.view(np.int32)
+    return torch.from_numpy(a).to(device)
+
+
+class DeviceModel:
+    """A workload's tensors, BatchNorm vectors and biases resident on one GPU."""
+
+    def __init__(self, wl, dtype: int = B.DNNS_F32, device="cuda:0", weights: Optional[List[np.ndarray]] = None,
+                 pinned_host: bool = False):
+        self.wl, self.dtype, self.device = wl, dtype, torch.device(device)
+        host_w = weights if weights is not None else wl.weights_as(dtype)
+        self.elem_bytes = 4 if dtype == B.DNNS_F32 else 2
+        # one allocation for all weights (256-byte aligned pieces) so that a host copy is one transfer
+        offs, o = [], 0
+        for w in host_w:
+            offs.append(o)
+            o = (o + w.size * self.elem_bytes + 255) // 256 * 256
+        self.weight_offsets, self.weight_bytes = offs, o
+        host = torch.zeros(o, dtype=torch.uint8)
+        hv = host.numpy()
+        for w, off in zip(host_w, offs):
+            hv[off: off + w.size * self.elem_bytes] = np.ascontiguousarray(w).view(np.uint8).ravel()
+        self.host_weights = host.pin_memory() if pinned_host else host
+        self.weights = torch.empty(o, dtype=torch.uint8, device=self.device)
+        self.weights.copy_(self.host_weights)
+        self.biases = [None if b is None else _to_dev(b.astype(np.float32), self.device) for b in wl.biases]
+        self.bn = [tuple(_to_dev(np.asarray(v, np.float32), self.device) for v in p) for p in wl.bn_params]
+        self._t = (B.dnns_tensor * len(wl.tensors))()
+        base = self.weights.data_ptr()
+        for i, t in enumerate(wl.tensors):
+            self._t[i] = B.dnns_tensor(base + offs[i], dtype, t.O, t.I, t.KH, t.KW, t.in_spatial, int(t.prunable),
+                                       t.out_group, t.in_group,
+                                       None if self.biases[i] is None else self.biases[i].data_ptr())
+        self._b = (B.dnns_bn * max(1, len(wl.bns)))()
+        for i, b in enumerate(wl.bns):
+            g, be, mu, va = self.bn[i]
+            self._b[i] = B.dnns_bn(g.data_ptr(), be.data_ptr(), mu.data_ptr(), va.data_ptr(), b.C, b.tensor, b.eps)
+        self._g = (B.dnns_group * len(wl.groups))()
+        for i, g in enumerate(wl.groups):
+            self._g[i] = B.dnns_group(g.C, g.flags)
+        self.c = B.dnns_model(len(wl.tensors), self._t, len(wl.bns), self._b, len(wl.groups), self._g)
+
+    def upload_weights(self):
+        """Host-to-device copy of all weights (one transfer from the host staging buffer)."""
+        self.weights.copy_(self.host_weights, non_blocking=True)
+
+
+class Session:
+    """A plan with its workspace and one set of output buffers for one variant at a time."""
+
+    def __init__(self, dm: DeviceModel, scope: int, max_variants: int, want_mask_bits: bool = True,
+                 want_nz_map: bool = True):
+        self.dm, self.scope, self.max_variants = dm, scope, max_variants
+        dev = dm.device
+        nbytes = B.dnns_workspace_bytes(dm.c, scope, max_variants)
+        if nbytes == 0:
+            raise B.DnnsError(B.DNNS_ERR_INVALID_ARG, "dnns_workspace_bytes")
+        self.ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        self.plan = B.dnns_plan_create(dm.c, scope, max_variants, self.ws.data_ptr(), nbytes, _stream())
+        L = B.dnns_plan_layout(self.plan)
+        self.L = L
+        T, G, S = L.n_tensors, L.n_groups, L.n_segments
+        self.n_segments = S
+        arr = lambda p, n, dt: np.array([p[i] for i in range(n)], dt)
+        self.arena_offset = arr(L.arena_offset, T, np.uint64)
+        self.mask_offset = arr(L.mask_offset, T, np.uint64)
+        self.nz_map_offset = arr(L.nz_map_offset, T, np.uint64)
+        self.out_nz_offset = arr(L.out_nz_offset, T, np.uint64)
+        self.in_nz_offset = arr(L.in_nz_offset, T, np.uint64)
+        self.keep_offset = arr(L.keep_offset, G, np.uint64)
+        self.keep_idx_offset = arr(L.keep_idx_offset, G, np.uint64)
+        self.segment_size = arr(L.segment_size, max(S, 1), np.uint64)
+        i32 = lambda n: torch.zeros(max(int(n), 1), dtype=torch.int32, device=dev)
+        self.thr = torch.zeros(max_variants * max(S, 1) * REC_DTYPE.itemsize, dtype=torch.uint8, device=dev)
+        self.masked = torch.empty(int(L.masked_arena_bytes), dtype=torch.uint8, device=dev)
+        self.mask_bits = i32(L.mask_words) if want_mask_bits else None
+        self.nz_map = i32(L.nz_map_words) if want_nz_map else None
+        self.out_nz, self.in_nz = i32(L.out_nz_words), i32(L.in_nz_words)
+        self.keep_bits, self.keep_idx = i32(L.keep_words), i32(L.keep_idx_len)
+        self.keep_count = i32(G)
+        self.stats = torch.zeros(4, dtype=torch.int64, device=dev)
+        self.compact_arena = torch.empty(int(L.compact_arena_bytes), dtype=torch.uint8, device=dev)
+        self.dst_offsets = torch.zeros(L.n_compact_items, dtype=torch.int64, device=dev)
+        self.dst_shapes = i32(2 * T)
+
+    def close(self):
+        if self.plan is not None:
+            B.dnns_plan_destroy(self.plan)
+            self.plan = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- the five steps -------------------------------------------------------------
+    def magnitude_threshold(self, ks: np.ndarray):
+        ks = np.ascontiguousarray(ks, np.uint64)
+        assert ks.ndim == 2 and ks.shape[1] == self.n_segments
+        self.n_k = ks.shape[0]
+        B.dnns_magnitude_threshold(self.plan, ks.ravel().tolist(), ks.shape[0], self.thr.data_ptr(), _stream())
+
+    def apply_mask(self, variant: int, in_place: bool = False):
+        B.dnns_apply_mask(self.plan, self.thr.data_ptr(), variant, 0 if in_place else self.masked.data_ptr(),
+                          0 if self.mask_bits is None else self.mask_bits.data_ptr(), _stream())
+
+    def zero_structures(self, from_model: bool = False):
+        B.dnns_zero_structures(self.plan, 0 if from_model else self.masked.data_ptr(),
+                               0 if self.nz_map is None else self.nz_map.data_ptr(), self.out_nz.data_ptr(),
+                               self.in_nz.data_ptr(), _stream())
+
+    def propagate_keep(self, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1):
+        B.dnns_propagate_keep(self.plan, self.out_nz.data_ptr(), self.in_nz.data_ptr(), policy, min_keep,
+                              self.keep_bits.data_ptr(), self.keep_idx.data_ptr(), self.keep_count.data_ptr(),
+                              self.stats.data_ptr(), _stream())
+
+    def compact(self, from_model: bool = False, dst_bytes: Optional[int] = None):
+        B.dnns_compact(self.plan, 0 if from_model else self.masked.data_ptr(), self.keep_idx.data_ptr(),
+                       self.keep_count.data_ptr(), self.compact_arena.data_ptr(),
+                       self.compact_arena.numel() if dst_bytes is None else dst_bytes, self.dst_offsets.data_ptr(),
+                       self.dst_shapes.data_ptr(), _stream())
+
+    def variant(self, v: int, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1):
+        """Steps 2-5 for variant v of the latest threshold call."""
+        self.apply_mask(v)
+        self.zero_structures()
+        self.propagate_keep(policy, min_keep)
+        self.compact()
+
+    def device_status(self) -> int:
+        return B.dnns_last_device_status(self.plan, _stream())
+
+    def launch_count(self) -> int:
+        return B.dnns_plan_launch_count(self.plan)
+
+    # ---- read-back (host copies, for tests and reports) ------------------------------------
+    def records(self) -> np.ndarray:
+        n = self.n_k * self.n_segments
+        raw = self.thr.cpu().numpy()[: n * REC_DTYPE.itemsize]
+        return raw.view(REC_DTYPE).reshape(self.n_k, self.n_segments).copy()
+
+    def _np_dtype(self):
+        return np.float32 if self.dm.dtype == B.DNNS_F32 else np.uint16
+
+    def masked_tensors(self, in_place: bool = False) -> List[np.ndarray]:
+        wl, eb = self.dm.wl, self.dm.elem_bytes
+        if in_place:
+            raw, offs = self.dm.weights.cpu().numpy(), self.dm.weight_offsets
+        else:
+            raw, offs = self.masked.cpu().numpy(), self.arena_offset
+        return [raw[int(o): int(o) + t.numel * eb].view(self._np_dtype()).reshape(t.O, t.I, t.KH, t.KW).copy()
+                for t, o in zip(wl.tensors, offs)]
+
+    def _split_words(self, buf, offsets, nbits) -> List[np.ndarray]:
+        raw = buf.cpu().numpy().view(np.uint32)
+        return [raw[int(o): int(o) + (n + 31) // 32].copy() for o, n in zip(offsets, nbits)]
+
+    def mask_words(self):
+        return self._split_words(self.mask_bits, self.mask_offset, [t.numel for t in self.dm.wl.tensors])
+
+    def structure_words(self):
+        wl = self.dm.wl
+        nz = None if self.nz_map is None else self._split_words(self.nz_map, self.nz_map_offset,
+                                                                 [t.O * t.I for t in wl.tensors])
+        return (nz, self._split_words(self.out_nz, self.out_nz_offset, [t.O for t in wl.tensors]),
+                self._split_words(self.in_nz, self.in_nz_offset, [t.I for t in wl.tensors]))
+
+    def keep_sets(self):
+        wl = self.dm.wl
+        bits = self._split_words(self.keep_bits, self.keep_offset, [g.C for g in wl.groups])
+        cnt = self.keep_count.cpu().numpy()[: len(wl.groups)].copy()
+        idx_raw = self.keep_idx.cpu().numpy()
+        idx = [idx_raw[int(o): int(o) + int(c)].copy() for o, c in zip(self.keep_idx_offset, cnt)]
+        return bits, idx, cnt, self.stats.cpu().numpy().view(np.uint64).copy()
+
+    def compacted(self):
+        """(weights [(O', I', KH, KW)], bn [(g, b, m, v)], biases, shapes (T, 2), offsets)."""
+        wl, eb = self.dm.wl, self.dm.elem_bytes
+        T = len(wl.tensors)
+        offs = self.dst_offsets.cpu().numpy().view(np.uint64)
+        shapes = self.dst_shapes.cpu().numpy()[: 2 * T].reshape(T, 2).copy()
+        raw = self.compact_arena.cpu().numpy()
+        ws = []
+        for i, t in enumerate(wl.tensors):
+            On, In = int(shapes[i, 0]), int(shapes[i, 1])
+            n = On * In * t.KH * t.KW
+            ws.append(raw[int(offs[i]): int(offs[i]) + n * eb].view(self._np_dtype()).reshape(On, In, t.KH, t.KW).copy())
+        cnt = self.keep_count.cpu().numpy()
+        bns, k = [], T
+        for b in wl.bns:
+            Cn = int(cnt[wl.tensors[b.tensor].out_group])
+            vecs = []
+            for _ in range(4):
+                vecs.append(raw[int(offs[k]): int(offs[k]) + 4 * Cn].view(np.float32).copy())
+                k += 1
+            bns.append(tuple(vecs))
+        biases = []
+        for i, t in enumerate(wl.tensors):
+            if wl.biases[i] is None:
+                biases.append(None)
+            else:
+                On = int(shapes[i, 0])
+                biases.append(raw[int(offs[k]): int(offs[k]) + 4 * On].view(np.float32).copy())
+                k += 1
+        return ws, bns, biases, shapes, offs.copy()

@@ -1,0 +1,75 @@
+"""Shared driver of the GPU parity tests: run the CUDA path and the oracle on the same seeded
+workload and compare every output bit for bit."""
+import numpy as np
+
+from oracle import oracle as O
+from paper_2309_06973_b200 import binding as B
+from paper_2309_06973_b200.runtime import DeviceModel, Session
+
+
+def assert_words(a, b, what):
+    assert len(a) == len(b), what
+    for i, (x, y) in enumerate(zip(a, b)):
+        assert np.array_equal(np.asarray(x).view(np.uint32), np.asarray(y).view(np.uint32)), f"{what}[{i}]"
+
+
+def bits_eq(a, b):
+    a, b = np.ascontiguousarray(a), np.ascontiguousarray(b)
+    return a.shape == b.shape and np.array_equal(a.view(np.uint8), b.view(np.uint8))
+
+
+def expected_offsets(sizes_bytes):
+    """Destination offsets rule: items in order, each at the next multiple of 256 bytes."""
+    out, o = [], 0
+    for s in sizes_bytes:
+        out.append(o)
+        o = (o + s + 255) // 256 * 256
+    return out
+
+
+def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCER | O.RULE_CONSUMER, min_keep=1,
+                      weights=None, check_structure_maps=True):
+    """Thresholds for all of wl.ks in one call, then steps 2-5 for the chosen variants."""
+    om = O.OracleModel(wl, dtype, weights)
+    dm = DeviceModel(wl, dtype, weights=weights)
+    ses = Session(dm, wl.scope, len(wl.ks))
+    ses.magnitude_threshold(wl.ks)
+    rec_gpu = ses.records()
+    rec_cpu = O.threshold(om, wl.scope, wl.ks)
+    for f in ("tau_bits", "n_below", "n_tie", "n_equal"):
+        assert np.array_equal(rec_gpu[f], rec_cpu[f]), f
+    eb = 4 if dtype == B.DNNS_F32 else 2
+    for v in (range(len(wl.ks)) if variants is None else variants):
+        ses.variant(v, policy, min_keep)
+        assert ses.device_status() == B.DNNS_OK
+        masked_cpu, bits_cpu = O.apply_mask(om, wl.scope, rec_cpu[v])
+        for i, (a, b) in enumerate(zip(ses.masked_tensors(), masked_cpu.weights)):
+            assert bits_eq(a, b), f"masked weights, variant {v}, tensor {i}"
+        assert_words(ses.mask_words(), bits_cpu, f"mask bits v{v}")
+        nz_c, out_c, in_c = O.zero_structures(masked_cpu)
+        nz_g, out_g, in_g = ses.structure_words()
+        if check_structure_maps:
+            assert_words(nz_g, nz_c, f"kernel map v{v}")
+        assert_words(out_g, out_c, f"out flags v{v}")
+        assert_words(in_g, in_c, f"in flags v{v}")
+        kb_c, ki_c, kc_c, st_c = O.propagate_keep(masked_cpu, out_c, in_c, policy, min_keep)
+        kb_g, ki_g, kc_g, st_g = ses.keep_sets()
+        assert np.array_equal(kc_g, kc_c), f"keep counts v{v}"
+        assert_words(kb_g, kb_c, f"keep bits v{v}")
+        for g, (a, b) in enumerate(zip(ki_g, ki_c)):
+            assert np.array_equal(a, b[: kc_c[g]]), f"keep idx v{v} group {g}"
+        assert st_g.tolist() == st_c.tolist(), f"stats v{v}"
+        cw_c, cbn_c, cb_c, sh_c = O.compact(masked_cpu, ki_c, kc_c)
+        cw_g, cbn_g, cb_g, sh_g, offs = ses.compacted()
+        assert np.array_equal(sh_g, sh_c), f"shapes v{v}"
+        for i, (a, b) in enumerate(zip(cw_g, cw_c)):
+            assert bits_eq(a, b), f"compacted weights v{v} tensor {i}"
+        for i, (a, b) in enumerate(zip(cbn_g, cbn_c)):
+            for x, y in zip(a, b):
+                assert bits_eq(x, y), f"compacted bn v{v} {i}"
+        for a, b in zip(cb_g, cb_c):
+            assert (a is None and b is None) or bits_eq(a, b)
+        sizes = [w.size * eb for w in cw_c] + [4 * len(x) for p in cbn_c for x in p] + \
+                [4 * len(b) for b in cb_c if b is not None]
+        assert offs.tolist() == expected_offsets(sizes), f"arena offsets v{v}"
+    return ses

@@ -1,0 +1,44 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration the benchmark uses: every
+output of the chosen variants is still compared element by element (the oracle needs some tens
+of seconds per model), plus the forward pass of the rebuilt model."""
+import numpy as np
+import pytest
+import torch
+
+from forward_ref import forward, silenced_reference
+from gpu_compare import compare_portfolio
+from paper_2309_06973_b200 import binding as B
+from paper_2309_06973_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def forward_check(wl, ses, dtype):
+    is_bf16 = dtype == B.DNNS_BF16
+    x = torch.from_numpy(np.random.default_rng(1).standard_normal((2, 3, wl.input_hw, wl.input_hw)).astype(np.float32))
+    cw, cbn, cb, _, _ = ses.compacted()
+    kb, _, _, _ = ses.keep_sets()
+    mw, mbn, mb = silenced_reference(wl, ses.masked_tensors(), wl.bn_params, wl.biases, kb)
+    y_ref = forward(wl, mw, mbn, mb, x, is_bf16)
+    y = forward(wl, cw, cbn, cb, x, is_bf16)
+    assert float((y - y_ref).abs().max()) <= 1e-5 * float(y_ref.abs().max())
+    assert float(y_ref.abs().max()) > 0
+
+
+def test_vgg16_per_layer_95():
+    wl = W.vgg16()
+    ses = compare_portfolio(wl, B.DNNS_F32, check_structure_maps=True)
+    forward_check(wl, ses, B.DNNS_F32)
+
+
+def test_resnet50_three_variants():
+    wl = W.resnet50()
+    ses = compare_portfolio(wl, B.DNNS_F32)
+    forward_check(wl, ses, B.DNNS_F32)
+
+
+@pytest.mark.parametrize("dtype", [B.DNNS_F32, B.DNNS_BF16])
+def test_resnet152_portfolio(dtype):
+    wl = W.resnet152()
+    ses = compare_portfolio(wl, dtype, variants=[0, 7])
+    forward_check(wl, ses, dtype)

@@ -1,0 +1,144 @@
+"""GPU parity: the CUDA path against the CPU oracle, element by element, on seeded workloads that
+span several tiles, ragged tails, odd shapes, both dtypes, both scopes and every policy."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_compare import compare_portfolio
+from oracle import oracle as O
+from paper_2309_06973_b200 import binding as B
+from paper_2309_06973_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("dtype", [B.DNNS_F32, B.DNNS_BF16])
+@pytest.mark.parametrize("make", [W.toy, lambda: W.small_resnet(seed=3), lambda: W.small_resnet(seed=4, bottleneck=False),
+                                  W.resnet56])
+def test_small_configs_every_variant(make, dtype):
+    compare_portfolio(make(), dtype)
+
+
+@pytest.mark.parametrize("policy", [O.RULE_PRODUCER, O.RULE_CONSUMER, O.RULE_PRODUCER | O.RULE_CONSUMER | O.SHIFT_STRICT])
+@pytest.mark.parametrize("min_keep", [0, 1, 5])
+def test_policies_and_min_keep(policy, min_keep):
+    wl = W.small_resnet(seed=8)
+    for (g, be, mu, va) in wl.bn_params:
+        be[::2] = 0.0
+        mu[::2] = 0.0
+    wl.ks = np.array([[W.k_fraction(wl.n_prunable, 97, 100)], [wl.n_prunable]], np.uint64)
+    compare_portfolio(wl, B.DNNS_F32, policy=policy, min_keep=min_keep)
+
+
+@pytest.mark.parametrize("dtype", [B.DNNS_F32, B.DNNS_BF16])
+def test_per_tensor_scope_and_odd_shapes(dtype):
+    # widths that are not multiples of 32, 5x5 kernels, ragged tiles
+    wl = W.chain([37, 70, 129, 33], seed=5, kernel=5, planted_frac=0.2)
+    wl.scope = W.SCOPE_PER_TENSOR
+    sizes = [t.numel for t in wl.tensors]
+    wl.ks = np.array([[0] * len(sizes), [n // 2 for n in sizes], [n * 9 // 10 for n in sizes],
+                      [n - 1 for n in sizes], sizes], np.uint64)
+    compare_portfolio(wl, dtype)
+
+
+def test_non_prunable_tensor_and_1x1_chain():
+    wl = W.chain([64, 96, 64, 256], seed=6, kernel=1, planted_frac=0.3)
+    wl.tensors[1].prunable = False
+    n = wl.n_prunable
+    wl.ks = np.array([[n // 3], [n * 19 // 20]], np.uint64)
+    compare_portfolio(wl, B.DNNS_F32)
+    compare_portfolio(wl, B.DNNS_BF16)
+
+
+def test_special_values_and_heavy_ties():
+    """Zeros, negative zeros, denormals, infinities, NaNs and many duplicates: ties split inside tiles."""
+    wl = W.chain([48, 64, 80], seed=7, planted_frac=0.5)
+    rng = np.random.default_rng(0)
+    for w in wl.weights:
+        flat = w.reshape(-1)
+        n = flat.size
+        flat[rng.integers(0, n, n // 8)] = -0.0
+        flat[rng.integers(0, n, n // 16)] = np.float32(1e-42)
+        flat[rng.integers(0, n, n // 32)] = np.inf
+        flat[rng.integers(0, n, n // 32)] = np.nan
+        flat[rng.integers(0, n, n // 4)] = np.float32(0.125)      # a big block of equal magnitudes
+        flat[rng.integers(0, n, n // 8)] = np.float32(-0.125)
+    n = wl.n_prunable
+    nz0 = sum(int(np.count_nonzero(w.view(np.uint32) & 0x7FFFFFFF == 0)) for w in wl.weights)
+    ks = [1, nz0 // 2, nz0, nz0 + 5, n // 2, n * 3 // 4, n - 3, n]
+    wl.ks = np.array(ks, np.uint64)[:, None]
+    ses = compare_portfolio(wl, B.DNNS_F32)
+    rec = ses.records()
+    assert (rec["n_tie"] < rec["n_equal"]).any()                   # the split-tie path really ran
+    compare_portfolio(wl, B.DNNS_BF16)
+
+
+def test_fc_with_spatial_columns():
+    b = W._Builder()
+    gi = b.group(3, frozen=True)
+    g1 = b.group(40)
+    gc = b.group(7, frozen=True)
+    b.conv_bn("c", "x", "a", gi, g1, 3, 1, 1)
+    b.fc("fc", "a", "out", g1, gc, in_spatial=9)
+    wl = W.Workload("fcS", 11, W.SCOPE_GLOBAL, b.tensors, b.bns, b.groups, b.ops, 3)
+    W._draw(wl, True, 0.5, 0.3)
+    wl.biases[1][:] = np.arange(7)
+    W._set_ks(wl, lambda n: [n // 2, n * 9 // 10])
+    compare_portfolio(wl, B.DNNS_F32)
+
+
+def test_sparse_model_straight_from_the_model_tensors():
+    """Phase 2 alone: structures and rebuild read the model's own (already sparse) tensors."""
+    from paper_2309_06973_b200.runtime import DeviceModel, Session
+    from gpu_compare import bits_eq
+    wl = W.small_resnet(seed=12)
+    om = O.OracleModel(wl)
+    rec = O.threshold(om, wl.scope, wl.ks)
+    sparse, _ = O.apply_mask(om, wl.scope, rec[-1])
+    dm = DeviceModel(wl, B.DNNS_F32, weights=sparse.weights)
+    ses = Session(dm, wl.scope, 1)
+    ses.zero_structures(from_model=True)
+    ses.propagate_keep()
+    ses.compact(from_model=True)
+    _, out_c, in_c = O.zero_structures(sparse)
+    kb, ki, kc, st = O.propagate_keep(sparse, out_c, in_c)
+    cw, *_ = O.compact(sparse, ki, kc)
+    for a, b in zip(ses.compacted()[0], cw):
+        assert bits_eq(a, b)
+
+
+def test_in_place_mask_and_small_destination_arena():
+    from paper_2309_06973_b200.runtime import DeviceModel, Session
+    from gpu_compare import bits_eq
+    wl = W.toy()
+    om = O.OracleModel(wl)
+    dm = DeviceModel(wl)
+    ses = Session(dm, wl.scope, 1)
+    ses.magnitude_threshold(wl.ks)
+    ses.apply_mask(0, in_place=True)
+    rec = O.threshold(om, wl.scope, wl.ks)
+    masked, _ = O.apply_mask(om, wl.scope, rec[0])
+    for a, b in zip(ses.masked_tensors(in_place=True), masked.weights):
+        assert bits_eq(a, b)
+    ses.zero_structures(from_model=True)
+    ses.propagate_keep()
+    ses.compact(from_model=True, dst_bytes=256)
+    assert ses.device_status() == B.DNNS_ERR_WORKSPACE            # reported, nothing copied
+    assert ses.device_status() == B.DNNS_OK                       # and cleared
+    with pytest.raises(B.DnnsError):
+        ses.magnitude_threshold(np.array([[wl.n_prunable + 1]], np.uint64))
+
+
+def test_two_runs_are_bit_identical():
+    wl = W.resnet56()
+    from paper_2309_06973_b200.runtime import DeviceModel, Session
+    outs = []
+    for _ in range(2):
+        dm = DeviceModel(wl, B.DNNS_BF16)
+        ses = Session(dm, wl.scope, len(wl.ks))
+        ses.magnitude_threshold(wl.ks)
+        ses.variant(7)
+        torch.cuda.synchronize()
+        outs.append((ses.masked.cpu(), ses.compact_arena.cpu()[: 1 << 20], ses.keep_idx.cpu(), ses.thr.cpu()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
