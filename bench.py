@@ -1,0 +1,338 @@
+#!/usr/bin/env python
+"""Benchmark of the portfolio-generation hot path: threshold once, then mask, zero-structure
+detection, keep propagation and compaction for every variant.
+
+One "step" is one whole portfolio on one model.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet152] [--dtype f32|bf16]
+  python bench.py --impl reference ...     # the CPU oracle, as it stands, on the host cores
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "ms per pruned variant (portfolio generation: threshold, mask, zero structures, keep propagation, compaction)"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return None
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            return None
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            p = [x.strip() for x in line.split(",")]
+            if len(p) < 7:
+                continue
+            try:
+                sm.append(float(p[0]))
+                mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, p[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return None
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------------
+# reference arm / CPU baseline: the oracle, unchanged, on the host
+# --------------------------------------------------------------------------------------------
+
+def oracle_portfolio(wl, dtype, variants):
+    """One pass of the whole path in the oracle for the given variant indices. Returns seconds."""
+    from oracle import oracle as O
+    om = O.OracleModel(wl, dtype)
+    t0 = time.perf_counter()
+    rec = O.threshold(om, wl.scope, wl.ks[variants])
+    for i in range(len(variants)):
+        masked, _ = O.apply_mask(om, wl.scope, rec[i])
+        _, out_nz, in_nz = O.zero_structures(masked)
+        _, ki, kc, _ = O.propagate_keep(masked, out_nz, in_nz)
+        O.compact(masked, ki, kc)
+    return time.perf_counter() - t0
+
+
+def run_reference(args, wl, dtype):
+    V = len(wl.ks)
+    variants = sorted({0, V - 1})
+    for _ in range(args.warmup):
+        oracle_portfolio(wl, dtype, variants)
+    times = [oracle_portfolio(wl, dtype, variants) for _ in range(args.steps)]
+    total = sum(times)
+    ms_per_variant = 1e3 * total / (args.steps * len(variants))
+    sample = f"variants {variants} of {V} (threshold sort shared by {len(variants)} instead of {V}), full weights"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": ms_per_variant, "unit": "ms", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u32 keys / fp32 words" if dtype == 0 else "u16 keys / bf16 words", "data": "synthetic",
+        "config": config_of(args, wl, dtype),
+        "cpu_baseline": {"value": ms_per_variant, "unit": "ms", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": ms_per_variant, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def config_of(args, wl, dtype):
+    return {"workload": f"{wl.name} ({'fp32' if dtype == 0 else 'bf16'}), {wl.n_prunable} prunable weights, "
+                        f"{len(wl.ks)} variants, {'global' if wl.scope == 0 else 'per-tensor'} ranking, seed {wl.seed}",
+            "variants": len(wl.ks), "prunable_weights": wl.n_prunable,
+            "l2": "weights larger than L2 (no flush)" if wl.n_prunable * (4 if dtype == 0 else 2) > 126e6
+                  else "L2 flushed between steps (256 MiB scratch write)"}
+
+
+# --------------------------------------------------------------------------------------------
+# the CUDA arm
+# --------------------------------------------------------------------------------------------
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="dnns", choices=["dnns", "reference"])
+    ap.add_argument("--workload", default="resnet152", choices=["toy", "vgg16", "resnet56", "resnet50", "resnet152"])
+    ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2309_06973_b200 import workloads as W
+    dtype = 0 if args.dtype == "f32" else 1
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        wl = W.BY_NAME[args.workload]()
+        run_reference(args, wl, dtype)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2309_06973_b200 import binding as B
+    from paper_2309_06973_b200.runtime import DeviceModel, Session
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    B.lib()  # fail loudly if the extension is missing
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    wl = W.BY_NAME[args.workload]()
+    V = len(wl.ks)
+    eb = 4 if dtype == 0 else 2
+    N = wl.n_prunable
+    dm = DeviceModel(wl, dtype, device=f"cuda:{local_rank}", pinned_host=True)
+    ses = Session(dm, wl.scope, V, want_mask_bits=True, want_nz_map=False)
+    need_flush = N * eb <= 126e6
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dm.device) if need_flush else None
+
+    names = ["threshold", "mask", "structures", "propagate", "compact"]
+    spans = {n: [] for n in names}
+
+    def step(record: bool):
+        def timed(name, fn, *a):
+            if not record:
+                return fn(*a)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn(*a)
+            e1.record()
+            spans[name].append((e0, e1))
+        timed("threshold", ses.magnitude_threshold, wl.ks)
+        for v in range(V):
+            timed("mask", ses.apply_mask, v)
+            timed("structures", ses.zero_structures)
+            timed("propagate", ses.propagate_keep)
+            timed("compact", ses.compact)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing --------------------------------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        step(False)
+    torch.cuda.synchronize()
+    assert ses.device_status() == B.DNNS_OK
+    # data-dependent sizes of every variant (outside the timed region): R = kept filter rows, N' = rebuilt size
+    R, Nn = [], []
+    for v in range(V):
+        ses.variant(v)
+        torch.cuda.synchronize()
+        sh = ses.dst_shapes.cpu().numpy()[: 2 * len(wl.tensors)].reshape(-1, 2)
+        R.append(sum(int(sh[i, 0]) * t.I * t.KH * t.KW for i, t in enumerate(wl.tensors)))
+        Nn.append(sum(int(sh[i, 0]) * int(sh[i, 1]) * t.KH * t.KW for i, t in enumerate(wl.tensors)))
+
+    launches0 = ses.launch_count()
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_ms = []
+    if need_flush:
+        # inputs fit in L2: flush between steps and time every step on its own
+        for _ in range(args.steps):
+            flush_buf.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            step(True)
+            b.record()
+            step_ms.append((a, b))
+        torch.cuda.synchronize()
+        total_ms = sum(a.elapsed_time(b) for a, b in step_ms)
+    else:
+        t_start.record()
+        for _ in range(args.steps):
+            step(True)
+        t_end.record()
+        torch.cuda.synchronize()
+        total_ms = t_start.elapsed_time(t_end)
+    clocks = sampler.stop()
+    barrier()
+    launches = ses.launch_count() - launches0
+    if world > 1:
+        t = torch.tensor([total_ms], device=dm.device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    assert ses.device_status() == B.DNNS_OK
+
+    ms_per_step = total_ms / args.steps
+    ms_per_variant = ms_per_step / V / world if world > 1 else ms_per_step / V
+    per_call = {n: statistics.mean(a.elapsed_time(b) for a, b in spans[n]) for n in names}
+    share = {n: per_call[n] * (1 if n == "threshold" else V) / ms_per_step for n in names}
+
+    # algorithmic bytes: one read of every input a step consumes, one write of every output
+    alg = {"threshold": N * eb, "mask": 2 * N * eb + N / 8, "structures": N * eb,
+           "propagate": 0, "compact": statistics.mean((r + n) * eb for r, n in zip(R, Nn))}
+    portfolio_bytes = alg["threshold"] + V * (alg["mask"] + alg["structures"]) + sum((r + n) * eb for r, n in zip(R, Nn))
+    peak, peak_kind = load_peaks()
+    dominant = max((n for n in names if alg[n] > 0), key=lambda n: share[n])
+    achieved = alg[dominant] / (per_call[dominant] * 1e-3) / 1e9
+    kernel_of = {"threshold": "k_hist1+k_hist2 (+select, ties)", "mask": "k_sweep<mask>", "structures": "k_sweep<structures>",
+                 "compact": "k_compact_gather"}
+
+    # ---- end to end through the C ABI with host buffers -----------------------------------------
+    small = torch.empty(1 << 16, dtype=torch.uint8).pin_memory()
+    host_out = torch.empty(ses.compact_arena.numel(), dtype=torch.uint8).pin_memory()
+    h2d = d2h = 0
+
+    def e2e_step():
+        nonlocal h2d, d2h
+        dm.upload_weights()
+        h2d += dm.weight_bytes
+        ses.magnitude_threshold(wl.ks)
+        for v in range(V):
+            ses.variant(v)
+            offs = ses.dst_offsets.cpu()           # synchronises: the sizes are only known on the device
+            shp = ses.dst_shapes.cpu()
+            cnt = ses.keep_count.cpu()
+            last_w = len(wl.tensors) - 1
+            used = int(offs[-1].item()) + 4 * max(int(cnt.max().item()), 1)
+            used = min((used + 255) // 256 * 256, host_out.numel())
+            host_out[:used].copy_(ses.compact_arena[:used], non_blocking=True)
+            d2h += used + offs.numel() * 8 + shp.numel() * 4 + cnt.numel() * 4
+        torch.cuda.synchronize()
+
+    for _ in range(2):
+        e2e_step()
+    h2d = d2h = 0
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        e2e_step()
+    barrier()
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dm.device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_per_variant = e2e_ms / args.steps / V / world
+
+    line = {
+        "metric": METRIC, "value": ms_per_variant, "unit": "ms", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u32 keys / fp32 words" if dtype == 0 else "u16 keys / bf16 words",
+        "data": "synthetic", "config": config_of(args, wl, dtype),
+        "effective_gbs": portfolio_bytes / (ms_per_step * 1e-3) / 1e9,
+        "effective_frac_of_peak": portfolio_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
+        "algorithmic_bytes_per_variant": portfolio_bytes / V,
+        "per_call_ms": per_call, "share": share,
+        "per_call_gbs": {n: (alg[n] / (per_call[n] * 1e-3) / 1e9 if alg[n] else None) for n in names},
+        "roofline": {"bound": "hbm", "kernel": kernel_of[dominant], "achieved": achieved, "peak": peak,
+                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": None},
+        "e2e": {"value": e2e_per_variant, "unit": "ms", "h2d_bytes_per_step": h2d // args.steps,
+                "d2h_bytes_per_step": d2h // args.steps},
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "context": {"paper_pruning_time_ms": 120, "paper_hardware": "not stated for that figure"},
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        t = oracle_portfolio(wl, dtype, list(range(V)))
+        line["cpu_baseline"] = {"value": 1e3 * t / V, "unit": "ms", "cores": 1, "kind": "oracle",
+                                "sample": f"the whole workload once: all {V} variants, full weights ({t:.1f} s)"}
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

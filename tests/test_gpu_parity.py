@@ -139,6 +139,7 @@ def test_two_runs_are_bit_identical():
         ses.magnitude_threshold(wl.ks)
         ses.variant(7)
         torch.cuda.synchronize()
-        outs.append((ses.masked.cpu(), ses.compact_arena.cpu()[: 1 << 20], ses.keep_idx.cpu(), ses.thr.cpu()))
+        # padding between arena items is never written: compare the tensors, not the raw arenas
+        outs.append(ses.masked_tensors() + ses.compacted()[0] + [ses.keep_idx.cpu().numpy(), ses.records()])
     for a, b in zip(*outs):
-        assert torch.equal(a, b)
+        assert np.array_equal(a.view(np.uint8), b.view(np.uint8))
