@@ -61,7 +61,8 @@ typedef enum {
     DNNS_ERR_WORKSPACE = 3,   /* workspace or destination arena too small                                   */
     DNNS_ERR_UNSUPPORTED = 4, /* mixed dtypes, unknown dtype, extents beyond the documented limits          */
     DNNS_ERR_CUDA = 5,        /* a CUDA runtime call failed                                                 */
-    DNNS_ERR_TIMEOUT = 6      /* reserved for bounded device-side waits (the current kernels have none)     */
+    DNNS_ERR_TIMEOUT = 6,     /* reserved for bounded device-side waits (the current kernels have none)     */
+    DNNS_ERR_STATIC_LIMIT = 7 /* input larger than the built-in scratch of a *_static entry point allows    */
 } dnns_status;
 
 typedef enum { DNNS_F32 = 0, DNNS_BF16 = 1 } dnns_dtype;
@@ -241,6 +242,32 @@ dnns_status dnns_compact(dnns_plan* plan, const void* masked_arena, const int32_
 dnns_status dnns_last_device_status(dnns_plan* plan, void* stream);
 
 const char* dnns_status_string(dnns_status s);
+
+/*
+ * The threshold of step 1 for ONE tensor, for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this is a packaging variant of dnns_magnitude_threshold.)
+ *
+ * Meant for code that runs where cudaMalloc is off limits: a plug-in inside another framework's
+ * memory-planned step, a callback invoked while that framework's allocator is locked, a process
+ * whose device memory was fully handed out at start-up.  Such callers own the weights and the
+ * result record but cannot supply the workspace a plan needs, so the histograms and tables live
+ * in a fixed array inside the library (about 0.6 MB, held by every GPU that loads the library
+ * until the process exits).  The call makes no allocation of any kind, on device or host.
+ *
+ * weights_dev: device, 16-byte aligned, numel elements of dtype (DNNS_F32 / DNNS_BF16), treated as
+ * one ranking segment in index order.  k: how many weights to mask, 0 <= k <= numel.  thr_dev:
+ * device, one record, same meaning as in dnns_magnitude_threshold.
+ * Limits and errors: numel > DNNS_STATIC_MAX_NUMEL returns DNNS_ERR_STATIC_LIMIT and launches
+ * nothing; INVALID_ARG (null or misaligned pointer, numel == 0, k > numel), UNSUPPORTED (dtype,
+ * device ordinal above 63), CUDA.
+ * The first call on each device resolves the array's device address and clears it; make that
+ * first call outside any stream capture.  All calls on a device share the one array and each call
+ * clears the parts it needs at its start: calls that overlap on the GPU (different streams
+ * without ordering between them) race on it and give wrong results; order them on one stream.
+ */
+#define DNNS_STATIC_MAX_NUMEL (1ull << 26)
+dnns_status dnns_magnitude_threshold_static(const void* weights_dev, int32_t dtype, uint64_t numel, uint64_t k,
+                                            dnns_threshold* thr_dev, void* stream);
 
 #ifdef __cplusplus
 }

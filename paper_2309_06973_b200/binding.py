@@ -15,11 +15,12 @@ DNNS_SCOPE_GLOBAL, DNNS_SCOPE_PER_TENSOR = 0, 1
 DNNS_RULE_PRODUCER, DNNS_RULE_CONSUMER, DNNS_SHIFT_STRICT = 1, 2, 4
 DNNS_GROUP_FROZEN = 1
 (DNNS_OK, DNNS_ERR_INVALID_ARG, DNNS_ERR_BAD_GRAPH, DNNS_ERR_WORKSPACE, DNNS_ERR_UNSUPPORTED, DNNS_ERR_CUDA,
- DNNS_ERR_TIMEOUT) = range(7)
+ DNNS_ERR_TIMEOUT, DNNS_ERR_STATIC_LIMIT) = range(8)
+DNNS_STATIC_MAX_NUMEL = 1 << 26
 
 EXPORTS = ["dnns_status_string", "dnns_workspace_bytes", "dnns_plan_create", "dnns_plan_destroy", "dnns_plan_layout",
            "dnns_plan_launch_count", "dnns_magnitude_threshold", "dnns_apply_mask", "dnns_zero_structures",
-           "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status"]
+           "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static"]
 
 
 class dnns_tensor(C.Structure):
@@ -94,6 +95,7 @@ def lib() -> C.CDLL:
         L.dnns_propagate_keep.argtypes = [vp, vp, vp, u32, i32, vp, vp, vp, vp, vp]
         L.dnns_compact.argtypes = [vp, vp, vp, vp, vp, C.c_size_t, vp, vp, vp]
         L.dnns_last_device_status.argtypes = [vp, vp]
+        L.dnns_magnitude_threshold_static.argtypes = [vp, i32, u64, u64, vp, vp]
         _lib = L
     return _lib
 
@@ -162,3 +164,10 @@ def dnns_compact(plan, masked_arena: int, keep_idx: int, keep_count: int, dst_ar
 
 def dnns_last_device_status(plan, stream: int = 0) -> int:
     return lib().dnns_last_device_status(plan, stream)
+
+
+def dnns_magnitude_threshold_static(weights_dev: int, dtype: int, numel: int, k: int, thr_dev: int,
+                                    stream: int = 0) -> None:
+    """Threshold of one tensor using the library's built-in scratch: nothing is allocated."""
+    _check(lib().dnns_magnitude_threshold_static(weights_dev, dtype, numel, k, thr_dev, stream),
+           "dnns_magnitude_threshold_static")

@@ -152,6 +152,7 @@ const char* dnns_status_string(dnns_status s) {
         case DNNS_ERR_UNSUPPORTED: return "unsupported dtype or extent";
         case DNNS_ERR_CUDA: return "CUDA runtime error";
         case DNNS_ERR_TIMEOUT: return "device-side wait expired";
+        case DNNS_ERR_STATIC_LIMIT: return "input exceeds the size limit of the built-in scratch (DNNS_STATIC_MAX_NUMEL)";
     }
     return "unknown status";
 }

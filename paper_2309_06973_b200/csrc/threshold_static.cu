@@ -1,0 +1,121 @@
+// dnns_magnitude_threshold_static: the k-th-magnitude threshold of ONE weight tensor with all of
+// its scratch memory inside this library instead of a caller-provided workspace.
+//
+// Who this is for: code that runs where device memory cannot be allocated - a plug-in called
+// inside someone else's memory-planned inference or training step, a callback that runs while
+// the host framework's allocator is locked, or a process whose memory budget was handed out in
+// full at start-up.  Such a caller owns the weights and the 32-byte result record and nothing
+// else; it cannot provide the few hundred kilobytes of histograms and tables that the plan-based
+// entry point keeps in its workspace.
+//
+// The scratch is the file-scope array below.  It is part of the library image: every GPU that
+// loads the library holds these ~0.6 MB until the process exits.  Host code must not pass the
+// array's name to a kernel (on the host that name is only a stand-in for the symbol); the device
+// address is obtained once per device with cudaGetSymbolAddress and handed to the kernels.
+#include <mutex>
+
+#include "dnns_internal.cuh"
+
+namespace {
+
+using namespace dnns;
+
+constexpr uint64_t kMaxNumel = DNNS_STATIC_MAX_NUMEL;
+constexpr uint32_t kMaxTiles = (uint32_t)(kMaxNumel * 4 / kTileBytes);  // fp32 is the wider case
+
+// Byte offsets inside the scratch array (every section 256-byte aligned).
+constexpr size_t kOffTensor = 0;                                  // TensorDesc[1]
+constexpr size_t kOffSeg = 256;                                   // SegDesc[1]
+constexpr size_t kOffK = 512;                                     // uint64 k
+constexpr size_t kOffSel = 768;                                   // SelectState[1]
+constexpr size_t kOffBitmap = 1024;                               // kBitmapWords words
+constexpr size_t kOffTileTensor = kOffBitmap + 4 * kBitmapWords;  // kMaxTiles words, always zero (tensor 0)
+constexpr size_t kOffTiePrefix = kOffTileTensor + 4 * (size_t)kMaxTiles;
+// --- everything from here on is cleared at the start of every call ---
+constexpr size_t kOffClear = kOffTiePrefix + 4 * (size_t)kMaxTiles;
+constexpr size_t kOffAnyNeed = kOffClear;
+constexpr size_t kOffNeed = kOffAnyNeed + 256;
+constexpr size_t kOffTileTies = kOffNeed + 256;
+constexpr size_t kOffHist1 = kOffTileTies + 4 * (size_t)kMaxTiles;
+constexpr size_t kOffHist2 = kOffHist1 + 4 * (size_t)kHistBins;
+constexpr size_t kScratchBytes = kOffHist2 + 4 * (size_t)kLowBins;
+
+static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_mutex;
+unsigned char* g_scratch_ptr[kMaxDevices] = {};  // device address of the array, per device ordinal
+int g_n_sm[kMaxDevices] = {};
+
+// One-time set-up on the current device: resolve the device address of the scratch array, zero
+// the part that stays constant, raise the shared-memory limit of the histogram kernel.
+dnns_status setup_device(int dev, cudaStream_t st) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_scratch_ptr[dev]) return DNNS_OK;
+    unsigned char* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_scratch) != cudaSuccess || !p) return DNNS_ERR_CUDA;
+    int n_sm = 0;
+    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DNNS_ERR_CUDA;
+    if (init_kernel_attributes() != cudaSuccess) return DNNS_ERR_CUDA;
+    if (cudaMemsetAsync(p, 0, kScratchBytes, st) != cudaSuccess) return DNNS_ERR_CUDA;
+    g_n_sm[dev] = n_sm;
+    g_scratch_ptr[dev] = p;
+    return DNNS_OK;
+}
+
+}  // namespace
+
+extern "C" dnns_status dnns_magnitude_threshold_static(const void* weights_dev, int32_t dtype, uint64_t numel,
+                                                       uint64_t k, dnns_threshold* thr_dev, void* stream) {
+    if (!weights_dev || !thr_dev || numel == 0) return DNNS_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(weights_dev) & 15) return DNNS_ERR_INVALID_ARG;
+    if (dtype != DNNS_F32 && dtype != DNNS_BF16) return DNNS_ERR_UNSUPPORTED;
+    if (numel > kMaxNumel) return DNNS_ERR_STATIC_LIMIT;
+    if (k > numel) return DNNS_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DNNS_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return DNNS_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dnns_status s = setup_device(dev, st);
+    if (s != DNNS_OK) return s;
+    unsigned char* base = g_scratch_ptr[dev];
+
+    const uint32_t elem_bytes = dtype == DNNS_F32 ? 4 : 2;
+    const uint32_t n_tiles = (uint32_t)((numel * elem_bytes + kTileBytes - 1) / kTileBytes);
+
+    // descriptors of the one tensor and its one ranking segment
+    TensorDesc td{};
+    td.src = weights_dev;
+    td.numel = (uint32_t)numel;
+    td.O = 1, td.I = (int32_t)numel, td.KK = 1, td.S = 1;
+    td.out_group = td.in_group = 0;
+    td.seg = 0, td.bn = -1;
+    td.tile0 = 0, td.n_tiles = n_tiles;
+    const SegDesc sd{0, n_tiles, numel};
+
+    // what must start at zero: histograms, tie tables and flags of the previous call
+    if (cudaMemsetAsync(base + kOffClear, 0, kScratchBytes - kOffClear, st) != cudaSuccess ||
+        cudaMemcpyAsync(base + kOffTensor, &td, sizeof(td), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(base + kOffSeg, &sd, sizeof(sd), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(base + kOffK, &k, sizeof(k), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return DNNS_ERR_CUDA;
+
+    Tables tb{};
+    tb.tensors = reinterpret_cast<const TensorDesc*>(base + kOffTensor);
+    tb.segs = reinterpret_cast<const SegDesc*>(base + kOffSeg);
+    tb.tile_tensor = reinterpret_cast<const uint32_t*>(base + kOffTileTensor);
+    tb.n_tensors = 1, tb.n_segs = 1, tb.n_tiles = n_tiles;
+    tb.tile_elems = kTileBytes / elem_bytes;
+    tb.dtype = dtype;
+    ThresholdWs ws{};
+    ws.k_dev = reinterpret_cast<uint64_t*>(base + kOffK);
+    ws.hist1 = reinterpret_cast<uint32_t*>(base + kOffHist1);
+    ws.hist2 = reinterpret_cast<uint32_t*>(base + kOffHist2);
+    ws.bitmap = reinterpret_cast<uint32_t*>(base + kOffBitmap);
+    ws.sel = reinterpret_cast<SelectState*>(base + kOffSel);
+    ws.need = reinterpret_cast<uint32_t*>(base + kOffNeed);
+    ws.any_need = reinterpret_cast<uint32_t*>(base + kOffAnyNeed);
+    ws.tile_ties = reinterpret_cast<uint32_t*>(base + kOffTileTies);
+    ws.tie_prefix = reinterpret_cast<uint32_t*>(base + kOffTiePrefix);
+    return launch_threshold(tb, ws, 1, 1, thr_dev, g_n_sm[dev], st) < 0 ? DNNS_ERR_CUDA : DNNS_OK;
+}
