@@ -144,6 +144,7 @@ def main():
     ap.add_argument("--workload", default="resnet152", choices=["toy", "vgg16", "resnet56", "resnet50", "resnet152"])
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stepwise", action="store_true", help="mask and zero-structure detection as two sweeps")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -182,7 +183,8 @@ def main():
     need_flush = N * eb <= 126e6
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dm.device) if need_flush else None
 
-    names = ["threshold", "mask", "structures", "propagate", "compact"]
+    names = (["threshold", "mask", "structures", "propagate", "compact"] if args.stepwise
+             else ["threshold", "mask+structures", "propagate", "compact"])
     spans = {n: [] for n in names}
 
     def step(record: bool):
@@ -196,8 +198,11 @@ def main():
             spans[name].append((e0, e1))
         timed("threshold", ses.magnitude_threshold, wl.ks)
         for v in range(V):
-            timed("mask", ses.apply_mask, v)
-            timed("structures", ses.zero_structures)
+            if args.stepwise:
+                timed("mask", ses.apply_mask, v)
+                timed("structures", ses.zero_structures)
+            else:
+                timed("mask+structures", ses.mask_and_structures, v)
             timed("propagate", ses.propagate_keep)
             timed("compact", ses.compact)
 
@@ -259,14 +264,17 @@ def main():
     share = {n: per_call[n] * (1 if n == "threshold" else V) / ms_per_step for n in names}
 
     # algorithmic bytes: one read of every input a step consumes, one write of every output
-    alg = {"threshold": N * eb, "mask": 2 * N * eb + N / 8, "structures": N * eb,
+    # (the fused sweep moves 2*N*b + N/8 per launch; the stepwise accounting B_v charges the path 3*N*b + N/8)
+    alg = {"threshold": N * eb, "mask": 2 * N * eb + N / 8, "structures": N * eb, "mask+structures": 2 * N * eb + N / 8,
            "propagate": 0, "compact": statistics.mean((r + n) * eb for r, n in zip(R, Nn))}
     portfolio_bytes = alg["threshold"] + V * (alg["mask"] + alg["structures"]) + sum((r + n) * eb for r, n in zip(R, Nn))
+    moved_bytes = alg["threshold"] + V * (alg["mask"] + (alg["structures"] if args.stepwise else 0)) + \
+        sum((r + n) * eb for r, n in zip(R, Nn))
     peak, peak_kind = load_peaks()
     dominant = max((n for n in names if alg[n] > 0), key=lambda n: share[n])
     achieved = alg[dominant] / (per_call[dominant] * 1e-3) / 1e9
     kernel_of = {"threshold": "k_hist1+k_hist2 (+select, ties)", "mask": "k_sweep<mask>", "structures": "k_sweep<structures>",
-                 "compact": "k_compact_gather"}
+                 "mask+structures": "k_sweep<mask+structures>", "compact": "k_compact_gather"}
 
     # ---- end to end through the C ABI with host buffers -----------------------------------------
     small = torch.empty(1 << 16, dtype=torch.uint8).pin_memory()
@@ -279,7 +287,7 @@ def main():
         h2d += dm.weight_bytes
         ses.magnitude_threshold(wl.ks)
         for v in range(V):
-            ses.variant(v)
+            ses.variant(v, fused=not args.stepwise)
             offs = ses.dst_offsets.cpu()           # synchronises: the sizes are only known on the device
             shp = ses.dst_shapes.cpu()
             cnt = ses.keep_count.cpu()
@@ -313,6 +321,7 @@ def main():
         "effective_gbs": portfolio_bytes / (ms_per_step * 1e-3) / 1e9,
         "effective_frac_of_peak": portfolio_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
         "algorithmic_bytes_per_variant": portfolio_bytes / V,
+        "moved_gbs": moved_bytes / (ms_per_step * 1e-3) / 1e9, "sweeps": "stepwise" if args.stepwise else "fused mask+structures",
         "per_call_ms": per_call, "share": share,
         "per_call_gbs": {n: (alg[n] / (per_call[n] * 1e-3) / 1e9 if alg[n] else None) for n in names},
         "roofline": {"bound": "hbm", "kernel": kernel_of[dominant], "achieved": achieved, "peak": peak,

@@ -205,6 +205,17 @@ dnns_status dnns_zero_structures(dnns_plan* plan, const void* masked_arena, uint
                                  uint32_t* in_nz, void* stream);
 
 /*
+ * Steps 2 and 3 in one sweep over the weights: the same outputs, bit for bit, as dnns_apply_mask
+ * followed by dnns_zero_structures on its result, but the masked weights are analysed while they
+ * are still in registers, which saves one full read of the model per variant (Module 2 only
+ * needs the sparse weights, Section III-D).  Arguments as in the two calls; masked_arena NULL
+ * masks in place.
+ */
+dnns_status dnns_mask_and_structures(dnns_plan* plan, const dnns_threshold* thr_dev, int32_t variant,
+                                     void* masked_arena, uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz,
+                                     uint32_t* in_nz, void* stream);
+
+/*
  * Step 4 - keep sets per channel group (Algorithm 1 generalised from a chain to groups).
  * Channel j of a group is removed when
  *   (policy & RULE_PRODUCER) and every producer's filter j is all zero [the paper's rule], and,

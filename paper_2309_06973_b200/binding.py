@@ -20,7 +20,7 @@ DNNS_STATIC_MAX_NUMEL = 1 << 26
 
 EXPORTS = ["dnns_status_string", "dnns_workspace_bytes", "dnns_plan_create", "dnns_plan_destroy", "dnns_plan_layout",
            "dnns_plan_launch_count", "dnns_magnitude_threshold", "dnns_apply_mask", "dnns_zero_structures",
-           "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static"]
+           "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures"]
 
 
 class dnns_tensor(C.Structure):
@@ -92,6 +92,7 @@ def lib() -> C.CDLL:
         L.dnns_magnitude_threshold.argtypes = [vp, C.POINTER(u64), i32, vp, vp]
         L.dnns_apply_mask.argtypes = [vp, vp, i32, vp, vp, vp]
         L.dnns_zero_structures.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.dnns_mask_and_structures.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.dnns_propagate_keep.argtypes = [vp, vp, vp, u32, i32, vp, vp, vp, vp, vp]
         L.dnns_compact.argtypes = [vp, vp, vp, vp, vp, C.c_size_t, vp, vp, vp]
         L.dnns_last_device_status.argtypes = [vp, vp]
@@ -148,6 +149,12 @@ def dnns_apply_mask(plan, thr_dev: int, variant: int, masked_arena: int, mask_bi
 def dnns_zero_structures(plan, masked_arena: int, nz_map: int, out_nz: int, in_nz: int, stream: int = 0) -> None:
     _check(lib().dnns_zero_structures(plan, masked_arena or None, nz_map or None, out_nz, in_nz, stream),
            "dnns_zero_structures")
+
+
+def dnns_mask_and_structures(plan, thr_dev: int, variant: int, masked_arena: int, mask_bits: int, nz_map: int,
+                             out_nz: int, in_nz: int, stream: int = 0) -> None:
+    _check(lib().dnns_mask_and_structures(plan, thr_dev, variant, masked_arena or None, mask_bits or None,
+                                          nz_map or None, out_nz, in_nz, stream), "dnns_mask_and_structures")
 
 
 def dnns_propagate_keep(plan, out_nz: int, in_nz: int, policy: int, min_keep: int, keep_bits: int, keep_idx: int,

@@ -19,7 +19,6 @@ constexpr uint32_t kHistBins = 32768;    // first radix digit: the top 15 bits o
 constexpr uint32_t kLowBins = 65536;     // second digit of a 31-bit key
 constexpr uint32_t kBitmapWords = kHistBins / 32;
 constexpr int kMaxVariants = 64;
-constexpr uint32_t kInSmemBits = 32768;  // input-column flags accumulate in shared memory up to this many columns
 
 struct TensorDesc {
     const void* src;        // the model's tensor

@@ -399,6 +399,24 @@ dnns_status dnns_zero_structures(dnns_plan* p, const void* masked_arena, uint32_
     return DNNS_OK;
 }
 
+dnns_status dnns_mask_and_structures(dnns_plan* p, const dnns_threshold* thr_dev, int32_t variant, void* masked_arena,
+                                     uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz,
+                                     void* stream) {
+    if (!p || !thr_dev || !out_nz || !in_nz || variant < 0 || variant >= p->maxv) return DNNS_ERR_INVALID_ARG;
+    if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dnns_layout& L = p->layout;
+    if (cudaMemsetAsync(out_nz, 0, 4 * L.out_nz_words, st) != cudaSuccess ||
+        cudaMemsetAsync(in_nz, 0, 4 * L.in_nz_words, st) != cudaSuccess ||
+        (nz_map && cudaMemsetAsync(nz_map, 0, 4 * L.nz_map_words, st) != cudaSuccess))
+        return DNNS_ERR_CUDA;
+    const int n = launch_tile_sweep(p->tb, p->tws, true, true, thr_dev, variant, nullptr, masked_arena, mask_bits,
+                                    nz_map, out_nz, in_nz, p->n_sm, st);
+    if (n < 0) return DNNS_ERR_CUDA;
+    p->launches += n;
+    return DNNS_OK;
+}
+
 dnns_status dnns_propagate_keep(dnns_plan* p, const uint32_t* out_nz, const uint32_t* in_nz, uint32_t policy,
                                 int32_t min_keep, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count,
                                 uint64_t* stats, void* stream) {

@@ -9,7 +9,7 @@
 //   structures (Module 2, Sparsity Analyser) - the non-zero bits of the tile's elements go to
 //              shared memory; from them the all-zero 2-D kernels, and from those the filters
 //              (rows) and input columns that still hold something, are OR-ed into the packed
-//              global flag arrays.
+//              global flag arrays (test first, atomic only when a bit is still missing).
 //
 // The same kernel runs either step alone or both in one sweep (the structures are then derived
 // from the masked values while they are still in registers).
@@ -44,70 +44,66 @@ __device__ __forceinline__ bool any_bits(const uint32_t* bits, uint32_t lo, uint
     return acc != 0;
 }
 
+// OR `bits` into a global flag word unless they are already there.  The plain read may be stale,
+// which only costs a redundant atomic; flags saturate early in a sweep, so almost every update
+// ends at the read.
+__device__ __forceinline__ void or_if_missing(uint32_t* word, uint32_t bits) {
+    if ((__ldcg(word) & bits) != bits) atomicOr(word, bits);
+}
+
 // From the element bits of one tile (elements [e0, e0+n_e) of tensor d) to kernel map, filter
 // flags and input-column flags.  Kernel q = (o, i) covers elements [q*KK, (q+1)*KK); a kernel cut
-// by the tile edge is OR-ed by both tiles.
+// by the tile edge is OR-ed by both tiles.  s_kbits receives the kernel bits of the tile, kernel
+// q at bit q - (q0 & ~31); for 1x1 kernels the element bits are used as they are.
+// Ends with a barrier, after which ebits and s_kbits may be overwritten.
 __device__ void tile_structures(const TensorDesc& d, uint32_t e0, uint32_t n_e, const uint32_t* ebits,
-                                uint32_t* s_in, uint32_t* s_out, uint32_t* nz_map, uint32_t* out_nz,
-                                uint32_t* in_nz) {
+                                uint32_t* s_kbits, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz) {
     const uint32_t KK = d.KK, I = d.I;
     const uint32_t q0 = e0 / KK, q1 = (e0 + n_e - 1) / KK;
-    const uint32_t row0 = q0 / I, row1 = q1 / I;
-    const bool in_smem = I <= kInSmemBits;
-    const uint32_t in_words = in_smem ? (I + 31) / 32 : 0;
-    const uint32_t out_words = (row1 - row0) / 32 + 1;
-    for (uint32_t w = threadIdx.x; w < in_words; w += kTileThreads) s_in[w] = 0;
-    for (uint32_t w = threadIdx.x; w < out_words; w += kTileThreads) s_out[w] = 0;
-    __syncthreads();
-    uint32_t* g_in = in_nz + d.off_innz;
-    uint32_t* g_out = out_nz + d.off_outnz;
-    uint32_t* g_map = nz_map ? nz_map + d.off_nzmap : nullptr;
-    const bool row_words = (I % 32 == 0);  // 32 consecutive kernels never cross a filter boundary
+    const uint32_t qa = q0 & ~31u;
+    const uint32_t n_words = ((q1 - qa) >> 5) + 1;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (uint32_t qb = (q0 & ~31u) + warp * 32; qb <= q1; qb += 32 * (kTileThreads / 32)) {
-        uint32_t bits;
-        if (KK == 1) {
-            bits = ebits[(qb - e0) >> 5];  // kernels are elements and the tile starts on a word
-        } else {
-            const uint32_t q = qb + lane;
+    const uint32_t* kbits = ebits;  // KK == 1: kernels are elements and the tile starts on a word
+    if (KK != 1) {
+        for (uint32_t w = warp; w < n_words; w += kTileThreads / 32) {
+            const uint32_t q = qa + 32 * w + lane;
             bool bit = false;
             if (q >= q0 && q <= q1) {
                 const uint32_t lo = max(q * KK, e0) - e0, hi = min((q + 1) * KK, e0 + n_e) - e0;
                 bit = any_bits(ebits, lo, hi);
             }
-            bits = __ballot_sync(kFull, bit);
+            const uint32_t word = __ballot_sync(kFull, bit);
+            if (lane == 0) s_kbits[w] = word;
         }
+        __syncthreads();
+        kbits = s_kbits;
+    }
+    uint32_t* g_in = in_nz + d.off_innz;
+    uint32_t* g_out = out_nz + d.off_outnz;
+    uint32_t* g_map = nz_map ? nz_map + d.off_nzmap : nullptr;
+    const bool row_words = (I % 32 == 0);  // 32 consecutive kernels never cross a filter boundary
+    for (uint32_t w = threadIdx.x; w < n_words; w += kTileThreads) {
+        uint32_t bits = kbits[w];
         if (!bits) continue;
-        if (g_map && lane == 0) {
-            if (KK == 1) g_map[qb >> 5] = bits;  // the word belongs to this tile alone
+        const uint32_t qb = qa + 32 * w;
+        if (g_map) {
+            // only the first and last word can hold kernels shared with a neighbouring tile
+            if (KK == 1 || (w != 0 && w != n_words - 1)) g_map[qb >> 5] = bits;
             else atomicOr(&g_map[qb >> 5], bits);
         }
         if (row_words) {
-            if (lane == 0) {
-                const uint32_t o = qb / I, r = o - row0, iw = (qb - o * I) >> 5;
-                atomicOr(&s_out[r >> 5], 1u << (r & 31));
-                if (in_smem) atomicOr(&s_in[iw], bits);
-                else atomicOr(&g_in[iw], bits);
+            const uint32_t o = qb / I, iw = (qb - o * I) >> 5;
+            or_if_missing(&g_in[iw], bits);
+            or_if_missing(&g_out[o >> 5], 1u << (o & 31));
+        } else {
+            while (bits) {
+                const uint32_t q = qb + __ffs(bits) - 1;
+                bits &= bits - 1;
+                const uint32_t o = q / I, i = q - o * I;
+                or_if_missing(&g_in[i >> 5], 1u << (i & 31));
+                or_if_missing(&g_out[o >> 5], 1u << (o & 31));
             }
-        } else if ((bits >> lane) & 1u) {
-            const uint32_t q = qb + lane, o = q / I, i = q - o * I, r = o - row0;
-            atomicOr(&s_out[r >> 5], 1u << (r & 31));
-            if (in_smem) atomicOr(&s_in[i >> 5], 1u << (i & 31));
-            else atomicOr(&g_in[i >> 5], 1u << (i & 31));
         }
-    }
-    __syncthreads();
-    for (uint32_t w = threadIdx.x; w < out_words; w += kTileThreads) {
-        const uint32_t v = s_out[w];
-        if (v) {
-            const uint32_t pos = row0 + 32 * w, sh = pos & 31;
-            atomicOr(&g_out[pos >> 5], v << sh);
-            if (sh && (v >> (32 - sh))) atomicOr(&g_out[(pos >> 5) + 1], v >> (32 - sh));
-        }
-    }
-    for (uint32_t w = threadIdx.x; w < in_words; w += kTileThreads) {
-        const uint32_t v = s_in[w];
-        if (v) atomicOr(&g_in[w], v);
     }
     __syncthreads();
 }
@@ -120,8 +116,7 @@ __global__ void __launch_bounds__(kTileThreads) k_sweep(Tables tb, ThresholdWs w
     constexpr int P = Elem<DT>::kPerVec;
     constexpr int G = 32 / P;  // lanes per bit word
     __shared__ uint32_t s_ebits[kTileBytes / Elem<DT>::kBytes / 32];
-    __shared__ uint32_t s_in[DO_STRUCT ? kInSmemBits / 32 : 1];
-    __shared__ uint32_t s_out[DO_STRUCT ? kTileBytes / Elem<DT>::kBytes / 32 + 2 : 1];
+    __shared__ uint32_t s_kbits[DO_STRUCT ? kTileBytes / Elem<DT>::kBytes / 32 + 1 : 1];
     __shared__ uint32_t scratch[33];
     const int lane = threadIdx.x & 31;
 
@@ -220,7 +215,7 @@ __global__ void __launch_bounds__(kTileThreads) k_sweep(Tables tb, ThresholdWs w
         }
         if (DO_STRUCT) {
             __syncthreads();
-            tile_structures(d, e0, n_e, s_ebits, s_in, s_out, nz_map, out_nz, in_nz);
+            tile_structures(d, e0, n_e, s_ebits, s_kbits, nz_map, out_nz, in_nz);
         }
     }
 }

@@ -138,6 +138,12 @@ class Session:
                                0 if self.nz_map is None else self.nz_map.data_ptr(), self.out_nz.data_ptr(),
                                self.in_nz.data_ptr(), _stream())
 
+    def mask_and_structures(self, variant: int, in_place: bool = False):
+        B.dnns_mask_and_structures(self.plan, self.thr.data_ptr(), variant, 0 if in_place else self.masked.data_ptr(),
+                                   0 if self.mask_bits is None else self.mask_bits.data_ptr(),
+                                   0 if self.nz_map is None else self.nz_map.data_ptr(), self.out_nz.data_ptr(),
+                                   self.in_nz.data_ptr(), _stream())
+
     def propagate_keep(self, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1):
         B.dnns_propagate_keep(self.plan, self.out_nz.data_ptr(), self.in_nz.data_ptr(), policy, min_keep,
                               self.keep_bits.data_ptr(), self.keep_idx.data_ptr(), self.keep_count.data_ptr(),
@@ -149,10 +155,14 @@ class Session:
                        self.compact_arena.numel() if dst_bytes is None else dst_bytes, self.dst_offsets.data_ptr(),
                        self.dst_shapes.data_ptr(), _stream())
 
-    def variant(self, v: int, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1):
-        """Steps 2-5 for variant v of the latest threshold call."""
-        self.apply_mask(v)
-        self.zero_structures()
+    def variant(self, v: int, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1,
+                fused: bool = False):
+        """Steps 2-5 for variant v of the latest threshold call (fused: steps 2 and 3 in one sweep)."""
+        if fused:
+            self.mask_and_structures(v)
+        else:
+            self.apply_mask(v)
+            self.zero_structures()
         self.propagate_keep(policy, min_keep)
         self.compact()
 

@@ -28,7 +28,7 @@ def expected_offsets(sizes_bytes):
 
 
 def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCER | O.RULE_CONSUMER, min_keep=1,
-                      weights=None, check_structure_maps=True):
+                      weights=None, check_structure_maps=True, fused=False):
     """Thresholds for all of wl.ks in one call, then steps 2-5 for the chosen variants."""
     om = O.OracleModel(wl, dtype, weights)
     dm = DeviceModel(wl, dtype, weights=weights)
@@ -40,7 +40,7 @@ def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCE
         assert np.array_equal(rec_gpu[f], rec_cpu[f]), f
     eb = 4 if dtype == B.DNNS_F32 else 2
     for v in (range(len(wl.ks)) if variants is None else variants):
-        ses.variant(v, policy, min_keep)
+        ses.variant(v, policy, min_keep, fused=fused)
         assert ses.device_status() == B.DNNS_OK
         masked_cpu, bits_cpu = O.apply_mask(om, wl.scope, rec_cpu[v])
         for i, (a, b) in enumerate(zip(ses.masked_tensors(), masked_cpu.weights)):

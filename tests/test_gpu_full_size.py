@@ -33,12 +33,13 @@ def test_vgg16_per_layer_95():
 
 def test_resnet50_three_variants():
     wl = W.resnet50()
-    ses = compare_portfolio(wl, B.DNNS_F32)
+    ses = compare_portfolio(wl, B.DNNS_F32, fused=True)
     forward_check(wl, ses, B.DNNS_F32)
 
 
 @pytest.mark.parametrize("dtype", [B.DNNS_F32, B.DNNS_BF16])
 def test_resnet152_portfolio(dtype):
     wl = W.resnet152()
-    ses = compare_portfolio(wl, dtype, variants=[0, 7])
+    ses = compare_portfolio(wl, dtype, variants=[0], fused=False)
+    ses = compare_portfolio(wl, dtype, variants=[7], fused=True)
     forward_check(wl, ses, dtype)

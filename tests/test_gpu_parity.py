@@ -12,11 +12,12 @@ from paper_2309_06973_b200 import workloads as W
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("dtype", [B.DNNS_F32, B.DNNS_BF16])
 @pytest.mark.parametrize("make", [W.toy, lambda: W.small_resnet(seed=3), lambda: W.small_resnet(seed=4, bottleneck=False),
                                   W.resnet56])
-def test_small_configs_every_variant(make, dtype):
-    compare_portfolio(make(), dtype)
+def test_small_configs_every_variant(make, dtype, fused):
+    compare_portfolio(make(), dtype, fused=fused)
 
 
 @pytest.mark.parametrize("policy", [O.RULE_PRODUCER, O.RULE_CONSUMER, O.RULE_PRODUCER | O.RULE_CONSUMER | O.SHIFT_STRICT])
@@ -39,6 +40,7 @@ def test_per_tensor_scope_and_odd_shapes(dtype):
     wl.ks = np.array([[0] * len(sizes), [n // 2 for n in sizes], [n * 9 // 10 for n in sizes],
                       [n - 1 for n in sizes], sizes], np.uint64)
     compare_portfolio(wl, dtype)
+    compare_portfolio(wl, dtype, variants=[1, 3], fused=True)
 
 
 def test_non_prunable_tensor_and_1x1_chain():
@@ -71,6 +73,7 @@ def test_special_values_and_heavy_ties():
     rec = ses.records()
     assert (rec["n_tie"] < rec["n_equal"]).any()                   # the split-tie path really ran
     compare_portfolio(wl, B.DNNS_BF16)
+    compare_portfolio(wl, B.DNNS_F32, fused=True)
 
 
 def test_fc_with_spatial_columns():
