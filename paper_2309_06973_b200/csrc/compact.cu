@@ -64,65 +64,137 @@ __device__ __forceinline__ uint32_t load_elem(const void* base, uint32_t idx) {
     return __ldg(static_cast<const uint16_t*>(base) + idx);
 }
 
-// Gather one unit of an item whose elements are BYTES wide.
+// Gather a run of consecutive units of one item whose elements are BYTES wide, starting at
+// destination element f0.  A unit is 4 x 16-byte destination vectors per thread.
 template <int BYTES>
-__device__ __forceinline__ void gather_unit(const ItemDesc& it, const char* src, char* dst, const int32_t* ko,
-                                            const int32_t* ki, uint32_t On, uint32_t Cn, uint32_t f0) {
+__device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, char* dst, const int32_t* ko,
+                                           const int32_t* ki, uint32_t On, uint32_t Cn, uint32_t f0, uint32_t n_units) {
     constexpr uint32_t VE = 16 / BYTES;  // elements per 16-byte vector
+    constexpr int U = kUnitBytes / 16 / kThreads;
+    constexpr uint32_t kUnitElems = kUnitBytes / BYTES;
+    constexpr uint32_t kNone = 0xFFFFFFFFu;
     const uint32_t blk = it.blk, Cin = it.Cin;
     const uint32_t Ln = Cn * blk, L = Cin * blk;  // new and old row length
     const uint32_t total = On * Ln;
-    const uint32_t f1 = min(total, f0 + kUnitBytes / BYTES);
-    const bool rows_intact = (Cn == Cin) && (L % VE == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0);
-    for (uint32_t f = f0 + threadIdx.x * VE; f < f1; f += kThreads * VE) {
-        uint32_t a = f / Ln, rem = f - a * Ln;
-        if (rows_intact && f + VE <= total) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(src + ((size_t)ko[a] * L + rem) * BYTES));
-            *reinterpret_cast<uint4*>(dst + (size_t)f * BYTES) = v;
-            continue;
-        }
-        uint32_t c = rem / blk, r = rem - c * blk;
-        uint32_t row = (uint32_t)ko[a] * Cin, col = ki ? (uint32_t)ki[c] : c;
-        uint32_t w[4] = {0, 0, 0, 0};
-        const uint32_t nv = min(VE, total - f);
-        for (uint32_t e = 0; e < nv; ++e) {
-            const uint32_t x = load_elem<BYTES>(src, (row + col) * blk + r);
-            if (BYTES == 4) w[e] = x;
-            else w[e >> 1] |= x << (16 * (e & 1));
-            if (++r == blk) {
-                r = 0;
-                if (++c == Cn) {
-                    c = 0;
-                    ++a;
-                    if (a < On) row = (uint32_t)ko[a] * Cin;
+    if ((Cn == Cin) && (L % VE == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0)) {
+        // Rows lose no input channel: every destination vector is one aligned source vector of row
+        // ko[a].  The loads of the next unit are issued before the current unit is stored.
+        uint4 nxt[U];
+        bool nxt_ok[U];
+        auto issue = [&](uint32_t fu) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t f = fu + (u * kThreads + threadIdx.x) * VE;
+                nxt_ok[u] = f < total;
+                if (nxt_ok[u]) {
+                    const uint32_t a = f / Ln, rem = f - a * Ln;
+                    nxt[u] = __ldg(reinterpret_cast<const uint4*>(src + ((size_t)(uint32_t)ko[a] * L + rem) * BYTES));
                 }
-                if (a < On) col = ki ? (uint32_t)ki[c] : c;
+            }
+        };
+        issue(f0);
+        for (uint32_t n = 0; n < n_units; ++n) {
+            uint4 cur[U];
+            bool ok[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) cur[u] = nxt[u], ok[u] = nxt_ok[u];
+            const uint32_t fu = f0 + n * kUnitElems;
+            if (n + 1 < n_units) issue(fu + kUnitElems);
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (ok[u]) *reinterpret_cast<uint4*>(dst + (size_t)(fu + (u * kThreads + threadIdx.x) * VE) * BYTES) = cur[u];
+        }
+        return;
+    }
+    // General case: element (a, c, r) of the new row-major layout reads (ko[a], ki[c], r).  Per
+    // pass: all source positions, then all 16 element loads of the thread, then the stores.
+    constexpr int UG = BYTES == 4 ? U : U / 2;
+#pragma unroll 1
+    for (uint32_t pass = 0; pass < n_units * (U / UG); ++pass) {
+        const uint32_t fp = f0 + pass * UG * kThreads * VE;
+        uint32_t idx[UG][VE];
+#pragma unroll
+        for (int u = 0; u < UG; ++u) {
+            const uint32_t f = fp + (u * kThreads + threadIdx.x) * VE;
+#pragma unroll
+            for (uint32_t e = 0; e < VE; ++e) idx[u][e] = kNone;
+            if (f >= total) continue;
+            uint32_t a = f / Ln, rem = f - a * Ln;
+            uint32_t c = rem / blk, r = rem - c * blk;
+            uint32_t row = (uint32_t)ko[a] * Cin, col = ki ? (uint32_t)ki[c] : c;
+            const uint32_t nv = min(VE, total - f);
+#pragma unroll
+            for (uint32_t e = 0; e < VE; ++e) {
+                if (e < nv) {
+                    idx[u][e] = (row + col) * blk + r;
+                    if (++r == blk) {
+                        r = 0;
+                        if (++c == Cn) {
+                            c = 0;
+                            ++a;
+                            if (a < On) row = (uint32_t)ko[a] * Cin;
+                        }
+                        if (a < On) col = ki ? (uint32_t)ki[c] : c;
+                    }
+                }
             }
         }
-        if (nv == VE) {
-            *reinterpret_cast<uint4*>(dst + (size_t)f * BYTES) = make_uint4(w[0], w[1], w[2], w[3]);
-        } else {
-            for (uint32_t e = 0; e < nv; ++e) {
-                if (BYTES == 4) reinterpret_cast<uint32_t*>(dst)[f + e] = w[e];
-                else reinterpret_cast<uint16_t*>(dst)[f + e] = (uint16_t)(w[e >> 1] >> (16 * (e & 1)));
+        uint32_t w[UG][4];
+#pragma unroll
+        for (int u = 0; u < UG; ++u) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) w[u][j] = 0;
+#pragma unroll
+            for (uint32_t e = 0; e < VE; ++e) {
+                const uint32_t x = idx[u][e] != kNone ? load_elem<BYTES>(src, idx[u][e]) : 0u;
+                if (BYTES == 4) w[u][e] = x;
+                else w[u][e >> 1] |= x << (16 * (e & 1));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UG; ++u) {
+            const uint32_t f = fp + (u * kThreads + threadIdx.x) * VE;
+            if (f >= total) continue;
+            if (f + VE <= total) {
+                *reinterpret_cast<uint4*>(dst + (size_t)f * BYTES) = make_uint4(w[u][0], w[u][1], w[u][2], w[u][3]);
+            } else {
+#pragma unroll
+                for (uint32_t e = 0; e < VE; ++e) {
+                    if (e < total - f) {
+                        if (BYTES == 4) reinterpret_cast<uint32_t*>(dst)[f + e] = w[u][e];
+                        else reinterpret_cast<uint16_t*>(dst)[f + e] = (uint16_t)(w[u][e >> 1] >> (16 * (e & 1)));
+                    }
+                }
             }
         }
     }
 }
 
-__global__ void __launch_bounds__(kThreads) k_compact_gather(Tables tb, CompactWs ws, const char* src_arena,
-                                                             const int32_t* __restrict__ keep_idx, char* dst_arena) {
+// Every block takes a contiguous range of gather units and walks the items that own them, so the
+// item's context (source, destination, keep lists, new extents) is fetched once per run.
+template <int WBYTES>  // element width of the weight tensors; BatchNorm vectors and biases are always 4 bytes
+__global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, CompactWs ws, const char* src_arena,
+                                                                const int32_t* __restrict__ keep_idx, char* dst_arena) {
     const uint32_t total_units = ws.unit_prefix[tb.n_items];
-    for (uint32_t unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
-        // the item holding this unit: last i with unit_prefix[i] <= unit
-        uint32_t lo = 0, hi = tb.n_items;
-        while (hi - lo > 1) {
-            const uint32_t mid = (lo + hi) >> 1;
-            if (ws.unit_prefix[mid] <= unit) lo = mid;
-            else hi = mid;
+    const uint32_t per = (total_units + gridDim.x - 1) / gridDim.x;
+    const uint32_t u_lo = min(total_units, blockIdx.x * per), u_hi = min(total_units, u_lo + per);
+    if (u_lo >= u_hi) return;
+    // the item holding the first unit: last i with unit_prefix[i] <= u_lo
+    uint32_t item = 0, hi = tb.n_items;
+    while (hi - item > 1) {
+        const uint32_t mid = (item + hi) >> 1;
+        if (ws.unit_prefix[mid] <= u_lo) item = mid;
+        else hi = mid;
+    }
+    uint32_t unit = u_lo;
+    while (unit < u_hi) {
+        const uint32_t item_begin = ws.unit_prefix[item], item_end = ws.unit_prefix[item + 1];
+        if (unit >= item_end) {  // items that shrank to nothing own no units
+            ++item;
+            continue;
         }
-        const ItemDesc& it = tb.items[lo];
-        const uint32_t On = ws.item_dims[2 * lo], Cn = ws.item_dims[2 * lo + 1];
+        const ItemDesc& it = tb.items[item];
+        const uint32_t On = ws.item_dims[2 * item], Cn = ws.item_dims[2 * item + 1];
         const char* src;
         if (it.tensor >= 0) {
             const TensorDesc& d = tb.tensors[it.tensor];
@@ -130,12 +202,14 @@ __global__ void __launch_bounds__(kThreads) k_compact_gather(Tables tb, CompactW
         } else {
             src = static_cast<const char*>(it.src);
         }
-        char* dst = dst_arena + ws.item_off[lo];
+        char* dst = dst_arena + ws.item_off[item];
         const int32_t* ko = keep_idx + tb.groups[it.out_group].off_idx;
         const int32_t* ki = it.in_group >= 0 ? keep_idx + tb.groups[it.in_group].off_idx : nullptr;
-        const uint32_t f0 = (unit - ws.unit_prefix[lo]) * (kUnitBytes / it.elem_bytes);
-        if (it.elem_bytes == 4) gather_unit<4>(it, src, dst, ko, ki, On, Cn, f0);
-        else gather_unit<2>(it, src, dst, ko, ki, On, Cn, f0);
+        const uint32_t run_end = min(u_hi, item_end);
+        const uint32_t f0 = (unit - item_begin) * (kUnitBytes / it.elem_bytes);
+        if (WBYTES == 4 || it.elem_bytes == 4) gather_run<4>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit);
+        else gather_run<2>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit);
+        unit = run_end;
     }
 }
 
@@ -145,7 +219,10 @@ int launch_compact(const Tables& tb, const CompactWs& ws, const void* src_arena,
                    const int32_t* keep_count, void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets,
                    int32_t* dst_shapes, int n_sm, cudaStream_t st) {
     k_compact_layout<<<1, 1024, 0, st>>>(tb, ws, keep_count, dst_bytes, dst_offsets, dst_shapes);
-    k_compact_gather<<<n_sm * 8, kThreads, 0, st>>>(tb, ws, (const char*)src_arena, keep_idx, (char*)dst_arena);
+    if (tb.dtype == DNNS_F32)
+        k_compact_gather<4><<<n_sm * 4, kThreads, 0, st>>>(tb, ws, (const char*)src_arena, keep_idx, (char*)dst_arena);
+    else
+        k_compact_gather<2><<<n_sm * 4, kThreads, 0, st>>>(tb, ws, (const char*)src_arena, keep_idx, (char*)dst_arena);
     return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 

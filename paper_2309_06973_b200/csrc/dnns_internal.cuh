@@ -91,6 +91,7 @@ struct ThresholdWs {
     uint32_t* hist1;        // [S][kHistBins]
     uint32_t* hist2;        // [S][n_k][kLowBins] (fp32 only)
     uint32_t* bitmap;       // [S][kBitmapWords]: first digits that some variant selected
+    uint32_t* tie_bitmap;   // [S][kBitmapWords]: low 15 bits of the thresholds that need tie tables
     SelectState* sel;       // [n_k][S]
     uint32_t* need;         // [n_k][S]: the variant masks only part of the weights equal to tau
     uint32_t* any_need;     // [1]

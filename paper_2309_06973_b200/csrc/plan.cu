@@ -20,7 +20,7 @@ struct WsMap {
     uint64_t tables_end;  // everything before this is uploaded once at plan creation
     uint64_t k_dev, bitmap, sel, tie_prefix, unit_prefix, item_off, item_dims;
     uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
-    uint64_t any_need, need, tile_ties, hist1, hist2;
+    uint64_t any_need, need, tie_bitmap, tile_ties, hist1, hist2;
     uint64_t total;
 };
 
@@ -114,6 +114,7 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.clear_begin = o;
     w.any_need = take(4);
     w.need = take(4 * vs);
+    w.tie_bitmap = take(4ull * kBitmapWords * (c.S ? c.S : 1));
     w.tile_ties = take(4ull * maxv * c.tiles);
     w.hist1 = take(4ull * kHistBins * (c.S ? c.S : 1));
     w.hist2 = take(c.dtype == DNNS_F32 ? 4ull * kLowBins * vs : 0);
@@ -311,6 +312,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     t.hist1 = reinterpret_cast<uint32_t*>(w + map.hist1);
     t.hist2 = reinterpret_cast<uint32_t*>(w + map.hist2);
     t.bitmap = reinterpret_cast<uint32_t*>(w + map.bitmap);
+    t.tie_bitmap = reinterpret_cast<uint32_t*>(w + map.tie_bitmap);
     t.sel = reinterpret_cast<SelectState*>(w + map.sel);
     t.need = reinterpret_cast<uint32_t*>(w + map.need);
     t.any_need = reinterpret_cast<uint32_t*>(w + map.any_need);

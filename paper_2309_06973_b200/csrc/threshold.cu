@@ -20,32 +20,106 @@ namespace {
 
 constexpr int kHistThreads = 1024;
 
-// Visit the vectors of elements [e0, e1) of one tensor with all threads of the block; e0 is a
-// multiple of the vector width.  f(vector, n_valid) is called once per vector.
-template <int DT, int THREADS, typename F>
-__device__ __forceinline__ void for_each_vec(const void* base, uint32_t e0, uint32_t e1, uint32_t numel, F f) {
-    constexpr uint32_t P = Elem<DT>::kPerVec;
-    constexpr int U = 4;
-    const uint32_t v0 = e0 / P, v1 = (e1 + P - 1) / P;
-    uint32_t i = v0 + threadIdx.x;
-    for (; i + (U - 1) * THREADS < v1; i += U * THREADS) {
-        uint4 v[U];
-        int n[U];
+// Bit `i` of a 32768-bit bitmap in shared memory, i = the 15 bits of x starting at bit SHIFT.
+template <int SHIFT>
+__device__ __forceinline__ uint32_t bitmap_test(const uint32_t* bm, uint32_t x) {
+    return (bm[(x >> (SHIFT + 5)) & 0x3FFu] >> ((x >> SHIFT) & 31u)) & 1u;
+}
+
+// Walk the block's contiguous share of the tile list.  For every run of tiles of one prunable
+// tensor: on_span(d) (block-uniform, may synchronise; false skips the run), then
+// on_tile(tile, n_e, v) per tile (n_e valid elements; vectors past the end hold zeros), with the
+// next tile's loads already in flight.
+template <int DT, typename SpanFn, typename TileFn>
+__device__ __forceinline__ void walk_prunable_tiles(const Tables& tb, SpanFn on_span, TileFn on_tile) {
+    constexpr int P = Elem<DT>::kPerVec;
+    constexpr uint32_t kTileElems = kTileBytes / Elem<DT>::kBytes;
+    const uint32_t per = (tb.n_tiles + gridDim.x - 1) / gridDim.x;
+    const uint32_t lo = min(tb.n_tiles, blockIdx.x * per), hi = min(tb.n_tiles, lo + per);
+    uint32_t tile = lo;
+    while (tile < hi) {
+        const TensorDesc& d = tb.tensors[tb.tile_tensor[tile]];
+        const uint32_t span_end = min(hi, d.tile0 + d.n_tiles);
+        if (d.seg < 0 || !on_span(d)) {
+            tile = span_end;
+            continue;
+        }
+        const uint32_t numel = d.numel, tile0 = d.tile0;
+        const char* src = static_cast<const char*>(d.src);
+        uint4 nxt[kVecPerThread];
+        auto issue = [&](uint32_t t) {
+            const uint32_t e0 = (t - tile0) * kTileElems;
+            if (e0 + kTileElems <= numel) {
+                const uint4* p = reinterpret_cast<const uint4*>(src + (size_t)e0 * Elem<DT>::kBytes) + threadIdx.x;
 #pragma unroll
-        for (int u = 0; u < U; ++u) n[u] = load_vec<DT>(base, (i + u * THREADS) * P, numel, v[u]);
+                for (int u = 0; u < kVecPerThread; ++u) nxt[u] = __ldg(p + u * kTileThreads);
+            } else {
 #pragma unroll
-        for (int u = 0; u < U; ++u) f(v[u], n[u]);
+                for (int u = 0; u < kVecPerThread; ++u)
+                    load_vec<DT>(src, e0 + (u * kTileThreads + threadIdx.x) * P, numel, nxt[u]);
+            }
+        };
+        issue(tile);
+        for (; tile < span_end; ++tile) {
+            uint4 v[kVecPerThread];
+#pragma unroll
+            for (int u = 0; u < kVecPerThread; ++u) v[u] = nxt[u];
+            if (tile + 1 < span_end) issue(tile + 1);
+            on_tile(tile, min(kTileElems, numel - (tile - tile0) * kTileElems), v);
+        }
     }
-    for (; i < v1; i += THREADS) {
-        uint4 v;
-        const int n = load_vec<DT>(base, i * P, numel, v);
-        f(v, n);
+}
+
+// The keys of a tile that pass a bitmap filter: f(key) is called by the thread holding the key.
+// SHIFT32 / the two 16-bit halves select which 15 bits of a stored word index the bitmap.
+template <int DT, int SHIFT32, typename F>
+__device__ __forceinline__ void for_filtered_keys(const uint4 (&v)[kVecPerThread], uint32_t n_e, const uint32_t* bm, F f) {
+    constexpr int P = Elem<DT>::kPerVec;
+    constexpr uint32_t kTileElems = kTileBytes / Elem<DT>::kBytes;
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; ++u) {
+        const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+        uint32_t hits = 0;
+        if (DT == DNNS_F32) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) hits |= bitmap_test<SHIFT32>(bm, w[j]) << j;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                hits |= (bitmap_test<0>(bm, w[j]) << (2 * j)) | (bitmap_test<16>(bm, w[j]) << (2 * j + 1));
+        }
+        if (n_e != kTileElems) {  // ragged tile: drop the slots past the end of the tensor
+            const uint32_t first = (u * kTileThreads + threadIdx.x) * P;
+            hits &= first >= n_e ? 0u : (n_e - first >= (uint32_t)P ? 0xFFu : ((1u << (n_e - first)) - 1u));
+        }
+        while (hits) {
+            const int j = __ffs(hits) - 1;
+            hits &= hits - 1;
+            uint32_t x = DT == DNNS_F32 ? j : j >> 1;
+            x = x == 0 ? w[0] : (x == 1 ? w[1] : (x == 2 ? w[2] : w[3]));
+            f(DT == DNNS_F32 ? (x & 0x7FFFFFFFu) : ((x >> (16 * (j & 1))) & 0x7FFFu));
+        }
     }
 }
 
 // ---------------------------------------------------------------- pass 1
+// Count one stored word's key(s) by first digit; digit 0 (exact zeros, mostly) in a register.
+template <int DT>
+__device__ __forceinline__ void count_word(uint32_t w, uint32_t* sh, uint32_t& zeros) {
+    const uint32_t hi = (w >> 14) & 0x1FFFCu;  // 4 * (bits 16..30)
+    if (hi == 0) ++zeros;
+    else atomicAdd(reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(sh) + hi), 1u);
+    if (DT == DNNS_BF16) {
+        const uint32_t lo = (w << 2) & 0x1FFFCu;  // 4 * (bits 0..14)
+        if (lo == 0) ++zeros;
+        else atomicAdd(reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(sh) + lo), 1u);
+    }
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kHistThreads, 1) k_hist1(Tables tb, uint32_t* __restrict__ hist1) {
+    constexpr uint32_t P = Elem<DT>::kPerVec;
+    constexpr int U = 4;
     extern __shared__ uint32_t sh[];  // kHistBins counters
     for (uint32_t b = threadIdx.x; b < kHistBins; b += kHistThreads) sh[b] = 0;
     __syncthreads();
@@ -53,7 +127,7 @@ __global__ void __launch_bounds__(kHistThreads, 1) k_hist1(Tables tb, uint32_t* 
     const uint32_t per = (tb.n_tiles + gridDim.x - 1) / gridDim.x;
     const uint32_t lo = min(tb.n_tiles, blockIdx.x * per), hi = min(tb.n_tiles, lo + per);
     int cur_seg = -1;
-    uint32_t zeros = 0;  // keys with first digit 0 (exact zeros, mostly): counted in a register
+    uint32_t zeros = 0;
 
     auto flush = [&](int seg) {
         // merge this block's counters into the segment's global histogram and clear them
@@ -84,20 +158,52 @@ __global__ void __launch_bounds__(kHistThreads, 1) k_hist1(Tables tb, uint32_t* 
                 flush(cur_seg);
                 cur_seg = d.seg;
             }
+            // elements [e0, e1) of this tensor: whole vectors in batches of U per thread with the
+            // next batch in flight, then the remaining vectors, then the last few elements
             const uint32_t e0 = (tile - d.tile0) * tb.tile_elems;
             const uint32_t e1 = min(d.numel, (span_end - d.tile0) * tb.tile_elems);
-            for_each_vec<DT, kHistThreads>(d.src, e0, e1, d.numel, [&](const uint4& v, int n) {
-                uint32_t key[Elem<DT>::kPerVec];
-                vec_keys<DT>(v, key);
+            const uint32_t n_vec = (e1 - e0) / P;
+            const uint4* p = reinterpret_cast<const uint4*>(static_cast<const char*>(d.src) + (size_t)e0 * Elem<DT>::kBytes);
+            const uint32_t n_batch = n_vec / (U * kHistThreads);
+            if (n_batch) {
+                uint4 nxt[U];
+                const uint4* q = p + threadIdx.x;
 #pragma unroll
-                for (int j = 0; j < Elem<DT>::kPerVec; ++j) {
-                    const uint32_t dg = digit_of<DT>(key[j]);
-                    if (j < n) {
-                        if (dg == 0) ++zeros;
-                        else atomicAdd(&sh[dg], 1u);
+                for (int u = 0; u < U; ++u) nxt[u] = __ldg(q + u * kHistThreads);
+                for (uint32_t b = 0; b < n_batch; ++b) {
+                    uint4 cur[U];
+#pragma unroll
+                    for (int u = 0; u < U; ++u) cur[u] = nxt[u];
+                    if (b + 1 < n_batch) {
+                        q += U * kHistThreads;
+#pragma unroll
+                        for (int u = 0; u < U; ++u) nxt[u] = __ldg(q + u * kHistThreads);
+                    }
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        count_word<DT>(cur[u].x, sh, zeros);
+                        count_word<DT>(cur[u].y, sh, zeros);
+                        count_word<DT>(cur[u].z, sh, zeros);
+                        count_word<DT>(cur[u].w, sh, zeros);
                     }
                 }
-            });
+            }
+            for (uint32_t i = n_batch * U * kHistThreads + threadIdx.x; i < n_vec; i += kHistThreads) {
+                const uint4 c = __ldg(p + i);
+                count_word<DT>(c.x, sh, zeros);
+                count_word<DT>(c.y, sh, zeros);
+                count_word<DT>(c.z, sh, zeros);
+                count_word<DT>(c.w, sh, zeros);
+            }
+            const uint32_t e = e0 + n_vec * P + threadIdx.x;
+            if (e < e1) {
+                uint32_t key;
+                if (DT == DNNS_F32) key = static_cast<const uint32_t*>(d.src)[e] & 0x7FFFFFFFu;
+                else key = static_cast<const uint16_t*>(d.src)[e] & 0x7FFFu;
+                const uint32_t dg = digit_of<DT>(key);
+                if (dg == 0) ++zeros;
+                else atomicAdd(&sh[dg], 1u);
+            }
         }
         tile = span_end;
     }
@@ -158,23 +264,21 @@ __global__ void __launch_bounds__(1024) k_select1(Tables tb, ThresholdWs ws, int
         }
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        // variants that selected the same first digit share one second-pass histogram
-        int n_slots = 0;
-        for (int v = 0; v < n_k; ++v) {
-            const uint32_t dg = s_digit[v];
-            if (dg == 0xFFFFFFFFu) continue;
-            int slot = -1;
-            for (int u = 0; u < v; ++u)
-                if (s_digit[u] == dg) {
-                    slot = (int)ws.sel[(size_t)u * S + seg].slot;
-                    break;
-                }
-            if (slot < 0) {
-                slot = n_slots++;
-                bm[dg >> 5] |= 1u << (dg & 31);
+    if ((int)threadIdx.x < n_k) {
+        // variants that selected the same first digit share one second-pass histogram: its slot is
+        // the rank of the digit among the distinct selected digits of the segment
+        const uint32_t dg = s_digit[threadIdx.x];
+        if (dg != 0xFFFFFFFFu) {
+            uint32_t slot = 0;
+            for (int u = 0; u < n_k; ++u) {
+                const uint32_t du = s_digit[u];
+                bool first = du != 0xFFFFFFFFu && du < dg;  // count each smaller digit once
+                for (int t = 0; t < u && first; ++t)
+                    if (s_digit[t] == du) first = false;
+                slot += first;
             }
-            ws.sel[(size_t)v * S + seg].slot = (uint32_t)slot;
+            ws.sel[(size_t)threadIdx.x * S + seg].slot = slot;
+            atomicOr(&bm[dg >> 5], 1u << (dg & 31));
         }
     }
     if (DT == DNNS_BF16) {
@@ -194,70 +298,72 @@ __global__ void __launch_bounds__(1024) k_select1(Tables tb, ThresholdWs ws, int
             }
             thr[(size_t)v * S + seg] = r;
             ws.need[(size_t)v * S + seg] = need;
-            if (need) atomicOr(ws.any_need, 1u);
+            if (need) {
+                atomicOr(ws.any_need, 1u);
+                atomicOr(&ws.tie_bitmap[(size_t)seg * kBitmapWords + (r.tau_bits >> 5)], 1u << (r.tau_bits & 31));
+            }
         }
     }
 }
 
 // ---------------------------------------------------------------- pass 2 (31-bit keys)
-__global__ void __launch_bounds__(kTileThreads) k_hist2(Tables tb, ThresholdWs ws, int n_k) {
-    __shared__ uint32_t s_bm[kBitmapWords];
-    __shared__ uint32_t s_digit[kMaxVariants], s_slot[kMaxVariants];
-    const uint32_t S = tb.n_segs;
-    int cur_seg = -1;
-    for (uint32_t tile = blockIdx.x; tile < tb.n_tiles; tile += gridDim.x) {
-        const TensorDesc& d = tb.tensors[tb.tile_tensor[tile]];
-        if (d.seg < 0) continue;
-        if (d.seg != cur_seg) {
-            __syncthreads();
-            cur_seg = d.seg;
-            for (uint32_t w = threadIdx.x; w < kBitmapWords; w += kTileThreads)
-                s_bm[w] = ws.bitmap[(size_t)cur_seg * kBitmapWords + w];
-            if ((int)threadIdx.x < n_k) {
-                const SelectState st = ws.sel[(size_t)threadIdx.x * S + cur_seg];
-                s_digit[threadIdx.x] = st.digit;
-                s_slot[threadIdx.x] = st.slot;
-            }
-            __syncthreads();
-        }
-        uint32_t* h2 = ws.hist2 + (size_t)cur_seg * n_k * kLowBins;
-        const uint32_t e0 = (tile - d.tile0) * tb.tile_elems;
-        uint4 v[kVecPerThread];
-        int n[kVecPerThread];
+// Load a segment's bitmap into shared memory together with, per word, the number of set bits in
+// earlier words, so that rank(digit) - the digit's histogram slot - is one popcount away.
+__device__ __forceinline__ void load_bitmap_with_ranks(const uint32_t* g_bm, uint32_t* s_bm, uint32_t* s_rank,
+                                                       uint32_t* scratch) {
+    constexpr int W = kBitmapWords / kTileThreads;  // words per thread
+    uint32_t w[W], c = 0;
 #pragma unroll
-        for (int u = 0; u < kVecPerThread; ++u)
-            n[u] = load_vec<DNNS_F32>(d.src, e0 + (u * kTileThreads + threadIdx.x) * 4, d.numel, v[u]);
-#pragma unroll
-        for (int u = 0; u < kVecPerThread; ++u) {
-            uint32_t key[4];
-            vec_keys<DNNS_F32>(v[u], key);
-            bool hit[4];
-            bool any = false;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t dg = key[j] >> 16;
-                hit[j] = j < n[u] && ((s_bm[dg >> 5] >> (dg & 31)) & 1u);
-                any |= hit[j];
-            }
-            if (!__any_sync(0xffffffffu, any)) continue;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const unsigned act = __ballot_sync(0xffffffffu, hit[j]);
-                if (!hit[j]) continue;
-                const unsigned peers = __match_any_sync(act, key[j]);
-                if ((threadIdx.x & 31) == (unsigned)(__ffs(peers) - 1)) {
-                    const uint32_t dg = key[j] >> 16;
-                    uint32_t slot = 0;
-                    for (int vv = 0; vv < n_k; ++vv)
-                        if (s_digit[vv] == dg) {
-                            slot = s_slot[vv];
-                            break;
-                        }
-                    atomicAdd(&h2[(size_t)slot * kLowBins + (key[j] & 0xFFFFu)], (uint32_t)__popc(peers));
-                }
-            }
-        }
+    for (int i = 0; i < W; ++i) {
+        w[i] = g_bm[threadIdx.x * W + i];
+        c += __popc(w[i]);
     }
+    uint32_t total;
+    uint32_t ex = block_exclusive_scan<uint32_t>(c, scratch, &total);
+#pragma unroll
+    for (int i = 0; i < W; ++i) {
+        s_bm[threadIdx.x * W + i] = w[i];
+        s_rank[threadIdx.x * W + i] = ex;
+        ex += __popc(w[i]);
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kTileThreads, 4) k_hist2(Tables tb, ThresholdWs ws, int n_k) {
+    __shared__ uint32_t s_bm[kBitmapWords], s_rank[kBitmapWords];
+    __shared__ uint32_t scratch[33];
+    int cur_seg = -1;
+    uint32_t* h2 = nullptr;
+    uint32_t zeros = 0;  // exact zeros among the selected keys: counted in a register, added once
+    auto flush_zeros = [&]() {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) zeros += __shfl_xor_sync(0xffffffffu, zeros, d);
+        if ((threadIdx.x & 31) == 0 && zeros) atomicAdd(&h2[0], zeros);  // digit 0 has rank 0, low digit 0
+        zeros = 0;
+    };
+    walk_prunable_tiles<DNNS_F32>(
+        tb,
+        [&](const TensorDesc& d) {
+            if (d.seg != cur_seg) {
+                if (cur_seg >= 0) flush_zeros();
+                cur_seg = d.seg;
+                load_bitmap_with_ranks(ws.bitmap + (size_t)cur_seg * kBitmapWords, s_bm, s_rank, scratch);
+                h2 = ws.hist2 + (size_t)cur_seg * n_k * kLowBins;
+            }
+            return true;
+        },
+        [&](uint32_t, uint32_t n_e, const uint4(&v)[kVecPerThread]) {
+            for_filtered_keys<DNNS_F32, 16>(v, n_e, s_bm, [&](uint32_t key) {
+                if (key == 0) {
+                    ++zeros;
+                    return;
+                }
+                const uint32_t dg = key >> 16;
+                const uint32_t slot = s_rank[dg >> 5] + __popc(s_bm[dg >> 5] & ((1u << (dg & 31)) - 1u));
+                atomicAdd(&h2[(size_t)slot * kLowBins + (key & 0xFFFFu)], 1u);
+            });
+        });
+    if (cur_seg >= 0) flush_zeros();
 }
 
 // ---------------------------------------------------------------- select 2 (31-bit keys)
@@ -304,66 +410,67 @@ __global__ void __launch_bounds__(1024) k_select2(Tables tb, ThresholdWs ws, int
         thr[idx] = r;
         const uint32_t need = r.n_tie < r.n_equal;
         ws.need[idx] = need;
-        if (need) atomicOr(ws.any_need, 1u);
+        if (need) {
+            const uint32_t low = r.tau_bits & 0x7FFFu;  // the tie sweep filters keys by these 15 bits
+            atomicOr(ws.any_need, 1u);
+            atomicOr(&ws.tie_bitmap[(size_t)seg * kBitmapWords + (low >> 5)], 1u << (low & 31));
+        }
     }
 }
 
 // ---------------------------------------------------------------- tie counts per tile
+// Keys are filtered by the low 15 bits of the thresholds that need tie tables (a 15-bit key is its
+// own filter), then compared exactly.  Counts go straight to the per-tile table in global memory;
+// exact zeros, the one value that can fill whole tiles, are counted per warp first.
 template <int DT>
-__global__ void __launch_bounds__(kTileThreads) k_ties(Tables tb, ThresholdWs ws, int n_k,
-                                                       const dnns_threshold* __restrict__ thr) {
+__global__ void __launch_bounds__(kTileThreads, 4) k_ties(Tables tb, ThresholdWs ws, int n_k,
+                                                          const dnns_threshold* __restrict__ thr) {
     if (*ws.any_need == 0) return;
     __shared__ uint32_t s_bm[kBitmapWords];
-    __shared__ uint32_t s_tau[kMaxVariants], s_need[kMaxVariants], s_cnt[kMaxVariants];
-    __shared__ uint32_t s_any;
+    __shared__ uint32_t s_tau[kMaxVariants], s_need[kMaxVariants];
+    __shared__ uint32_t s_any, s_zero_tau;
     const uint32_t S = tb.n_segs;
     int cur_seg = -1;
-    for (uint32_t tile = blockIdx.x; tile < tb.n_tiles; tile += gridDim.x) {
-        const TensorDesc& d = tb.tensors[tb.tile_tensor[tile]];
-        if (d.seg < 0) continue;
-        if (d.seg != cur_seg) {
-            __syncthreads();
-            cur_seg = d.seg;
-            if (threadIdx.x == 0) s_any = 0;
-            __syncthreads();
-            for (uint32_t w = threadIdx.x; w < kBitmapWords; w += kTileThreads)
-                s_bm[w] = ws.bitmap[(size_t)cur_seg * kBitmapWords + w];
-            if ((int)threadIdx.x < n_k) {
-                const size_t idx = (size_t)threadIdx.x * S + cur_seg;
-                s_tau[threadIdx.x] = thr[idx].tau_bits;
-                s_need[threadIdx.x] = ws.need[idx];
-                s_cnt[threadIdx.x] = 0;
-                if (ws.need[idx]) s_any = 1;
-            }
-            __syncthreads();
-        }
-        if (!s_any) continue;
-        const uint32_t e0 = (tile - d.tile0) * tb.tile_elems;
-        uint4 v[kVecPerThread];
-        int n[kVecPerThread];
-#pragma unroll
-        for (int u = 0; u < kVecPerThread; ++u)
-            n[u] = load_vec<DT>(d.src, e0 + (u * kTileThreads + threadIdx.x) * Elem<DT>::kPerVec, d.numel, v[u]);
-#pragma unroll
-        for (int u = 0; u < kVecPerThread; ++u) {
-            uint32_t key[Elem<DT>::kPerVec];
-            vec_keys<DT>(v[u], key);
-#pragma unroll
-            for (int j = 0; j < Elem<DT>::kPerVec; ++j) {
-                const uint32_t dg = digit_of<DT>(key[j]);
-                if (j < n[u] && ((s_bm[dg >> 5] >> (dg & 31)) & 1u)) {
-                    for (int vv = 0; vv < n_k; ++vv)
-                        if (s_need[vv] && s_tau[vv] == key[j]) atomicAdd(&s_cnt[vv], 1u);
+    walk_prunable_tiles<DT>(
+        tb,
+        [&](const TensorDesc& d) {
+            if (d.seg != cur_seg) {
+                __syncthreads();
+                cur_seg = d.seg;
+                if (threadIdx.x == 0) s_any = s_zero_tau = 0;
+                __syncthreads();
+                for (uint32_t w = threadIdx.x; w < kBitmapWords; w += kTileThreads)
+                    s_bm[w] = ws.tie_bitmap[(size_t)cur_seg * kBitmapWords + w];
+                if ((int)threadIdx.x < n_k) {
+                    const size_t idx = (size_t)threadIdx.x * S + cur_seg;
+                    const uint32_t need = ws.need[idx], tau = thr[idx].tau_bits;
+                    s_tau[threadIdx.x] = tau;
+                    s_need[threadIdx.x] = need;
+                    if (need) s_any = 1;
+                    if (need && tau == 0) s_zero_tau = 1;
                 }
+                __syncthreads();
             }
-        }
-        __syncthreads();
-        if ((int)threadIdx.x < n_k) {
-            ws.tile_ties[(size_t)threadIdx.x * tb.n_tiles + tile] = s_cnt[threadIdx.x];
-            s_cnt[threadIdx.x] = 0;
-        }
-        __syncthreads();
-    }
+            return s_any != 0;  // no variant of this segment splits its ties: nothing to count
+        },
+        [&](uint32_t tile, uint32_t n_e, const uint4(&v)[kVecPerThread]) {
+            uint32_t zeros = 0;
+            for_filtered_keys<DT, 0>(v, n_e, s_bm, [&](uint32_t key) {
+                if (key == 0) {
+                    ++zeros;
+                    return;
+                }
+                for (int vv = 0; vv < n_k; ++vv)
+                    if (s_need[vv] && s_tau[vv] == key) atomicAdd(&ws.tile_ties[(size_t)vv * tb.n_tiles + tile], 1u);
+            });
+            if (s_zero_tau) {
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) zeros += __shfl_xor_sync(0xffffffffu, zeros, d);
+                if ((threadIdx.x & 31) == 0 && zeros)
+                    for (int vv = 0; vv < n_k; ++vv)
+                        if (s_need[vv] && s_tau[vv] == 0) atomicAdd(&ws.tile_ties[(size_t)vv * tb.n_tiles + tile], zeros);
+            }
+        });
 }
 
 // Exclusive scan of the tile counts over the tiles of a segment, one block per (variant, segment).
@@ -400,7 +507,7 @@ int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, int /*n_k
                      int n_sm, cudaStream_t st) {
     const uint32_t S = tb.n_segs;
     const int hist_grid = (int)min((uint32_t)n_sm, tb.n_tiles);
-    const int sweep_grid = (int)min((uint32_t)n_sm * 8u, tb.n_tiles);
+    const int sweep_grid = (int)min((uint32_t)n_sm * 4u, tb.n_tiles);
     int launches = 0;
     if (tb.dtype == DNNS_F32) {
         k_hist1<DNNS_F32><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws.hist1);

@@ -35,7 +35,8 @@ constexpr size_t kOffTiePrefix = kOffTileTensor + 4 * (size_t)kMaxTiles;
 constexpr size_t kOffClear = kOffTiePrefix + 4 * (size_t)kMaxTiles;
 constexpr size_t kOffAnyNeed = kOffClear;
 constexpr size_t kOffNeed = kOffAnyNeed + 256;
-constexpr size_t kOffTileTies = kOffNeed + 256;
+constexpr size_t kOffTieBitmap = kOffNeed + 256;
+constexpr size_t kOffTileTies = kOffTieBitmap + 4 * kBitmapWords;
 constexpr size_t kOffHist1 = kOffTileTies + 4 * (size_t)kMaxTiles;
 constexpr size_t kOffHist2 = kOffHist1 + 4 * (size_t)kHistBins;
 constexpr size_t kScratchBytes = kOffHist2 + 4 * (size_t)kLowBins;
@@ -112,6 +113,7 @@ extern "C" dnns_status dnns_magnitude_threshold_static(const void* weights_dev, 
     ws.hist1 = reinterpret_cast<uint32_t*>(base + kOffHist1);
     ws.hist2 = reinterpret_cast<uint32_t*>(base + kOffHist2);
     ws.bitmap = reinterpret_cast<uint32_t*>(base + kOffBitmap);
+    ws.tie_bitmap = reinterpret_cast<uint32_t*>(base + kOffTieBitmap);
     ws.sel = reinterpret_cast<SelectState*>(base + kOffSel);
     ws.need = reinterpret_cast<uint32_t*>(base + kOffNeed);
     ws.any_need = reinterpret_cast<uint32_t*>(base + kOffAnyNeed);
