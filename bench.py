@@ -219,7 +219,7 @@ def main():
     # data-dependent sizes of every variant (outside the timed region): R = kept filter rows, N' = rebuilt size
     R, Nn = [], []
     for v in range(V):
-        ses.variant(v)
+        ses.variant(v, fused=not args.stepwise)
         torch.cuda.synchronize()
         sh = ses.dst_shapes.cpu().numpy()[: 2 * len(wl.tensors)].reshape(-1, 2)
         R.append(sum(int(sh[i, 0]) * t.I * t.KH * t.KW for i, t in enumerate(wl.tensors)))

@@ -76,30 +76,43 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
     const uint32_t blk = it.blk, Cin = it.Cin;
     const uint32_t Ln = Cn * blk, L = Cin * blk;  // new and old row length
     const uint32_t total = On * Ln;
+    // A thread's destination vectors are kStride elements apart, unit after unit, so its position
+    // (row a, offset rem in the row) is advanced with one add and one compare instead of a division.
+    constexpr uint32_t kStride = kThreads * VE;
+    const uint32_t step_a = kStride / Ln, step_rem = kStride - step_a * Ln;
+    uint32_t pos_f = f0 + threadIdx.x * VE;
+    uint32_t pos_a = pos_f / Ln, pos_rem = pos_f - pos_a * Ln;
+    auto advance = [&]() {
+        pos_f += kStride;
+        pos_a += step_a;
+        pos_rem += step_rem;
+        if (pos_rem >= Ln) {
+            pos_rem -= Ln;
+            ++pos_a;
+        }
+    };
     if ((Cn == Cin) && (L % VE == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0)) {
         // Rows lose no input channel: every destination vector is one aligned source vector of row
         // ko[a].  The loads of the next unit are issued before the current unit is stored.
         uint4 nxt[U];
         bool nxt_ok[U];
-        auto issue = [&](uint32_t fu) {
+        auto issue = [&]() {
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const uint32_t f = fu + (u * kThreads + threadIdx.x) * VE;
-                nxt_ok[u] = f < total;
-                if (nxt_ok[u]) {
-                    const uint32_t a = f / Ln, rem = f - a * Ln;
-                    nxt[u] = __ldg(reinterpret_cast<const uint4*>(src + ((size_t)(uint32_t)ko[a] * L + rem) * BYTES));
-                }
+                nxt_ok[u] = pos_f < total;
+                if (nxt_ok[u])
+                    nxt[u] = __ldg(reinterpret_cast<const uint4*>(src + ((size_t)(uint32_t)ko[pos_a] * L + pos_rem) * BYTES));
+                advance();
             }
         };
-        issue(f0);
+        issue();
         for (uint32_t n = 0; n < n_units; ++n) {
             uint4 cur[U];
             bool ok[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) cur[u] = nxt[u], ok[u] = nxt_ok[u];
             const uint32_t fu = f0 + n * kUnitElems;
-            if (n + 1 < n_units) issue(fu + kUnitElems);
+            if (n + 1 < n_units) issue();
 #pragma unroll
             for (int u = 0; u < U; ++u)
                 if (ok[u]) *reinterpret_cast<uint4*>(dst + (size_t)(fu + (u * kThreads + threadIdx.x) * VE) * BYTES) = cur[u];
@@ -118,9 +131,11 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
             const uint32_t f = fp + (u * kThreads + threadIdx.x) * VE;
 #pragma unroll
             for (uint32_t e = 0; e < VE; ++e) idx[u][e] = kNone;
+            uint32_t a = pos_a;
+            const uint32_t rem = pos_rem;
+            advance();
             if (f >= total) continue;
-            uint32_t a = f / Ln, rem = f - a * Ln;
-            uint32_t c = rem / blk, r = rem - c * blk;
+            uint32_t c = blk == 1 ? rem : (blk == 9 ? rem / 9u : rem / blk), r = rem - c * blk;
             uint32_t row = (uint32_t)ko[a] * Cin, col = ki ? (uint32_t)ki[c] : c;
             const uint32_t nv = min(VE, total - f);
 #pragma unroll

@@ -19,6 +19,7 @@ constexpr uint32_t kHistBins = 32768;    // first radix digit: the top 15 bits o
 constexpr uint32_t kLowBins = 65536;     // second digit of a 31-bit key
 constexpr uint32_t kBitmapWords = kHistBins / 32;
 constexpr int kMaxVariants = 64;
+constexpr uint32_t kFlagRows = 8;         // filters per unit of the flag kernel (divides 32)
 
 struct TensorDesc {
     const void* src;        // the model's tensor
@@ -80,8 +81,10 @@ struct Tables {
     const uint32_t* tile_tensor;
     const int32_t* prod_list;
     const int32_t* cons_list;
+    const uint32_t* flag_prefix;  // [n_tensors + 1] units of the flag kernel before each tensor
+    uint32_t* ebits;        // packed "element is non-zero" bits of the latest sweep (same packing as the mask bits)
     uint32_t* status;       // device status word (a dnns_status, 0 = ok)
-    uint32_t n_tensors, n_groups, n_bn, n_segs, n_items, n_tiles;
+    uint32_t n_tensors, n_groups, n_bn, n_segs, n_items, n_tiles, n_flag_units;
     uint32_t tile_elems;    // 4096 (fp32) or 8192 (bf16)
     int32_t dtype;
 };
@@ -110,8 +113,8 @@ int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, int n_k_s
                      int n_sm, cudaStream_t st);
 int launch_tile_sweep(const Tables& tb, const ThresholdWs& ws, bool do_mask, bool do_struct,
                       const dnns_threshold* thr_dev, int variant, const void* src_arena, void* dst_arena,
-                      uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz, int n_sm,
-                      cudaStream_t st);
+                      uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz, uint32_t n_out_words,
+                      uint32_t n_in_words, int n_sm, cudaStream_t st);
 int launch_propagate(const Tables& tb, const uint32_t* out_nz, const uint32_t* in_nz, uint32_t policy,
                      int32_t min_keep, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count, uint64_t* stats,
                      cudaStream_t st);

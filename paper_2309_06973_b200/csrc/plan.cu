@@ -16,9 +16,9 @@ inline uint64_t align_up(uint64_t x, uint64_t a = kAlign) { return (x + a - 1) /
 
 // Byte offsets of every section of the workspace.
 struct WsMap {
-    uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, status;
+    uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, flag_prefix, status;
     uint64_t tables_end;  // everything before this is uploaded once at plan creation
-    uint64_t k_dev, bitmap, sel, tie_prefix, unit_prefix, item_off, item_dims;
+    uint64_t k_dev, bitmap, sel, tie_prefix, unit_prefix, item_off, item_dims, ebits;
     uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
     uint64_t any_need, need, tie_bitmap, tile_ties, hist1, hist2;
     uint64_t total;
@@ -26,6 +26,7 @@ struct WsMap {
 
 struct Counts {
     uint32_t T = 0, G = 0, B = 0, S = 0, items = 0, tiles = 0, n_bias = 0;
+    uint64_t mask_words = 0;
     int dtype = 0, elem_bytes = 4;
 };
 
@@ -60,6 +61,7 @@ dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts*
         const uint64_t numel = (uint64_t)t.O * t.I * t.KH * t.KW;
         if (numel >= (1ull << 31)) return DNNS_ERR_UNSUPPORTED;
         c->tiles += (uint32_t)((numel * c->elem_bytes + kTileBytes - 1) / kTileBytes);
+        c->mask_words += (numel + 31) / 32;
         if (t.bias) ++c->n_bias;
         if (t.prunable) {
             n_prunable += numel;
@@ -101,6 +103,7 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.tile_tensor = take(4ull * c.tiles);
     w.prod_list = take(4ull * c.T);
     w.cons_list = take(4ull * c.T);
+    w.flag_prefix = take(4ull * (c.T + 1));
     w.status = take(4);
     w.tables_end = o;
     const uint64_t vs = (uint64_t)maxv * (c.S ? c.S : 1);
@@ -111,6 +114,7 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.unit_prefix = take(4ull * (c.items + 1));
     w.item_off = take(8ull * c.items);
     w.item_dims = take(8ull * c.items);
+    w.ebits = take(4ull * c.mask_words);
     w.clear_begin = o;
     w.any_need = take(4);
     w.need = take(4 * vs);
@@ -197,11 +201,12 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     auto* tile_tensor = reinterpret_cast<uint32_t*>(host.data() + map.tile_tensor);
     auto* prod_list = reinterpret_cast<int32_t*>(host.data() + map.prod_list);
     auto* cons_list = reinterpret_cast<int32_t*>(host.data() + map.cons_list);
+    auto* flag_prefix = reinterpret_cast<uint32_t*>(host.data() + map.flag_prefix);
 
     p->arena_off.resize(c.T), p->mask_off.resize(c.T), p->nzmap_off.resize(c.T), p->outnz_off.resize(c.T);
     p->innz_off.resize(c.T), p->seg_of_tensor.assign(c.T, -1), p->keep_off.resize(c.G), p->keepidx_off.resize(c.G);
     p->seg_size.assign(c.S ? c.S : 1, 0);
-    uint64_t arena = 0, mask_w = 0, map_w = 0, out_w = 0, in_w = 0, compact_bytes = 0, n_prunable = 0;
+    uint64_t arena = 0, mask_w = 0, map_w = 0, out_w = 0, in_w = 0, compact_bytes = 0, n_prunable = 0, flag_units = 0;
     uint32_t tile = 0, seg = 0;
     for (uint32_t S = 0; S < c.S; ++S) sd[S] = SegDesc{0xFFFFFFFFu, 0, 0};
     for (uint32_t i = 0; i < c.T; ++i) {
@@ -233,6 +238,19 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
             n_prunable += d.numel;
         }
         tile += d.n_tiles;
+        // units of the flag kernel: kFlagRows filters x 32 map words when a filter is a power-of-two number
+        // of kernel-map words, else 32 kernels
+        const uint64_t n_kernels = (uint64_t)t.O * t.I, wpr = t.I / 32;
+        flag_prefix[i] = (uint32_t)flag_units;
+        if (t.I % 32 == 0 && (wpr & (wpr - 1)) == 0)
+            flag_units += (((uint64_t)t.O + kFlagRows - 1) / kFlagRows) * ((wpr + 31) / 32);
+        else
+            flag_units += (n_kernels + 31) / 32;
+    }
+    flag_prefix[c.T] = (uint32_t)flag_units;
+    if (flag_units >= (1ull << 32)) {
+        delete p;
+        return DNNS_ERR_UNSUPPORTED;
     }
     if (mask_w >= (1ull << 32) || map_w >= (1ull << 32)) {
         delete p;
@@ -304,6 +322,9 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     tb.prod_list = reinterpret_cast<int32_t*>(w + map.prod_list);
     tb.cons_list = reinterpret_cast<int32_t*>(w + map.cons_list);
     tb.status = reinterpret_cast<uint32_t*>(w + map.status);
+    tb.flag_prefix = reinterpret_cast<uint32_t*>(w + map.flag_prefix);
+    tb.ebits = reinterpret_cast<uint32_t*>(w + map.ebits);
+    tb.n_flag_units = (uint32_t)flag_units;
     tb.n_tensors = c.T, tb.n_groups = c.G, tb.n_bn = c.B, tb.n_segs = c.S, tb.n_items = c.items, tb.n_tiles = c.tiles;
     tb.tile_elems = kTileBytes / c.elem_bytes;
     tb.dtype = c.dtype;
@@ -378,7 +399,7 @@ dnns_status dnns_apply_mask(dnns_plan* p, const dnns_threshold* thr_dev, int32_t
     if (!p || !thr_dev || variant < 0 || variant >= p->maxv) return DNNS_ERR_INVALID_ARG;
     if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
     const int n = launch_tile_sweep(p->tb, p->tws, true, false, thr_dev, variant, nullptr, masked_arena, mask_bits,
-                                    nullptr, nullptr, nullptr, p->n_sm, static_cast<cudaStream_t>(stream));
+                                    nullptr, nullptr, nullptr, 0, 0, p->n_sm, static_cast<cudaStream_t>(stream));
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
     return DNNS_OK;
@@ -390,12 +411,9 @@ dnns_status dnns_zero_structures(dnns_plan* p, const void* masked_arena, uint32_
     if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const dnns_layout& L = p->layout;
-    if (cudaMemsetAsync(out_nz, 0, 4 * L.out_nz_words, st) != cudaSuccess ||
-        cudaMemsetAsync(in_nz, 0, 4 * L.in_nz_words, st) != cudaSuccess ||
-        (nz_map && cudaMemsetAsync(nz_map, 0, 4 * L.nz_map_words, st) != cudaSuccess))
-        return DNNS_ERR_CUDA;
+    // (the sweep clears the flag words before the flag kernel ORs into them)
     const int n = launch_tile_sweep(p->tb, p->tws, false, true, nullptr, 0, masked_arena, nullptr, nullptr, nz_map,
-                                    out_nz, in_nz, p->n_sm, st);
+                                    out_nz, in_nz, (uint32_t)L.out_nz_words, (uint32_t)L.in_nz_words, p->n_sm, st);
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
     return DNNS_OK;
@@ -408,12 +426,9 @@ dnns_status dnns_mask_and_structures(dnns_plan* p, const dnns_threshold* thr_dev
     if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const dnns_layout& L = p->layout;
-    if (cudaMemsetAsync(out_nz, 0, 4 * L.out_nz_words, st) != cudaSuccess ||
-        cudaMemsetAsync(in_nz, 0, 4 * L.in_nz_words, st) != cudaSuccess ||
-        (nz_map && cudaMemsetAsync(nz_map, 0, 4 * L.nz_map_words, st) != cudaSuccess))
-        return DNNS_ERR_CUDA;
+    // the flag words are OR-ed into; the kernel map is stored word by word and needs no clearing
     const int n = launch_tile_sweep(p->tb, p->tws, true, true, thr_dev, variant, nullptr, masked_arena, mask_bits,
-                                    nz_map, out_nz, in_nz, p->n_sm, st);
+                                    nz_map, out_nz, in_nz, (uint32_t)L.out_nz_words, (uint32_t)L.in_nz_words, p->n_sm, st);
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
     return DNNS_OK;

@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(kThreads) k_propagate(Tables tb, const uint32_
         }
     }
     if (threadIdx.x == 0) keep_count[g] = (int32_t)carry;
-    if (stats) {
+    if (stats) {  // cleared by the entry point before the launch
         if (lost_pairs) atomicAdd(&stats[0], lost_pairs);
         if (threadIdx.x == 0) {
             if (C - (int)carry) atomicAdd(&stats[1], (unsigned long long)(C - (int)carry));

@@ -1,4 +1,4 @@
-// Steps 2 and 3 as one tile kernel.
+// Steps 2 and 3.
 //
 //   mask       (Section III-C: the insignificant weights are set to zero, the sparse model keeps
 //              its size) - a weight survives when its magnitude key is above tau, or equals tau
@@ -6,13 +6,14 @@
 //              written by the threshold step tell every tile, without looking at any other
 //              tile, whether its ties are all masked, all kept, or split (one tile per segment
 //              at most, which then ranks its ties with a block scan).
-//   structures (Module 2, Sparsity Analyser) - the non-zero bits of the tile's elements go to
-//              shared memory; from them the all-zero 2-D kernels, and from those the filters
-//              (rows) and input columns that still hold something, are OR-ed into the packed
-//              global flag arrays (test first, atomic only when a bit is still missing).
+//   structures (Module 2, Sparsity Analyser) in two kernels: the sweep over the weights packs one
+//              "non-zero" bit per element into the workspace (32 times less data than the
+//              weights, still in L2 when it is read back); k_flags turns those bits into the
+//              all-zero 2-D kernels and from those into the filters (rows) and input columns that
+//              still hold something.
 //
-// The same kernel runs either step alone or both in one sweep (the structures are then derived
-// from the masked values while they are still in registers).
+// The sweep kernel runs either step alone or both at once (the non-zero bits are then taken from
+// the masked values while they are still in registers).
 #include "dnns_internal.cuh"
 
 namespace dnns {
@@ -32,7 +33,7 @@ __device__ __forceinline__ uint32_t gather_word(uint32_t bits, int lane) {
     return v;
 }
 
-// Any bit set in [lo, hi) of a shared-memory bit array.
+// Any bit set in [lo, hi) of a packed bit array.
 __device__ __forceinline__ bool any_bits(const uint32_t* bits, uint32_t lo, uint32_t hi) {
     uint32_t acc = 0;
     while (lo < hi) {
@@ -44,66 +45,121 @@ __device__ __forceinline__ bool any_bits(const uint32_t* bits, uint32_t lo, uint
     return acc != 0;
 }
 
-// From the element bits of one tile (elements [e0, e0+n_e) of tensor d) to kernel map, filter
-// flags and input-column flags.  Kernel q = (o, i) covers elements [q*KK, (q+1)*KK); a kernel cut
-// by the tile edge is OR-ed by both tiles.  kbits_buf receives the kernel bits of the tile, kernel
-// q at bit q - (q0 & ~31); for 1x1 kernels the element bits are used as they are.
-// Global flag words are read first and only updated (atomicOr) when a bit is still missing: a
-// stale read costs a redundant atomic at worst, and flags saturate early in a sweep.
-// There is no barrier at the end: the caller alternates between two sets of bit buffers.
-__device__ __forceinline__ void tile_structures(const TensorDesc& d, uint32_t e0, uint32_t n_e, const uint32_t* ebits,
-                                                uint32_t* kbits_buf, uint32_t* nz_map, uint32_t* out_nz,
-                                                uint32_t* in_nz) {
-    const uint32_t KK = d.KK, I = d.I;
-    const uint32_t q0 = e0 / KK, q1 = (e0 + n_e - 1) / KK;
-    const uint32_t qa = q0 & ~31u;
-    const uint32_t n_words = ((q1 - qa) >> 5) + 1;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t* kbits = ebits;  // KK == 1: kernels are elements and the tile starts on a word
-    if (KK != 1) {
-        for (uint32_t w = warp; w < n_words; w += kTileThreads / 32) {
-            const uint32_t q = qa + 32 * w + lane;
-            bool bit = false;
-            if (q >= q0 && q <= q1) {
-                const uint32_t lo = max(q * KK, e0) - e0, hi = min((q + 1) * KK, e0 + n_e) - e0;
-                bit = any_bits(ebits, lo, hi);
-            }
-            const uint32_t word = __ballot_sync(kFull, bit);
-            if (lane == 0) kbits_buf[w] = word;
-        }
-        __syncthreads();
-        kbits = kbits_buf;
+// The kernel-map word of 32 consecutive 3x3 kernels from their 288 element bits (9 words): the
+// position of every 9-bit field is a compile-time constant, so a field costs a funnel shift, a
+// mask and a compare.
+__device__ __forceinline__ uint32_t kernel_word_3x3(const uint32_t* p) {
+    uint32_t w[10];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) w[i] = __ldg(p + i);
+    w[9] = 0;
+    uint32_t word = 0;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const int idx = (9 * j) >> 5, off = (9 * j) & 31;
+        const uint32_t field = __funnelshift_r(w[idx], w[idx + 1], off) & 0x1FFu;
+        word |= field ? (1u << j) : 0u;
     }
-    uint32_t* g_in = in_nz + d.off_innz;
-    uint32_t* g_out = out_nz + d.off_outnz;
-    uint32_t* g_map = nz_map ? nz_map + d.off_nzmap : nullptr;
-    const bool row_words = (I % 32 == 0);  // 32 consecutive kernels never cross a filter boundary
-    for (uint32_t w = threadIdx.x; w < n_words; w += kTileThreads) {
-        uint32_t bits = kbits[w];
-        if (!bits) continue;
-        const uint32_t qb = qa + 32 * w;
-        if (g_map) {
-            // only the first and last word can hold kernels shared with a neighbouring tile
-            if (KK == 1 || (w != 0 && w != n_words - 1)) g_map[qb >> 5] = bits;
-            else atomicOr(&g_map[qb >> 5], bits);
+    return word;
+}
+
+// OR `bits` into a global flag word unless they are already there.  The plain read may be stale,
+// which only costs a redundant atomic; flags saturate early, so almost every update ends at the read.
+__device__ __forceinline__ void or_if_missing(uint32_t* word, uint32_t bits) {
+    if ((__ldcg(word) & bits) != bits) atomicOr(word, bits);
+}
+
+// From the packed element bits to kernel map, filter flags and input-column flags.
+//
+// Tensors whose filters are a power-of-two number of kernel-map words (I = 32, 64, 128, ...) are cut
+// into units of kFlagRows filters x up to 32 map words per filter; one warp per unit.  In every
+// step the 32 lanes build 32 consecutive words of the unit (a copy of the element bits for 1x1
+// kernels, else one test per 2-D kernel) and store them plainly, as the unit owns them.  A lane
+// always meets the same input-column word, so the column OR stays in a register until the end of
+// the unit and costs one shuffle reduction and at most one atomic per word; filter flags cost at
+// most one atomic per step.  This keeps the number of atomics on the few flag words small even
+// though every unit of a tensor runs at the same time.
+// Other shapes take units of 32 kernels, one per lane, each kernel setting its own two flags.
+__global__ void __launch_bounds__(256) k_flags(Tables tb, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz) {
+    const int lane = threadIdx.x & 31;
+    const uint32_t n_warps = gridDim.x * (blockDim.x >> 5), warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const uint32_t per = (tb.n_flag_units + n_warps - 1) / n_warps;
+    const uint32_t lo = min(tb.n_flag_units, warp * per), hi = min(tb.n_flag_units, lo + per);
+    if (lo >= hi) return;
+    uint32_t t = 0, top = tb.n_tensors;  // tensor holding unit lo: last t with flag_prefix[t] <= lo
+    while (top - t > 1) {
+        const uint32_t mid = (t + top) >> 1;
+        if (tb.flag_prefix[mid] <= lo) t = mid;
+        else top = mid;
+    }
+    uint32_t unit = lo;
+    while (unit < hi) {
+        const uint32_t t_begin = tb.flag_prefix[t], t_end = tb.flag_prefix[t + 1];
+        if (unit >= t_end) {
+            ++t;
+            continue;
         }
-        if (row_words) {
-            const uint32_t o = qb / I, iw = (qb - o * I) >> 5, ob = 1u << (o & 31);
-            uint32_t* pi = &g_in[iw];
-            uint32_t* po = &g_out[o >> 5];
-            const uint32_t gi = __ldcg(pi), go = __ldcg(po);  // both reads in flight together
-            if ((gi & bits) != bits) atomicOr(pi, bits);
-            if (!(go & ob)) atomicOr(po, ob);
+        const TensorDesc& d = tb.tensors[t];
+        const uint32_t KK = d.KK, I = d.I, O = d.O, n_kernels = O * I;
+        const uint32_t* ebits = tb.ebits + d.off_mask;
+        uint32_t* g_in = in_nz + d.off_innz;
+        uint32_t* g_out = out_nz + d.off_outnz;
+        uint32_t* g_map = nz_map ? nz_map + d.off_nzmap : nullptr;
+        const uint32_t wpr = (I % 32 == 0 && ((I / 32) & (I / 32 - 1)) == 0) ? I / 32 : 0;  // map words per filter
+        const uint32_t run_end = min(hi, t_end);
+        if (wpr) {
+            const uint32_t n_chunks = (wpr + 31) / 32, cw = min(wpr, 32u);  // column chunks per filter block, words in each
+            const int cw_shift = __ffs(cw) - 1;
+            for (; unit < run_end; ++unit) {
+                const uint32_t local = unit - t_begin, rb = local / n_chunks, cc = local - rb * n_chunks;
+                const uint32_t row0 = rb * kFlagRows, iw = cc * 32 + (lane & (cw - 1));
+                uint32_t acc = 0, rows = 0;  // column OR of this lane's words; filters of the unit that hold something
+                // (the trip count is the same in every lane: the loop body holds a warp-wide vote)
+                constexpr int kMaxSteps = kFlagRows;  // cw <= 32 words per filter and chunk
+#pragma unroll
+                for (int step = 0; step < kMaxSteps; ++step) {
+                    const uint32_t base = step * 32;
+                    if (base >= kFlagRows * cw) break;
+                    const uint32_t k = base + lane;
+                    const uint32_t o = row0 + (k >> cw_shift);
+                    uint32_t word = 0;
+                    if (k < kFlagRows * cw && o < O) {
+                        const uint32_t gw = o * wpr + iw;  // this lane's word of the kernel map
+                        if (KK == 1) {
+                            word = __ldg(ebits + gw);
+                        } else if (KK == 9) {
+                            word = kernel_word_3x3(ebits + (size_t)gw * 9);
+                        } else {
+                            const uint32_t q0 = gw * 32;
+                            for (uint32_t j = 0; j < 32; ++j)
+                                word |= (uint32_t)any_bits(ebits, (q0 + j) * KK, (q0 + j + 1) * KK) << j;
+                        }
+                        if (g_map) g_map[gw] = word;
+                    }
+                    acc |= word;
+                    // one bit per group of cw lanes = per filter of this step
+                    const uint32_t nzl = __ballot_sync(kFull, word != 0);
+                    const uint32_t group_mask = cw == 32 ? 0xffffffffu : ((1u << cw) - 1u);
+                    for (uint32_t g = 0; g < min(32u >> cw_shift, kFlagRows); ++g)
+                        if ((nzl >> (g << cw_shift)) & group_mask) rows |= 1u << ((base >> cw_shift) + g);
+                }
+                // kFlagRows divides 32, so the filters of a unit share one flag word
+                if (lane == 0 && rows) or_if_missing(&g_out[row0 >> 5], rows << (row0 & 31));
+                for (uint32_t sft = cw; sft < 32; sft <<= 1) acc |= __shfl_xor_sync(kFull, acc, sft);
+                if ((uint32_t)lane < cw && acc) or_if_missing(&g_in[iw], acc);
+            }
         } else {
-            while (bits) {
-                const uint32_t q = qb + __ffs(bits) - 1;
-                bits &= bits - 1;
-                const uint32_t o = q / I, i = q - o * I;
-                uint32_t* pi = &g_in[i >> 5];
-                uint32_t* po = &g_out[o >> 5];
-                const uint32_t gi = __ldcg(pi), go = __ldcg(po);
-                if (!((gi >> (i & 31)) & 1u)) atomicOr(pi, 1u << (i & 31));
-                if (!((go >> (o & 31)) & 1u)) atomicOr(po, 1u << (o & 31));
+            // one kernel per lane, every kernel sets its own two flags
+            for (; unit < run_end; ++unit) {
+                const uint32_t q = (unit - t_begin) * 32 + lane;
+                const bool bit = q < n_kernels && any_bits(ebits, q * KK, (q + 1) * KK);
+                const uint32_t word = __ballot_sync(kFull, bit);
+                if (lane == 0 && g_map) g_map[unit - t_begin] = word;
+                if (bit) {
+                    const uint32_t o = q / I, i = q - o * I;
+                    or_if_missing(&g_in[i >> 5], 1u << (i & 31));
+                    or_if_missing(&g_out[o >> 5], 1u << (o & 31));
+                }
             }
         }
     }
@@ -111,24 +167,26 @@ __device__ __forceinline__ void tile_structures(const TensorDesc& d, uint32_t e0
 
 // Each block owns a contiguous range of tiles.  Inside a tensor the loop is software-pipelined:
 // the 16-byte loads of the next tile (and its two tie-table words) are issued before the current
-// tile is processed, so a block always has a tile in flight while it masks, stores and updates
-// the flags of the previous one.  Whole tiles whose ties do not split take a lean path; the last
+// tile is processed, so a block always has a tile in flight while it masks and stores the
+// previous one.  Whole tiles whose ties do not split take a lean path; the last
 // (ragged) tile of a tensor and the one tile per segment that ranks its ties take the general one.
 template <int DT, bool DO_MASK, bool DO_STRUCT>
 __global__ void __launch_bounds__(kTileThreads, 4) k_sweep(Tables tb, ThresholdWs ws, const dnns_threshold* __restrict__ thr,
                                                            int variant, const char* src_arena, char* dst_arena,
-                                                           uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz,
-                                                           uint32_t* in_nz) {
+                                                           uint32_t* mask_bits, uint32_t* clear_a, uint32_t n_clear_a,
+                                                           uint32_t* clear_b, uint32_t n_clear_b) {
     constexpr int P = Elem<DT>::kPerVec;
+    if (DO_STRUCT) {
+        // the flag words that k_flags (the next kernel in the stream) ORs into start at zero
+        for (uint32_t i = blockIdx.x * kTileThreads + threadIdx.x; i < n_clear_a; i += gridDim.x * kTileThreads) clear_a[i] = 0;
+        for (uint32_t i = blockIdx.x * kTileThreads + threadIdx.x; i < n_clear_b; i += gridDim.x * kTileThreads) clear_b[i] = 0;
+    }
     constexpr int G = 32 / P;  // lanes per bit word
     constexpr uint32_t kTileElems = kTileBytes / Elem<DT>::kBytes;
     constexpr uint32_t kKeyMask = DT == DNNS_F32 ? 0x7FFFFFFFu : 0x7FFF7FFFu;
-    __shared__ uint32_t s_ebits[2][kTileElems / 32];
-    __shared__ uint32_t s_kbits[2][DO_STRUCT ? kTileElems / 32 + 1 : 1];
     __shared__ uint32_t scratch[33];
     const int lane = threadIdx.x & 31;
     const bool word_lane = (lane & (G - 1)) == 0;
-    int buf = 0;
 
     const uint32_t per = (tb.n_tiles + gridDim.x - 1) / gridDim.x;
     const uint32_t lo = min(tb.n_tiles, blockIdx.x * per), hi = min(tb.n_tiles, lo + per);
@@ -161,6 +219,7 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_sweep(Tables tb, ThresholdW
         const uint32_t* tie_before = ws.tie_prefix + (size_t)variant * tb.n_tiles;
         const uint32_t* tie_here = ws.tile_ties + (size_t)variant * tb.n_tiles;
         uint32_t* mask_words = mask_bits ? mask_bits + d.off_mask : nullptr;
+        uint32_t* nz_words = DO_STRUCT ? tb.ebits + d.off_mask : nullptr;  // same packing as the mask bits
 
         uint4 nxt[kVecPerThread];
         uint32_t nxt_before = 0, nxt_here = 0;
@@ -202,7 +261,6 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_sweep(Tables tb, ThresholdW
                     quota = (uint32_t)(n_tie - before);
                 }
             }
-            uint32_t* ebits = s_ebits[buf];
 
             if (n_e == kTileElems && !split) {
                 // ---- lean path: a whole tile, one threshold for all its keys
@@ -243,7 +301,7 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_sweep(Tables tb, ThresholdW
                     if (DO_MASK && mask_words && word_lane) mask_words[e0 / 32 + vi / G] = keep_word;
                     if (DO_STRUCT) {
                         const uint32_t nz_word = zeros_survive ? gather_word<P>(nz, lane) : keep_word;
-                        if (word_lane) ebits[vi / G] = nz_word;
+                        if (word_lane) nz_words[e0 / 32 + vi / G] = nz_word;
                     }
                 }
             } else {
@@ -298,14 +356,9 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_sweep(Tables tb, ThresholdW
                     }
                     if (DO_STRUCT) {
                         const uint32_t word = gather_word<P>(nz, lane);
-                        if (word_lane) ebits[vi / G] = word;
+                        if (word_lane && (vi / G) * 32 < n_e) nz_words[e0 / 32 + vi / G] = word;
                     }
                 }
-            }
-            if (DO_STRUCT) {
-                __syncthreads();
-                tile_structures(d, e0, n_e, ebits, s_kbits[buf], nz_map, out_nz, in_nz);
-                buf ^= 1;
             }
         }
     }
@@ -314,32 +367,36 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_sweep(Tables tb, ThresholdW
 template <int DT>
 void launch_dt(bool do_mask, bool do_struct, dim3 grid, cudaStream_t st, const Tables& tb, const ThresholdWs& ws,
                const dnns_threshold* thr, int variant, const char* src_arena, char* dst_arena, uint32_t* mask_bits,
-               uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz) {
+               uint32_t* out_nz, uint32_t n_out, uint32_t* in_nz, uint32_t n_in) {
     if (do_mask && do_struct)
         k_sweep<DT, true, true><<<grid, kTileThreads, 0, st>>>(tb, ws, thr, variant, src_arena, dst_arena, mask_bits,
-                                                               nz_map, out_nz, in_nz);
+                                                               out_nz, n_out, in_nz, n_in);
     else if (do_mask)
         k_sweep<DT, true, false><<<grid, kTileThreads, 0, st>>>(tb, ws, thr, variant, src_arena, dst_arena, mask_bits,
-                                                                nz_map, out_nz, in_nz);
+                                                                nullptr, 0, nullptr, 0);
     else
         k_sweep<DT, false, true><<<grid, kTileThreads, 0, st>>>(tb, ws, thr, variant, src_arena, dst_arena, mask_bits,
-                                                                nz_map, out_nz, in_nz);
+                                                                out_nz, n_out, in_nz, n_in);
 }
 
 }  // namespace
 
 int launch_tile_sweep(const Tables& tb, const ThresholdWs& ws, bool do_mask, bool do_struct,
                       const dnns_threshold* thr_dev, int variant, const void* src_arena, void* dst_arena,
-                      uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz, int n_sm,
-                      cudaStream_t st) {
+                      uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz, uint32_t n_out_words,
+                      uint32_t n_in_words, int n_sm, cudaStream_t st) {
     const dim3 grid(min((uint32_t)n_sm * 4u, tb.n_tiles));
     if (tb.dtype == DNNS_F32)
         launch_dt<DNNS_F32>(do_mask, do_struct, grid, st, tb, ws, thr_dev, variant, (const char*)src_arena,
-                            (char*)dst_arena, mask_bits, nz_map, out_nz, in_nz);
+                            (char*)dst_arena, mask_bits, out_nz, n_out_words, in_nz, n_in_words);
     else
         launch_dt<DNNS_BF16>(do_mask, do_struct, grid, st, tb, ws, thr_dev, variant, (const char*)src_arena,
-                             (char*)dst_arena, mask_bits, nz_map, out_nz, in_nz);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+                             (char*)dst_arena, mask_bits, out_nz, n_out_words, in_nz, n_in_words);
+    if (do_struct) {
+        const uint32_t blocks = min((uint32_t)n_sm * 64u, (tb.n_flag_units + 7) / 8);  // one unit per warp if possible
+        k_flags<<<max(blocks, 1u), 256, 0, st>>>(tb, nz_map, out_nz, in_nz);
+    }
+    return cudaGetLastError() == cudaSuccess ? (do_struct ? 2 : 1) : -1;
 }
 
 }  // namespace dnns

@@ -216,7 +216,9 @@ template <int DT>
 __global__ void __launch_bounds__(1024) k_select1(Tables tb, ThresholdWs ws, int n_k, dnns_threshold* __restrict__ thr) {
     __shared__ uint64_t scratch[33];
     __shared__ uint32_t s_digit[kMaxVariants];
+    __shared__ uint64_t s_k[kMaxVariants];
     const uint32_t seg = blockIdx.x, S = tb.n_segs;
+    if ((int)threadIdx.x < n_k) s_k[threadIdx.x] = ws.k_dev[(size_t)threadIdx.x * S + seg];  // one round trip for all k
     const uint32_t* h = ws.hist1 + (size_t)seg * kHistBins;
     uint32_t c[32];
     uint64_t sum = 0;
@@ -231,7 +233,7 @@ __global__ void __launch_bounds__(1024) k_select1(Tables tb, ThresholdWs ws, int
     uint32_t* bm = ws.bitmap + (size_t)seg * kBitmapWords;
     bm[threadIdx.x] = 0;  // 1024 words
     for (int v = 0; v < n_k; ++v) {
-        const uint64_t k = ws.k_dev[(size_t)v * S + seg];
+        const uint64_t k = s_k[v];  // published by the barriers of the scan above
         SelectState* st = &ws.sel[(size_t)v * S + seg];
         if (k == 0) {
             if (threadIdx.x == 0) {
@@ -390,16 +392,28 @@ __global__ void __launch_bounds__(1024) k_select2(Tables tb, ThresholdWs ws, int
     uint64_t total;
     const uint64_t excl = st.below + block_exclusive_scan<uint64_t>(sum, scratch, &total);
     if (excl < st.k && st.k <= excl + sum) {
+        // this thread's 64 bins again, as independent vector loads, then a search in registers
+        uint4 q[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) q[j] = reinterpret_cast<const uint4*>(h)[threadIdx.x * 16 + j];
         uint64_t cum = excl;
         uint32_t b = 0, cnt = 0;
-        for (int j = 0; j < 64; ++j) {
-            const uint32_t cj = h[threadIdx.x * 64 + j];
-            if (cum + cj >= st.k) {
-                b = j;
-                cnt = cj;
-                break;
+        bool found = false;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const uint32_t c4[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                if (!found) {
+                    if (cum + c4[t] >= st.k) {
+                        b = 4 * j + t;
+                        cnt = c4[t];
+                        found = true;
+                    } else {
+                        cum += c4[t];
+                    }
+                }
             }
-            cum += cj;
         }
         dnns_threshold r;
         r.tau_bits = (st.digit << 16) | (threadIdx.x * 64 + b);
@@ -474,6 +488,7 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_ties(Tables tb, ThresholdWs
 }
 
 // Exclusive scan of the tile counts over the tiles of a segment, one block per (variant, segment).
+// Every thread owns a contiguous run of tiles: one pass of independent loads, one block scan.
 __global__ void __launch_bounds__(1024) k_tie_scan(Tables tb, ThresholdWs ws) {
     if (*ws.any_need == 0) return;
     __shared__ uint32_t scratch[33];
@@ -483,14 +498,16 @@ __global__ void __launch_bounds__(1024) k_tie_scan(Tables tb, ThresholdWs ws) {
     const SegDesc sd = tb.segs[seg];
     const uint32_t* cnt = ws.tile_ties + (size_t)v * tb.n_tiles;
     uint32_t* pre = ws.tie_prefix + (size_t)v * tb.n_tiles;
-    uint32_t carry = 0;
-    for (uint32_t base = sd.tile_begin; base < sd.tile_end; base += 1024) {
-        const uint32_t t = base + threadIdx.x;
-        const uint32_t x = t < sd.tile_end ? cnt[t] : 0;
-        uint32_t total;
-        const uint32_t ex = block_exclusive_scan<uint32_t>(x, scratch, &total);
-        if (t < sd.tile_end) pre[t] = carry + ex;
-        carry += total;
+    const uint32_t n = sd.tile_end - sd.tile_begin;
+    const uint32_t run = (n + 1023) / 1024;
+    const uint32_t t0 = min(sd.tile_end, sd.tile_begin + threadIdx.x * run), t1 = min(sd.tile_end, t0 + run);
+    uint32_t sum = 0;
+    for (uint32_t t = t0; t < t1; ++t) sum += cnt[t];
+    uint32_t total;
+    uint32_t ex = block_exclusive_scan<uint32_t>(sum, scratch, &total);
+    for (uint32_t t = t0; t < t1; ++t) {
+        pre[t] = ex;
+        ex += cnt[t];
     }
 }
 
