@@ -145,6 +145,7 @@ def main():
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--stepwise", action="store_true", help="mask and zero-structure detection as two sweeps")
+    ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph replay")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -225,43 +226,71 @@ def main():
         R.append(sum(int(sh[i, 0]) * t.I * t.KH * t.KW for i, t in enumerate(wl.tensors)))
         Nn.append(sum(int(sh[i, 0]) * int(sh[i, 1]) * t.KH * t.KW for i, t in enumerate(wl.tensors)))
 
-    launches0 = ses.launch_count()
+    # One portfolio captured once as a CUDA graph (the calls are plain stream work: no allocation, no
+    # synchronisation), replayed for the timed steps.  A second, plain pass with an event pair around
+    # every call gives the per-call durations; its total is reported as ms_per_step_plain.
+    graph = None
+    launches_per_step = None
+    if not args.no_graph:
+        try:
+            l0 = ses.launch_count()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step(False)
+            launches_per_step = ses.launch_count() - l0
+            graph.replay()
+            torch.cuda.synchronize()
+        except Exception as e:  # capture refused: fall back to plain launches and say so
+            print(f"bench: CUDA graph capture failed ({e}); timing plain launches", file=sys.stderr)
+            graph = None
+
+    def timed_steps(run_step):
+        """K steps; returns total ms.  Models that fit in L2 get a flush before every step."""
+        if need_flush:
+            pairs = []
+            for _ in range(args.steps):
+                flush_buf.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                run_step()
+                b.record()
+                pairs.append((a, b))
+            torch.cuda.synchronize()
+            return sum(a.elapsed_time(b) for a, b in pairs)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.steps):
+            run_step()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
+
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
-    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    step_ms = []
-    if need_flush:
-        # inputs fit in L2: flush between steps and time every step on its own
-        for _ in range(args.steps):
-            flush_buf.fill_(1)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            step(True)
-            b.record()
-            step_ms.append((a, b))
-        torch.cuda.synchronize()
-        total_ms = sum(a.elapsed_time(b) for a, b in step_ms)
+    launches0 = ses.launch_count()
+    plain_ms = timed_steps(lambda: step(True))
+    launches_plain = ses.launch_count() - launches0
+    if graph is not None:
+        barrier()
+        total_ms = timed_steps(graph.replay)
+        launches = launches_per_step * args.steps
     else:
-        t_start.record()
-        for _ in range(args.steps):
-            step(True)
-        t_end.record()
-        torch.cuda.synchronize()
-        total_ms = t_start.elapsed_time(t_end)
+        total_ms = plain_ms
+        launches = launches_plain
     clocks = sampler.stop()
     barrier()
-    launches = ses.launch_count() - launches0
     if world > 1:
-        t = torch.tensor([total_ms], device=dm.device)
+        t = torch.tensor([total_ms, plain_ms], device=dm.device)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+        total_ms, plain_ms = float(t[0].item()), float(t[1].item())
     assert ses.device_status() == B.DNNS_OK
 
     ms_per_step = total_ms / args.steps
     ms_per_variant = ms_per_step / V / world if world > 1 else ms_per_step / V
     per_call = {n: statistics.mean(a.elapsed_time(b) for a, b in spans[n]) for n in names}
-    share = {n: per_call[n] * (1 if n == "threshold" else V) / ms_per_step for n in names}
+    plain_per_step = plain_ms / args.steps
+    share = {n: per_call[n] * (1 if n == "threshold" else V) / plain_per_step for n in names}
 
     # algorithmic bytes: one read of every input a step consumes, one write of every output
     # (the fused sweep moves 2*N*b + N/8 per launch; the stepwise accounting B_v charges the path 3*N*b + N/8)
@@ -322,6 +351,7 @@ def main():
         "effective_frac_of_peak": portfolio_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
         "algorithmic_bytes_per_variant": portfolio_bytes / V,
         "moved_gbs": moved_bytes / (ms_per_step * 1e-3) / 1e9, "sweeps": "stepwise" if args.stepwise else "fused mask+structures",
+        "launch": "cuda graph replay" if graph is not None else "plain stream launches", "ms_per_step_plain": plain_per_step,
         "per_call_ms": per_call, "share": share,
         "per_call_gbs": {n: (alg[n] / (per_call[n] * 1e-3) / 1e9 if alg[n] else None) for n in names},
         "roofline": {"bound": "hbm", "kernel": kernel_of[dominant], "achieved": achieved, "peak": peak,

@@ -109,7 +109,7 @@ struct CompactWs {
 };
 
 // ---- launch wrappers (each returns the number of kernels it launched, or -1 on a CUDA error) ----
-int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, int n_k_stride, dnns_threshold* thr_dev,
+int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, const uint64_t* k_host, dnns_threshold* thr_dev,
                      int n_sm, cudaStream_t st);
 int launch_tile_sweep(const Tables& tb, const ThresholdWs& ws, bool do_mask, bool do_struct,
                       const dnns_threshold* thr_dev, int variant, const void* src_arena, void* dst_arena,

@@ -386,8 +386,7 @@ dnns_status dnns_magnitude_threshold(dnns_plan* p, const uint64_t* k, int32_t n_
     const uint64_t clear_end = p->map.hist2 + (p->c.dtype == DNNS_F32 ? 4ull * kLowBins * S * n_k : 0);
     if (cudaMemsetAsync(p->ws + p->map.clear_begin, 0, clear_end - p->map.clear_begin, st) != cudaSuccess)
         return DNNS_ERR_CUDA;
-    if (cudaMemcpyAsync(p->tws.k_dev, k, 8ull * n_k * S, cudaMemcpyHostToDevice, st) != cudaSuccess) return DNNS_ERR_CUDA;
-    const int n = launch_threshold(p->tb, p->tws, n_k, n_k, thr_dev, p->n_sm, st);
+    const int n = launch_threshold(p->tb, p->tws, n_k, k, thr_dev, p->n_sm, st);
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
     p->last_n_k = n_k;

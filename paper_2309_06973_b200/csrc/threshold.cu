@@ -212,13 +212,23 @@ __global__ void __launch_bounds__(kHistThreads, 1) k_hist1(Tables tb, uint32_t* 
 
 // ---------------------------------------------------------------- select 1
 // One block per segment.  Thread t owns bins [32t, 32t+32).
+// Prune counts handed over as a kernel argument (no copy to stage, nothing to capture but the launch).
+constexpr int kInlineCounts = 64;
+struct InlineCounts {
+    uint64_t k[kInlineCounts];
+};
+
 template <int DT>
-__global__ void __launch_bounds__(1024) k_select1(Tables tb, ThresholdWs ws, int n_k, dnns_threshold* __restrict__ thr) {
+__global__ void __launch_bounds__(1024) k_select1(Tables tb, ThresholdWs ws, int n_k, dnns_threshold* __restrict__ thr,
+                                                  InlineCounts counts, bool counts_inline) {
     __shared__ uint64_t scratch[33];
     __shared__ uint32_t s_digit[kMaxVariants];
     __shared__ uint64_t s_k[kMaxVariants];
     const uint32_t seg = blockIdx.x, S = tb.n_segs;
-    if ((int)threadIdx.x < n_k) s_k[threadIdx.x] = ws.k_dev[(size_t)threadIdx.x * S + seg];  // one round trip for all k
+    if ((int)threadIdx.x < n_k) {
+        const size_t idx = (size_t)threadIdx.x * S + seg;
+        s_k[threadIdx.x] = counts_inline ? counts.k[idx] : ws.k_dev[idx];  // one round trip for all k
+    }
     const uint32_t* h = ws.hist1 + (size_t)seg * kHistBins;
     uint32_t c[32];
     uint64_t sum = 0;
@@ -520,22 +530,30 @@ cudaError_t init_kernel_attributes() {
     return cudaFuncSetAttribute(k_hist1<DNNS_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kHistBins * 4));
 }
 
-int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, int /*n_k_stride*/, dnns_threshold* thr_dev,
+int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, const uint64_t* k_host, dnns_threshold* thr_dev,
                      int n_sm, cudaStream_t st) {
     const uint32_t S = tb.n_segs;
+    // few counts travel as a kernel argument, many through the workspace
+    InlineCounts counts{};
+    const bool counts_inline = (size_t)n_k * S <= kInlineCounts;
+    if (counts_inline) {
+        for (size_t i = 0; i < (size_t)n_k * S; ++i) counts.k[i] = k_host[i];
+    } else if (cudaMemcpyAsync(ws.k_dev, k_host, 8ull * n_k * S, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        return -1;
+    }
     const int hist_grid = (int)min((uint32_t)n_sm, tb.n_tiles);
     const int sweep_grid = (int)min((uint32_t)n_sm * 4u, tb.n_tiles);
     int launches = 0;
     if (tb.dtype == DNNS_F32) {
         k_hist1<DNNS_F32><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws.hist1);
-        k_select1<DNNS_F32><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev);
+        k_select1<DNNS_F32><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline);
         k_hist2<<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k);
         k_select2<<<S * n_k, 1024, 0, st>>>(tb, ws, n_k, thr_dev);
         k_ties<DNNS_F32><<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k, thr_dev);
         launches = 5;
     } else {
         k_hist1<DNNS_BF16><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws.hist1);
-        k_select1<DNNS_BF16><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev);
+        k_select1<DNNS_BF16><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline);
         k_ties<DNNS_BF16><<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k, thr_dev);
         launches = 3;
     }

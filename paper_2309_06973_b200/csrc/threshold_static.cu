@@ -97,8 +97,7 @@ extern "C" dnns_status dnns_magnitude_threshold_static(const void* weights_dev, 
     // what must start at zero: histograms, tie tables and flags of the previous call
     if (cudaMemsetAsync(base + kOffClear, 0, kScratchBytes - kOffClear, st) != cudaSuccess ||
         cudaMemcpyAsync(base + kOffTensor, &td, sizeof(td), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(base + kOffSeg, &sd, sizeof(sd), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(base + kOffK, &k, sizeof(k), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        cudaMemcpyAsync(base + kOffSeg, &sd, sizeof(sd), cudaMemcpyHostToDevice, st) != cudaSuccess)
         return DNNS_ERR_CUDA;
 
     Tables tb{};
@@ -119,5 +118,5 @@ extern "C" dnns_status dnns_magnitude_threshold_static(const void* weights_dev, 
     ws.any_need = reinterpret_cast<uint32_t*>(base + kOffAnyNeed);
     ws.tile_ties = reinterpret_cast<uint32_t*>(base + kOffTileTies);
     ws.tie_prefix = reinterpret_cast<uint32_t*>(base + kOffTiePrefix);
-    return launch_threshold(tb, ws, 1, 1, thr_dev, g_n_sm[dev], st) < 0 ? DNNS_ERR_CUDA : DNNS_OK;
+    return launch_threshold(tb, ws, 1, &k, thr_dev, g_n_sm[dev], st) < 0 ? DNNS_ERR_CUDA : DNNS_OK;
 }
