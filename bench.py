@@ -36,6 +36,15 @@ def load_peaks():
     return 6650.0, "fallback"
 
 
+def measured_traffic(workload: str, dtype: str, kernel: str):
+    """DRAM bytes per launch of `kernel` from the committed ncu summary, or None when there is none."""
+    try:
+        table = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic.json")))
+        return table[f"{workload}_{dtype}"][kernel]
+    except Exception:
+        return None
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -355,7 +364,9 @@ def main():
         "per_call_ms": per_call, "share": share,
         "per_call_gbs": {n: (alg[n] / (per_call[n] * 1e-3) / 1e9 if alg[n] else None) for n in names},
         "roofline": {"bound": "hbm", "kernel": kernel_of[dominant], "achieved": achieved, "peak": peak,
-                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": None},
+                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                     "algorithmic_bytes": alg[dominant],
+                     "traffic": measured_traffic(args.workload, args.dtype, kernel_of[dominant])},
         "e2e": {"value": e2e_per_variant, "unit": "ms", "h2d_bytes_per_step": h2d // args.steps,
                 "d2h_bytes_per_step": d2h // args.steps},
         "gpu_launches": launches,
