@@ -187,10 +187,70 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
 
 // Every block takes a contiguous range of gather units and walks the items that own them, so the
 // item's context (source, destination, keep lists, new extents) is fetched once per run.
-template <int WBYTES>  // element width of the weight tensors; BatchNorm vectors and biases are always 4 bytes
+//
+// INLINE_LAYOUT (models of up to kInlineItems items): every block derives the destination layout
+// itself, in shared memory, from the keep counts - a few hundred items, one scan - instead of waiting
+// for a separate one-block kernel; block 0 also writes the offsets and shapes the caller asked for.
+constexpr uint32_t kInlineItems = 1024;
+
+template <int WBYTES, bool INLINE_LAYOUT>  // WBYTES: element width of the weight tensors (BatchNorm, bias: 4 bytes)
 __global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, CompactWs ws, const char* src_arena,
-                                                                const int32_t* __restrict__ keep_idx, char* dst_arena) {
-    const uint32_t total_units = ws.unit_prefix[tb.n_items];
+                                                                const int32_t* __restrict__ keep_idx, char* dst_arena,
+                                                                const int32_t* __restrict__ keep_count, uint64_t dst_bytes,
+                                                                uint64_t* dst_offsets, int32_t* dst_shapes) {
+    __shared__ uint32_t s_unit_prefix[INLINE_LAYOUT ? kInlineItems + 1 : 1];
+    __shared__ uint64_t s_item_off[INLINE_LAYOUT ? kInlineItems : 1];
+    __shared__ int32_t s_item_dims[INLINE_LAYOUT ? 2 * kInlineItems : 1];
+    __shared__ uint64_t scratch[33];
+    if (INLINE_LAYOUT) {
+        constexpr uint32_t kPer = kInlineItems / kThreads;  // consecutive items per thread
+        uint64_t bytes[kPer], units[kPer], sum_b = 0, sum_u = 0;
+#pragma unroll
+        for (uint32_t k = 0; k < kPer; ++k) {
+            const uint32_t i = threadIdx.x * kPer + k;
+            bytes[k] = units[k] = 0;
+            if (i < tb.n_items) {
+                const ItemDesc& it = tb.items[i];
+                const int64_t On = keep_count[it.out_group];
+                const int64_t Cn = it.in_group >= 0 ? keep_count[it.in_group] : it.Cin;
+                const uint64_t raw = (uint64_t)(On * Cn * it.blk) * it.elem_bytes;
+                bytes[k] = (raw + 255) & ~(uint64_t)255;
+                units[k] = (raw + kUnitBytes - 1) / kUnitBytes;
+                s_item_dims[2 * i] = (int32_t)On;
+                s_item_dims[2 * i + 1] = (int32_t)Cn;
+                if (blockIdx.x == 0 && it.tensor >= 0) {
+                    dst_shapes[2 * it.tensor] = (int32_t)On;
+                    dst_shapes[2 * it.tensor + 1] = (int32_t)(Cn * tb.tensors[it.tensor].S);
+                }
+            }
+            sum_b += bytes[k];
+            sum_u += units[k];
+        }
+        uint64_t tot_b, tot_u;
+        uint64_t ex_b = block_exclusive_scan<uint64_t>(sum_b, scratch, &tot_b);
+        uint64_t ex_u = block_exclusive_scan<uint64_t>(sum_u, scratch, &tot_u);
+        const bool fits = tot_b <= dst_bytes;
+#pragma unroll
+        for (uint32_t k = 0; k < kPer; ++k) {
+            const uint32_t i = threadIdx.x * kPer + k;
+            if (i < tb.n_items) {
+                s_item_off[i] = ex_b;
+                s_unit_prefix[i] = (uint32_t)ex_u;
+                if (blockIdx.x == 0) dst_offsets[i] = ex_b;
+            }
+            ex_b += bytes[k];
+            ex_u += units[k];
+        }
+        if (threadIdx.x == 0) {
+            s_unit_prefix[tb.n_items] = fits ? (uint32_t)tot_u : 0u;  // too small an arena: nothing is copied
+            if (!fits && blockIdx.x == 0) atomicCAS(tb.status, 0u, (uint32_t)DNNS_ERR_WORKSPACE);
+        }
+        __syncthreads();
+    }
+    const uint32_t* unit_prefix = INLINE_LAYOUT ? s_unit_prefix : ws.unit_prefix;
+    const uint64_t* item_off = INLINE_LAYOUT ? s_item_off : ws.item_off;
+    const int32_t* item_dims = INLINE_LAYOUT ? s_item_dims : ws.item_dims;
+    const uint32_t total_units = unit_prefix[tb.n_items];
     const uint32_t per = (total_units + gridDim.x - 1) / gridDim.x;
     const uint32_t u_lo = min(total_units, blockIdx.x * per), u_hi = min(total_units, u_lo + per);
     if (u_lo >= u_hi) return;
@@ -198,18 +258,18 @@ __global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, Compa
     uint32_t item = 0, hi = tb.n_items;
     while (hi - item > 1) {
         const uint32_t mid = (item + hi) >> 1;
-        if (ws.unit_prefix[mid] <= u_lo) item = mid;
+        if (unit_prefix[mid] <= u_lo) item = mid;
         else hi = mid;
     }
     uint32_t unit = u_lo;
     while (unit < u_hi) {
-        const uint32_t item_begin = ws.unit_prefix[item], item_end = ws.unit_prefix[item + 1];
+        const uint32_t item_begin = unit_prefix[item], item_end = unit_prefix[item + 1];
         if (unit >= item_end) {  // items that shrank to nothing own no units
             ++item;
             continue;
         }
         const ItemDesc& it = tb.items[item];
-        const uint32_t On = ws.item_dims[2 * item], Cn = ws.item_dims[2 * item + 1];
+        const uint32_t On = item_dims[2 * item], Cn = item_dims[2 * item + 1];
         const char* src;
         if (it.tensor >= 0) {
             const TensorDesc& d = tb.tensors[it.tensor];
@@ -217,7 +277,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, Compa
         } else {
             src = static_cast<const char*>(it.src);
         }
-        char* dst = dst_arena + ws.item_off[item];
+        char* dst = dst_arena + item_off[item];
         const int32_t* ko = keep_idx + tb.groups[it.out_group].off_idx;
         const int32_t* ki = it.in_group >= 0 ? keep_idx + tb.groups[it.in_group].off_idx : nullptr;
         const uint32_t run_end = min(u_hi, item_end);
@@ -233,12 +293,24 @@ __global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, Compa
 int launch_compact(const Tables& tb, const CompactWs& ws, const void* src_arena, const int32_t* keep_idx,
                    const int32_t* keep_count, void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets,
                    int32_t* dst_shapes, int n_sm, cudaStream_t st) {
-    k_compact_layout<<<1, 1024, 0, st>>>(tb, ws, keep_count, dst_bytes, dst_offsets, dst_shapes);
-    if (tb.dtype == DNNS_F32)
-        k_compact_gather<4><<<n_sm * 4, kThreads, 0, st>>>(tb, ws, (const char*)src_arena, keep_idx, (char*)dst_arena);
-    else
-        k_compact_gather<2><<<n_sm * 4, kThreads, 0, st>>>(tb, ws, (const char*)src_arena, keep_idx, (char*)dst_arena);
-    return cudaGetLastError() == cudaSuccess ? 2 : -1;
+    const char* src = (const char*)src_arena;
+    char* dst = (char*)dst_arena;
+    const int grid = n_sm * 4;
+    int launches = 1;
+    if (tb.n_items <= kInlineItems) {
+        if (tb.dtype == DNNS_F32)
+            k_compact_gather<4, true><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, dst_shapes);
+        else
+            k_compact_gather<2, true><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, dst_shapes);
+    } else {
+        k_compact_layout<<<1, 1024, 0, st>>>(tb, ws, keep_count, dst_bytes, dst_offsets, dst_shapes);
+        if (tb.dtype == DNNS_F32)
+            k_compact_gather<4, false><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, dst_shapes);
+        else
+            k_compact_gather<2, false><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, dst_shapes);
+        launches = 2;
+    }
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
 }  // namespace dnns

@@ -48,6 +48,18 @@ struct BnDesc {
     int32_t C, tensor;
 };
 
+// What the keep propagation needs of one producer / consumer of a group, next to the lists of
+// tensor ids, so that a flag word is two dependent loads away instead of four.
+struct ProducerDesc {
+    const float *beta, *gamma, *mean, *bias;  // BatchNorm after the producer (beta null: none) and its bias (nullable)
+    uint32_t off_outnz;
+    uint32_t pad;
+};
+struct ConsumerDesc {
+    uint32_t off_innz;
+    int32_t S;
+};
+
 struct SegDesc {
     uint32_t tile_begin, tile_end;  // tiles [begin, end) cover the segment (tiles of other tensors in between count 0)
     uint64_t size;
@@ -81,6 +93,8 @@ struct Tables {
     const uint32_t* tile_tensor;
     const int32_t* prod_list;
     const int32_t* cons_list;
+    const ProducerDesc* producers;  // parallel to prod_list
+    const ConsumerDesc* consumers;  // parallel to cons_list
     const uint32_t* flag_prefix;  // [n_tensors + 1] units of the flag kernel before each tensor
     uint32_t* ebits;        // packed "element is non-zero" bits of the latest sweep (same packing as the mask bits)
     uint32_t* status;       // device status word (a dnns_status, 0 = ok)

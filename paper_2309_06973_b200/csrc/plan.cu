@@ -16,7 +16,7 @@ inline uint64_t align_up(uint64_t x, uint64_t a = kAlign) { return (x + a - 1) /
 
 // Byte offsets of every section of the workspace.
 struct WsMap {
-    uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, flag_prefix, status;
+    uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, producers, consumers, flag_prefix, status;
     uint64_t tables_end;  // everything before this is uploaded once at plan creation
     uint64_t k_dev, bitmap, sel, tie_prefix, unit_prefix, item_off, item_dims, ebits;
     uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
@@ -103,6 +103,8 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.tile_tensor = take(4ull * c.tiles);
     w.prod_list = take(4ull * c.T);
     w.cons_list = take(4ull * c.T);
+    w.producers = take(sizeof(ProducerDesc) * c.T);
+    w.consumers = take(sizeof(ConsumerDesc) * c.T);
     w.flag_prefix = take(4ull * (c.T + 1));
     w.status = take(4);
     w.tables_end = o;
@@ -202,6 +204,8 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     auto* prod_list = reinterpret_cast<int32_t*>(host.data() + map.prod_list);
     auto* cons_list = reinterpret_cast<int32_t*>(host.data() + map.cons_list);
     auto* flag_prefix = reinterpret_cast<uint32_t*>(host.data() + map.flag_prefix);
+    auto* producers = reinterpret_cast<ProducerDesc*>(host.data() + map.producers);
+    auto* consumers = reinterpret_cast<ConsumerDesc*>(host.data() + map.consumers);
 
     p->arena_off.resize(c.T), p->mask_off.resize(c.T), p->nzmap_off.resize(c.T), p->outnz_off.resize(c.T);
     p->innz_off.resize(c.T), p->seg_of_tensor.assign(c.T, -1), p->keep_off.resize(c.G), p->keepidx_off.resize(c.G);
@@ -282,6 +286,13 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
         bd[b] = BnDesc{bn.gamma, bn.beta, bn.mean, bn.var, bn.C, bn.tensor};
         td[bn.tensor].bn = (int32_t)b;
     }
+    for (int i = 0; i < np; ++i) {
+        const TensorDesc& d = td[prod_list[i]];
+        ProducerDesc pd{nullptr, nullptr, nullptr, d.bias, d.off_outnz, 0};
+        if (d.bn >= 0) pd.beta = bd[d.bn].beta, pd.gamma = bd[d.bn].gamma, pd.mean = bd[d.bn].mean;
+        producers[i] = pd;
+    }
+    for (int i = 0; i < nc; ++i) consumers[i] = ConsumerDesc{td[cons_list[i]].off_innz, td[cons_list[i]].S};
     // gather items: weights, then BN vectors, then biases
     uint32_t n_it = 0;
     for (uint32_t i = 0; i < c.T; ++i) {
@@ -321,6 +332,8 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     tb.tile_tensor = reinterpret_cast<uint32_t*>(w + map.tile_tensor);
     tb.prod_list = reinterpret_cast<int32_t*>(w + map.prod_list);
     tb.cons_list = reinterpret_cast<int32_t*>(w + map.cons_list);
+    tb.producers = reinterpret_cast<ProducerDesc*>(w + map.producers);
+    tb.consumers = reinterpret_cast<ConsumerDesc*>(w + map.consumers);
     tb.status = reinterpret_cast<uint32_t*>(w + map.status);
     tb.flag_prefix = reinterpret_cast<uint32_t*>(w + map.flag_prefix);
     tb.ebits = reinterpret_cast<uint32_t*>(w + map.ebits);

@@ -16,14 +16,12 @@ constexpr int kMaxGroupWords = 65536 / 32;
 
 __device__ __forceinline__ bool get_bit(const uint32_t* w, uint32_t b) { return (w[b >> 5] >> (b & 31)) & 1u; }
 
-// The constant a zero filter of producer `t` still emits on channel j is structurally zero.
-__device__ __forceinline__ bool shift_zero(const Tables& tb, int t, int j) {
-    const TensorDesc& d = tb.tensors[t];
+// The constant a zero filter of producer p (an index into the producer list) still emits on channel
+// j is structurally zero.
+__device__ __forceinline__ bool shift_zero(const Tables& tb, int p, int j) {
+    const ProducerDesc d = tb.producers[p];
     const float bias = d.bias ? d.bias[j] : 0.0f;
-    if (d.bn >= 0) {
-        const BnDesc& b = tb.bns[d.bn];
-        return b.beta[j] == 0.0f && (b.gamma[j] == 0.0f || b.mean[j] == bias);
-    }
+    if (d.beta) return d.beta[j] == 0.0f && (d.gamma[j] == 0.0f || d.mean[j] == bias);
     return bias == 0.0f;
 }
 
@@ -50,13 +48,13 @@ __global__ void __launch_bounds__(kThreads) k_propagate(Tables tb, const uint32_
         // producers: OR of the filter flags, one (producer, word) pair per thread and step
         for (int it = threadIdx.x; it < n_prod * n_words; it += kThreads) {
             const int p = it / n_words, w = it - p * n_words;
-            const uint32_t x = out_nz[tb.tensors[tb.prod_list[gd.prod_begin + p]].off_outnz + w];
+            const uint32_t x = out_nz[tb.producers[gd.prod_begin + p].off_outnz + w];
             if (x) atomicOr(&s_prod[w], x);
         }
         // consumers: OR of the input-column flags; with S columns per channel the S bits are folded
         for (int it = threadIdx.x; it < n_cons * n_words; it += kThreads) {
             const int q = it / n_words, w = it - q * n_words;
-            const TensorDesc& d = tb.tensors[tb.cons_list[gd.cons_begin + q]];
+            const ConsumerDesc d = tb.consumers[gd.cons_begin + q];
             uint32_t x = 0;
             if (d.S == 1) {
                 x = in_nz[d.off_innz + w];
@@ -80,7 +78,7 @@ __global__ void __launch_bounds__(kThreads) k_propagate(Tables tb, const uint32_
             for (uint32_t m = prod_dead; m; m &= m - 1) {
                 const int j = w * 32 + __ffs(m) - 1;
                 for (int p = gd.prod_begin; p < gd.prod_end; ++p)
-                    if (!shift_zero(tb, tb.prod_list[p], j)) shift_bad |= 1u << (j & 31);
+                    if (!shift_zero(tb, p, j)) shift_bad |= 1u << (j & 31);
             }
         }
         const uint32_t rem = ((policy & DNNS_RULE_PRODUCER) ? prod_dead & ~shift_bad : 0u) |
@@ -131,7 +129,7 @@ __global__ void __launch_bounds__(kThreads) k_propagate(Tables tb, const uint32_
             keep_idx[gd.off_idx + s_pre[j >> 5] + __popc(~rem & (bit - 1u))] = j;
         } else if (stats && (s_prod[j >> 5] & bit)) {
             for (int p = gd.prod_begin; p < gd.prod_end; ++p)
-                if (!shift_zero(tb, tb.prod_list[p], j)) ++lost_pairs;
+                if (!shift_zero(tb, p, j)) ++lost_pairs;
         }
     }
     if (threadIdx.x == 0) keep_count[g] = (int32_t)carry;

@@ -76,6 +76,14 @@ def test_special_values_and_heavy_ties():
     compare_portfolio(wl, B.DNNS_F32, fused=True)
 
 
+def test_deep_chain_with_more_than_1024_gather_items():
+    """260 convs + BN = 1300 gather items: the layout is then computed by its own kernel."""
+    wl = W.chain([8] * 260, seed=21, kernel=1, planted_frac=0.25)
+    n = wl.n_prunable
+    wl.ks = np.array([[n // 2]], np.uint64)
+    compare_portfolio(wl, B.DNNS_F32, fused=True)
+
+
 def test_fc_with_spatial_columns():
     b = W._Builder()
     gi = b.group(3, frozen=True)
