@@ -135,6 +135,25 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
             const uint32_t rem = pos_rem;
             advance();
             if (f >= total) continue;
+            if (rem + VE <= Ln && blk == 1) {
+                // 1x1 kernels, vector inside one filter: one kept-channel lookup per element
+                const uint32_t row = (uint32_t)ko[a] * Cin;
+#pragma unroll
+                for (uint32_t e = 0; e < VE; ++e) idx[u][e] = row + (ki ? (uint32_t)ki[rem + e] : rem + e);
+                continue;
+            }
+            if (rem + VE <= Ln && blk >= VE) {
+                // vector inside one filter and at most two input channels: two lookups
+                const uint32_t c0 = blk == 9 ? rem / 9u : rem / blk, r0 = rem - c0 * blk, n0 = blk - r0;
+                const uint32_t row = (uint32_t)ko[a] * Cin;
+                const uint32_t base0 = (row + (ki ? (uint32_t)ki[c0] : c0)) * blk + r0;
+                uint32_t base1 = 0;
+                if (n0 < VE) base1 = (row + (ki ? (uint32_t)ki[c0 + 1] : c0 + 1)) * blk - n0;
+#pragma unroll
+                for (uint32_t e = 0; e < VE; ++e) idx[u][e] = (e < n0 ? base0 : base1) + e;
+                continue;
+            }
+            // vectors that cross a filter boundary or the end of the item: walk element by element
             uint32_t c = blk == 1 ? rem : (blk == 9 ? rem / 9u : rem / blk), r = rem - c * blk;
             uint32_t row = (uint32_t)ko[a] * Cin, col = ki ? (uint32_t)ki[c] : c;
             const uint32_t nv = min(VE, total - f);
@@ -185,8 +204,7 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
     }
 }
 
-// Every block takes a contiguous range of gather units and walks the items that own them, so the
-// item's context (source, destination, keep lists, new extents) is fetched once per run.
+// Blocks take chunks of consecutive gather units and walk the items that own them.
 //
 // INLINE_LAYOUT (models of up to kInlineItems items): every block derives the destination layout
 // itself, in shared memory, from the keep counts - a few hundred items, one scan - instead of waiting
@@ -251,40 +269,43 @@ __global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, Compa
     const uint64_t* item_off = INLINE_LAYOUT ? s_item_off : ws.item_off;
     const int32_t* item_dims = INLINE_LAYOUT ? s_item_dims : ws.item_dims;
     const uint32_t total_units = unit_prefix[tb.n_items];
-    const uint32_t per = (total_units + gridDim.x - 1) / gridDim.x;
-    const uint32_t u_lo = min(total_units, blockIdx.x * per), u_hi = min(total_units, u_lo + per);
-    if (u_lo >= u_hi) return;
-    // the item holding the first unit: last i with unit_prefix[i] <= u_lo
-    uint32_t item = 0, hi = tb.n_items;
-    while (hi - item > 1) {
-        const uint32_t mid = (item + hi) >> 1;
-        if (unit_prefix[mid] <= u_lo) item = mid;
-        else hi = mid;
-    }
-    uint32_t unit = u_lo;
-    while (unit < u_hi) {
-        const uint32_t item_begin = unit_prefix[item], item_end = unit_prefix[item + 1];
-        if (unit >= item_end) {  // items that shrank to nothing own no units
-            ++item;
-            continue;
+    // Units are dealt to the blocks in chunks, round robin: items differ a lot in cost per unit (plain
+    // row copies against element gathers), and interleaving evens that out without any shared counter.
+    constexpr uint32_t kChunkUnits = 2;
+    for (uint32_t u_lo = blockIdx.x * kChunkUnits; u_lo < total_units; u_lo += gridDim.x * kChunkUnits) {
+        const uint32_t u_hi = min(total_units, u_lo + kChunkUnits);
+        // the item holding the first unit: last i with unit_prefix[i] <= u_lo
+        uint32_t item = 0, hi = tb.n_items;
+        while (hi - item > 1) {
+            const uint32_t mid = (item + hi) >> 1;
+            if (unit_prefix[mid] <= u_lo) item = mid;
+            else hi = mid;
         }
-        const ItemDesc& it = tb.items[item];
-        const uint32_t On = item_dims[2 * item], Cn = item_dims[2 * item + 1];
-        const char* src;
-        if (it.tensor >= 0) {
-            const TensorDesc& d = tb.tensors[it.tensor];
-            src = src_arena ? src_arena + d.arena_off : static_cast<const char*>(d.src);
-        } else {
-            src = static_cast<const char*>(it.src);
+        uint32_t unit = u_lo;
+        while (unit < u_hi) {
+            const uint32_t item_begin = unit_prefix[item], item_end = unit_prefix[item + 1];
+            if (unit >= item_end) {  // items that shrank to nothing own no units
+                ++item;
+                continue;
+            }
+            const ItemDesc& it = tb.items[item];
+            const uint32_t On = item_dims[2 * item], Cn = item_dims[2 * item + 1];
+            const char* src;
+            if (it.tensor >= 0) {
+                const TensorDesc& d = tb.tensors[it.tensor];
+                src = src_arena ? src_arena + d.arena_off : static_cast<const char*>(d.src);
+            } else {
+                src = static_cast<const char*>(it.src);
+            }
+            char* dst = dst_arena + item_off[item];
+            const int32_t* ko = keep_idx + tb.groups[it.out_group].off_idx;
+            const int32_t* ki = it.in_group >= 0 ? keep_idx + tb.groups[it.in_group].off_idx : nullptr;
+            const uint32_t run_end = min(u_hi, item_end);
+            const uint32_t f0 = (unit - item_begin) * (kUnitBytes / it.elem_bytes);
+            if (WBYTES == 4 || it.elem_bytes == 4) gather_run<4>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit);
+            else gather_run<2>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit);
+            unit = run_end;
         }
-        char* dst = dst_arena + item_off[item];
-        const int32_t* ko = keep_idx + tb.groups[it.out_group].off_idx;
-        const int32_t* ki = it.in_group >= 0 ? keep_idx + tb.groups[it.in_group].off_idx : nullptr;
-        const uint32_t run_end = min(u_hi, item_end);
-        const uint32_t f0 = (unit - item_begin) * (kUnitBytes / it.elem_bytes);
-        if (WBYTES == 4 || it.elem_bytes == 4) gather_run<4>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit);
-        else gather_run<2>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit);
-        unit = run_end;
     }
 }
 

@@ -114,17 +114,18 @@ __global__ void __launch_bounds__(256) k_flags(Tables tb, uint32_t* nz_map, uint
                 const uint32_t local = unit - t_begin, rb = local / n_chunks, cc = local - rb * n_chunks;
                 const uint32_t row0 = rb * kFlagRows, iw = cc * 32 + (lane & (cw - 1));
                 uint32_t acc = 0, rows = 0;  // column OR of this lane's words; filters of the unit that hold something
-                // (the trip count is the same in every lane: the loop body holds a warp-wide vote)
                 constexpr int kMaxSteps = kFlagRows;  // cw <= 32 words per filter and chunk
+                const uint32_t n_steps = (kFlagRows * cw + 31) / 32;
+                // first all the words of the unit (their loads are independent and overlap) ...
+                uint32_t words[kMaxSteps];
 #pragma unroll
                 for (int step = 0; step < kMaxSteps; ++step) {
-                    const uint32_t base = step * 32;
-                    if (base >= kFlagRows * cw) break;
-                    const uint32_t k = base + lane;
+                    words[step] = 0;
+                    const uint32_t k = step * 32 + lane;
                     const uint32_t o = row0 + (k >> cw_shift);
-                    uint32_t word = 0;
-                    if (k < kFlagRows * cw && o < O) {
+                    if ((uint32_t)step < n_steps && k < kFlagRows * cw && o < O) {
                         const uint32_t gw = o * wpr + iw;  // this lane's word of the kernel map
+                        uint32_t word = 0;
                         if (KK == 1) {
                             word = __ldg(ebits + gw);
                         } else if (KK == 9) {
@@ -135,13 +136,19 @@ __global__ void __launch_bounds__(256) k_flags(Tables tb, uint32_t* nz_map, uint
                                 word |= (uint32_t)any_bits(ebits, (q0 + j) * KK, (q0 + j + 1) * KK) << j;
                         }
                         if (g_map) g_map[gw] = word;
+                        words[step] = word;
                     }
-                    acc |= word;
-                    // one bit per group of cw lanes = per filter of this step
-                    const uint32_t nzl = __ballot_sync(kFull, word != 0);
-                    const uint32_t group_mask = cw == 32 ? 0xffffffffu : ((1u << cw) - 1u);
+                    acc |= words[step];
+                }
+                // ... then one vote per step: one bit per group of cw lanes = per filter of the step
+                // (the trip count is the same in every lane)
+                const uint32_t group_mask = cw == 32 ? 0xffffffffu : ((1u << cw) - 1u);
+#pragma unroll
+                for (int step = 0; step < kMaxSteps; ++step) {
+                    if ((uint32_t)step >= n_steps) break;
+                    const uint32_t nzl = __ballot_sync(kFull, words[step] != 0);
                     for (uint32_t g = 0; g < min(32u >> cw_shift, kFlagRows); ++g)
-                        if ((nzl >> (g << cw_shift)) & group_mask) rows |= 1u << ((base >> cw_shift) + g);
+                        if ((nzl >> (g << cw_shift)) & group_mask) rows |= 1u << (((step * 32) >> cw_shift) + g);
                 }
                 // kFlagRows divides 32, so the filters of a unit share one flag word
                 if (lane == 0 && rows) or_if_missing(&g_out[row0 >> 5], rows << (row0 & 31));
