@@ -58,7 +58,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -176,6 +176,7 @@ def main():
     import torch.distributed as dist
     from paper_2309_06973_b200 import binding as B
     from paper_2309_06973_b200.runtime import DeviceModel, Session
+    from paper_2309_06973_b200.dist_util import max_over_ranks, ms_per_variant as whole_job_ms_per_variant
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
@@ -289,14 +290,11 @@ def main():
         launches = launches_plain
     clocks = sampler.stop()
     barrier()
-    if world > 1:
-        t = torch.tensor([total_ms, plain_ms], device=dm.device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, plain_ms = float(t[0].item()), float(t[1].item())
+    total_ms, plain_ms = max_over_ranks([total_ms, plain_ms], dm.device)
     assert ses.device_status() == B.DNNS_OK
 
     ms_per_step = total_ms / args.steps
-    ms_per_variant = ms_per_step / V / world if world > 1 else ms_per_step / V
+    ms_per_variant = whole_job_ms_per_variant(ms_per_step, V, world)
     per_call = {n: statistics.mean(a.elapsed_time(b) for a, b in spans[n]) for n in names}
     plain_per_step = plain_ms / args.steps
     share = {n: per_call[n] * (1 if n == "threshold" else V) / plain_per_step for n in names}
@@ -345,11 +343,8 @@ def main():
         e2e_step()
     barrier()
     e2e_ms = (time.perf_counter() - t0) * 1e3
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dm.device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_per_variant = e2e_ms / args.steps / V / world
+    e2e_ms = max_over_ranks([e2e_ms], dm.device)[0]
+    e2e_per_variant = whole_job_ms_per_variant(e2e_ms / args.steps, V, world)
 
     line = {
         "metric": METRIC, "value": ms_per_variant, "unit": "ms", "n_gpus": world, "steps": args.steps,
