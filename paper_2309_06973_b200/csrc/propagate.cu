@@ -45,15 +45,18 @@ __global__ void __launch_bounds__(kThreads) k_propagate(Tables tb, const uint32_
     for (int w = threadIdx.x; w < n_words; w += kThreads) s_prod[w] = s_cons[w] = 0;
     __syncthreads();
     if (!frozen) {
-        // producers: OR of the filter flags, one (producer, word) pair per thread and step
-        for (int it = threadIdx.x; it < n_prod * n_words; it += kThreads) {
-            const int p = it / n_words, w = it - p * n_words;
-            const uint32_t x = out_nz[tb.producers[gd.prod_begin + p].off_outnz + w];
-            if (x) atomicOr(&s_prod[w], x);
-        }
-        // consumers: OR of the input-column flags; with S columns per channel the S bits are folded
-        for (int it = threadIdx.x; it < n_cons * n_words; it += kThreads) {
-            const int q = it / n_words, w = it - q * n_words;
+        // One (tensor, word) pair per thread and step, producers first, then consumers: all flag
+        // words of the group are requested in one go.  Producers OR their filter flags; consumers OR
+        // their input-column flags (with S columns per channel the S bits are folded).
+        const int n_pw = n_prod * n_words;
+        for (int it = threadIdx.x; it < n_pw + n_cons * n_words; it += kThreads) {
+            if (it < n_pw) {
+                const int p = it / n_words, w = it - p * n_words;
+                const uint32_t x = out_nz[tb.producers[gd.prod_begin + p].off_outnz + w];
+                if (x) atomicOr(&s_prod[w], x);
+                continue;
+            }
+            const int q = (it - n_pw) / n_words, w = (it - n_pw) - q * n_words;
             const ConsumerDesc d = tb.consumers[gd.cons_begin + q];
             uint32_t x = 0;
             if (d.S == 1) {

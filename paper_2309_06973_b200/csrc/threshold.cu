@@ -394,35 +394,37 @@ __global__ void __launch_bounds__(1024) k_select2(Tables tb, ThresholdWs ws, int
         return;
     }
     const uint32_t* h = ws.hist2 + ((size_t)seg * n_k + st.slot) * kLowBins;
+    uint32_t part[16];  // this thread's 64 bins in groups of four
     uint64_t sum = 0;
+#pragma unroll
     for (int j = 0; j < 16; ++j) {
         const uint4 q = reinterpret_cast<const uint4*>(h)[threadIdx.x * 16 + j];
-        sum += (uint64_t)q.x + q.y + q.z + q.w;
+        part[j] = q.x + q.y + q.z + q.w;
+        sum += part[j];
     }
     uint64_t total;
     const uint64_t excl = st.below + block_exclusive_scan<uint64_t>(sum, scratch, &total);
     if (excl < st.k && st.k <= excl + sum) {
-        // this thread's 64 bins again, as independent vector loads, then a search in registers
-        uint4 q[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) q[j] = reinterpret_cast<const uint4*>(h)[threadIdx.x * 16 + j];
+        // the group of four that holds the k-th key, then one more load for its bins
         uint64_t cum = excl;
-        uint32_t b = 0, cnt = 0;
+        int jj = 0;
         bool found = false;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-            const uint32_t c4[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+            if (!found) {
+                if (cum + part[j] >= st.k) jj = j, found = true;
+                else cum += part[j];
+            }
+        }
+        const uint4 q = reinterpret_cast<const uint4*>(h)[threadIdx.x * 16 + jj];
+        const uint32_t c4[4] = {q.x, q.y, q.z, q.w};
+        uint32_t b = 0, cnt = 0;
+        found = false;
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                if (!found) {
-                    if (cum + c4[t] >= st.k) {
-                        b = 4 * j + t;
-                        cnt = c4[t];
-                        found = true;
-                    } else {
-                        cum += c4[t];
-                    }
-                }
+        for (int t = 0; t < 4; ++t) {
+            if (!found) {
+                if (cum + c4[t] >= st.k) b = 4 * jj + t, cnt = c4[t], found = true;
+                else cum += c4[t];
             }
         }
         dnns_threshold r;
