@@ -454,8 +454,11 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_ties(Tables tb, ThresholdWs
     if (*ws.any_need == 0) return;
     __shared__ uint32_t s_bm[kBitmapWords];
     __shared__ uint32_t s_tau[kMaxVariants], s_need[kMaxVariants];
+    __shared__ uint32_t s_cnt[kTileThreads / 32][kMaxVariants];  // per warp: ties of the current tile, per variant
     __shared__ uint32_t s_any, s_zero_tau;
     const uint32_t S = tb.n_segs;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = threadIdx.x; i < (kTileThreads / 32) * kMaxVariants; i += kTileThreads) (&s_cnt[0][0])[i] = 0;
     int cur_seg = -1;
     walk_prunable_tiles<DT>(
         tb,
@@ -487,8 +490,19 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_ties(Tables tb, ThresholdWs
                     return;
                 }
                 for (int vv = 0; vv < n_k; ++vv)
-                    if (s_need[vv] && s_tau[vv] == key) atomicAdd(&ws.tile_ties[(size_t)vv * tb.n_tiles + tile], 1u);
+                    if (s_need[vv] && s_tau[vv] == key) atomicAdd(&s_cnt[warp][vv], 1u);
             });
+            // a warp sends its counts of the tile to the table in one atomic per variant: keys equal to
+            // tau are common in 15-bit keys, and thousands of single atomics on one word would queue up
+            __syncwarp();
+            for (int vv = lane; vv < n_k; vv += 32) {
+                const uint32_t c = s_cnt[warp][vv];
+                if (c) {
+                    atomicAdd(&ws.tile_ties[(size_t)vv * tb.n_tiles + tile], c);
+                    s_cnt[warp][vv] = 0;
+                }
+            }
+            __syncwarp();
             if (s_zero_tau) {
 #pragma unroll
                 for (int d = 16; d > 0; d >>= 1) zeros += __shfl_xor_sync(0xffffffffu, zeros, d);
