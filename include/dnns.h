@@ -249,6 +249,18 @@ dnns_status dnns_compact(dnns_plan* plan, const void* masked_arena, const int32_
                          const int32_t* keep_count, void* dst_arena, size_t dst_bytes, uint64_t* dst_offsets_dev,
                          int32_t* dst_shapes_dev, void* stream);
 
+/*
+ * Module 1, Model Pre-Processor (Section III-D): fold every BatchNorm into the convolution it
+ * follows, on a rebuilt variant as dnns_compact left it (same dst_arena, dst_offsets_dev,
+ * dst_shapes_dev).  In place, fp32 arithmetic (bf16 weights are widened, scaled, rounded to nearest
+ * even):  s_o = gamma_o / sqrt(var_o + eps);  W[o] <- W[o] * s_o;  the arena slot of gamma receives
+ * s, the slot of beta receives the folded bias beta_o + (bias_o - mean_o) * s_o (bias_o = 0 when the
+ * layer has none).  mean and var are left as they are; tensors without BatchNorm are untouched.
+ * Floating point: results agree with an fp64 evaluation to a few fp32 units in the last place.
+ */
+dnns_status dnns_fold_batchnorm(dnns_plan* plan, void* dst_arena, const uint64_t* dst_offsets_dev,
+                                const int32_t* dst_shapes_dev, void* stream);
+
 /* Synchronises `stream`, then returns (and clears) the status recorded by the plan's kernels. */
 dnns_status dnns_last_device_status(dnns_plan* plan, void* stream);
 

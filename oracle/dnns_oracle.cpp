@@ -24,6 +24,8 @@
 //   O5 orc_compact         - Module 4 (Model Pruner, Algorithm 2): rebuild each
 //                            layer with |C'_in| x |C'_out| channels and move the
 //                            surviving out-channels, biases and in-channels over.
+//   O7 orc_fold_batchnorm  - Module 1 (Model Pre-Processor): fuse each convolution
+//                            with the batch normalisation that follows it.
 //
 // Parity against numbers printed in the paper: unpinned (every number the paper
 // prints depends on trained weights).  The functions are pinned instead by brute
@@ -36,6 +38,7 @@
 // the set stored at word b/32, position b%32.
 
 #include <algorithm>
+#include <cmath>
 #include <cstdint>
 #include <cstring>
 #include <vector>
@@ -354,6 +357,43 @@ void orc_compact(const orc_model* m, int32_t* const* keep_idx, const int32_t* ke
         const float* src[4] = {B.gamma, B.beta, B.mean, B.var};
         for (int v = 0; v < 4; ++v)
             for (int a = 0; a < keep_count[g]; ++a) dst_bn[4 * b + v][a] = src[v][keep_idx[g][a]];
+    }
+}
+
+// O7.  Module 1 fuses a convolution with the batch normalisation behind it.  BN maps the
+// conv output y_o (plus the conv bias) to gamma_o * (y_o + bias_o - mean_o) / sqrt(var_o + eps) +
+// beta_o, which is a convolution again with
+//   scale_o = gamma_o / sqrt(var_o + eps),  W_f[o] = W[o] * scale_o,
+//   b_f[o]  = beta_o + (bias_o - mean_o) * scale_o        (bias_o = 0 without a bias),
+// evaluated here in double precision.  folded_w[t] (numel doubles) is filled for tensors that
+// have a BN and may be null for the others; scale[b], folded_bias[b] hold C doubles per BN.
+void orc_fold_batchnorm(const orc_model* m, double* const* folded_w, double* const* scale, double* const* folded_bias) {
+    for (int b = 0; b < m->n_bn; ++b) {
+        const orc_bn& B = m->bns[b];
+        const orc_tensor& T = m->tensors[B.tensor];
+        const int64_t row = (int64_t)T.I * T.KH * T.KW;
+        for (int64_t o = 0; o < T.O; ++o) {
+            const double s = (double)B.gamma[o] / std::sqrt((double)B.var[o] + (double)B.eps);
+            const double bias = T.bias ? (double)T.bias[o] : 0.0;
+            scale[b][o] = s;
+            folded_bias[b][o] = (double)B.beta[o] + (bias - (double)B.mean[o]) * s;
+            for (int64_t r = 0; r < row; ++r) {
+                double w;
+                if (T.dtype == ORC_F32) {
+                    float f;
+                    std::memcpy(&f, (const char*)T.data + 4 * (o * row + r), 4);
+                    w = f;
+                } else {
+                    uint16_t h;
+                    std::memcpy(&h, (const char*)T.data + 2 * (o * row + r), 2);
+                    const uint32_t u = (uint32_t)h << 16;
+                    float f;
+                    std::memcpy(&f, &u, 4);
+                    w = f;
+                }
+                folded_w[B.tensor][o * row + r] = w * s;
+            }
+        }
     }
 }
 

@@ -170,3 +170,14 @@ def compact(om: OracleModel, keep_idx, keep_count):
                       _ptr_array(dst_bn) if dst_bn else None, _ptr_array(dst_bias), C.c_void_p(shapes.ctypes.data))
     bns = [tuple(dst_bn[4 * i: 4 * i + 4]) for i in range(len(wl.bns))]
     return dst_w, bns, dst_bias, shapes
+
+
+def fold_batchnorm(om: OracleModel):
+    """Returns (folded weights as float64 arrays or None per tensor, scale per BN, folded bias per BN)."""
+    wl = om.wl
+    has_bn = {b.tensor for b in wl.bns}
+    fw = [np.zeros(w.shape, np.float64) if i in has_bn else None for i, w in enumerate(om.weights)]
+    scale = [np.zeros(b.C, np.float64) for b in wl.bns]
+    fbias = [np.zeros(b.C, np.float64) for b in wl.bns]
+    lib().orc_fold_batchnorm(C.byref(om.c), _ptr_array(fw), _ptr_array(scale), _ptr_array(fbias))
+    return fw, scale, fbias

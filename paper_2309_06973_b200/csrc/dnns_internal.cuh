@@ -46,6 +46,8 @@ struct GroupDesc {
 struct BnDesc {
     const float *gamma, *beta, *mean, *var;
     int32_t C, tensor;
+    int32_t bias_item;  // gather item of the tensor's bias, -1 when it has none
+    float eps;
 };
 
 // What the keep propagation needs of one producer / consumer of a group, next to the lists of
@@ -135,6 +137,7 @@ int launch_propagate(const Tables& tb, const uint32_t* out_nz, const uint32_t* i
 int launch_compact(const Tables& tb, const CompactWs& ws, const void* src_arena, const int32_t* keep_idx,
                    const int32_t* keep_count, void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets,
                    int32_t* dst_shapes, int n_sm, cudaStream_t st);
+int launch_fold(const Tables& tb, void* arena, const uint64_t* offsets, const int32_t* shapes, cudaStream_t st);
 cudaError_t init_kernel_attributes();
 
 // ---- small device helpers ----

@@ -283,7 +283,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     }
     for (uint32_t b = 0; b < c.B; ++b) {
         const dnns_bn& bn = m->bns[b];
-        bd[b] = BnDesc{bn.gamma, bn.beta, bn.mean, bn.var, bn.C, bn.tensor};
+        bd[b] = BnDesc{bn.gamma, bn.beta, bn.mean, bn.var, bn.C, bn.tensor, -1, bn.eps};
         td[bn.tensor].bn = (int32_t)b;
     }
     for (int i = 0; i < np; ++i) {
@@ -311,6 +311,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     }
     for (uint32_t i = 0; i < c.T; ++i)
         if (m->tensors[i].bias) {
+            if (td[i].bn >= 0) bd[td[i].bn].bias_item = (int32_t)n_it;
             id[n_it++] = ItemDesc{m->tensors[i].bias, -1, m->tensors[i].O, 1, 1, m->tensors[i].out_group, -1, 4};
             compact_bytes += align_up(4ull * m->tensors[i].O);
         }
@@ -468,6 +469,16 @@ dnns_status dnns_compact(dnns_plan* p, const void* masked_arena, const int32_t* 
         return DNNS_ERR_INVALID_ARG;
     const int n = launch_compact(p->tb, p->cws, masked_arena, keep_idx, keep_count, dst_arena, dst_bytes,
                                  dst_offsets_dev, dst_shapes_dev, p->n_sm, static_cast<cudaStream_t>(stream));
+    if (n < 0) return DNNS_ERR_CUDA;
+    p->launches += n;
+    return DNNS_OK;
+}
+
+dnns_status dnns_fold_batchnorm(dnns_plan* p, void* dst_arena, const uint64_t* dst_offsets_dev,
+                                const int32_t* dst_shapes_dev, void* stream) {
+    if (!p || !dst_arena || !dst_offsets_dev || !dst_shapes_dev) return DNNS_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) return DNNS_ERR_INVALID_ARG;
+    const int n = launch_fold(p->tb, dst_arena, dst_offsets_dev, dst_shapes_dev, static_cast<cudaStream_t>(stream));
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
     return DNNS_OK;

@@ -155,6 +155,11 @@ class Session:
                        self.compact_arena.numel() if dst_bytes is None else dst_bytes, self.dst_offsets.data_ptr(),
                        self.dst_shapes.data_ptr(), _stream())
 
+    def fold_batchnorm(self):
+        """Fold the BatchNorms of the variant in the destination arena into its convolutions (in place)."""
+        B.dnns_fold_batchnorm(self.plan, self.compact_arena.data_ptr(), self.dst_offsets.data_ptr(),
+                              self.dst_shapes.data_ptr(), _stream())
+
     def variant(self, v: int, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1,
                 fused: bool = False):
         """Steps 2-5 for variant v of the latest threshold call (fused: steps 2 and 3 in one sweep)."""
