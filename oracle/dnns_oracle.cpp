@@ -24,6 +24,9 @@
 //   O5 orc_compact         - Module 4 (Model Pruner, Algorithm 2): rebuild each
 //                            layer with |C'_in| x |C'_out| channels and move the
 //                            surviving out-channels, biases and in-channels over.
+//   O8 orc_propagate_keep_cascade - Algorithm 1 applied again and again: once channels
+//                            are gone, filters that only read removed channels (and input
+//                            columns only read by removed filters) are zero channels too.
 //   O7 orc_fold_batchnorm  - Module 1 (Model Pre-Processor): fuse each convolution
 //                            with the batch normalisation that follows it.
 //
@@ -357,6 +360,96 @@ void orc_compact(const orc_model* m, int32_t* const* keep_idx, const int32_t* ke
         const float* src[4] = {B.gamma, B.beta, B.mean, B.var};
         for (int v = 0; v < 4; ++v)
             for (int a = 0; a < keep_count[g]; ++a) dst_bn[4 * b + v][a] = src[v][keep_idx[g][a]];
+    }
+}
+
+// O8.  Fixed point of the plan.  Algorithm 1 looks at the zero channels once; but a filter whose
+// only non-zero 2-D kernels sit in input channels that are being removed is as good as zero, and
+// an input column that only removed filters read is as good as unread.  Pass p evaluates the rule of
+// O4 for every channel with "zero" judged on the kernel maps restricted to what pass p-1 kept:
+//   prod_dead  - every producer's filter j has no non-zero kernel in a kept input channel,
+//   cons_dead  - no kept filter of any consumer has a non-zero kernel in the columns of channel j,
+// all channels judged against the same previous sets (simultaneous update), removed channels stay
+// removed.  Passes stop when nothing changes or after max_passes.  Pass 1 is O4's single pass.
+// min_keep is applied once, at the end.  nz_map[t]: O*I bits as written by orc_zero_structures.
+// stats: [0] as in O4, judged in the last pass, [1] channels removed, [2] taken back by min_keep,
+// [3] passes that removed something.
+void orc_propagate_keep_cascade(const orc_model* m, uint32_t* const* nz_map, uint32_t policy, int32_t min_keep,
+                                int32_t max_passes, uint32_t* const* keep_bits, int32_t* const* keep_idx,
+                                int32_t* keep_count, uint64_t* stats) {
+    const int G = m->n_groups;
+    std::vector<std::vector<char>> removed(G), lost(G);
+    for (int g = 0; g < G; ++g) removed[g].assign(m->groups[g].C, 0), lost[g].assign(m->groups[g].C, 0);
+    auto shift_zero = [&](int p, int j) {
+        const orc_tensor& T = m->tensors[p];
+        const float bias = T.bias ? T.bias[j] : 0.0f;
+        for (int b = 0; b < m->n_bn; ++b)
+            if (m->bns[b].tensor == p) {
+                const orc_bn& B = m->bns[b];
+                return B.beta[j] == 0.0f && (B.gamma[j] == 0.0f || B.mean[j] == bias);
+            }
+        return bias == 0.0f;
+    };
+    uint64_t passes = 0;
+    for (int pass = 0; pass < max_passes; ++pass) {
+        std::vector<std::vector<char>> next = removed;
+        bool changed = false;
+        for (int g = 0; g < G; ++g) {
+            if (m->groups[g].flags & ORC_GROUP_FROZEN) continue;
+            std::vector<int> producers, consumers;
+            for (int t = 0; t < m->n_tensors; ++t) {
+                if (m->tensors[t].out_group == g) producers.push_back(t);
+                if (m->tensors[t].in_group == g) consumers.push_back(t);
+            }
+            for (int j = 0; j < m->groups[g].C; ++j) {
+                bool prod_dead = !producers.empty();
+                for (int p : producers) {
+                    const orc_tensor& T = m->tensors[p];
+                    for (int i = 0; i < T.I; ++i)
+                        if (!removed[T.in_group][i / T.in_spatial] && get_bit(nz_map[p], (int64_t)j * T.I + i)) prod_dead = false;
+                }
+                bool cons_dead = !consumers.empty();
+                for (int q : consumers) {
+                    const orc_tensor& T = m->tensors[q];
+                    for (int o = 0; o < T.O; ++o)
+                        for (int s2 = 0; s2 < T.in_spatial; ++s2)
+                            if (!removed[T.out_group][o] && get_bit(nz_map[q], (int64_t)o * T.I + (int64_t)j * T.in_spatial + s2))
+                                cons_dead = false;
+                }
+                bool shift_ok = true;
+                if (policy & ORC_SHIFT_STRICT)
+                    for (int p : producers)
+                        if (!shift_zero(p, j)) shift_ok = false;
+                const bool rule = ((policy & ORC_RULE_PRODUCER) && prod_dead && shift_ok) ||
+                                  ((policy & ORC_RULE_CONSUMER) && cons_dead);
+                lost[g][j] = prod_dead && !cons_dead;
+                if (rule && !removed[g][j]) next[g][j] = 1, changed = true;
+            }
+        }
+        removed.swap(next);
+        if (!changed) break;
+        ++passes;
+    }
+    if (stats) stats[0] = stats[1] = stats[2] = 0, stats[3] = passes;
+    for (int g = 0; g < G; ++g) {
+        const int C = m->groups[g].C;
+        int kept = 0;
+        for (int j = 0; j < C; ++j) kept += !removed[g][j];
+        const int floor_keep = std::min<int>(std::max<int>(min_keep, 0), C);
+        for (int j = 0; j < C && kept < floor_keep; ++j)
+            if (removed[g][j]) { removed[g][j] = 0; ++kept; if (stats) ++stats[2]; }
+        std::memset(keep_bits[g], 0, (size_t)((C + 31) / 32) * 4);
+        int n = 0;
+        for (int j = 0; j < C; ++j) {
+            if (!removed[g][j]) { set_bit(keep_bits[g], j); keep_idx[g][n++] = j; continue; }
+            if (stats) {
+                ++stats[1];
+                if (lost[g][j])
+                    for (int t = 0; t < m->n_tensors; ++t)
+                        if (m->tensors[t].out_group == g && !shift_zero(t, j)) ++stats[0];
+            }
+        }
+        keep_count[g] = n;
     }
 }
 

@@ -181,3 +181,16 @@ def fold_batchnorm(om: OracleModel):
     fbias = [np.zeros(b.C, np.float64) for b in wl.bns]
     lib().orc_fold_batchnorm(C.byref(om.c), _ptr_array(fw), _ptr_array(scale), _ptr_array(fbias))
     return fw, scale, fbias
+
+
+def propagate_keep_cascade(om: OracleModel, nz_map, policy: int = RULE_PRODUCER | RULE_CONSUMER, min_keep: int = 1,
+                           max_passes: int = 64):
+    wl = om.wl
+    keep_bits = [_bitwords(g.C) for g in wl.groups]
+    keep_idx = [np.full(g.C, -1, np.int32) for g in wl.groups]
+    keep_count = np.zeros(len(wl.groups), np.int32)
+    stats = np.zeros(4, np.uint64)
+    lib().orc_propagate_keep_cascade(C.byref(om.c), _ptr_array(nz_map), C.c_uint32(policy), C.c_int32(min_keep),
+                                     C.c_int32(max_passes), _ptr_array(keep_bits), _ptr_array(keep_idx),
+                                     C.c_void_p(keep_count.ctypes.data), C.c_void_p(stats.ctypes.data))
+    return keep_bits, keep_idx, keep_count, stats

@@ -2,8 +2,6 @@
 Tolerance: the kernel works in fp32 (one division, one square root, one multiply per value), so a
 result may differ from the fp64 value by a few fp32 units in the last place; bf16 weights add the
 final rounding to 8 significant bits."""
-import copy
-
 import numpy as np
 import pytest
 
@@ -11,25 +9,12 @@ from oracle import oracle as O
 from paper_2309_06973_b200 import binding as B
 from paper_2309_06973_b200 import workloads as W
 from paper_2309_06973_b200.runtime import DeviceModel, Session
+from model_utils import compacted_workload
 
-pytestmark = pytest.mark.gpu
+pytestmark = pytest.mark.gpu  # (compacted_workload below is also used by CPU tests)
 
 F32_RTOL = 4 * 2.0 ** -24      # division, square root and product, each within half an ulp
 BF16_RTOL = 2.0 ** -8 + F32_RTOL
-
-
-def compacted_workload(wl, keep_count, weights, bn_params, biases):
-    """The rebuilt variant as a workload of its own (smaller extents, same wiring)."""
-    cw = copy.deepcopy(wl)
-    for g, c in zip(cw.groups, keep_count):
-        g.C = int(c)
-    for t in cw.tensors:
-        t.O = cw.groups[t.out_group].C
-        t.I = cw.groups[t.in_group].C * t.in_spatial
-    for b in cw.bns:
-        b.C = cw.groups[cw.tensors[b.tensor].out_group].C
-    cw.weights, cw.bn_params, cw.biases = weights, bn_params, biases
-    return cw
 
 
 def close(got, want, rtol):
