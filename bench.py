@@ -324,6 +324,34 @@ def main():
         fold_ms.append(a.elapsed_time(b))
     fold_ms = statistics.median(fold_ms)
 
+    # ---- fixed-point keep propagation on the last variant (not part of the portfolio step)
+    def params_of(session):
+        sh = session.dst_shapes.cpu().numpy()[: 2 * len(wl.tensors)].reshape(-1, 2)
+        return sum(int(sh[i, 0]) * int(sh[i, 1]) * t.KH * t.KW for i, t in enumerate(wl.tensors))
+
+    ses2 = Session(dm, wl.scope, V, want_mask_bits=False, want_nz_map=True)
+    ses2.magnitude_threshold(wl.ks)
+    ses2.mask_and_structures(V - 1)
+    ses2.propagate_keep()
+    ses2.compact()
+    torch.cuda.synchronize()
+    params_single = params_of(ses2)
+    casc_ms = []
+    for _ in range(5):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        ses2.propagate_keep_cascade(max_passes=8)
+        b.record()
+        torch.cuda.synchronize()
+        casc_ms.append(a.elapsed_time(b))
+    ses2.compact()
+    torch.cuda.synchronize()
+    cascade = {"ms": statistics.median(casc_ms), "max_passes": 8,
+               "passes_that_removed": int(ses2.stats.cpu().numpy().view(np.uint64)[3]),
+               "weights_after_single_pass": params_single, "weights_after_cascade": params_of(ses2),
+               "what": "last variant: rule of Algorithm 1 applied to a fixed point on the kernel maps"}
+    ses2.close()
+
     # ---- end to end through the C ABI with host buffers -----------------------------------------
     small = torch.empty(1 << 16, dtype=torch.uint8).pin_memory()
     host_out = torch.empty(ses.compact_arena.numel(), dtype=torch.uint8).pin_memory()
@@ -377,6 +405,7 @@ def main():
         "e2e": {"value": e2e_per_variant, "unit": "ms", "h2d_bytes_per_step": h2d // args.steps,
                 "d2h_bytes_per_step": d2h // args.steps},
         "gpu_launches": launches,
+        "cascade": cascade,
         "fold_batchnorm": {"ms": fold_ms, "gbs": 2 * Nn[-1] * eb / (fold_ms * 1e-3) / 1e9,
                            "what": "conv + BatchNorm fusion of the last variant in place (read + write of its weights)"},
         "clocks": clocks,

@@ -235,6 +235,22 @@ dnns_status dnns_propagate_keep(dnns_plan* plan, const uint32_t* out_nz, const u
                                 uint64_t* stats, void* stream);
 
 /*
+ * Step 4 applied to a fixed point.  Algorithm 1 looks at the zero channels once; once channels are
+ * gone, a filter whose only non-zero 2-D kernels sit in removed input channels is a zero channel
+ * too, and an input column that only removed filters read is unread.  Pass p judges every channel by
+ * the rule of dnns_propagate_keep on the kernel maps restricted to what pass p-1 kept (all channels
+ * against the same previous sets; removal only grows); passes end when nothing changes or after
+ * max_passes (1..64; pass 1 alone is dnns_propagate_keep).  min_keep is applied once, at the end.
+ * nz_map (device): the packed kernel maps written by dnns_zero_structures / dnns_mask_and_structures.
+ * Outputs as in dnns_propagate_keep; stats[0] is judged in the last pass, stats[3] = passes that
+ * removed something.  The launches of all max_passes passes are enqueued; those after the last
+ * change return at once.
+ */
+dnns_status dnns_propagate_keep_cascade(dnns_plan* plan, const uint32_t* nz_map, uint32_t policy, int32_t min_keep,
+                                        int32_t max_passes, uint32_t* keep_bits, int32_t* keep_idx,
+                                        int32_t* keep_count, uint64_t* stats, void* stream);
+
+/*
  * Step 5 - rebuild every tensor with its kept channels only (Algorithm 2):
  *   W'[a][c][s][y][x] = W[keep_out[a]][keep_in[c]][s][y][x],  v'[a] = v[keep_out[a]] for every
  * BatchNorm vector and bias.  masked_arena as in step 3.  The destination arena receives, at

@@ -20,7 +20,7 @@ DNNS_STATIC_MAX_NUMEL = 1 << 26
 
 EXPORTS = ["dnns_status_string", "dnns_workspace_bytes", "dnns_plan_create", "dnns_plan_destroy", "dnns_plan_layout",
            "dnns_plan_launch_count", "dnns_magnitude_threshold", "dnns_apply_mask", "dnns_zero_structures",
-           "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures", "dnns_fold_batchnorm"]
+           "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures", "dnns_fold_batchnorm", "dnns_propagate_keep_cascade"]
 
 
 class dnns_tensor(C.Structure):
@@ -97,6 +97,7 @@ def lib() -> C.CDLL:
         L.dnns_compact.argtypes = [vp, vp, vp, vp, vp, C.c_size_t, vp, vp, vp]
         L.dnns_last_device_status.argtypes = [vp, vp]
         L.dnns_fold_batchnorm.argtypes = [vp, vp, vp, vp, vp]
+        L.dnns_propagate_keep_cascade.argtypes = [vp, vp, u32, i32, i32, vp, vp, vp, vp, vp]
         L.dnns_magnitude_threshold_static.argtypes = [vp, i32, u64, u64, vp, vp]
         _lib = L
     return _lib
@@ -183,3 +184,9 @@ def dnns_magnitude_threshold_static(weights_dev: int, dtype: int, numel: int, k:
 
 def dnns_fold_batchnorm(plan, dst_arena: int, dst_offsets_dev: int, dst_shapes_dev: int, stream: int = 0) -> None:
     _check(lib().dnns_fold_batchnorm(plan, dst_arena, dst_offsets_dev, dst_shapes_dev, stream), "dnns_fold_batchnorm")
+
+
+def dnns_propagate_keep_cascade(plan, nz_map: int, policy: int, min_keep: int, max_passes: int, keep_bits: int,
+                                keep_idx: int, keep_count: int, stats: int, stream: int = 0) -> None:
+    _check(lib().dnns_propagate_keep_cascade(plan, nz_map, policy, min_keep, max_passes, keep_bits, keep_idx,
+                                             keep_count, stats or None, stream), "dnns_propagate_keep_cascade")

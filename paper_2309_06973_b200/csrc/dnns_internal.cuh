@@ -118,6 +118,17 @@ struct ThresholdWs {
     uint32_t* tie_prefix;   // [max_variants][n_tiles]: those in earlier tiles of the segment
 };
 
+constexpr int kMaxCascadePasses = 64;
+
+// Scratch of the fixed-point keep propagation.
+struct CascadeWs {
+    uint32_t* rem[2];        // removal words of all groups (packed like the keep bits), previous / next pass
+    uint32_t* lost;          // dead channels that somebody still reads, as judged by the last pass
+    uint32_t* live;          // filter flags, then (at live_in_offset words) input-column flags of the current pass
+    uint32_t live_in_offset;
+    uint32_t* changed;       // [kMaxCascadePasses + 1] pass p removed something
+};
+
 struct CompactWs {
     uint32_t* unit_prefix;  // [n_items + 1] gather units before each item
     uint64_t* item_off;     // [n_items] byte offset in the destination arena
@@ -134,6 +145,10 @@ int launch_tile_sweep(const Tables& tb, const ThresholdWs& ws, bool do_mask, boo
 int launch_propagate(const Tables& tb, const uint32_t* out_nz, const uint32_t* in_nz, uint32_t policy,
                      int32_t min_keep, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count, uint64_t* stats,
                      cudaStream_t st);
+int launch_propagate_cascade(const Tables& tb, const CascadeWs& cw, const uint32_t* nz_map, uint32_t policy,
+                             int32_t min_keep, int32_t max_passes, uint32_t* keep_bits, int32_t* keep_idx,
+                             int32_t* keep_count, uint64_t* stats, uint32_t n_keep_words, uint32_t n_live_words, int n_sm,
+                             cudaStream_t st);
 int launch_compact(const Tables& tb, const CompactWs& ws, const void* src_arena, const int32_t* keep_idx,
                    const int32_t* keep_count, void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets,
                    int32_t* dst_shapes, int n_sm, cudaStream_t st);

@@ -19,6 +19,7 @@ struct WsMap {
     uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, producers, consumers, flag_prefix, status;
     uint64_t tables_end;  // everything before this is uploaded once at plan creation
     uint64_t k_dev, bitmap, sel, tie_prefix, unit_prefix, item_off, item_dims, ebits;
+    uint64_t casc_rem0, casc_rem1, casc_lost, casc_live, casc_changed;
     uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
     uint64_t any_need, need, tie_bitmap, tile_ties, hist1, hist2;
     uint64_t total;
@@ -26,7 +27,7 @@ struct WsMap {
 
 struct Counts {
     uint32_t T = 0, G = 0, B = 0, S = 0, items = 0, tiles = 0, n_bias = 0;
-    uint64_t mask_words = 0;
+    uint64_t mask_words = 0, keep_words = 0, out_words = 0, in_words = 0;
     int dtype = 0, elem_bytes = 4;
 };
 
@@ -47,6 +48,7 @@ dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts*
     for (int g = 0; g < m->n_groups; ++g) {
         if (m->groups[g].C <= 0) return DNNS_ERR_INVALID_ARG;
         if (m->groups[g].C > 65536) return DNNS_ERR_UNSUPPORTED;
+        c->keep_words += ((uint64_t)m->groups[g].C + 31) / 32;
     }
     uint64_t n_prunable = 0, seg_count = 0;
     for (int i = 0; i < m->n_tensors; ++i) {
@@ -62,6 +64,8 @@ dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts*
         if (numel >= (1ull << 31)) return DNNS_ERR_UNSUPPORTED;
         c->tiles += (uint32_t)((numel * c->elem_bytes + kTileBytes - 1) / kTileBytes);
         c->mask_words += (numel + 31) / 32;
+        c->out_words += ((uint64_t)t.O + 31) / 32;
+        c->in_words += ((uint64_t)t.I + 31) / 32;
         if (t.bias) ++c->n_bias;
         if (t.prunable) {
             n_prunable += numel;
@@ -117,6 +121,11 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.item_off = take(8ull * c.items);
     w.item_dims = take(8ull * c.items);
     w.ebits = take(4ull * c.mask_words);
+    w.casc_rem0 = take(4ull * c.keep_words);
+    w.casc_rem1 = take(4ull * c.keep_words);
+    w.casc_lost = take(4ull * c.keep_words);
+    w.casc_live = take(4ull * (c.out_words + c.in_words));
+    w.casc_changed = take(4ull * (kMaxCascadePasses + 1));
     w.clear_begin = o;
     w.any_need = take(4);
     w.need = take(4 * vs);
@@ -140,6 +149,7 @@ struct dnns_plan {
     Tables tb;
     ThresholdWs tws;
     CompactWs cws;
+    CascadeWs kws;
     uint64_t launches;
     int last_n_k;
     // host-side layout, handed out by dnns_plan_layout
@@ -356,6 +366,12 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     p->cws.unit_prefix = reinterpret_cast<uint32_t*>(w + map.unit_prefix);
     p->cws.item_off = reinterpret_cast<uint64_t*>(w + map.item_off);
     p->cws.item_dims = reinterpret_cast<int32_t*>(w + map.item_dims);
+    p->kws.rem[0] = reinterpret_cast<uint32_t*>(w + map.casc_rem0);
+    p->kws.rem[1] = reinterpret_cast<uint32_t*>(w + map.casc_rem1);
+    p->kws.lost = reinterpret_cast<uint32_t*>(w + map.casc_lost);
+    p->kws.live = reinterpret_cast<uint32_t*>(w + map.casc_live);
+    p->kws.live_in_offset = (uint32_t)c.out_words;
+    p->kws.changed = reinterpret_cast<uint32_t*>(w + map.casc_changed);
 
     dnns_layout& L = p->layout;
     L.n_tensors = c.T, L.n_bn = c.B, L.n_groups = c.G, L.n_segments = c.S, L.n_bias = c.n_bias;
@@ -455,6 +471,23 @@ dnns_status dnns_propagate_keep(dnns_plan* p, const uint32_t* out_nz, const uint
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (stats && cudaMemsetAsync(stats, 0, 32, st) != cudaSuccess) return DNNS_ERR_CUDA;
     const int n = launch_propagate(p->tb, out_nz, in_nz, policy, min_keep, keep_bits, keep_idx, keep_count, stats, st);
+    if (n < 0) return DNNS_ERR_CUDA;
+    p->launches += n;
+    return DNNS_OK;
+}
+
+dnns_status dnns_propagate_keep_cascade(dnns_plan* p, const uint32_t* nz_map, uint32_t policy, int32_t min_keep,
+                                        int32_t max_passes, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count,
+                                        uint64_t* stats, void* stream) {
+    if (!p || !nz_map || !keep_bits || !keep_idx || !keep_count) return DNNS_ERR_INVALID_ARG;
+    if (policy & ~(uint32_t)(DNNS_RULE_PRODUCER | DNNS_RULE_CONSUMER | DNNS_SHIFT_STRICT)) return DNNS_ERR_INVALID_ARG;
+    if (max_passes < 1 || max_passes > kMaxCascadePasses) return DNNS_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (stats && cudaMemsetAsync(stats, 0, 32, st) != cudaSuccess) return DNNS_ERR_CUDA;
+    const dnns_layout& L = p->layout;
+    const int n = launch_propagate_cascade(p->tb, p->kws, nz_map, policy, min_keep, max_passes, keep_bits, keep_idx,
+                                           keep_count, stats, (uint32_t)L.keep_words,
+                                           (uint32_t)(L.out_nz_words + L.in_nz_words), p->n_sm, st);
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
     return DNNS_OK;

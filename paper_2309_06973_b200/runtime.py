@@ -155,6 +155,12 @@ class Session:
                        self.compact_arena.numel() if dst_bytes is None else dst_bytes, self.dst_offsets.data_ptr(),
                        self.dst_shapes.data_ptr(), _stream())
 
+    def propagate_keep_cascade(self, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1,
+                               max_passes: int = 8):
+        B.dnns_propagate_keep_cascade(self.plan, self.nz_map.data_ptr(), policy, min_keep, max_passes,
+                                      self.keep_bits.data_ptr(), self.keep_idx.data_ptr(), self.keep_count.data_ptr(),
+                                      self.stats.data_ptr(), _stream())
+
     def fold_batchnorm(self):
         """Fold the BatchNorms of the variant in the destination arena into its convolutions (in place)."""
         B.dnns_fold_batchnorm(self.plan, self.compact_arena.data_ptr(), self.dst_offsets.data_ptr(),
