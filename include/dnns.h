@@ -277,6 +277,43 @@ dnns_status dnns_compact(dnns_plan* plan, const void* masked_arena, const int32_
 dnns_status dnns_fold_batchnorm(dnns_plan* plan, void* dst_arena, const uint64_t* dst_offsets_dev,
                                 const int32_t* dst_shapes_dev, void* stream);
 
+/*
+ * Phase 3, Module 7 (Model Deflater) and the inflation of Module 8 (Section III-E): a rebuilt variant
+ * that is not in use is packed with the lossless DEFLATE format (RFC 1951) - the zeroed weights that
+ * survive the rebuild repeat - and unpacked when it is switched in.  Both calls work on plain byte
+ * buffers (a destination arena of dnns_compact, or anything else) and need no plan.
+ *
+ * dnns_deflate writes a raw RFC 1951 stream that any inflater can read.  The encoder's choices:
+ * the input is cut into chunks of DNNS_DEFLATE_CHUNK bytes, each one block (fixed Huffman codes, or
+ * stored when that is shorter) followed - except after the last - by an empty stored block, so every
+ * chunk starts on a byte boundary; inside a chunk, sub-blocks of DNNS_DEFLATE_SUB bytes are coded on
+ * their own: every run of equal bytes is a literal followed by matches at distance 1 (258 at a time,
+ * then one match of the 3..257 repeats left, else literals).  An empty input is one empty final block.
+ *   src_dev (device, 16-byte aligned, n_bytes), stream_dev (device, 16-byte aligned, capacity at
+ *   least dnns_deflate_bound(n_bytes) rounded up to 4), chunk_offset_dev (device,
+ *   dnns_deflate_chunks(n_bytes) + 1 entries: byte offset of every chunk, the last entry is the
+ *   stream's size), sub_bits_dev (device, 32 entries per chunk: bit offset, from the chunk's first
+ *   byte, of the first token of every sub-block; for a stored chunk, of its first byte), ws_dev
+ *   (device, 16-byte aligned scratch of dnns_deflate_workspace_bytes(n_bytes), contents undefined
+ *   afterwards).  Enqueues three kernels on `stream`; nothing is read back.
+ * dnns_inflate restores the n_bytes from a stream, its two index arrays and its size, all as
+ * dnns_deflate left them (stream_dev readable up to stream_bytes rounded up to 4, dst_dev 16-byte
+ * aligned).  It decodes the streams dnns_deflate writes, not arbitrary DEFLATE: a block type, symbol
+ * or distance the encoder never emits sets *status_dev (device word, cleared by the caller) to
+ * DNNS_ERR_UNSUPPORTED and leaves that sub-block incomplete; nothing traps.
+ * Errors of both: INVALID_ARG (null or misaligned pointer), WORKSPACE (capacity or scratch too
+ * small), UNSUPPORTED (more than 2^40 bytes), CUDA.
+ */
+#define DNNS_DEFLATE_CHUNK 16384
+#define DNNS_DEFLATE_SUB 512
+size_t dnns_deflate_chunks(size_t n_bytes);          /* max(1, ceil(n_bytes / DNNS_DEFLATE_CHUNK))   */
+size_t dnns_deflate_bound(size_t n_bytes);           /* largest possible stream: n_bytes + 5 * chunks */
+size_t dnns_deflate_workspace_bytes(size_t n_bytes); /* device scratch of dnns_deflate                */
+dnns_status dnns_deflate(const void* src_dev, size_t n_bytes, void* stream_dev, size_t stream_capacity,
+                         uint64_t* chunk_offset_dev, uint32_t* sub_bits_dev, void* ws_dev, size_t ws_bytes, void* stream);
+dnns_status dnns_inflate(const void* stream_dev, size_t stream_bytes, const uint64_t* chunk_offset_dev,
+                         const uint32_t* sub_bits_dev, size_t n_bytes, void* dst_dev, uint32_t* status_dev, void* stream);
+
 /* Synchronises `stream`, then returns (and clears) the status recorded by the plan's kernels. */
 dnns_status dnns_last_device_status(dnns_plan* plan, void* stream);
 

@@ -17,10 +17,12 @@ DNNS_GROUP_FROZEN = 1
 (DNNS_OK, DNNS_ERR_INVALID_ARG, DNNS_ERR_BAD_GRAPH, DNNS_ERR_WORKSPACE, DNNS_ERR_UNSUPPORTED, DNNS_ERR_CUDA,
  DNNS_ERR_TIMEOUT, DNNS_ERR_STATIC_LIMIT) = range(8)
 DNNS_STATIC_MAX_NUMEL = 1 << 26
+DNNS_DEFLATE_CHUNK, DNNS_DEFLATE_SUB = 16384, 512
 
 EXPORTS = ["dnns_status_string", "dnns_workspace_bytes", "dnns_plan_create", "dnns_plan_destroy", "dnns_plan_layout",
            "dnns_plan_launch_count", "dnns_magnitude_threshold", "dnns_apply_mask", "dnns_zero_structures",
-           "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures", "dnns_fold_batchnorm", "dnns_propagate_keep_cascade"]
+           "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures", "dnns_fold_batchnorm", "dnns_propagate_keep_cascade",
+           "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
 
 
 class dnns_tensor(C.Structure):
@@ -99,6 +101,11 @@ def lib() -> C.CDLL:
         L.dnns_fold_batchnorm.argtypes = [vp, vp, vp, vp, vp]
         L.dnns_propagate_keep_cascade.argtypes = [vp, vp, u32, i32, i32, vp, vp, vp, vp, vp]
         L.dnns_magnitude_threshold_static.argtypes = [vp, i32, u64, u64, vp, vp]
+        for name in ("dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes"):
+            getattr(L, name).restype = C.c_size_t
+            getattr(L, name).argtypes = [C.c_size_t]
+        L.dnns_deflate.argtypes = [vp, C.c_size_t, vp, C.c_size_t, vp, vp, vp, C.c_size_t, vp]
+        L.dnns_inflate.argtypes = [vp, C.c_size_t, vp, vp, C.c_size_t, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -190,3 +197,27 @@ def dnns_propagate_keep_cascade(plan, nz_map: int, policy: int, min_keep: int, m
                                 keep_idx: int, keep_count: int, stats: int, stream: int = 0) -> None:
     _check(lib().dnns_propagate_keep_cascade(plan, nz_map, policy, min_keep, max_passes, keep_bits, keep_idx,
                                              keep_count, stats or None, stream), "dnns_propagate_keep_cascade")
+
+
+def dnns_deflate_chunks(n_bytes: int) -> int:
+    return lib().dnns_deflate_chunks(n_bytes)
+
+
+def dnns_deflate_bound(n_bytes: int) -> int:
+    return lib().dnns_deflate_bound(n_bytes)
+
+
+def dnns_deflate_workspace_bytes(n_bytes: int) -> int:
+    return lib().dnns_deflate_workspace_bytes(n_bytes)
+
+
+def dnns_deflate(src_dev: int, n_bytes: int, stream_dev: int, stream_capacity: int, chunk_offset_dev: int,
+                 sub_bits_dev: int, ws_dev: int, ws_bytes: int, stream: int = 0) -> None:
+    _check(lib().dnns_deflate(src_dev or None, n_bytes, stream_dev, stream_capacity, chunk_offset_dev, sub_bits_dev,
+                              ws_dev, ws_bytes, stream), "dnns_deflate")
+
+
+def dnns_inflate(stream_dev: int, stream_bytes: int, chunk_offset_dev: int, sub_bits_dev: int, n_bytes: int,
+                 dst_dev: int, status_dev: int, stream: int = 0) -> None:
+    _check(lib().dnns_inflate(stream_dev, stream_bytes, chunk_offset_dev, sub_bits_dev, n_bytes, dst_dev or None,
+                              status_dev, stream), "dnns_inflate")

@@ -1,0 +1,468 @@
+// Deflation of inactive variants - Phase 3, Module 7 (Model Deflater) and the inflation of
+// Module 8 (Section III-E): a rebuilt variant still holds the zeroed weights of its surviving
+// channels, and those repeat, so the variant is packed as a DEFLATE stream (RFC 1951) while it is
+// not in use and unpacked when it is switched in.
+//
+// The stream is plain RFC 1951 (any inflater reads it); the encoder's free choices are made so
+// that both directions run in parallel:
+//   chunk      16384 input bytes = one block (fixed Huffman codes, or stored when that is shorter),
+//              followed - unless it is the last - by an empty stored block, which puts the next
+//              chunk on a byte boundary;
+//   sub-block  512 input bytes: runs of equal bytes are coded as a literal plus matches at
+//              distance 1 and never reach back across the start of a sub-block.
+// One warp takes a chunk, one lane a sub-block.  Beside the stream the encoder writes the byte
+// offset of every chunk and the bit offset of every sub-block, which is all the decoder needs to
+// start 32 lanes per chunk at once.
+//
+//   k_deflate_encode  per chunk: count the bits of every sub-block, scan, write the bits into a
+//                     shared-memory image of the block, copy it to the chunk's slot of the workspace;
+//   k_deflate_scan    exclusive scan of the chunk sizes -> chunk offsets;
+//   k_deflate_pack    moves every slot to its byte offset in the stream;
+//   k_inflate         per chunk: every lane decodes its sub-block straight into the destination.
+#include "dnns_internal.cuh"
+
+namespace dnns {
+
+namespace {
+
+constexpr uint32_t kChunk = DNNS_DEFLATE_CHUNK;
+constexpr uint32_t kSub = DNNS_DEFLATE_SUB;
+constexpr uint32_t kSubs = kChunk / kSub;           // 32: one lane each
+constexpr uint32_t kSlotBytes = kChunk + 32;        // image of one chunk: at most 5 + 16384 bytes, padded
+constexpr uint32_t kSlotWords = kSlotBytes / 4;
+constexpr int kWarpsPerBlock = 4;
+constexpr unsigned kFull = 0xffffffffu;
+
+static_assert(kSubs == 32, "one lane per sub-block");
+
+// ---- token costs and codes (RFC 1951, sections 3.2.5 and 3.2.6) ----
+__device__ __forceinline__ uint32_t literal_bits(uint32_t v) { return v < 144 ? 8u : 9u; }
+
+// A match of `len` (3..258) at distance 1: Huffman code of the length symbol (most significant bit
+// first, hence reversed here), its extra bits, then the 5-bit distance code 0.  Returns the bit
+// string (first bit = bit 0) and its length.
+__device__ __forceinline__ uint32_t match_code(uint32_t len, uint32_t& n_bits) {
+    const uint32_t x = len - 3;
+    uint32_t sym, e = 0, extra = 0;
+    if (len == 258) {
+        sym = 285;
+    } else if (x < 8) {
+        sym = 257 + x;
+    } else {
+        e = (31 - __clz(x)) - 2;               // lengths come in groups of four codes per power of two
+        sym = 257 + 4 * (e + 1) + ((x >> e) & 3u);
+        extra = x & ((1u << e) - 1u);
+    }
+    uint32_t code, nb;
+    if (sym <= 279) code = sym - 256, nb = 7;
+    else code = 0xC0 + (sym - 280), nb = 8;
+    n_bits = nb + e + 5;
+    return (__brev(code) >> (32 - nb)) | (extra << nb);
+}
+
+__device__ __forceinline__ uint32_t literal_code(uint32_t v, uint32_t& n_bits) {
+    if (v < 144) {
+        n_bits = 8;
+        return __brev(0x30 + v) >> 24;
+    }
+    n_bits = 9;
+    return __brev(0x190 + (v - 144)) >> 23;
+}
+
+struct CountSink {
+    uint32_t bits = 0;
+    __device__ __forceinline__ void literal(uint32_t v, uint32_t times) { bits += times * literal_bits(v); }
+    __device__ __forceinline__ void match(uint32_t len) {
+        uint32_t n;
+        match_code(len, n);
+        bits += n;
+    }
+};
+
+// Appends bit strings at a bit position of a zeroed shared-memory image.  Neighbouring lanes
+// share the words at their borders, so words are merged with atomicOr.
+struct WriteSink {
+    uint32_t* words;
+    uint32_t widx, fill;
+    uint64_t acc = 0;
+    __device__ __forceinline__ WriteSink(uint32_t* w, uint32_t bit_pos) : words(w), widx(bit_pos >> 5), fill(bit_pos & 31) {}
+    __device__ __forceinline__ void put(uint32_t v, uint32_t n) {
+        acc |= (uint64_t)v << fill;
+        fill += n;
+        if (fill >= 32) {
+            atomicOr(&words[widx++], (uint32_t)acc);
+            acc >>= 32;
+            fill -= 32;
+        }
+    }
+    __device__ __forceinline__ void literal(uint32_t v, uint32_t times) {
+        uint32_t n;
+        const uint32_t c = literal_code(v, n);
+        for (uint32_t t = 0; t < times; ++t) put(c, n);
+    }
+    __device__ __forceinline__ void match(uint32_t len) {
+        uint32_t n;
+        const uint32_t c = match_code(len, n);
+        put(c, n);
+    }
+    __device__ __forceinline__ void finish() {
+        if (fill) atomicOr(&words[widx], (uint32_t)acc);
+    }
+};
+
+// A run of `len` equal bytes: one literal, then its repeats as matches of 258, one shorter match
+// when at least 3 repeats remain, else literals.
+template <typename Sink>
+__device__ __forceinline__ void emit_run(Sink& s, uint32_t v, uint32_t len) {
+    uint32_t rep = len - 1;
+    s.literal(v, 1);
+    while (rep >= 258) {
+        s.match(258);
+        rep -= 258;
+    }
+    if (rep >= 3) s.match(rep);
+    else if (rep) s.literal(v, rep);
+}
+
+// Walk the n (<= 512) bytes of a sub-block at p (16-byte aligned) and hand its runs to the sink.
+template <typename Sink>
+__device__ __forceinline__ void parse_sub_block(Sink& s, const uint8_t* p, uint32_t n) {
+    uint32_t run_val = 0, run_len = 0;
+    for (uint32_t i = 0; i < n; i += 16) {
+        uint32_t w[4];
+        if (i + 16 <= n) {
+            const uint4 q = __ldg(reinterpret_cast<const uint4*>(p + i));
+            w[0] = q.x, w[1] = q.y, w[2] = q.z, w[3] = q.w;
+            const uint32_t splat = run_val * 0x01010101u;
+            if (run_len && w[0] == splat && w[1] == splat && w[2] == splat && w[3] == splat) {
+                run_len += 16;  // sixteen more of the same (long runs of zeros are the common case)
+                continue;
+            }
+        } else {
+            w[0] = w[1] = w[2] = w[3] = 0;
+            for (uint32_t j = 0; i + j < n; ++j) w[j >> 2] |= (uint32_t)p[i + j] << (8 * (j & 3));
+        }
+        const uint32_t m = min(16u, n - i);
+        for (uint32_t j = 0; j < m; ++j) {
+            const uint32_t b = (w[j >> 2] >> (8 * (j & 3))) & 0xFFu;
+            if (run_len && b == run_val) {
+                ++run_len;
+            } else {
+                if (run_len) emit_run(s, run_val, run_len);
+                run_val = b;
+                run_len = 1;
+            }
+        }
+    }
+    if (run_len) emit_run(s, run_val, run_len);
+}
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32) k_deflate_encode(const uint8_t* __restrict__ src, uint64_t n_bytes,
+                                                                         uint32_t n_chunks, uint8_t* slots,
+                                                                         uint32_t* sizes, uint32_t* sub_bits) {
+    extern __shared__ uint32_t sh_img[];  // kWarpsPerBlock images of kSlotWords words
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t* img = sh_img + warp * kSlotWords;
+    for (uint32_t c = blockIdx.x * kWarpsPerBlock + warp; c < n_chunks; c += gridDim.x * kWarpsPerBlock) {
+        const uint64_t c0 = (uint64_t)c * kChunk;
+        const uint32_t n = (uint32_t)min((uint64_t)kChunk, n_bytes - c0);  // an empty input has one chunk of 0 bytes
+        const bool last = c + 1 == n_chunks;
+        const uint32_t lo = min(n, lane * kSub), n_lane = min(n - lo, kSub);
+        const uint8_t* p = src + c0 + lo;
+
+        CountSink cnt;
+        parse_sub_block(cnt, p, n_lane);
+        uint32_t incl = cnt.bits;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(kFull, incl, d);
+            if (lane >= d) incl += y;
+        }
+        const uint32_t tokens = __shfl_sync(kFull, incl, 31);
+        const uint32_t start = 3 + incl - cnt.bits;       // after the 3 header bits
+        const uint32_t block_bits = 3 + tokens + 7;       // header, tokens, end-of-block symbol
+        const uint32_t fixed_bytes = last ? (block_bits + 7) / 8 : (block_bits + 3 + 7) / 8 + 4;
+        const uint32_t stored_bytes = 5 + n;
+        const bool fixed = fixed_bytes <= stored_bytes;
+        const uint32_t bytes = fixed ? fixed_bytes : stored_bytes;
+        const uint32_t words = (bytes + 3) / 4;
+
+        for (uint32_t i = lane; i < words + 1; i += 32) img[i] = 0;
+        __syncwarp();
+        if (fixed) {
+            WriteSink wr(img, start);
+            if (lane == 0) atomicOr(&img[0], (last ? 1u : 0u) | 2u);  // BFINAL, BTYPE = 01 (low bit first)
+            parse_sub_block(wr, p, n_lane);
+            wr.finish();
+            // the end-of-block symbol and the empty stored block's header are zero bits: already there
+            if (!last && lane == 0) {
+                const uint32_t at = bytes - 2;            // NLEN = 0xFFFF closes the empty stored block
+                atomicOr(&img[at >> 2], 0xFFu << (8 * (at & 3)));
+                atomicOr(&img[(at + 1) >> 2], 0xFFu << (8 * ((at + 1) & 3)));
+            }
+            sub_bits[(size_t)c * kSubs + lane] = start;
+        } else {
+            uint8_t* b = reinterpret_cast<uint8_t*>(img);
+            if (lane == 0) {
+                b[0] = last ? 1 : 0;                      // BFINAL, BTYPE = 00, padding
+                b[1] = (uint8_t)n, b[2] = (uint8_t)(n >> 8);
+                b[3] = (uint8_t)~n, b[4] = (uint8_t)(~n >> 8);
+            }
+            for (uint32_t i = lane * 16; i < n; i += 32 * 16) {
+                if (i + 16 <= n) {
+                    const uint4 q = __ldg(reinterpret_cast<const uint4*>(src + c0 + i));
+                    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+                    for (int j = 0; j < 16; ++j) b[5 + i + j] = (uint8_t)(w[j >> 2] >> (8 * (j & 3)));
+                } else {
+                    for (uint32_t j = i; j < n; ++j) b[5 + j] = src[c0 + j];
+                }
+            }
+            sub_bits[(size_t)c * kSubs + lane] = 8 * (5 + lo);
+        }
+        __syncwarp();
+        uint32_t* slot = reinterpret_cast<uint32_t*>(slots + (size_t)c * kSlotBytes);
+        for (uint32_t i = lane; i < words + 1; i += 32) slot[i] = img[i];
+        if (lane == 0) sizes[c] = bytes;
+        __syncwarp();
+    }
+}
+
+__global__ void __launch_bounds__(1024) k_deflate_scan(const uint32_t* __restrict__ sizes, uint32_t n_chunks,
+                                                       uint64_t* chunk_offset) {
+    __shared__ uint64_t scratch[33];
+    uint64_t carry = 0;
+    for (uint32_t base = 0; base < n_chunks; base += 1024) {
+        const uint32_t i = base + threadIdx.x;
+        const uint64_t x = i < n_chunks ? sizes[i] : 0;
+        uint64_t total;
+        const uint64_t ex = block_exclusive_scan<uint64_t>(x, scratch, &total);
+        if (i < n_chunks) chunk_offset[i] = carry + ex;
+        carry += total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) chunk_offset[n_chunks] = carry;
+}
+
+// Word j of a byte string that starts `shift` bytes into aligned word array w.
+__device__ __forceinline__ uint32_t unaligned_word(const uint32_t* w, uint32_t j, uint32_t shift) {
+    return shift ? __funnelshift_r(w[j], w[j + 1], 8 * shift) : w[j];
+}
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32) k_deflate_pack(const uint8_t* __restrict__ slots,
+                                                                       const uint32_t* __restrict__ sizes,
+                                                                       const uint64_t* __restrict__ chunk_offset,
+                                                                       uint32_t n_chunks, uint8_t* stream) {
+    const int lane = threadIdx.x & 31;
+    for (uint32_t c = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); c < n_chunks; c += gridDim.x * kWarpsPerBlock) {
+        const uint32_t* slot = reinterpret_cast<const uint32_t*>(slots + (size_t)c * kSlotBytes);
+        const uint8_t* slot_b = reinterpret_cast<const uint8_t*>(slot);
+        const uint32_t n = sizes[c];
+        uint8_t* d = stream + chunk_offset[c];
+        // bytes up to the first aligned destination word, then whole words, then the rest
+        const uint32_t head = min(n, (uint32_t)((4 - (reinterpret_cast<uintptr_t>(d) & 3)) & 3));
+        if ((uint32_t)lane < head) d[lane] = slot_b[lane];
+        const uint32_t n_words = (n - head) / 4;
+        uint32_t* dw = reinterpret_cast<uint32_t*>(d + head);
+        for (uint32_t j = lane; j < n_words; j += 32) dw[j] = unaligned_word(slot, j, head);  // the slot has a spare word
+        const uint32_t done = head + 4 * n_words;
+        if (done + lane < n) d[done + lane] = slot_b[done + lane];
+    }
+}
+
+// One lane's output: bytes gathered into 16-byte vectors and stored into its own 512 bytes.
+struct ByteOut {
+    uint8_t* dst;
+    uint32_t n = 0;
+    uint32_t w[4] = {0, 0, 0, 0};
+    __device__ __forceinline__ explicit ByteOut(uint8_t* d) : dst(d) {}
+    __device__ __forceinline__ void push(uint32_t b) {
+        const uint32_t k = n & 15;
+        const uint32_t v = b << (8 * (k & 3));
+        if ((k >> 2) == 0) w[0] |= v;
+        else if ((k >> 2) == 1) w[1] |= v;
+        else if ((k >> 2) == 2) w[2] |= v;
+        else w[3] |= v;
+        if ((++n & 15) == 0) {
+            *reinterpret_cast<uint4*>(dst + n - 16) = make_uint4(w[0], w[1], w[2], w[3]);
+            w[0] = w[1] = w[2] = w[3] = 0;
+        }
+    }
+    __device__ __forceinline__ void repeat(uint32_t b, uint32_t times) {
+        while (times && (n & 15)) push(b), --times;
+        const uint32_t s = b * 0x01010101u;
+        for (; times >= 16; times -= 16, n += 16) *reinterpret_cast<uint4*>(dst + n) = make_uint4(s, s, s, s);
+        while (times) push(b), --times;
+    }
+    __device__ __forceinline__ void finish() {  // the last sub-block of the data may end inside a vector
+        const uint32_t k = n & 15;
+        for (uint32_t j = 0; j < k; ++j) dst[n - k + j] = (uint8_t)(w[j >> 2] >> (8 * (j & 3)));
+    }
+};
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32) k_inflate(const uint32_t* __restrict__ stream_w, uint64_t stream_bytes,
+                                                                  const uint64_t* __restrict__ chunk_offset,
+                                                                  const uint32_t* __restrict__ sub_bits, uint64_t n_bytes,
+                                                                  uint32_t n_chunks, uint8_t* dst, uint32_t* status) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t n_words = (stream_bytes + 3) / 4;
+    auto word = [&](uint64_t i) -> uint32_t { return i < n_words ? __ldg(stream_w + i) : 0u; };
+    auto fail = [&]() { atomicCAS(status, 0u, (uint32_t)DNNS_ERR_UNSUPPORTED); };
+    for (uint32_t c = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); c < n_chunks; c += gridDim.x * kWarpsPerBlock) {
+        const uint64_t c0 = (uint64_t)c * kChunk;
+        const uint32_t n = (uint32_t)min((uint64_t)kChunk, n_bytes - c0);
+        const uint32_t lo = min(n, lane * kSub), n_lane = min(n - lo, kSub);
+        const uint64_t off = chunk_offset[c];
+        if (off >= stream_bytes) {
+            fail();
+            continue;
+        }
+        const uint32_t type = ((word(off >> 2) >> (8 * (off & 3))) >> 1) & 3u;
+        uint8_t* out = dst + c0 + lo;
+        if (type == 0) {
+            // stored: the lane's bytes start 5 + lo bytes into the chunk
+            const uint64_t a = off + 5 + lo;
+            const uint32_t shift = (uint32_t)(a & 3);
+            const uint64_t w0 = a >> 2;
+            for (uint32_t j = 0; j < n_lane / 4; ++j) {
+                const uint32_t x = shift ? __funnelshift_r(word(w0 + j), word(w0 + j + 1), 8 * shift) : word(w0 + j);
+                reinterpret_cast<uint32_t*>(out)[j] = x;
+            }
+            for (uint32_t j = n_lane & ~3u; j < n_lane; ++j) {
+                const uint64_t b = a + j;
+                out[j] = (uint8_t)(word(b >> 2) >> (8 * (b & 3)));
+            }
+            continue;
+        }
+        if (type != 1) {
+            fail();
+            continue;
+        }
+        // fixed Huffman codes: the lane reads tokens from its bit offset until its bytes are there
+        const uint64_t pos = off * 8 + sub_bits[(size_t)c * kSubs + lane];
+        uint64_t wi = pos >> 5;
+        uint64_t buf = (uint64_t)word(wi) >> (pos & 31);
+        uint32_t have = 32 - (uint32_t)(pos & 31);
+        ByteOut bo(out);
+        uint32_t prev = 0;
+        bool ok = true;
+        while (bo.n < n_lane) {
+            if (have <= 32) {
+                buf |= (uint64_t)word(++wi) << have;
+                have += 32;
+            }
+            const uint32_t code9 = __brev((uint32_t)buf) >> 23;  // the next 9 bits as a code, first bit on top
+            uint32_t sym, used;
+            if ((code9 >> 2) <= 0x17) sym = 256 + (code9 >> 2), used = 7;
+            else if ((code9 >> 1) <= 0xBF) sym = (code9 >> 1) - 0x30, used = 8;
+            else if ((code9 >> 1) <= 0xC7) sym = 280 + (code9 >> 1) - 0xC0, used = 8;
+            else sym = 144 + code9 - 0x190, used = 9;
+            if (sym < 256) {
+                buf >>= used, have -= used;
+                bo.push(sym);
+                prev = sym;
+                continue;
+            }
+            const uint32_t idx = sym - 257;
+            if (sym == 256 || idx > 28 || bo.n == 0) {  // early end of block, unassigned symbol, nothing to repeat
+                ok = false;
+                break;
+            }
+            uint32_t len, e = 0;
+            if (idx < 8) len = 3 + idx;
+            else if (idx == 28) len = 258;
+            else {
+                e = (idx >> 2) - 1;
+                len = 3 + ((4 + (idx & 3)) << e);
+            }
+            const uint32_t rest = (uint32_t)(buf >> used);
+            len += rest & ((1u << e) - 1u);
+            const uint32_t dist_code = (rest >> e) & 31u;
+            used += e + 5;
+            if (dist_code != 0 || bo.n + len > n_lane) {  // only distance 1 is decoded here
+                ok = false;
+                break;
+            }
+            buf >>= used, have -= used;
+            bo.repeat(prev, len);
+        }
+        bo.finish();
+        if (!ok) fail();
+    }
+}
+
+int launch_deflate(const void* src, uint64_t n_bytes, uint32_t n_chunks, void* stream_out, uint64_t* chunk_offset,
+                   uint32_t* sub_bits, void* ws, int n_sm, cudaStream_t st) {
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+    constexpr int smem = kWarpsPerBlock * kSlotBytes;
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(k_deflate_encode, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -1;
+        attr_set[dev] = true;
+    }
+    uint8_t* slots = static_cast<uint8_t*>(ws);
+    uint32_t* sizes = reinterpret_cast<uint32_t*>(slots + (size_t)n_chunks * kSlotBytes);
+    const uint32_t blocks = (n_chunks + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const uint32_t grid = min(blocks, (uint32_t)n_sm * 3u * 8u);
+    k_deflate_encode<<<grid, kWarpsPerBlock * 32, smem, st>>>(static_cast<const uint8_t*>(src), n_bytes, n_chunks, slots,
+                                                              sizes, sub_bits);
+    k_deflate_scan<<<1, 1024, 0, st>>>(sizes, n_chunks, chunk_offset);
+    k_deflate_pack<<<grid, kWarpsPerBlock * 32, 0, st>>>(slots, sizes, chunk_offset, n_chunks,
+                                                         static_cast<uint8_t*>(stream_out));
+    return cudaGetLastError() == cudaSuccess ? 3 : -1;
+}
+
+size_t deflate_workspace_bytes(uint32_t n_chunks) { return (size_t)n_chunks * kSlotBytes + (((size_t)n_chunks * 4 + 255) & ~(size_t)255); }
+
+int launch_inflate(const void* stream_in, uint64_t stream_bytes, const uint64_t* chunk_offset, const uint32_t* sub_bits,
+                   uint64_t n_bytes, uint32_t n_chunks, void* dst, uint32_t* status, cudaStream_t st) {
+    const uint32_t blocks = (n_chunks + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    k_inflate<<<blocks, kWarpsPerBlock * 32, 0, st>>>(static_cast<const uint32_t*>(stream_in), stream_bytes, chunk_offset,
+                                                      sub_bits, n_bytes, n_chunks, static_cast<uint8_t*>(dst), status);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+}  // namespace
+
+}  // namespace dnns
+
+extern "C" {
+
+size_t dnns_deflate_chunks(size_t n_bytes) { return n_bytes == 0 ? 1 : (n_bytes + DNNS_DEFLATE_CHUNK - 1) / DNNS_DEFLATE_CHUNK; }
+
+size_t dnns_deflate_bound(size_t n_bytes) { return n_bytes + 5 * dnns_deflate_chunks(n_bytes); }
+
+size_t dnns_deflate_workspace_bytes(size_t n_bytes) {
+    return dnns::deflate_workspace_bytes((uint32_t)dnns_deflate_chunks(n_bytes));
+}
+
+static bool deflate_size_ok(size_t n_bytes) { return n_bytes <= ((size_t)1 << 40); }
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+dnns_status dnns_deflate(const void* src_dev, size_t n_bytes, void* stream_dev, size_t stream_capacity,
+                         uint64_t* chunk_offset_dev, uint32_t* sub_bits_dev, void* ws_dev, size_t ws_bytes, void* stream) {
+    if (!stream_dev || !chunk_offset_dev || !sub_bits_dev || !ws_dev || (n_bytes && !src_dev)) return DNNS_ERR_INVALID_ARG;
+    if (!aligned16(src_dev) || !aligned16(stream_dev) || !aligned16(ws_dev)) return DNNS_ERR_INVALID_ARG;
+    if (!deflate_size_ok(n_bytes)) return DNNS_ERR_UNSUPPORTED;
+    if (stream_capacity < ((dnns_deflate_bound(n_bytes) + 3) & ~(size_t)3) || ws_bytes < dnns_deflate_workspace_bytes(n_bytes))
+        return DNNS_ERR_WORKSPACE;
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return DNNS_ERR_CUDA;
+    const int n = dnns::launch_deflate(src_dev, n_bytes, (uint32_t)dnns_deflate_chunks(n_bytes), stream_dev, chunk_offset_dev,
+                                       sub_bits_dev, ws_dev, n_sm, static_cast<cudaStream_t>(stream));
+    return n < 0 ? DNNS_ERR_CUDA : DNNS_OK;
+}
+
+dnns_status dnns_inflate(const void* stream_dev, size_t stream_bytes, const uint64_t* chunk_offset_dev,
+                         const uint32_t* sub_bits_dev, size_t n_bytes, void* dst_dev, uint32_t* status_dev, void* stream) {
+    if (!stream_dev || !chunk_offset_dev || !sub_bits_dev || !status_dev || (n_bytes && !dst_dev)) return DNNS_ERR_INVALID_ARG;
+    if (!aligned16(stream_dev) || !aligned16(dst_dev) || stream_bytes == 0) return DNNS_ERR_INVALID_ARG;
+    if (!deflate_size_ok(n_bytes)) return DNNS_ERR_UNSUPPORTED;
+    const int n = dnns::launch_inflate(stream_dev, stream_bytes, chunk_offset_dev, sub_bits_dev, n_bytes,
+                                       (uint32_t)dnns_deflate_chunks(n_bytes), dst_dev, status_dev,
+                                       static_cast<cudaStream_t>(stream));
+    return n < 0 ? DNNS_ERR_CUDA : DNNS_OK;
+}
+
+}  // extern "C"

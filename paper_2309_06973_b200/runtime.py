@@ -253,3 +253,39 @@ class Session:
                 biases.append(raw[int(offs[k]): int(offs[k]) + 4 * On].view(np.float32).copy())
                 k += 1
         return ws, bns, biases, shapes, offs.copy()
+
+
+class Deflater:
+    """Buffers for dnns_deflate / dnns_inflate of byte strings of up to `max_bytes` (device memory only)."""
+
+    def __init__(self, max_bytes: int, device="cuda:0"):
+        self.device, self.max_bytes = torch.device(device), max_bytes
+        nc = B.dnns_deflate_chunks(max_bytes)
+        u8 = lambda n: torch.empty(max(int(n), 16), dtype=torch.uint8, device=self.device)
+        self.capacity = (B.dnns_deflate_bound(max_bytes) + 3) // 4 * 4
+        self.stream = u8(self.capacity)
+        self.ws_bytes = B.dnns_deflate_workspace_bytes(max_bytes)
+        self.ws = u8(self.ws_bytes)
+        self.chunk_offset = torch.zeros(nc + 1, dtype=torch.int64, device=self.device)
+        self.sub_bits = torch.zeros(32 * nc, dtype=torch.int32, device=self.device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
+        self.n_bytes = 0
+
+    def deflate(self, src: torch.Tensor, n_bytes: int):
+        assert n_bytes <= self.max_bytes
+        self.n_bytes = n_bytes
+        B.dnns_deflate(src.data_ptr() if n_bytes else 0, n_bytes, self.stream.data_ptr(), self.capacity,
+                       self.chunk_offset.data_ptr(), self.sub_bits.data_ptr(), self.ws.data_ptr(), self.ws_bytes, _stream())
+
+    def stream_bytes(self) -> int:
+        """Size of the latest stream (synchronises: the size is computed on the device)."""
+        return int(self.chunk_offset[B.dnns_deflate_chunks(self.n_bytes)].item())
+
+    def inflate(self, dst: torch.Tensor, stream_bytes: int):
+        B.dnns_inflate(self.stream.data_ptr(), stream_bytes, self.chunk_offset.data_ptr(), self.sub_bits.data_ptr(),
+                       self.n_bytes, dst.data_ptr() if self.n_bytes else 0, self.status.data_ptr(), _stream())
+
+    def index(self):
+        nc = B.dnns_deflate_chunks(self.n_bytes)
+        return (self.chunk_offset[: nc + 1].cpu().numpy().view(np.uint64).copy(),
+                self.sub_bits[: 32 * nc].cpu().numpy().view(np.uint32).copy())
