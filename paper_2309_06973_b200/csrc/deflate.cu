@@ -14,8 +14,8 @@
 // offset of every chunk and the bit offset of every sub-block, which is all the decoder needs to
 // start 32 lanes per chunk at once.
 //
-//   k_deflate_encode  per chunk: count the bits of every sub-block, scan, write the bits into a
-//                     shared-memory image of the block, copy it to the chunk's slot of the workspace;
+//   k_deflate_encode  per chunk: count the bits of every sub-block, scan, then write the bits into the
+//                     chunk's (zeroed) slot of the workspace;
 //   k_deflate_scan    exclusive scan of the chunk sizes -> chunk offsets;
 //   k_deflate_pack    moves every slot to its byte offset in the stream;
 //   k_inflate         per chunk: every lane decodes its sub-block straight into the destination.
@@ -29,7 +29,6 @@ constexpr uint32_t kChunk = DNNS_DEFLATE_CHUNK;
 constexpr uint32_t kSub = DNNS_DEFLATE_SUB;
 constexpr uint32_t kSubs = kChunk / kSub;           // 32: one lane each
 constexpr uint32_t kSlotBytes = kChunk + 32;        // image of one chunk: at most 5 + 16384 bytes, padded
-constexpr uint32_t kSlotWords = kSlotBytes / 4;
 constexpr int kWarpsPerBlock = 4;
 constexpr unsigned kFull = 0xffffffffu;
 
@@ -79,8 +78,8 @@ struct CountSink {
     }
 };
 
-// Appends bit strings at a bit position of a zeroed shared-memory image.  Neighbouring lanes
-// share the words at their borders, so words are merged with atomicOr.
+// Appends bit strings at a bit position of a zeroed image of the block.  Neighbouring lanes
+// share the words at their borders, so words are merged with atomicOr (no value comes back).
 struct WriteSink {
     uint32_t* words;
     uint32_t widx, fill;
@@ -125,44 +124,54 @@ __device__ __forceinline__ void emit_run(Sink& s, uint32_t v, uint32_t len) {
 }
 
 // Walk the n (<= 512) bytes of a sub-block at p (16-byte aligned) and hand its runs to the sink.
+// The next 16 bytes are requested before the current ones are walked.
 template <typename Sink>
 __device__ __forceinline__ void parse_sub_block(Sink& s, const uint8_t* p, uint32_t n) {
     uint32_t run_val = 0, run_len = 0;
-    for (uint32_t i = 0; i < n; i += 16) {
-        uint32_t w[4];
-        if (i + 16 <= n) {
-            const uint4 q = __ldg(reinterpret_cast<const uint4*>(p + i));
-            w[0] = q.x, w[1] = q.y, w[2] = q.z, w[3] = q.w;
-            const uint32_t splat = run_val * 0x01010101u;
-            if (run_len && w[0] == splat && w[1] == splat && w[2] == splat && w[3] == splat) {
-                run_len += 16;  // sixteen more of the same (long runs of zeros are the common case)
-                continue;
-            }
+    auto step = [&](uint32_t b) {
+        if (run_len && b == run_val) {
+            ++run_len;
         } else {
-            w[0] = w[1] = w[2] = w[3] = 0;
-            for (uint32_t j = 0; i + j < n; ++j) w[j >> 2] |= (uint32_t)p[i + j] << (8 * (j & 3));
+            if (run_len) emit_run(s, run_val, run_len);
+            run_val = b;
+            run_len = 1;
         }
-        const uint32_t m = min(16u, n - i);
-        for (uint32_t j = 0; j < m; ++j) {
-            const uint32_t b = (w[j >> 2] >> (8 * (j & 3))) & 0xFFu;
-            if (run_len && b == run_val) {
-                ++run_len;
-            } else {
-                if (run_len) emit_run(s, run_val, run_len);
-                run_val = b;
-                run_len = 1;
-            }
+    };
+    const uint32_t n_vec = n / 16;
+    const uint4* pv = reinterpret_cast<const uint4*>(p);
+    uint4 nxt = n_vec ? __ldg(pv) : make_uint4(0, 0, 0, 0);
+    for (uint32_t v = 0; v < n_vec; ++v) {
+        const uint4 q = nxt;
+        if (v + 1 < n_vec) nxt = __ldg(pv + v + 1);
+        const uint32_t splat = run_val * 0x01010101u;
+        if (run_len && q.x == splat && q.y == splat && q.z == splat && q.w == splat) {
+            run_len += 16;  // sixteen more of the same (long runs of zeros are the common case)
+            continue;
+        }
+        uint32_t w0 = q.x, w1 = q.y, w2 = q.z, w3 = q.w;
+#pragma unroll 1
+        for (uint32_t j = 0; j < 16; ++j) {
+            step(w0 & 0xFFu);
+            w0 >>= 8;
+            if ((j & 3) == 3) w0 = w1, w1 = w2, w2 = w3;
         }
     }
+    for (uint32_t i = n_vec * 16; i < n; ++i) step(p[i]);  // only the very end of the data
     if (run_len) emit_run(s, run_val, run_len);
+}
+
+// Bytes [4k, 4k+4) of a chunk of n bytes at p (4-byte aligned) as a word; bytes past the end read as 0.
+__device__ __forceinline__ uint32_t chunk_word(const uint8_t* p, uint32_t n, uint32_t k) {
+    if (4 * k + 4 <= n) return __ldg(reinterpret_cast<const uint32_t*>(p) + k);
+    uint32_t w = 0;
+    for (uint32_t j = 4 * k; j < n; ++j) w |= (uint32_t)p[j] << (8 * (j & 3));
+    return w;
 }
 
 __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_deflate_encode(const uint8_t* __restrict__ src, uint64_t n_bytes,
                                                                          uint32_t n_chunks, uint8_t* slots,
                                                                          uint32_t* sizes, uint32_t* sub_bits) {
-    extern __shared__ uint32_t sh_img[];  // kWarpsPerBlock images of kSlotWords words
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t* img = sh_img + warp * kSlotWords;
     for (uint32_t c = blockIdx.x * kWarpsPerBlock + warp; c < n_chunks; c += gridDim.x * kWarpsPerBlock) {
         const uint64_t c0 = (uint64_t)c * kChunk;
         const uint32_t n = (uint32_t)min((uint64_t)kChunk, n_bytes - c0);  // an empty input has one chunk of 0 bytes
@@ -186,10 +195,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_deflate_encode(const ui
         const bool fixed = fixed_bytes <= stored_bytes;
         const uint32_t bytes = fixed ? fixed_bytes : stored_bytes;
         const uint32_t words = (bytes + 3) / 4;
+        uint32_t* img = reinterpret_cast<uint32_t*>(slots + (size_t)c * kSlotBytes);  // the chunk's slot
 
-        for (uint32_t i = lane; i < words + 1; i += 32) img[i] = 0;
-        __syncwarp();
         if (fixed) {
+            for (uint32_t i = lane; i < words + 1; i += 32) img[i] = 0;
+            __syncwarp();  // orders the zeroes before the other lanes' ORs
             WriteSink wr(img, start);
             if (lane == 0) atomicOr(&img[0], (last ? 1u : 0u) | 2u);  // BFINAL, BTYPE = 01 (low bit first)
             parse_sub_block(wr, p, n_lane);
@@ -202,28 +212,20 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_deflate_encode(const ui
             }
             sub_bits[(size_t)c * kSubs + lane] = start;
         } else {
-            uint8_t* b = reinterpret_cast<uint8_t*>(img);
-            if (lane == 0) {
-                b[0] = last ? 1 : 0;                      // BFINAL, BTYPE = 00, padding
-                b[1] = (uint8_t)n, b[2] = (uint8_t)(n >> 8);
-                b[3] = (uint8_t)~n, b[4] = (uint8_t)(~n >> 8);
-            }
-            for (uint32_t i = lane * 16; i < n; i += 32 * 16) {
-                if (i + 16 <= n) {
-                    const uint4 q = __ldg(reinterpret_cast<const uint4*>(src + c0 + i));
-                    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-                    for (int j = 0; j < 16; ++j) b[5 + i + j] = (uint8_t)(w[j >> 2] >> (8 * (j & 3)));
-                } else {
-                    for (uint32_t j = i; j < n; ++j) b[5 + j] = src[c0 + j];
-                }
+            // stored: BFINAL / BTYPE 00 / padding in one byte, LEN, NLEN, then the chunk's bytes, which
+            // sit 5 bytes into the image: image word j holds chunk bytes [4j - 5, 4j - 1)
+            const uint8_t* q = src + c0;
+            const uint32_t len = n & 0xFFFFu, nlen = ~n & 0xFFFFu;
+            for (uint32_t j = lane; j < words + 1; j += 32) {
+                uint32_t w;
+                if (j == 0) w = (last ? 1u : 0u) | (len << 8) | (nlen << 24);
+                else if (j == 1) w = (nlen >> 8) | (chunk_word(q, n, 0) << 8);
+                else w = __funnelshift_r(chunk_word(q, n, j - 2), chunk_word(q, n, j - 1), 24);
+                img[j] = w;
             }
             sub_bits[(size_t)c * kSubs + lane] = 8 * (5 + lo);
         }
-        __syncwarp();
-        uint32_t* slot = reinterpret_cast<uint32_t*>(slots + (size_t)c * kSlotBytes);
-        for (uint32_t i = lane; i < words + 1; i += 32) slot[i] = img[i];
         if (lane == 0) sizes[c] = bytes;
-        __syncwarp();
     }
 }
 
@@ -269,33 +271,20 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_deflate_pack(const uint
     }
 }
 
-// One lane's output: bytes gathered into 16-byte vectors and stored into its own 512 bytes.
+// One lane's output, written straight into its own 512 bytes of the destination (16-byte aligned):
+// literals byte by byte, repeats as words and vectors once aligned.  L2 merges the partial lines.
 struct ByteOut {
     uint8_t* dst;
     uint32_t n = 0;
-    uint32_t w[4] = {0, 0, 0, 0};
     __device__ __forceinline__ explicit ByteOut(uint8_t* d) : dst(d) {}
-    __device__ __forceinline__ void push(uint32_t b) {
-        const uint32_t k = n & 15;
-        const uint32_t v = b << (8 * (k & 3));
-        if ((k >> 2) == 0) w[0] |= v;
-        else if ((k >> 2) == 1) w[1] |= v;
-        else if ((k >> 2) == 2) w[2] |= v;
-        else w[3] |= v;
-        if ((++n & 15) == 0) {
-            *reinterpret_cast<uint4*>(dst + n - 16) = make_uint4(w[0], w[1], w[2], w[3]);
-            w[0] = w[1] = w[2] = w[3] = 0;
-        }
-    }
+    __device__ __forceinline__ void push(uint32_t b) { dst[n++] = (uint8_t)b; }
     __device__ __forceinline__ void repeat(uint32_t b, uint32_t times) {
-        while (times && (n & 15)) push(b), --times;
+        while (times && (n & 3)) dst[n++] = (uint8_t)b, --times;
         const uint32_t s = b * 0x01010101u;
+        while (times >= 4 && (n & 15)) *reinterpret_cast<uint32_t*>(dst + n) = s, n += 4, times -= 4;
         for (; times >= 16; times -= 16, n += 16) *reinterpret_cast<uint4*>(dst + n) = make_uint4(s, s, s, s);
-        while (times) push(b), --times;
-    }
-    __device__ __forceinline__ void finish() {  // the last sub-block of the data may end inside a vector
-        const uint32_t k = n & 15;
-        for (uint32_t j = 0; j < k; ++j) dst[n - k + j] = (uint8_t)(w[j >> 2] >> (8 * (j & 3)));
+        for (; times >= 4; times -= 4, n += 4) *reinterpret_cast<uint32_t*>(dst + n) = s;
+        while (times) dst[n++] = (uint8_t)b, --times;
     }
 };
 
@@ -342,13 +331,15 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_inflate(const uint32_t*
         uint64_t wi = pos >> 5;
         uint64_t buf = (uint64_t)word(wi) >> (pos & 31);
         uint32_t have = 32 - (uint32_t)(pos & 31);
+        uint32_t ahead = word(wi + 1);  // always one word ahead of the bit buffer
         ByteOut bo(out);
         uint32_t prev = 0;
         bool ok = true;
         while (bo.n < n_lane) {
             if (have <= 32) {
-                buf |= (uint64_t)word(++wi) << have;
+                buf |= (uint64_t)ahead << have;
                 have += 32;
+                ahead = word(++wi + 1);
             }
             const uint32_t code9 = __brev((uint32_t)buf) >> 23;  // the next 9 bits as a code, first bit on top
             uint32_t sym, used;
@@ -385,26 +376,17 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_inflate(const uint32_t*
             buf >>= used, have -= used;
             bo.repeat(prev, len);
         }
-        bo.finish();
         if (!ok) fail();
     }
 }
 
 int launch_deflate(const void* src, uint64_t n_bytes, uint32_t n_chunks, void* stream_out, uint64_t* chunk_offset,
                    uint32_t* sub_bits, void* ws, int n_sm, cudaStream_t st) {
-    static bool attr_set[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
-    constexpr int smem = kWarpsPerBlock * kSlotBytes;
-    if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(k_deflate_encode, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -1;
-        attr_set[dev] = true;
-    }
     uint8_t* slots = static_cast<uint8_t*>(ws);
     uint32_t* sizes = reinterpret_cast<uint32_t*>(slots + (size_t)n_chunks * kSlotBytes);
     const uint32_t blocks = (n_chunks + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    const uint32_t grid = min(blocks, (uint32_t)n_sm * 3u * 8u);
-    k_deflate_encode<<<grid, kWarpsPerBlock * 32, smem, st>>>(static_cast<const uint8_t*>(src), n_bytes, n_chunks, slots,
+    const uint32_t grid = min(blocks, (uint32_t)n_sm * 16u * 8u);
+    k_deflate_encode<<<grid, kWarpsPerBlock * 32, 0, st>>>(static_cast<const uint8_t*>(src), n_bytes, n_chunks, slots,
                                                               sizes, sub_bits);
     k_deflate_scan<<<1, 1024, 0, st>>>(sizes, n_chunks, chunk_offset);
     k_deflate_pack<<<grid, kWarpsPerBlock * 32, 0, st>>>(slots, sizes, chunk_offset, n_chunks,
