@@ -175,7 +175,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2309_06973_b200 import binding as B
-    from paper_2309_06973_b200.runtime import DeviceModel, Session
+    from paper_2309_06973_b200.runtime import Deflater, DeviceModel, Session
     from paper_2309_06973_b200.dist_util import max_over_ranks, ms_per_variant as whole_job_ms_per_variant
 
     if not torch.cuda.is_available():
@@ -352,6 +352,46 @@ def main():
                "what": "last variant: rule of Algorithm 1 applied to a fixed point on the kernel maps"}
     ses2.close()
 
+    # ---- Module 7 / 8 on the rebuilt variants (not part of the portfolio step): every variant deflated into
+    # one package, smallest first; timings for the last variant (deflate) and its inflation
+    deflater = Deflater(ses.compact_arena.numel(), dm.device)
+    raw_sizes, packed_sizes, codec_ms = [], [], {"deflate": [], "inflate": []}
+    restored = torch.empty_like(ses.compact_arena)
+    for v in range(V):
+        ses.variant(v, fused=not args.stepwise)
+        torch.cuda.synchronize()
+        offs = ses.dst_offsets.cpu().numpy().view(np.uint64)
+        cnt = ses.keep_count.cpu().numpy()
+        used = min((int(offs[-1]) + 4 * max(int(cnt.max()), 1) + 255) // 256 * 256, ses.compact_arena.numel())
+        reps = 5 if v == V - 1 else 1
+        for _ in range(reps):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            ev[0].record()
+            deflater.deflate(ses.compact_arena, used)
+            ev[1].record()
+            size = deflater.stream_bytes()
+            ev[2].record()
+            deflater.inflate(restored, size)
+            ev[3].record()
+            torch.cuda.synchronize()
+            if v == V - 1:
+                codec_ms["deflate"].append(ev[0].elapsed_time(ev[1]))
+                codec_ms["inflate"].append(ev[2].elapsed_time(ev[3]))
+        assert int(deflater.status.item()) == B.DNNS_OK and torch.equal(restored[:used], ses.compact_arena[:used])
+        raw_sizes.append(used)
+        packed_sizes.append(size + 8 * (B.dnns_deflate_chunks(used) + 1) + 4 * 32 * B.dnns_deflate_chunks(used))
+    order = sorted(range(V), key=lambda v: raw_sizes[v])           # Module 7 sorts the portfolio by model size
+    dms, ims = statistics.median(codec_ms["deflate"]), statistics.median(codec_ms["inflate"])
+    deflate_info = {"package_order": order, "raw_bytes": [raw_sizes[v] for v in order],
+                    "packed_bytes_with_index": [packed_sizes[v] for v in order],
+                    "package_ratio": sum(packed_sizes) / sum(raw_sizes),
+                    "last_variant": {"deflate_ms": dms, "inflate_ms": ims,
+                                     "deflate_gbs": (raw_sizes[-1] + packed_sizes[-1]) / (dms * 1e-3) / 1e9,
+                                     "inflate_gbs": (raw_sizes[-1] + packed_sizes[-1]) / (ims * 1e-3) / 1e9},
+                    "what": "RFC 1951 streams (fixed Huffman / stored blocks, runs as distance-1 matches) plus chunk and "
+                            "sub-block index; paper context: 43 ms to switch a VGG-16 variant in (Table V)"}
+    del restored
+
     # ---- end to end through the C ABI with host buffers -----------------------------------------
     small = torch.empty(1 << 16, dtype=torch.uint8).pin_memory()
     host_out = torch.empty(ses.compact_arena.numel(), dtype=torch.uint8).pin_memory()
@@ -408,6 +448,7 @@ def main():
         "cascade": cascade,
         "fold_batchnorm": {"ms": fold_ms, "gbs": 2 * Nn[-1] * eb / (fold_ms * 1e-3) / 1e9,
                            "what": "conv + BatchNorm fusion of the last variant in place (read + write of its weights)"},
+        "deflate": deflate_info,
         "clocks": clocks,
         "context": {"paper_pruning_time_ms": 120, "paper_hardware": "not stated for that figure"},
     }

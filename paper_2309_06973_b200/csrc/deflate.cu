@@ -124,7 +124,6 @@ __device__ __forceinline__ void emit_run(Sink& s, uint32_t v, uint32_t len) {
 }
 
 // Walk the n (<= 512) bytes of a sub-block at p (16-byte aligned) and hand its runs to the sink.
-// The next 16 bytes are requested before the current ones are walked.
 template <typename Sink>
 __device__ __forceinline__ void parse_sub_block(Sink& s, const uint8_t* p, uint32_t n) {
     uint32_t run_val = 0, run_len = 0;
@@ -139,10 +138,14 @@ __device__ __forceinline__ void parse_sub_block(Sink& s, const uint8_t* p, uint3
     };
     const uint32_t n_vec = n / 16;
     const uint4* pv = reinterpret_cast<const uint4*>(p);
-    uint4 nxt = n_vec ? __ldg(pv) : make_uint4(0, 0, 0, 0);
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    // four vectors (64 bytes) are always in flight ahead of the walk
+    uint4 q0 = n_vec > 0 ? __ldg(pv) : zero4, q1 = n_vec > 1 ? __ldg(pv + 1) : zero4;
+    uint4 q2 = n_vec > 2 ? __ldg(pv + 2) : zero4, q3 = n_vec > 3 ? __ldg(pv + 3) : zero4;
     for (uint32_t v = 0; v < n_vec; ++v) {
-        const uint4 q = nxt;
-        if (v + 1 < n_vec) nxt = __ldg(pv + v + 1);
+        const uint4 q = q0;
+        q0 = q1, q1 = q2, q2 = q3;
+        if (v + 4 < n_vec) q3 = __ldg(pv + v + 4);
         const uint32_t splat = run_val * 0x01010101u;
         if (run_len && q.x == splat && q.y == splat && q.z == splat && q.w == splat) {
             run_len += 16;  // sixteen more of the same (long runs of zeros are the common case)
@@ -272,19 +275,29 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_deflate_pack(const uint
 }
 
 // One lane's output, written straight into its own 512 bytes of the destination (16-byte aligned):
-// literals byte by byte, repeats as words and vectors once aligned.  L2 merges the partial lines.
+// literals are collected into words, repeats go out as words and vectors once aligned.  L2 merges
+// the partial lines.
 struct ByteOut {
     uint8_t* dst;
-    uint32_t n = 0;
+    uint32_t n = 0, acc = 0;
     __device__ __forceinline__ explicit ByteOut(uint8_t* d) : dst(d) {}
-    __device__ __forceinline__ void push(uint32_t b) { dst[n++] = (uint8_t)b; }
+    __device__ __forceinline__ void push(uint32_t b) {
+        acc |= b << (8 * (n & 3));
+        if ((++n & 3) == 0) {
+            *reinterpret_cast<uint32_t*>(dst + n - 4) = acc;
+            acc = 0;
+        }
+    }
     __device__ __forceinline__ void repeat(uint32_t b, uint32_t times) {
-        while (times && (n & 3)) dst[n++] = (uint8_t)b, --times;
+        while (times && (n & 3)) push(b), --times;
         const uint32_t s = b * 0x01010101u;
         while (times >= 4 && (n & 15)) *reinterpret_cast<uint32_t*>(dst + n) = s, n += 4, times -= 4;
         for (; times >= 16; times -= 16, n += 16) *reinterpret_cast<uint4*>(dst + n) = make_uint4(s, s, s, s);
         for (; times >= 4; times -= 4, n += 4) *reinterpret_cast<uint32_t*>(dst + n) = s;
-        while (times) dst[n++] = (uint8_t)b, --times;
+        while (times) push(b), --times;
+    }
+    __device__ __forceinline__ void finish() {  // the data may end inside a word
+        for (uint32_t j = 0; j < (n & 3); ++j) dst[(n & ~3u) + j] = (uint8_t)(acc >> (8 * j));
     }
 };
 
@@ -331,15 +344,25 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_inflate(const uint32_t*
         uint64_t wi = pos >> 5;
         uint64_t buf = (uint64_t)word(wi) >> (pos & 31);
         uint32_t have = 32 - (uint32_t)(pos & 31);
-        uint32_t ahead = word(wi + 1);  // always one word ahead of the bit buffer
+        // the stream words behind the bit buffer: four being used up, four more already requested
+        uint32_t a0 = word(wi + 1), a1 = word(wi + 2), a2 = word(wi + 3), a3 = word(wi + 4);
+        uint32_t b0 = word(wi + 5), b1 = word(wi + 6), b2 = word(wi + 7), b3 = word(wi + 8);
+        uint32_t left = 4;
+        wi += 9;  // the next word to request
         ByteOut bo(out);
         uint32_t prev = 0;
         bool ok = true;
         while (bo.n < n_lane) {
             if (have <= 32) {
-                buf |= (uint64_t)ahead << have;
+                buf |= (uint64_t)a0 << have;
                 have += 32;
-                ahead = word(++wi + 1);
+                a0 = a1, a1 = a2, a2 = a3;
+                if (--left == 0) {
+                    a0 = b0, a1 = b1, a2 = b2, a3 = b3;
+                    b0 = word(wi), b1 = word(wi + 1), b2 = word(wi + 2), b3 = word(wi + 3);
+                    wi += 4;
+                    left = 4;
+                }
             }
             const uint32_t code9 = __brev((uint32_t)buf) >> 23;  // the next 9 bits as a code, first bit on top
             uint32_t sym, used;
@@ -376,6 +399,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_inflate(const uint32_t*
             buf >>= used, have -= used;
             bo.repeat(prev, len);
         }
+        bo.finish();
         if (!ok) fail();
     }
 }

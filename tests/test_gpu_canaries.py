@@ -84,3 +84,15 @@ def test_workspace_is_not_overrun():
     torch.cuda.synchronize()
     r = raw.cpu().numpy()
     assert np.all(r[:GUARD] == PATTERN) and np.all(r[-GUARD:] == PATTERN)
+
+
+def test_codec_buffers_are_not_overrun():
+    """dnns_deflate / dnns_inflate with every buffer sized exactly as the size queries say, between guards:
+    dense bytes (every chunk stored, the largest stream and the fullest slots), sparse bytes, a ragged end."""
+    from runtime_guard_codec import run_guarded_codec
+    rng = np.random.default_rng(9)
+    dense = rng.integers(0, 256, 5 * B.DNNS_DEFLATE_CHUNK + 333, dtype=np.uint8)
+    sparse = dense.copy()
+    sparse[rng.random(sparse.size) < 0.9] = 0
+    for data in (dense, sparse, dense[:7], sparse[: B.DNNS_DEFLATE_CHUNK]):
+        run_guarded_codec(data, Guarded)
