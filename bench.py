@@ -281,6 +281,17 @@ def main():
     launches0 = ses.launch_count()
     plain_ms = timed_steps(lambda: step(True))
     launches_plain = ses.launch_count() - launches0
+    # the same steps once more with an event pair around every single kernel (dnns_plan_profile)
+    kernel_names = ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_ties", "k_tie_scan", "k_sweep", "k_flags",
+                    "k_propagate", "k_compact_layout", "k_compact_gather"]
+    ses.profile(True)
+    timed_steps(lambda: step(False))
+    ses.profile(False)
+    kernel_ms = {}
+    for kn in kernel_names:
+        ms, n = ses.kernel_time(kn)
+        if n:
+            kernel_ms[kn] = {"avg_ms": ms / n, "launches_per_step": n / args.steps, "ms_per_step": ms / args.steps}
     if graph is not None:
         barrier()
         total_ms = timed_steps(graph.replay)
@@ -307,10 +318,21 @@ def main():
     moved_bytes = alg["threshold"] + V * (alg["mask"] + (alg["structures"] if args.stepwise else 0)) + \
         sum((r + n) * eb for r, n in zip(R, Nn))
     peak, peak_kind = load_peaks()
-    dominant = max((n for n in names if alg[n] > 0), key=lambda n: share[n])
-    achieved = alg[dominant] / (per_call[dominant] * 1e-3) / 1e9
-    kernel_of = {"threshold": "k_hist1+k_hist2 (+select, ties)", "mask": "k_sweep<mask>", "structures": "k_sweep<structures>",
-                 "mask+structures": "k_sweep<mask+structures>", "compact": "k_compact_gather"}
+    # the dominant kernel: largest share of the summed kernel time; its algorithmic bytes per launch
+    kernel_alg = {"k_hist1": N * eb, "k_hist2": N * eb, "k_ties": N * eb,
+                  "k_sweep": alg["mask"] if args.stepwise else alg["mask+structures"] + N / 8,  # + the element bits it packs
+                  "k_compact_gather": alg["compact"]}
+    if args.stepwise:
+        kernel_alg["k_sweep"] = (alg["mask"] + alg["structures"] + N / 8) / 2   # two sweeps per variant, averaged
+    kernel_total = sum(k["ms_per_step"] for k in kernel_ms.values())
+    for k in kernel_ms.values():
+        k["share"] = k["ms_per_step"] / kernel_total
+    dominant = max((kn for kn in kernel_ms if kn in kernel_alg), key=lambda kn: kernel_ms[kn]["ms_per_step"])
+    achieved = kernel_alg[dominant] / (kernel_ms[dominant]["avg_ms"] * 1e-3) / 1e9
+    for kn, k in kernel_ms.items():
+        if kn in kernel_alg:
+            k["gbs"] = kernel_alg[kn] / (k["avg_ms"] * 1e-3) / 1e9
+    kernel_label = {"k_sweep": "k_sweep<mask>+<structures>" if args.stepwise else "k_sweep<mask+structures>"}
 
     # ---- Module 1 on a rebuilt variant (not part of the portfolio step): conv + BatchNorm fusion in place
     fold_ms = []
@@ -438,10 +460,14 @@ def main():
         "launch": "cuda graph replay" if graph is not None else "plain stream launches", "ms_per_step_plain": plain_per_step,
         "per_call_ms": per_call, "share": share,
         "per_call_gbs": {n: (alg[n] / (per_call[n] * 1e-3) / 1e9 if alg[n] else None) for n in names},
-        "roofline": {"bound": "hbm", "kernel": kernel_of[dominant], "achieved": achieved, "peak": peak,
+        "kernel_ms": kernel_ms,
+        "roofline": {"bound": "hbm", "kernel": kernel_label.get(dominant, dominant), "achieved": achieved, "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                     "algorithmic_bytes": alg[dominant],
-                     "traffic": measured_traffic(args.workload, args.dtype, kernel_of[dominant])},
+                     "algorithmic_bytes": kernel_alg[dominant],
+                     "avg_launch_ms": kernel_ms[dominant]["avg_ms"],
+                     "timed_by": "CUDA event pair around every launch of the kernel on its stream, "
+                                 f"{args.steps} steps of plain launches",
+                     "traffic": measured_traffic(args.workload, args.dtype, kernel_label.get(dominant, dominant))},
         "e2e": {"value": e2e_per_variant, "unit": "ms", "h2d_bytes_per_step": h2d // args.steps,
                 "d2h_bytes_per_step": d2h // args.steps},
         "gpu_launches": launches,

@@ -169,6 +169,19 @@ dnns_status dnns_plan_layout(const dnns_plan* plan, dnns_layout* out);
 uint64_t dnns_plan_launch_count(const dnns_plan* plan);
 
 /*
+ * Per-kernel timing of a plan's calls, for reports (the paper's Module 5 profiles models; this profiles
+ * the conversion itself).  dnns_plan_profile(plan, 1) synchronises the device, drops earlier records and,
+ * from then on, brackets every kernel the plan's calls launch with a pair of CUDA events on the launching
+ * stream (two event creations per launch: host work, so switch it off for timed runs and do not switch it
+ * on while a stream is being captured); dnns_plan_profile(plan, 0) stops recording.
+ * dnns_plan_profile_read synchronises the device and returns the summed device time and the number of
+ * recorded launches of the kernels whose name starts with `kernel` ("k_sweep", "k_compact_gather",
+ * "k_flags", "k_propagate", "k_hist1", "k_hist2", "k_ties", "k_select1", "k_select2", "k_tie_scan").
+ */
+dnns_status dnns_plan_profile(dnns_plan* plan, int32_t enable);
+dnns_status dnns_plan_profile_read(dnns_plan* plan, const char* kernel, double* total_ms, uint64_t* launches);
+
+/*
  * Step 1 - exact k-th-magnitude threshold by radix select over the magnitude keys.
  * k (host): k[v*n_segments + s] = how many weights of segment s variant v masks, 0 <= k <= the
  * segment's size, 1 <= n_k <= max_variants.  thr_dev (device, n_k*n_segments records, same

@@ -22,7 +22,7 @@ DNNS_DEFLATE_CHUNK, DNNS_DEFLATE_SUB = 16384, 512
 EXPORTS = ["dnns_status_string", "dnns_workspace_bytes", "dnns_plan_create", "dnns_plan_destroy", "dnns_plan_layout",
            "dnns_plan_launch_count", "dnns_magnitude_threshold", "dnns_apply_mask", "dnns_zero_structures",
            "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures", "dnns_fold_batchnorm", "dnns_propagate_keep_cascade",
-           "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
+           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
 
 
 class dnns_tensor(C.Structure):
@@ -101,6 +101,8 @@ def lib() -> C.CDLL:
         L.dnns_fold_batchnorm.argtypes = [vp, vp, vp, vp, vp]
         L.dnns_propagate_keep_cascade.argtypes = [vp, vp, u32, i32, i32, vp, vp, vp, vp, vp]
         L.dnns_magnitude_threshold_static.argtypes = [vp, i32, u64, u64, vp, vp]
+        L.dnns_plan_profile.argtypes = [vp, i32]
+        L.dnns_plan_profile_read.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(u64)]
         for name in ("dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
             getattr(L, name).argtypes = [C.c_size_t]
@@ -221,3 +223,14 @@ def dnns_inflate(stream_dev: int, stream_bytes: int, chunk_offset_dev: int, sub_
                  dst_dev: int, status_dev: int, stream: int = 0) -> None:
     _check(lib().dnns_inflate(stream_dev, stream_bytes, chunk_offset_dev, sub_bits_dev, n_bytes, dst_dev or None,
                               status_dev, stream), "dnns_inflate")
+
+
+def dnns_plan_profile(plan, enable: bool) -> None:
+    _check(lib().dnns_plan_profile(plan, int(enable)), "dnns_plan_profile")
+
+
+def dnns_plan_profile_read(plan, kernel: str):
+    """(total device milliseconds, launches) of the recorded kernels whose name starts with `kernel`."""
+    ms, n = C.c_double(0), C.c_uint64(0)
+    _check(lib().dnns_plan_profile_read(plan, kernel.encode(), C.byref(ms), C.byref(n)), "dnns_plan_profile_read")
+    return ms.value, n.value

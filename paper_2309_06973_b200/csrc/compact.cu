@@ -319,12 +319,17 @@ int launch_compact(const Tables& tb, const CompactWs& ws, const void* src_arena,
     const int grid = n_sm * 4;
     int launches = 1;
     if (tb.n_items <= kInlineItems) {
+        ScopedKernel timed("k_compact_gather", st);
         if (tb.dtype == DNNS_F32)
             k_compact_gather<4, true><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, dst_shapes);
         else
             k_compact_gather<2, true><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, dst_shapes);
     } else {
-        k_compact_layout<<<1, 1024, 0, st>>>(tb, ws, keep_count, dst_bytes, dst_offsets, dst_shapes);
+        {
+            ScopedKernel timed_layout("k_compact_layout", st);
+            k_compact_layout<<<1, 1024, 0, st>>>(tb, ws, keep_count, dst_bytes, dst_offsets, dst_shapes);
+        }
+        ScopedKernel timed("k_compact_gather", st);
         if (tb.dtype == DNNS_F32)
             k_compact_gather<4, false><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, dst_shapes);
         else

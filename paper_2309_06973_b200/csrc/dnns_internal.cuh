@@ -135,6 +135,17 @@ struct CompactWs {
     int32_t* item_dims;     // [n_items][2] rows', input channels' of the rebuilt item
 };
 
+// ---- optional per-kernel timing (dnns_plan_profile): while a plan's profile is on, every kernel launch
+// of its calls is bracketed by a pair of CUDA events on the launching stream.
+struct KernelTimer;
+struct ScopedKernel {
+    KernelTimer* t;
+    cudaStream_t st;
+    int rec;
+    ScopedKernel(const char* name, cudaStream_t stream);  // records the start event when a profile is on
+    ~ScopedKernel();                                       // records the stop event
+};
+
 // ---- launch wrappers (each returns the number of kernels it launched, or -1 on a CUDA error) ----
 int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, const uint64_t* k_host, dnns_threshold* thr_dev,
                      int n_sm, cudaStream_t st);

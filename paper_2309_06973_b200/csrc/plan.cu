@@ -5,9 +5,50 @@
 #include <new>
 #include <vector>
 
+#include <string>
+
 #include "dnns_internal.cuh"
 
 using namespace dnns;
+
+namespace dnns {
+
+struct KernelTimer {
+    struct Rec {
+        const char* name;
+        cudaEvent_t start, stop;
+    };
+    bool on = false;
+    std::vector<Rec> recs;
+    void clear() {
+        for (Rec& r : recs) {
+            cudaEventDestroy(r.start);
+            cudaEventDestroy(r.stop);
+        }
+        recs.clear();
+    }
+};
+
+static thread_local KernelTimer* g_timer = nullptr;  // the profile of the plan whose call is running on this thread
+
+ScopedKernel::ScopedKernel(const char* name, cudaStream_t stream) : t(g_timer), st(stream), rec(-1) {
+    if (!t || !t->on) return;
+    KernelTimer::Rec r{name, nullptr, nullptr};
+    if (cudaEventCreate(&r.start) != cudaSuccess) return;
+    if (cudaEventCreate(&r.stop) != cudaSuccess) {
+        cudaEventDestroy(r.start);
+        return;
+    }
+    t->recs.push_back(r);
+    rec = (int)t->recs.size() - 1;
+    cudaEventRecord(r.start, st);
+}
+
+ScopedKernel::~ScopedKernel() {
+    if (rec >= 0) cudaEventRecord(t->recs[rec].stop, st);
+}
+
+}  // namespace dnns
 
 namespace {
 
@@ -152,11 +193,19 @@ struct dnns_plan {
     CascadeWs kws;
     uint64_t launches;
     int last_n_k;
+    KernelTimer timer;
     // host-side layout, handed out by dnns_plan_layout
     std::vector<uint64_t> arena_off, mask_off, nzmap_off, outnz_off, innz_off, keep_off, keepidx_off, seg_size;
     std::vector<int32_t> seg_of_tensor;
     dnns_layout layout;
 };
+
+namespace {
+struct ProfileScope {  // makes the plan's profile the active one for the launches of one call
+    explicit ProfileScope(dnns_plan* p) { dnns::g_timer = p ? &p->timer : nullptr; }
+    ~ProfileScope() { dnns::g_timer = nullptr; }
+};
+}  // namespace
 
 extern "C" {
 
@@ -393,6 +442,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
 void dnns_plan_destroy(dnns_plan* plan) {
     if (!plan) return;
     cudaDeviceSynchronize();
+    plan->timer.clear();
     delete plan;
 }
 
@@ -416,6 +466,7 @@ dnns_status dnns_magnitude_threshold(dnns_plan* p, const uint64_t* k, int32_t n_
     const uint64_t clear_end = p->map.hist2 + (p->c.dtype == DNNS_F32 ? 4ull * kLowBins * S * n_k : 0);
     if (cudaMemsetAsync(p->ws + p->map.clear_begin, 0, clear_end - p->map.clear_begin, st) != cudaSuccess)
         return DNNS_ERR_CUDA;
+    ProfileScope profile_scope(p);
     const int n = launch_threshold(p->tb, p->tws, n_k, k, thr_dev, p->n_sm, st);
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
@@ -427,6 +478,7 @@ dnns_status dnns_apply_mask(dnns_plan* p, const dnns_threshold* thr_dev, int32_t
                             uint32_t* mask_bits, void* stream) {
     if (!p || !thr_dev || variant < 0 || variant >= p->maxv) return DNNS_ERR_INVALID_ARG;
     if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
+    ProfileScope profile_scope(p);
     const int n = launch_tile_sweep(p->tb, p->tws, true, false, thr_dev, variant, nullptr, masked_arena, mask_bits,
                                     nullptr, nullptr, nullptr, 0, 0, p->n_sm, static_cast<cudaStream_t>(stream));
     if (n < 0) return DNNS_ERR_CUDA;
@@ -441,6 +493,7 @@ dnns_status dnns_zero_structures(dnns_plan* p, const void* masked_arena, uint32_
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const dnns_layout& L = p->layout;
     // (the sweep clears the flag words before the flag kernel ORs into them)
+    ProfileScope profile_scope(p);
     const int n = launch_tile_sweep(p->tb, p->tws, false, true, nullptr, 0, masked_arena, nullptr, nullptr, nz_map,
                                     out_nz, in_nz, (uint32_t)L.out_nz_words, (uint32_t)L.in_nz_words, p->n_sm, st);
     if (n < 0) return DNNS_ERR_CUDA;
@@ -456,6 +509,7 @@ dnns_status dnns_mask_and_structures(dnns_plan* p, const dnns_threshold* thr_dev
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const dnns_layout& L = p->layout;
     // the flag words are OR-ed into; the kernel map is stored word by word and needs no clearing
+    ProfileScope profile_scope(p);
     const int n = launch_tile_sweep(p->tb, p->tws, true, true, thr_dev, variant, nullptr, masked_arena, mask_bits,
                                     nz_map, out_nz, in_nz, (uint32_t)L.out_nz_words, (uint32_t)L.in_nz_words, p->n_sm, st);
     if (n < 0) return DNNS_ERR_CUDA;
@@ -470,6 +524,7 @@ dnns_status dnns_propagate_keep(dnns_plan* p, const uint32_t* out_nz, const uint
     if (policy & ~(uint32_t)(DNNS_RULE_PRODUCER | DNNS_RULE_CONSUMER | DNNS_SHIFT_STRICT)) return DNNS_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (stats && cudaMemsetAsync(stats, 0, 32, st) != cudaSuccess) return DNNS_ERR_CUDA;
+    ProfileScope profile_scope(p);
     const int n = launch_propagate(p->tb, out_nz, in_nz, policy, min_keep, keep_bits, keep_idx, keep_count, stats, st);
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
@@ -485,6 +540,7 @@ dnns_status dnns_propagate_keep_cascade(dnns_plan* p, const uint32_t* nz_map, ui
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (stats && cudaMemsetAsync(stats, 0, 32, st) != cudaSuccess) return DNNS_ERR_CUDA;
     const dnns_layout& L = p->layout;
+    ProfileScope profile_scope(p);
     const int n = launch_propagate_cascade(p->tb, p->kws, nz_map, policy, min_keep, max_passes, keep_bits, keep_idx,
                                            keep_count, stats, (uint32_t)L.keep_words,
                                            (uint32_t)(L.out_nz_words + L.in_nz_words), p->n_sm, st);
@@ -500,6 +556,7 @@ dnns_status dnns_compact(dnns_plan* p, const void* masked_arena, const int32_t* 
     if ((reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) ||
         (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)))
         return DNNS_ERR_INVALID_ARG;
+    ProfileScope profile_scope(p);
     const int n = launch_compact(p->tb, p->cws, masked_arena, keep_idx, keep_count, dst_arena, dst_bytes,
                                  dst_offsets_dev, dst_shapes_dev, p->n_sm, static_cast<cudaStream_t>(stream));
     if (n < 0) return DNNS_ERR_CUDA;
@@ -511,9 +568,38 @@ dnns_status dnns_fold_batchnorm(dnns_plan* p, void* dst_arena, const uint64_t* d
                                 const int32_t* dst_shapes_dev, void* stream) {
     if (!p || !dst_arena || !dst_offsets_dev || !dst_shapes_dev) return DNNS_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) return DNNS_ERR_INVALID_ARG;
+    ProfileScope profile_scope(p);
     const int n = launch_fold(p->tb, dst_arena, dst_offsets_dev, dst_shapes_dev, static_cast<cudaStream_t>(stream));
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
+    return DNNS_OK;
+}
+
+dnns_status dnns_plan_profile(dnns_plan* p, int32_t enable) {
+    if (!p) return DNNS_ERR_INVALID_ARG;
+    if (enable) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return DNNS_ERR_CUDA;
+        p->timer.clear();
+    }
+    p->timer.on = enable != 0;
+    return DNNS_OK;
+}
+
+dnns_status dnns_plan_profile_read(dnns_plan* p, const char* kernel, double* total_ms, uint64_t* launches) {
+    if (!p || !kernel || !total_ms || !launches) return DNNS_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return DNNS_ERR_CUDA;
+    const size_t n = strlen(kernel);
+    double sum = 0;
+    uint64_t cnt = 0;
+    for (const KernelTimer::Rec& r : p->timer.recs) {
+        if (strncmp(r.name, kernel, n) != 0) continue;
+        float ms = 0;
+        if (cudaEventElapsedTime(&ms, r.start, r.stop) != cudaSuccess) return DNNS_ERR_CUDA;
+        sum += ms;
+        ++cnt;
+    }
+    *total_ms = sum;
+    *launches = cnt;
     return DNNS_OK;
 }
 

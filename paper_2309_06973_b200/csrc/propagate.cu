@@ -308,6 +308,7 @@ __global__ void __launch_bounds__(kThreads) k_cascade_finish(Tables tb, const ui
 int launch_propagate(const Tables& tb, const uint32_t* out_nz, const uint32_t* in_nz, uint32_t policy,
                      int32_t min_keep, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count, uint64_t* stats,
                      cudaStream_t st) {
+    ScopedKernel timed("k_propagate", st);
     k_propagate<<<tb.n_groups, kThreads, 0, st>>>(tb, out_nz, in_nz, policy, min_keep, keep_bits, keep_idx,
                                                   keep_count, reinterpret_cast<unsigned long long*>(stats));
     return cudaGetLastError() == cudaSuccess ? 1 : -1;

@@ -375,6 +375,7 @@ template <int DT>
 void launch_dt(bool do_mask, bool do_struct, dim3 grid, cudaStream_t st, const Tables& tb, const ThresholdWs& ws,
                const dnns_threshold* thr, int variant, const char* src_arena, char* dst_arena, uint32_t* mask_bits,
                uint32_t* out_nz, uint32_t n_out, uint32_t* in_nz, uint32_t n_in) {
+    ScopedKernel timed(do_mask && do_struct ? "k_sweep<mask+structures>" : (do_mask ? "k_sweep<mask>" : "k_sweep<structures>"), st);
     if (do_mask && do_struct)
         k_sweep<DT, true, true><<<grid, kTileThreads, 0, st>>>(tb, ws, thr, variant, src_arena, dst_arena, mask_bits,
                                                                out_nz, n_out, in_nz, n_in);
@@ -401,6 +402,7 @@ int launch_tile_sweep(const Tables& tb, const ThresholdWs& ws, bool do_mask, boo
                              (char*)dst_arena, mask_bits, out_nz, n_out_words, in_nz, n_in_words);
     if (do_struct) {
         const uint32_t blocks = min((uint32_t)n_sm * 64u, (tb.n_flag_units + 7) / 8);  // one unit per warp if possible
+        ScopedKernel timed("k_flags", st);
         k_flags<<<max(blocks, 1u), 256, 0, st>>>(tb, nz_map, out_nz, in_nz);
     }
     return cudaGetLastError() == cudaSuccess ? (do_struct ? 2 : 1) : -1;

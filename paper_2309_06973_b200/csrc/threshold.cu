@@ -561,19 +561,19 @@ int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, const uin
     const int sweep_grid = (int)min((uint32_t)n_sm * 4u, tb.n_tiles);
     int launches = 0;
     if (tb.dtype == DNNS_F32) {
-        k_hist1<DNNS_F32><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws.hist1);
-        k_select1<DNNS_F32><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline);
-        k_hist2<<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k);
-        k_select2<<<S * n_k, 1024, 0, st>>>(tb, ws, n_k, thr_dev);
-        k_ties<DNNS_F32><<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k, thr_dev);
+        { ScopedKernel t("k_hist1", st); k_hist1<DNNS_F32><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws.hist1); }
+        { ScopedKernel t("k_select1", st); k_select1<DNNS_F32><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline); }
+        { ScopedKernel t("k_hist2", st); k_hist2<<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k); }
+        { ScopedKernel t("k_select2", st); k_select2<<<S * n_k, 1024, 0, st>>>(tb, ws, n_k, thr_dev); }
+        { ScopedKernel t("k_ties", st); k_ties<DNNS_F32><<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k, thr_dev); }
         launches = 5;
     } else {
-        k_hist1<DNNS_BF16><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws.hist1);
-        k_select1<DNNS_BF16><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline);
-        k_ties<DNNS_BF16><<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k, thr_dev);
+        { ScopedKernel t("k_hist1", st); k_hist1<DNNS_BF16><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws.hist1); }
+        { ScopedKernel t("k_select1", st); k_select1<DNNS_BF16><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline); }
+        { ScopedKernel t("k_ties", st); k_ties<DNNS_BF16><<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k, thr_dev); }
         launches = 3;
     }
-    k_tie_scan<<<S * n_k, 1024, 0, st>>>(tb, ws);
+    { ScopedKernel t("k_tie_scan", st); k_tie_scan<<<S * n_k, 1024, 0, st>>>(tb, ws); }
     ++launches;
     return cudaGetLastError() == cudaSuccess ? launches : -1;
 }

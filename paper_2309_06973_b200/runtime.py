@@ -183,6 +183,13 @@ class Session:
     def launch_count(self) -> int:
         return B.dnns_plan_launch_count(self.plan)
 
+    def profile(self, enable: bool):
+        B.dnns_plan_profile(self.plan, enable)
+
+    def kernel_time(self, kernel: str):
+        """(total ms, launches) of a kernel since the profile was switched on."""
+        return B.dnns_plan_profile_read(self.plan, kernel)
+
     # ---- read-back (host copies, for tests and reports) ------------------------------------
     def records(self) -> np.ndarray:
         n = self.n_k * self.n_segments
