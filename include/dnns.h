@@ -229,6 +229,22 @@ dnns_status dnns_mask_and_structures(dnns_plan* plan, const dnns_threshold* thr_
                                      uint32_t* in_nz, void* stream);
 
 /*
+ * Steps 2 and 3 for up to DNNS_MULTI_MAX variants of the latest threshold call in ONE sweep over the
+ * dense weights: variants first_variant .. first_variant + n_variants - 1, each with outputs of its own,
+ * bit for bit what dnns_mask_and_structures gives for that variant.  The portfolio's variants all start
+ * from the same dense model (Section III-C: every iteration's sparse model joins the portfolio), so the
+ * model is read once per group of variants instead of once per variant.
+ * masked_arenas, out_nz, in_nz: host arrays of n_variants device pointers, all distinct; mask_bits, nz_map:
+ * host arrays of n_variants device pointers, or NULL (entries of mask_bits may be NULL too).  In-place
+ * masking is not offered here.  Errors: INVALID_ARG, CUDA.
+ */
+#define DNNS_MULTI_MAX 4
+dnns_status dnns_mask_and_structures_multi(dnns_plan* plan, const dnns_threshold* thr_dev, int32_t first_variant,
+                                           int32_t n_variants, void* const* masked_arenas, uint32_t* const* mask_bits,
+                                           uint32_t* const* nz_map, uint32_t* const* out_nz, uint32_t* const* in_nz,
+                                           void* stream);
+
+/*
  * Step 4 - keep sets per channel group (Algorithm 1 generalised from a chain to groups).
  * Channel j of a group is removed when
  *   (policy & RULE_PRODUCER) and every producer's filter j is all zero [the paper's rule], and,

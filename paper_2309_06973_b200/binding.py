@@ -18,11 +18,12 @@ DNNS_GROUP_FROZEN = 1
  DNNS_ERR_TIMEOUT, DNNS_ERR_STATIC_LIMIT) = range(8)
 DNNS_STATIC_MAX_NUMEL = 1 << 26
 DNNS_DEFLATE_CHUNK, DNNS_DEFLATE_SUB = 16384, 512
+DNNS_MULTI_MAX = 4
 
 EXPORTS = ["dnns_status_string", "dnns_workspace_bytes", "dnns_plan_create", "dnns_plan_destroy", "dnns_plan_layout",
            "dnns_plan_launch_count", "dnns_magnitude_threshold", "dnns_apply_mask", "dnns_zero_structures",
            "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures", "dnns_fold_batchnorm", "dnns_propagate_keep_cascade",
-           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
+           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_mask_and_structures_multi", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
 
 
 class dnns_tensor(C.Structure):
@@ -101,6 +102,7 @@ def lib() -> C.CDLL:
         L.dnns_fold_batchnorm.argtypes = [vp, vp, vp, vp, vp]
         L.dnns_propagate_keep_cascade.argtypes = [vp, vp, u32, i32, i32, vp, vp, vp, vp, vp]
         L.dnns_magnitude_threshold_static.argtypes = [vp, i32, u64, u64, vp, vp]
+        L.dnns_mask_and_structures_multi.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp, vp]
         L.dnns_plan_profile.argtypes = [vp, i32]
         L.dnns_plan_profile_read.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(u64)]
         for name in ("dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes"):
@@ -234,3 +236,18 @@ def dnns_plan_profile_read(plan, kernel: str):
     ms, n = C.c_double(0), C.c_uint64(0)
     _check(lib().dnns_plan_profile_read(plan, kernel.encode(), C.byref(ms), C.byref(n)), "dnns_plan_profile_read")
     return ms.value, n.value
+
+
+def _ptr_array(ptrs):
+    """A host array of device pointers (None -> NULL entry); None for the whole list -> NULL."""
+    if ptrs is None:
+        return None
+    return (C.c_void_p * len(ptrs))(*[p or None for p in ptrs])
+
+
+def dnns_mask_and_structures_multi(plan, thr_dev: int, first_variant: int, n_variants: int, masked_arenas, mask_bits,
+                                   nz_map, out_nz, in_nz, stream: int = 0) -> None:
+    """masked_arenas, out_nz, in_nz: lists of n_variants device addresses; mask_bits, nz_map: lists or None."""
+    arrays = [_ptr_array(a) for a in (masked_arenas, mask_bits, nz_map, out_nz, in_nz)]
+    _check(lib().dnns_mask_and_structures_multi(plan, thr_dev, first_variant, n_variants, *arrays, stream),
+           "dnns_mask_and_structures_multi")

@@ -118,6 +118,18 @@ struct ThresholdWs {
     uint32_t* tie_prefix;   // [max_variants][n_tiles]: those in earlier tiles of the segment
 };
 
+constexpr int kMultiMax = DNNS_MULTI_MAX;  // variants one multi-variant sweep can produce
+
+// Per-variant arguments of the multi-variant sweep (unused slots repeat slot 0).
+struct MultiSweepArgs {
+    int32_t variant[kMultiMax];
+    char* dst[kMultiMax];            // masked arenas
+    uint32_t* mask_bits[kMultiMax];  // nullable
+    uint32_t* ebits[kMultiMax];      // packed element bits in the workspace, one buffer per slot
+    uint32_t* clear_a[kMultiMax];    // filter flags (out_nz) ...
+    uint32_t* clear_b[kMultiMax];    // ... and input-column flags (in_nz): cleared by the sweep, OR-ed by k_flags
+};
+
 constexpr int kMaxCascadePasses = 64;
 
 // Scratch of the fixed-point keep propagation.
@@ -153,6 +165,9 @@ int launch_tile_sweep(const Tables& tb, const ThresholdWs& ws, bool do_mask, boo
                       const dnns_threshold* thr_dev, int variant, const void* src_arena, void* dst_arena,
                       uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz, uint32_t n_out_words,
                       uint32_t n_in_words, int n_sm, cudaStream_t st);
+int launch_multi_sweep(const Tables& tb, const ThresholdWs& ws, const dnns_threshold* thr_dev, const MultiSweepArgs& ma,
+                       int n_variants, uint32_t* const* nz_map, uint32_t n_out_words, uint32_t n_in_words, int n_sm,
+                       cudaStream_t st);
 int launch_propagate(const Tables& tb, const uint32_t* out_nz, const uint32_t* in_nz, uint32_t policy,
                      int32_t min_keep, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count, uint64_t* stats,
                      cudaStream_t st);

@@ -161,7 +161,7 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.unit_prefix = take(4ull * (c.items + 1));
     w.item_off = take(8ull * c.items);
     w.item_dims = take(8ull * c.items);
-    w.ebits = take(4ull * c.mask_words);
+    w.ebits = take(4ull * c.mask_words * kMultiMax);  // one buffer per slot of the multi-variant sweep
     w.casc_rem0 = take(4ull * c.keep_words);
     w.casc_rem1 = take(4ull * c.keep_words);
     w.casc_lost = take(4ull * c.keep_words);
@@ -512,6 +512,36 @@ dnns_status dnns_mask_and_structures(dnns_plan* p, const dnns_threshold* thr_dev
     ProfileScope profile_scope(p);
     const int n = launch_tile_sweep(p->tb, p->tws, true, true, thr_dev, variant, nullptr, masked_arena, mask_bits,
                                     nz_map, out_nz, in_nz, (uint32_t)L.out_nz_words, (uint32_t)L.in_nz_words, p->n_sm, st);
+    if (n < 0) return DNNS_ERR_CUDA;
+    p->launches += n;
+    return DNNS_OK;
+}
+
+dnns_status dnns_mask_and_structures_multi(dnns_plan* p, const dnns_threshold* thr_dev, int32_t first_variant,
+                                           int32_t n_variants, void* const* masked_arenas, uint32_t* const* mask_bits,
+                                           uint32_t* const* nz_map, uint32_t* const* out_nz, uint32_t* const* in_nz,
+                                           void* stream) {
+    if (!p || !thr_dev || !masked_arenas || !out_nz || !in_nz || n_variants < 1 || n_variants > kMultiMax ||
+        first_variant < 0 || first_variant + n_variants > p->maxv)
+        return DNNS_ERR_INVALID_ARG;
+    MultiSweepArgs ma;
+    for (int g = 0; g < kMultiMax; ++g) {
+        const int s = g < n_variants ? g : 0;
+        if (!masked_arenas[s] || (reinterpret_cast<uintptr_t>(masked_arenas[s]) & 15) || !out_nz[s] || !in_nz[s])
+            return DNNS_ERR_INVALID_ARG;
+        for (int h = 0; h < s; ++h)  // every variant needs buffers of its own
+            if (masked_arenas[h] == masked_arenas[s] || out_nz[h] == out_nz[s] || in_nz[h] == in_nz[s]) return DNNS_ERR_INVALID_ARG;
+        ma.variant[g] = first_variant + s;
+        ma.dst[g] = static_cast<char*>(masked_arenas[s]);
+        ma.mask_bits[g] = mask_bits ? mask_bits[s] : nullptr;
+        ma.ebits[g] = p->tb.ebits + (size_t)s * p->c.mask_words;
+        ma.clear_a[g] = out_nz[s];
+        ma.clear_b[g] = in_nz[s];
+    }
+    const dnns_layout& L = p->layout;
+    ProfileScope profile_scope(p);
+    const int n = launch_multi_sweep(p->tb, p->tws, thr_dev, ma, n_variants, nz_map, (uint32_t)L.out_nz_words,
+                                     (uint32_t)L.in_nz_words, p->n_sm, static_cast<cudaStream_t>(stream));
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
     return DNNS_OK;

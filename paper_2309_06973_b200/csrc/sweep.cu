@@ -80,7 +80,8 @@ __device__ __forceinline__ void or_if_missing(uint32_t* word, uint32_t bits) {
 // most one atomic per step.  This keeps the number of atomics on the few flag words small even
 // though every unit of a tensor runs at the same time.
 // Other shapes take units of 32 kernels, one per lane, each kernel setting its own two flags.
-__global__ void __launch_bounds__(256) k_flags(Tables tb, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz) {
+__global__ void __launch_bounds__(256) k_flags(Tables tb, const uint32_t* __restrict__ ebits_all, uint32_t* nz_map,
+                                               uint32_t* out_nz, uint32_t* in_nz) {
     const int lane = threadIdx.x & 31;
     const uint32_t n_warps = gridDim.x * (blockDim.x >> 5), warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const uint32_t per = (tb.n_flag_units + n_warps - 1) / n_warps;
@@ -101,7 +102,7 @@ __global__ void __launch_bounds__(256) k_flags(Tables tb, uint32_t* nz_map, uint
         }
         const TensorDesc& d = tb.tensors[t];
         const uint32_t KK = d.KK, I = d.I, O = d.O, n_kernels = O * I;
-        const uint32_t* ebits = tb.ebits + d.off_mask;
+        const uint32_t* ebits = ebits_all + d.off_mask;
         uint32_t* g_in = in_nz + d.off_innz;
         uint32_t* g_out = out_nz + d.off_outnz;
         uint32_t* g_map = nz_map ? nz_map + d.off_nzmap : nullptr;
@@ -371,6 +372,202 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_sweep(Tables tb, ThresholdW
     }
 }
 
+
+// The fused sweep for up to kMultiMax variants of one portfolio at once: every tile of the dense weights is
+// read once and masked against each variant's threshold in turn, so a variant costs one write of the
+// model plus 1/G of a read instead of a read and a write.  Same tile walk and the same two paths as
+// k_sweep<mask, structures>; the per-variant state (threshold, tie tables, destinations) is an array.
+template <int DT, int G>
+__global__ void __launch_bounds__(kTileThreads, G == 1 ? 4 : 3) k_sweep_multi(Tables tb, ThresholdWs ws, const dnns_threshold* __restrict__ thr,
+                                                                 MultiSweepArgs ma, uint32_t n_clear_a, uint32_t n_clear_b) {
+    constexpr int P = Elem<DT>::kPerVec;
+    constexpr int GL = 32 / P;  // lanes per bit word
+    constexpr uint32_t kTileElems = kTileBytes / Elem<DT>::kBytes;
+    constexpr uint32_t kKeyMask = DT == DNNS_F32 ? 0x7FFFFFFFu : 0x7FFF7FFFu;
+    __shared__ uint32_t scratch[33];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        for (uint32_t i = blockIdx.x * kTileThreads + threadIdx.x; i < n_clear_a; i += gridDim.x * kTileThreads) ma.clear_a[g][i] = 0;
+        for (uint32_t i = blockIdx.x * kTileThreads + threadIdx.x; i < n_clear_b; i += gridDim.x * kTileThreads) ma.clear_b[g][i] = 0;
+    }
+    const int lane = threadIdx.x & 31;
+    const bool word_lane = (lane & (GL - 1)) == 0;
+    const uint32_t per = (tb.n_tiles + gridDim.x - 1) / gridDim.x;
+    const uint32_t lo = min(tb.n_tiles, blockIdx.x * per), hi = min(tb.n_tiles, lo + per);
+    uint32_t tile = lo;
+    while (tile < hi) {
+        const TensorDesc& d = tb.tensors[tb.tile_tensor[tile]];
+        const uint32_t span_end = min(hi, d.tile0 + d.n_tiles);
+        const uint32_t numel = d.numel, tile0 = d.tile0;
+        const char* src = static_cast<const char*>(d.src);
+        const uint64_t arena_off = d.arena_off;
+        const uint32_t off_mask = d.off_mask;
+        uint32_t tau[G], thr_uniform[G], n_tie[G];  // n_tie saturated to 32 bits: tile counts never reach it otherwise
+        bool use_tables[G];
+        bool any_tables = false;
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            tau[g] = thr_uniform[g] = n_tie[g] = 0;
+            use_tables[g] = false;
+            if (d.seg >= 0) {
+                const dnns_threshold r = thr[(size_t)ma.variant[g] * tb.n_segs + d.seg];
+                tau[g] = r.tau_bits;
+                n_tie[g] = (uint32_t)min(r.n_tie, (uint64_t)0xFFFFFFFFu);
+                if (r.n_below + r.n_tie == 0) thr_uniform[g] = 0;
+                else if (r.n_tie >= r.n_equal) thr_uniform[g] = tau[g] + 1;
+                else use_tables[g] = true;
+                any_tables |= use_tables[g];
+            }
+        }
+        uint4 nxt[kVecPerThread];
+        uint32_t nxt_before[G], nxt_here[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) nxt_before[g] = nxt_here[g] = 0;
+        auto issue = [&](uint32_t t) {
+            const uint32_t e0 = (t - tile0) * kTileElems;
+            if (e0 + kTileElems <= numel) {
+                const uint4* p = reinterpret_cast<const uint4*>(src + (size_t)e0 * Elem<DT>::kBytes) + threadIdx.x;
+#pragma unroll
+                for (int u = 0; u < kVecPerThread; ++u) nxt[u] = __ldg(p + u * kTileThreads);
+            } else {
+#pragma unroll
+                for (int u = 0; u < kVecPerThread; ++u)
+                    load_vec<DT>(src, e0 + (u * kTileThreads + threadIdx.x) * P, numel, nxt[u]);
+            }
+            if (any_tables) {
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    if (use_tables[g]) {
+                        nxt_before[g] = ws.tie_prefix[(size_t)ma.variant[g] * tb.n_tiles + t];
+                        nxt_here[g] = ws.tile_ties[(size_t)ma.variant[g] * tb.n_tiles + t];
+                    }
+                }
+            }
+        };
+        issue(tile);
+        for (; tile < span_end; ++tile) {
+            uint4 v[kVecPerThread];
+#pragma unroll
+            for (int u = 0; u < kVecPerThread; ++u) v[u] = nxt[u];
+            uint32_t thr_eff[G], quota[G];
+            bool any_split = false;
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                thr_eff[g] = thr_uniform[g];
+                quota[g] = 0xFFFFFFFFu;  // no split
+                if (use_tables[g]) {
+                    const uint32_t before = nxt_before[g], here = nxt_here[g];
+                    if (before >= n_tie[g]) thr_eff[g] = tau[g];
+                    else {
+                        thr_eff[g] = tau[g] + 1;
+                        if ((uint64_t)before + here > n_tie[g]) {
+                            quota[g] = n_tie[g] - before;  // this tile ranks its ties: those below quota are masked
+                            any_split = true;
+                        }
+                    }
+                }
+            }
+            if (tile + 1 < span_end) issue(tile + 1);
+
+            const uint32_t e0 = (tile - tile0) * kTileElems;
+            const uint32_t n_e = min(kTileElems, numel - e0);
+            if (n_e == kTileElems && !any_split) {
+                // ---- lean path: a whole tile, one threshold per variant
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    uint4* out = reinterpret_cast<uint4*>(ma.dst[g] + arena_off + (size_t)e0 * Elem<DT>::kBytes) + threadIdx.x;
+                    uint32_t* mask_words = ma.mask_bits[g] ? ma.mask_bits[g] + off_mask : nullptr;
+                    uint32_t* nz_words = ma.ebits[g] + off_mask;
+                    const uint32_t te = thr_eff[g];
+                    const bool zeros_survive = te == 0;
+#pragma unroll
+                    for (int u = 0; u < kVecPerThread; ++u) {
+                        const uint32_t vi = u * kTileThreads + threadIdx.x;
+                        uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                        uint32_t keep = 0, nz = 0;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t m = w[j] & kKeyMask;
+                            if (DT == DNNS_F32) {
+                                const bool k = m >= te;
+                                w[j] = k ? w[j] : 0u;
+                                keep |= k ? (1u << j) : 0u;
+                                if (zeros_survive) nz |= m != 0 ? (1u << j) : 0u;
+                            } else {
+                                const uint32_t m0 = m & 0xFFFFu, m1 = m >> 16;
+                                const bool k0 = m0 >= te, k1 = m1 >= te;
+                                w[j] &= (k0 ? 0x0000FFFFu : 0u) | (k1 ? 0xFFFF0000u : 0u);
+                                keep |= (k0 ? (1u << (2 * j)) : 0u) | (k1 ? (2u << (2 * j)) : 0u);
+                                if (zeros_survive) nz |= (m0 != 0 ? (1u << (2 * j)) : 0u) | (m1 != 0 ? (2u << (2 * j)) : 0u);
+                            }
+                        }
+                        out[u * kTileThreads] = make_uint4(w[0], w[1], w[2], w[3]);
+                        // survivors of a non-zero threshold are non-zero: their keep bits are their non-zero bits
+                        const uint32_t keep_word = (mask_words || !zeros_survive) ? gather_word<P>(keep, lane) : 0u;
+                        const uint32_t nz_word = zeros_survive ? gather_word<P>(nz, lane) : keep_word;
+                        if (word_lane) {
+                            if (mask_words) mask_words[e0 / 32 + vi / GL] = keep_word;
+                            nz_words[e0 / 32 + vi / GL] = nz_word;
+                        }
+                    }
+                }
+            } else {
+                // ---- general path: ragged last tile of a tensor, or a tile that ranks the ties of some variant
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    char* dst = ma.dst[g] + arena_off;
+                    uint32_t* mask_words = ma.mask_bits[g] ? ma.mask_bits[g] + off_mask : nullptr;
+                    uint32_t* nz_words = ma.ebits[g] + off_mask;
+                    const uint32_t te = thr_eff[g], tg = tau[g], qg = quota[g];
+                    const bool split = qg != 0xFFFFFFFFu;
+                    uint32_t tie_carry = 0;
+#pragma unroll
+                    for (int u = 0; u < kVecPerThread; ++u) {
+                        const uint32_t vi = u * kTileThreads + threadIdx.x;
+                        const uint32_t e = e0 + vi * P;
+                        const int n = e >= numel ? 0 : (int)min((uint32_t)P, numel - e);
+                        uint32_t key[P];
+                        vec_keys<DT>(v[u], key);
+                        uint32_t tie_rank = 0;
+                        if (split) {
+                            uint32_t c = 0;
+#pragma unroll
+                            for (int j = 0; j < P; ++j) c += (j < n && key[j] == tg);
+                            uint32_t total;
+                            tie_rank = tie_carry + block_exclusive_scan<uint32_t>(c, scratch, &total);
+                            tie_carry += total;
+                        }
+                        uint32_t keep = 0, nz = 0;
+#pragma unroll
+                        for (int j = 0; j < P; ++j) {
+                            bool k = key[j] >= te;
+                            if (split && key[j] == tg) k = tie_rank++ >= qg;
+                            k = k && j < n;
+                            keep |= (uint32_t)k << j;
+                            nz |= (uint32_t)(k && key[j] != 0) << j;
+                        }
+                        uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                        if (DT == DNNS_F32) {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) w[j] = (keep >> j) & 1u ? w[j] : 0u;
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                w[j] &= ((keep >> (2 * j)) & 1u ? 0x0000FFFFu : 0u) | ((keep >> (2 * j + 1)) & 1u ? 0xFFFF0000u : 0u);
+                        }
+                        store_vec<DT>(dst, e, numel, make_uint4(w[0], w[1], w[2], w[3]));
+                        const uint32_t keep_word = gather_word<P>(keep, lane), nz_word = gather_word<P>(nz, lane);
+                        if (word_lane && (vi / GL) * 32 < n_e) {
+                            if (mask_words) mask_words[e0 / 32 + vi / GL] = keep_word;
+                            nz_words[e0 / 32 + vi / GL] = nz_word;
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
 template <int DT>
 void launch_dt(bool do_mask, bool do_struct, dim3 grid, cudaStream_t st, const Tables& tb, const ThresholdWs& ws,
                const dnns_threshold* thr, int variant, const char* src_arena, char* dst_arena, uint32_t* mask_bits,
@@ -403,9 +600,38 @@ int launch_tile_sweep(const Tables& tb, const ThresholdWs& ws, bool do_mask, boo
     if (do_struct) {
         const uint32_t blocks = min((uint32_t)n_sm * 64u, (tb.n_flag_units + 7) / 8);  // one unit per warp if possible
         ScopedKernel timed("k_flags", st);
-        k_flags<<<max(blocks, 1u), 256, 0, st>>>(tb, nz_map, out_nz, in_nz);
+        k_flags<<<max(blocks, 1u), 256, 0, st>>>(tb, tb.ebits, nz_map, out_nz, in_nz);
     }
     return cudaGetLastError() == cudaSuccess ? (do_struct ? 2 : 1) : -1;
+}
+
+
+int launch_multi_sweep(const Tables& tb, const ThresholdWs& ws, const dnns_threshold* thr_dev, const MultiSweepArgs& ma,
+                       int n_variants, uint32_t* const* nz_map, uint32_t n_out_words, uint32_t n_in_words, int n_sm,
+                       cudaStream_t st) {
+    const dim3 grid(min((uint32_t)n_sm * (n_variants == 1 ? 4u : 3u), tb.n_tiles));  // resident blocks per SM
+    {
+        ScopedKernel timed("k_sweep_multi", st);
+#define DNNS_LAUNCH_MULTI(DT, G) k_sweep_multi<DT, G><<<grid, kTileThreads, 0, st>>>(tb, ws, thr_dev, ma, n_out_words, n_in_words)
+        if (tb.dtype == DNNS_F32) {
+            if (n_variants == 1) DNNS_LAUNCH_MULTI(DNNS_F32, 1);
+            else if (n_variants == 2) DNNS_LAUNCH_MULTI(DNNS_F32, 2);
+            else if (n_variants == 3) DNNS_LAUNCH_MULTI(DNNS_F32, 3);
+            else DNNS_LAUNCH_MULTI(DNNS_F32, 4);
+        } else {
+            if (n_variants == 1) DNNS_LAUNCH_MULTI(DNNS_BF16, 1);
+            else if (n_variants == 2) DNNS_LAUNCH_MULTI(DNNS_BF16, 2);
+            else if (n_variants == 3) DNNS_LAUNCH_MULTI(DNNS_BF16, 3);
+            else DNNS_LAUNCH_MULTI(DNNS_BF16, 4);
+        }
+#undef DNNS_LAUNCH_MULTI
+    }
+    const uint32_t blocks = min((uint32_t)n_sm * 64u, (tb.n_flag_units + 7) / 8);
+    for (int g = 0; g < n_variants; ++g) {
+        ScopedKernel timed("k_flags", st);
+        k_flags<<<max(blocks, 1u), 256, 0, st>>>(tb, ma.ebits[g], nz_map ? nz_map[g] : nullptr, ma.clear_a[g], ma.clear_b[g]);
+    }
+    return cudaGetLastError() == cudaSuccess ? 1 + n_variants : -1;
 }
 
 }  // namespace dnns

@@ -77,8 +77,9 @@ class Session:
     """A plan with its workspace and one set of output buffers for one variant at a time."""
 
     def __init__(self, dm: DeviceModel, scope: int, max_variants: int, want_mask_bits: bool = True,
-                 want_nz_map: bool = True):
-        self.dm, self.scope, self.max_variants = dm, scope, max_variants
+                 want_nz_map: bool = True, slots: int = 1):
+        """slots > 1 adds that many more sets of per-variant buffers for the multi-variant sweep."""
+        self.dm, self.scope, self.max_variants, self.slots = dm, scope, max_variants, slots
         dev = dm.device
         nbytes = B.dnns_workspace_bytes(dm.c, scope, max_variants)
         if nbytes == 0:
@@ -110,6 +111,17 @@ class Session:
         self.compact_arena = torch.empty(int(L.compact_arena_bytes), dtype=torch.uint8, device=dev)
         self.dst_offsets = torch.zeros(L.n_compact_items, dtype=torch.int64, device=dev)
         self.dst_shapes = i32(2 * T)
+        # slot 0 is the set above; slots 1.. are further sets of what differs per variant before the rebuild
+        self.extra = []
+        for _ in range(1, slots):
+            self.extra.append({
+                "masked": torch.empty(int(L.masked_arena_bytes), dtype=torch.uint8, device=dev),
+                "mask_bits": i32(L.mask_words) if want_mask_bits else None,
+                "nz_map": i32(L.nz_map_words) if want_nz_map else None,
+                "out_nz": i32(L.out_nz_words), "in_nz": i32(L.in_nz_words)})
+
+    def _slot(self, name: str, slot: int):
+        return getattr(self, name) if slot == 0 else self.extra[slot - 1][name]
 
     def close(self):
         if self.plan is not None:
@@ -144,13 +156,21 @@ class Session:
                                    0 if self.nz_map is None else self.nz_map.data_ptr(), self.out_nz.data_ptr(),
                                    self.in_nz.data_ptr(), _stream())
 
-    def propagate_keep(self, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1):
-        B.dnns_propagate_keep(self.plan, self.out_nz.data_ptr(), self.in_nz.data_ptr(), policy, min_keep,
+    def mask_and_structures_multi(self, first_variant: int, n_variants: int):
+        """Steps 2 and 3 of n_variants consecutive variants in one sweep; variant first_variant + g lands in slot g."""
+        ptrs = lambda name: [None if self._slot(name, g) is None else self._slot(name, g).data_ptr() for g in range(n_variants)]
+        B.dnns_mask_and_structures_multi(self.plan, self.thr.data_ptr(), first_variant, n_variants, ptrs("masked"),
+                                         None if self.mask_bits is None else ptrs("mask_bits"),
+                                         None if self.nz_map is None else ptrs("nz_map"), ptrs("out_nz"), ptrs("in_nz"),
+                                         _stream())
+
+    def propagate_keep(self, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1, slot: int = 0):
+        B.dnns_propagate_keep(self.plan, self._slot("out_nz", slot).data_ptr(), self._slot("in_nz", slot).data_ptr(), policy, min_keep,
                               self.keep_bits.data_ptr(), self.keep_idx.data_ptr(), self.keep_count.data_ptr(),
                               self.stats.data_ptr(), _stream())
 
-    def compact(self, from_model: bool = False, dst_bytes: Optional[int] = None):
-        B.dnns_compact(self.plan, 0 if from_model else self.masked.data_ptr(), self.keep_idx.data_ptr(),
+    def compact(self, from_model: bool = False, dst_bytes: Optional[int] = None, slot: int = 0):
+        B.dnns_compact(self.plan, 0 if from_model else self._slot("masked", slot).data_ptr(), self.keep_idx.data_ptr(),
                        self.keep_count.data_ptr(), self.compact_arena.data_ptr(),
                        self.compact_arena.numel() if dst_bytes is None else dst_bytes, self.dst_offsets.data_ptr(),
                        self.dst_shapes.data_ptr(), _stream())
@@ -199,12 +219,12 @@ class Session:
     def _np_dtype(self):
         return np.float32 if self.dm.dtype == B.DNNS_F32 else np.uint16
 
-    def masked_tensors(self, in_place: bool = False) -> List[np.ndarray]:
+    def masked_tensors(self, in_place: bool = False, slot: int = 0) -> List[np.ndarray]:
         wl, eb = self.dm.wl, self.dm.elem_bytes
         if in_place:
             raw, offs = self.dm.weights.cpu().numpy(), self.dm.weight_offsets
         else:
-            raw, offs = self.masked.cpu().numpy(), self.arena_offset
+            raw, offs = self._slot("masked", slot).cpu().numpy(), self.arena_offset
         return [raw[int(o): int(o) + t.numel * eb].view(self._np_dtype()).reshape(t.O, t.I, t.KH, t.KW).copy()
                 for t, o in zip(wl.tensors, offs)]
 
@@ -212,15 +232,15 @@ class Session:
         raw = buf.cpu().numpy().view(np.uint32)
         return [raw[int(o): int(o) + (n + 31) // 32].copy() for o, n in zip(offsets, nbits)]
 
-    def mask_words(self):
-        return self._split_words(self.mask_bits, self.mask_offset, [t.numel for t in self.dm.wl.tensors])
+    def mask_words(self, slot: int = 0):
+        return self._split_words(self._slot("mask_bits", slot), self.mask_offset, [t.numel for t in self.dm.wl.tensors])
 
-    def structure_words(self):
+    def structure_words(self, slot: int = 0):
         wl = self.dm.wl
-        nz = None if self.nz_map is None else self._split_words(self.nz_map, self.nz_map_offset,
+        nz = None if self.nz_map is None else self._split_words(self._slot("nz_map", slot), self.nz_map_offset,
                                                                  [t.O * t.I for t in wl.tensors])
-        return (nz, self._split_words(self.out_nz, self.out_nz_offset, [t.O for t in wl.tensors]),
-                self._split_words(self.in_nz, self.in_nz_offset, [t.I for t in wl.tensors]))
+        return (nz, self._split_words(self._slot("out_nz", slot), self.out_nz_offset, [t.O for t in wl.tensors]),
+                self._split_words(self._slot("in_nz", slot), self.in_nz_offset, [t.I for t in wl.tensors]))
 
     def keep_sets(self):
         wl = self.dm.wl

@@ -28,26 +28,38 @@ def expected_offsets(sizes_bytes):
 
 
 def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCER | O.RULE_CONSUMER, min_keep=1,
-                      weights=None, check_structure_maps=True, fused=False):
-    """Thresholds for all of wl.ks in one call, then steps 2-5 for the chosen variants."""
+                      weights=None, check_structure_maps=True, fused=False, multi=0):
+    """Thresholds for all of wl.ks in one call, then steps 2-5 for the chosen variants.
+    multi = G > 0: steps 2 and 3 of G consecutive variants at a time through the multi-variant sweep."""
     om = O.OracleModel(wl, dtype, weights)
     dm = DeviceModel(wl, dtype, weights=weights)
-    ses = Session(dm, wl.scope, len(wl.ks))
+    ses = Session(dm, wl.scope, len(wl.ks), slots=max(multi, 1))
     ses.magnitude_threshold(wl.ks)
     rec_gpu = ses.records()
     rec_cpu = O.threshold(om, wl.scope, wl.ks)
     for f in ("tau_bits", "n_below", "n_tie", "n_equal"):
         assert np.array_equal(rec_gpu[f], rec_cpu[f]), f
     eb = 4 if dtype == B.DNNS_F32 else 2
-    for v in (range(len(wl.ks)) if variants is None else variants):
-        ses.variant(v, policy, min_keep, fused=fused)
+    todo = list(range(len(wl.ks)) if variants is None else variants)
+    for pos, v in enumerate(todo):
+        slot = 0
+        if multi:
+            slot = pos % multi
+            if slot == 0:
+                n = min(multi, len(todo) - pos)
+                assert todo[pos: pos + n] == list(range(v, v + n)), "the multi-variant sweep takes consecutive variants"
+                ses.mask_and_structures_multi(v, n)
+            ses.propagate_keep(policy, min_keep, slot=slot)
+            ses.compact(slot=slot)
+        else:
+            ses.variant(v, policy, min_keep, fused=fused)
         assert ses.device_status() == B.DNNS_OK
         masked_cpu, bits_cpu = O.apply_mask(om, wl.scope, rec_cpu[v])
-        for i, (a, b) in enumerate(zip(ses.masked_tensors(), masked_cpu.weights)):
+        for i, (a, b) in enumerate(zip(ses.masked_tensors(slot=slot), masked_cpu.weights)):
             assert bits_eq(a, b), f"masked weights, variant {v}, tensor {i}"
-        assert_words(ses.mask_words(), bits_cpu, f"mask bits v{v}")
+        assert_words(ses.mask_words(slot), bits_cpu, f"mask bits v{v}")
         nz_c, out_c, in_c = O.zero_structures(masked_cpu)
-        nz_g, out_g, in_g = ses.structure_words()
+        nz_g, out_g, in_g = ses.structure_words(slot)
         if check_structure_maps:
             assert_words(nz_g, nz_c, f"kernel map v{v}")
         assert_words(out_g, out_c, f"out flags v{v}")

@@ -20,6 +20,14 @@ def test_small_configs_every_variant(make, dtype, fused):
     compare_portfolio(make(), dtype, fused=fused)
 
 
+@pytest.mark.parametrize("multi", [1, 2, 3, 4])
+@pytest.mark.parametrize("dtype", [B.DNNS_F32, B.DNNS_BF16])
+@pytest.mark.parametrize("make", [W.toy, lambda: W.small_resnet(seed=3), W.resnet56])
+def test_multi_variant_sweep_every_variant(make, dtype, multi):
+    """Groups of up to four variants masked and analysed in one sweep: each variant as from its own sweep."""
+    compare_portfolio(make(), dtype, multi=multi)
+
+
 @pytest.mark.parametrize("policy", [O.RULE_PRODUCER, O.RULE_CONSUMER, O.RULE_PRODUCER | O.RULE_CONSUMER | O.SHIFT_STRICT])
 @pytest.mark.parametrize("min_keep", [0, 1, 5])
 def test_policies_and_min_keep(policy, min_keep):
@@ -41,6 +49,7 @@ def test_per_tensor_scope_and_odd_shapes(dtype):
                       [n - 1 for n in sizes], sizes], np.uint64)
     compare_portfolio(wl, dtype)
     compare_portfolio(wl, dtype, variants=[1, 3], fused=True)
+    compare_portfolio(wl, dtype, multi=2)
 
 
 def test_non_prunable_tensor_and_1x1_chain():
@@ -74,6 +83,8 @@ def test_special_values_and_heavy_ties():
     assert (rec["n_tie"] < rec["n_equal"]).any()                   # the split-tie path really ran
     compare_portfolio(wl, B.DNNS_BF16)
     compare_portfolio(wl, B.DNNS_F32, fused=True)
+    compare_portfolio(wl, B.DNNS_F32, multi=4)     # tiles that rank the ties of several variants at once
+    compare_portfolio(wl, B.DNNS_BF16, multi=3)
 
 
 def test_deep_chain_with_more_than_1024_gather_items():
