@@ -154,6 +154,8 @@ def main():
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--stepwise", action="store_true", help="mask and zero-structure detection as two sweeps")
+    ap.add_argument("--multi", type=int, default=-1,
+                    help="variants per sweep over the dense weights (1..4; 0: one fused call per variant; default 4 for f32, 2 for bf16)")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph replay")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -190,13 +192,20 @@ def main():
     eb = 4 if dtype == 0 else 2
     N = wl.n_prunable
     dm = DeviceModel(wl, dtype, device=f"cuda:{local_rank}", pinned_host=True)
-    ses = Session(dm, wl.scope, V, want_mask_bits=True, want_nz_map=False)
+    G = args.multi if args.multi >= 0 else (4 if dtype == 0 else 2)
+    G = 0 if args.stepwise else min(G, 4, V)
+    groups = [(v0, min(G, V - v0)) for v0 in range(0, V, G)] if G else []
+    ses = Session(dm, wl.scope, V, want_mask_bits=True, want_nz_map=False, slots=max(G, 1))
     need_flush = N * eb <= 126e6
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dm.device) if need_flush else None
 
     names = (["threshold", "mask", "structures", "propagate", "compact"] if args.stepwise
              else ["threshold", "mask+structures", "propagate", "compact"])
     spans = {n: [] for n in names}
+    calls_per_step = {n: V for n in names}
+    calls_per_step["threshold"] = 1
+    if G:
+        calls_per_step["mask+structures"] = len(groups)
 
     def step(record: bool):
         def timed(name, fn, *a):
@@ -208,7 +217,12 @@ def main():
             e1.record()
             spans[name].append((e0, e1))
         timed("threshold", ses.magnitude_threshold, wl.ks)
-        for v in range(V):
+        for v0, n in groups:                       # n variants per read of the dense weights
+            timed("mask+structures", ses.mask_and_structures_multi, v0, n)
+            for g in range(n):
+                timed("propagate", lambda: ses.propagate_keep(slot=g))
+                timed("compact", lambda: ses.compact(slot=g))
+        for v in (range(V) if not G else ()):
             if args.stepwise:
                 timed("mask", ses.apply_mask, v)
                 timed("structures", ses.zero_structures)
@@ -282,7 +296,7 @@ def main():
     plain_ms = timed_steps(lambda: step(True))
     launches_plain = ses.launch_count() - launches0
     # the same steps once more with an event pair around every single kernel (dnns_plan_profile)
-    kernel_names = ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_ties", "k_tie_scan", "k_sweep", "k_flags",
+    kernel_names = ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_ties", "k_tie_scan", "k_sweep<", "k_sweep_multi", "k_flags",
                     "k_propagate", "k_compact_layout", "k_compact_gather"]
     ses.profile(True)
     timed_steps(lambda: step(False))
@@ -308,7 +322,7 @@ def main():
     ms_per_variant = whole_job_ms_per_variant(ms_per_step, V, world)
     per_call = {n: statistics.mean(a.elapsed_time(b) for a, b in spans[n]) for n in names}
     plain_per_step = plain_ms / args.steps
-    share = {n: per_call[n] * (1 if n == "threshold" else V) / plain_per_step for n in names}
+    share = {n: per_call[n] * calls_per_step[n] / plain_per_step for n in names}
 
     # algorithmic bytes: one read of every input a step consumes, one write of every output
     # (the fused sweep moves 2*N*b + N/8 per launch; the stepwise accounting B_v charges the path 3*N*b + N/8)
@@ -317,13 +331,19 @@ def main():
     portfolio_bytes = alg["threshold"] + V * (alg["mask"] + alg["structures"]) + sum((r + n) * eb for r, n in zip(R, Nn))
     moved_bytes = alg["threshold"] + V * (alg["mask"] + (alg["structures"] if args.stepwise else 0)) + \
         sum((r + n) * eb for r, n in zip(R, Nn))
+    if G:   # one read of the dense weights per group, one write (+ mask bits) per variant
+        multi_bytes = sum(N * eb + n * (N * eb + N / 8) for _, n in groups)
+        alg["mask+structures"] = multi_bytes / len(groups)
+        moved_bytes = alg["threshold"] + multi_bytes + sum((r + n) * eb for r, n in zip(R, Nn))
     peak, peak_kind = load_peaks()
     # the dominant kernel: largest share of the summed kernel time; its algorithmic bytes per launch
     kernel_alg = {"k_hist1": N * eb, "k_hist2": N * eb, "k_ties": N * eb,
-                  "k_sweep": alg["mask"] if args.stepwise else alg["mask+structures"] + N / 8,  # + the element bits it packs
+                  "k_sweep<": 2 * N * eb + N / 4,          # weights in and out, mask bits, the element bits it packs
                   "k_compact_gather": alg["compact"]}
     if args.stepwise:
-        kernel_alg["k_sweep"] = (alg["mask"] + alg["structures"] + N / 8) / 2   # two sweeps per variant, averaged
+        kernel_alg["k_sweep<"] = (alg["mask"] + alg["structures"] + N / 8) / 2   # two sweeps per variant, averaged
+    if G:   # per launch: one read, n writes with their mask and element bits
+        kernel_alg["k_sweep_multi"] = sum(N * eb + n * (N * eb + N / 4) for _, n in groups) / len(groups)
     kernel_total = sum(k["ms_per_step"] for k in kernel_ms.values())
     for k in kernel_ms.values():
         k["share"] = k["ms_per_step"] / kernel_total
@@ -332,7 +352,8 @@ def main():
     for kn, k in kernel_ms.items():
         if kn in kernel_alg:
             k["gbs"] = kernel_alg[kn] / (k["avg_ms"] * 1e-3) / 1e9
-    kernel_label = {"k_sweep": "k_sweep<mask>+<structures>" if args.stepwise else "k_sweep<mask+structures>"}
+    kernel_label = {"k_sweep<": "k_sweep<mask>+<structures>" if args.stepwise else "k_sweep<mask+structures>",
+                    "k_sweep_multi": f"k_sweep_multi<{G}>"}
 
     # ---- Module 1 on a rebuilt variant (not part of the portfolio step): conv + BatchNorm fusion in place
     fold_ms = []
@@ -425,7 +446,13 @@ def main():
         h2d += dm.weight_bytes
         ses.magnitude_threshold(wl.ks)
         for v in range(V):
-            ses.variant(v, fused=not args.stepwise)
+            if G:
+                if v % G == 0:
+                    ses.mask_and_structures_multi(v, min(G, V - v))
+                ses.propagate_keep(slot=v % G)
+                ses.compact(slot=v % G)
+            else:
+                ses.variant(v, fused=not args.stepwise)
             offs = ses.dst_offsets.cpu()           # synchronises: the sizes are only known on the device
             shp = ses.dst_shapes.cpu()
             cnt = ses.keep_count.cpu()
@@ -456,7 +483,9 @@ def main():
         "effective_gbs": portfolio_bytes / (ms_per_step * 1e-3) / 1e9,
         "effective_frac_of_peak": portfolio_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
         "algorithmic_bytes_per_variant": portfolio_bytes / V,
-        "moved_gbs": moved_bytes / (ms_per_step * 1e-3) / 1e9, "sweeps": "stepwise" if args.stepwise else "fused mask+structures",
+        "moved_gbs": moved_bytes / (ms_per_step * 1e-3) / 1e9,
+        "sweeps": "stepwise" if args.stepwise else (f"fused mask+structures, {G} variants per read of the dense weights" if G
+                                                    else "fused mask+structures"),
         "launch": "cuda graph replay" if graph is not None else "plain stream launches", "ms_per_step_plain": plain_per_step,
         "per_call_ms": per_call, "share": share,
         "per_call_gbs": {n: (alg[n] / (per_call[n] * 1e-3) / 1e9 if alg[n] else None) for n in names},

@@ -479,6 +479,7 @@ __global__ void __launch_bounds__(kTileThreads, G == 1 ? 4 : 3) k_sweep_multi(Ta
                     uint32_t* mask_words = ma.mask_bits[g] ? ma.mask_bits[g] + off_mask : nullptr;
                     uint32_t* nz_words = ma.ebits[g] + off_mask;
                     const uint32_t te = thr_eff[g];
+                    const uint32_t te2 = te * 0x00010001u;  // the threshold in both halves of a word (16-bit keys)
                     const bool zeros_survive = te == 0;
 #pragma unroll
                     for (int u = 0; u < kVecPerThread; ++u) {
@@ -494,11 +495,16 @@ __global__ void __launch_bounds__(kTileThreads, G == 1 ? 4 : 3) k_sweep_multi(Ta
                                 keep |= k ? (1u << j) : 0u;
                                 if (zeros_survive) nz |= m != 0 ? (1u << j) : 0u;
                             } else {
-                                const uint32_t m0 = m & 0xFFFFu, m1 = m >> 16;
-                                const bool k0 = m0 >= te, k1 = m1 >= te;
-                                w[j] &= (k0 ? 0x0000FFFFu : 0u) | (k1 ? 0xFFFF0000u : 0u);
-                                keep |= (k0 ? (1u << (2 * j)) : 0u) | (k1 ? (2u << (2 * j)) : 0u);
-                                if (zeros_survive) nz |= (m0 != 0 ? (1u << (2 * j)) : 0u) | (m1 != 0 ? (2u << (2 * j)) : 0u);
+                                // both 15-bit keys of the word at once: with bit 15 of each half set, subtracting
+                                // the threshold leaves that bit standing exactly where key >= threshold, and no
+                                // borrow crosses into the other half (te <= 0x8000)
+                                const uint32_t ge = (((m | 0x80008000u) - te2) >> 15) & 0x00010001u;
+                                w[j] &= ge * 0xFFFFu;
+                                keep |= ((ge | (ge >> 15)) & 3u) << (2 * j);
+                                if (zeros_survive) {
+                                    const uint32_t ne = (((m | 0x80008000u) - 0x00010001u) >> 15) & 0x00010001u;  // key >= 1
+                                    nz |= ((ne | (ne >> 15)) & 3u) << (2 * j);
+                                }
                             }
                         }
                         out[u * kTileThreads] = make_uint4(w[0], w[1], w[2], w[3]);
