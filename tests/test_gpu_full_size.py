@@ -13,12 +13,13 @@ from paper_2309_06973_b200 import workloads as W
 pytestmark = pytest.mark.gpu
 
 
-def forward_check(wl, ses, dtype):
+def forward_check(wl, ses, dtype, slot=0):
+    """slot: which buffer set of the session holds the masked weights of the variant rebuilt last."""
     is_bf16 = dtype == B.DNNS_BF16
     x = torch.from_numpy(np.random.default_rng(1).standard_normal((2, 3, wl.input_hw, wl.input_hw)).astype(np.float32))
     cw, cbn, cb, _, _ = ses.compacted()
     kb, _, _, _ = ses.keep_sets()
-    mw, mbn, mb = silenced_reference(wl, ses.masked_tensors(), wl.bn_params, wl.biases, kb)
+    mw, mbn, mb = silenced_reference(wl, ses.masked_tensors(slot=slot), wl.bn_params, wl.biases, kb)
     y_ref = forward(wl, mw, mbn, mb, x, is_bf16)
     y = forward(wl, cw, cbn, cb, x, is_bf16)
     assert float((y - y_ref).abs().max()) <= 1e-5 * float(y_ref.abs().max())
@@ -35,6 +36,8 @@ def test_resnet50_three_variants():
     wl = W.resnet50()
     ses = compare_portfolio(wl, B.DNNS_F32, fused=True)
     forward_check(wl, ses, B.DNNS_F32)
+    ses = compare_portfolio(wl, B.DNNS_F32, multi=3)          # all three variants from one read of the weights
+    forward_check(wl, ses, B.DNNS_F32, slot=2)
 
 
 @pytest.mark.parametrize("dtype", [B.DNNS_F32, B.DNNS_BF16])
@@ -43,3 +46,7 @@ def test_resnet152_portfolio(dtype):
     ses = compare_portfolio(wl, dtype, variants=[0], fused=False)
     ses = compare_portfolio(wl, dtype, variants=[7], fused=True)
     forward_check(wl, ses, dtype)
+    # the benchmark's configuration: four (fp32) or two (bf16) variants per sweep
+    G = 4 if dtype == B.DNNS_F32 else 2
+    ses = compare_portfolio(wl, dtype, variants=list(range(8 - G, 8)), multi=G)
+    forward_check(wl, ses, dtype, slot=G - 1)
