@@ -153,7 +153,23 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
                 for (uint32_t e = 0; e < VE; ++e) idx[u][e] = (e < n0 ? base0 : base1) + e;
                 continue;
             }
-            // vectors that cross a filter boundary or the end of the item: walk element by element
+            if (Ln >= VE) {
+                // vectors that cross into the next filter or reach the end of the item: one formula per element
+                // (element e sits at offset rem + e of row a, or past its end in row a + 1), no walk
+                const uint32_t row0 = (uint32_t)ko[a] * Cin;
+                const uint32_t row1 = a + 1 < On ? (uint32_t)ko[a + 1] * Cin : 0u;
+#pragma unroll
+                for (uint32_t e = 0; e < VE; ++e) {
+                    uint32_t re = rem + e;
+                    const bool wrap = re >= Ln;
+                    re = wrap ? re - Ln : re;
+                    const uint32_t c = blk == 1 ? re : (blk == 9 ? re / 9u : re / blk), r = re - c * blk;
+                    const uint32_t col = ki ? (uint32_t)ki[c] : c;
+                    if (f + e < total) idx[u][e] = ((wrap ? row1 : row0) + col) * blk + r;
+                }
+                continue;
+            }
+            // rows shorter than a vector: walk element by element
             uint32_t c = blk == 1 ? rem : (blk == 9 ? rem / 9u : rem / blk), r = rem - c * blk;
             uint32_t row = (uint32_t)ko[a] * Cin, col = ki ? (uint32_t)ki[c] : c;
             const uint32_t nv = min(VE, total - f);
