@@ -123,44 +123,53 @@ __device__ __forceinline__ void emit_run(Sink& s, uint32_t v, uint32_t len) {
     else if (rep) s.literal(v, rep);
 }
 
-// Walk the n (<= 512) bytes of a sub-block at p (16-byte aligned) and hand its runs to the sink.
+// Bit i of the result: byte i of w differs from the byte before it (byte 0 from the top byte of `before`).
+__device__ __forceinline__ uint32_t run_starts(uint32_t w, uint32_t before) {
+    const uint32_t diff = w ^ __funnelshift_l(before, w, 8);  // every byte against its predecessor
+    const uint32_t nz = (((diff & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | diff) & 0x80808080u;  // top bit of every non-zero byte
+    return (((nz >> 7) * 0x00204081u) >> 21) & 0xFu;  // the four flags side by side
+}
+
+// Walk the n (<= 512) bytes of a sub-block at p (16-byte aligned) and hand its runs to the sink.  Sixteen
+// bytes at a time: the positions where a run starts are found with word operations, and only those are
+// visited (a lane steps from run to run, not from byte to byte).  Four vectors are always in flight.
 template <typename Sink>
 __device__ __forceinline__ void parse_sub_block(Sink& s, const uint8_t* p, uint32_t n) {
-    uint32_t run_val = 0, run_len = 0;
-    auto step = [&](uint32_t b) {
-        if (run_len && b == run_val) {
-            ++run_len;
-        } else {
-            if (run_len) emit_run(s, run_val, run_len);
-            run_val = b;
-            run_len = 1;
-        }
-    };
+    uint32_t run_val = 0, run_start = 0;  // the open run: its byte and where it began
+    bool open = false;
     const uint32_t n_vec = n / 16;
     const uint4* pv = reinterpret_cast<const uint4*>(p);
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
-    // four vectors (64 bytes) are always in flight ahead of the walk
     uint4 q0 = n_vec > 0 ? __ldg(pv) : zero4, q1 = n_vec > 1 ? __ldg(pv + 1) : zero4;
     uint4 q2 = n_vec > 2 ? __ldg(pv + 2) : zero4, q3 = n_vec > 3 ? __ldg(pv + 3) : zero4;
+    uint32_t last = 0;  // the word before the current vector
     for (uint32_t v = 0; v < n_vec; ++v) {
         const uint4 q = q0;
         q0 = q1, q1 = q2, q2 = q3;
         if (v + 4 < n_vec) q3 = __ldg(pv + v + 4);
-        const uint32_t splat = run_val * 0x01010101u;
-        if (run_len && q.x == splat && q.y == splat && q.z == splat && q.w == splat) {
-            run_len += 16;  // sixteen more of the same (long runs of zeros are the common case)
-            continue;
-        }
-        uint32_t w0 = q.x, w1 = q.y, w2 = q.z, w3 = q.w;
-#pragma unroll 1
-        for (uint32_t j = 0; j < 16; ++j) {
-            step(w0 & 0xFFu);
-            w0 >>= 8;
-            if ((j & 3) == 3) w0 = w1, w1 = w2, w2 = w3;
+        uint32_t heads = run_starts(q.x, last) | (run_starts(q.y, q.x) << 4) | (run_starts(q.z, q.y) << 8) |
+                         (run_starts(q.w, q.z) << 12);
+        if (v == 0) heads |= 1u;  // the first byte of the sub-block always starts a run
+        last = q.w;
+        while (heads) {
+            const uint32_t j = __ffs(heads) - 1;
+            heads &= heads - 1;
+            const uint32_t pos = v * 16 + j;
+            if (open) emit_run(s, run_val, pos - run_start);
+            const uint32_t word = j < 8 ? (j < 4 ? q.x : q.y) : (j < 12 ? q.z : q.w);
+            run_val = (word >> (8 * (j & 3))) & 0xFFu;
+            run_start = pos;
+            open = true;
         }
     }
-    for (uint32_t i = n_vec * 16; i < n; ++i) step(p[i]);  // only the very end of the data
-    if (run_len) emit_run(s, run_val, run_len);
+    for (uint32_t i = n_vec * 16; i < n; ++i) {  // only the very end of the data
+        const uint32_t b = p[i];
+        if (!open || b != run_val) {
+            if (open) emit_run(s, run_val, i - run_start);
+            run_val = b, run_start = i, open = true;
+        }
+    }
+    if (open) emit_run(s, run_val, n - run_start);
 }
 
 // Bytes [4k, 4k+4) of a chunk of n bytes at p (4-byte aligned) as a word; bytes past the end read as 0.
