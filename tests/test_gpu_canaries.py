@@ -37,6 +37,12 @@ def guard_session(ses):
         g = Guarded(getattr(ses, n))
         setattr(ses, n, g.view)
         guards[n] = g
+    for i, extra in enumerate(ses.extra):           # the further buffer sets of the multi-variant sweep
+        for n in list(extra):
+            if extra[n] is not None:
+                g = Guarded(extra[n])
+                extra[n] = g.view
+                guards[f"slot{i + 1}.{n}"] = g
     return guards
 
 
@@ -46,9 +52,14 @@ def guard_session(ses):
 def test_guards_survive_every_entry_point(make, dtype):
     wl = make()
     dm = DeviceModel(wl, dtype)
-    ses = Session(dm, wl.scope, len(wl.ks))
+    n_multi = min(len(wl.ks), B.DNNS_MULTI_MAX)
+    ses = Session(dm, wl.scope, len(wl.ks), slots=n_multi)
     guards = guard_session(ses)
     ses.magnitude_threshold(wl.ks)
+    ses.mask_and_structures_multi(len(wl.ks) - n_multi, n_multi)
+    for g in range(n_multi):
+        ses.propagate_keep(slot=g)
+        ses.compact(slot=g)
     for v in sorted({0, len(wl.ks) - 1}):
         ses.apply_mask(v)
         ses.zero_structures()
