@@ -486,25 +486,36 @@ __global__ void __launch_bounds__(kTileThreads, G == 1 ? 4 : 3) k_sweep_multi(Ta
                         const uint32_t vi = u * kTileThreads + threadIdx.x;
                         uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
                         uint32_t keep = 0, nz = 0;
+                        if (DT == DNNS_F32) {
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t m = w[j] & kKeyMask;
-                            if (DT == DNNS_F32) {
+                            for (int j = 0; j < 4; ++j) {
+                                const uint32_t m = w[j] & kKeyMask;
                                 const bool k = m >= te;
                                 w[j] = k ? w[j] : 0u;
                                 keep |= k ? (1u << j) : 0u;
                                 if (zeros_survive) nz |= m != 0 ? (1u << j) : 0u;
-                            } else {
-                                // both 15-bit keys of the word at once: with bit 15 of each half set, subtracting
-                                // the threshold leaves that bit standing exactly where key >= threshold, and no
-                                // borrow crosses into the other half (te <= 0x8000)
-                                const uint32_t ge = (((m | 0x80008000u) - te2) >> 15) & 0x00010001u;
-                                w[j] &= ge * 0xFFFFu;
-                                keep |= ((ge | (ge >> 15)) & 3u) << (2 * j);
-                                if (zeros_survive) {
-                                    const uint32_t ne = (((m | 0x80008000u) - 0x00010001u) >> 15) & 0x00010001u;  // key >= 1
-                                    nz |= ((ne | (ne >> 15)) & 3u) << (2 * j);
-                                }
+                            }
+                        } else {
+                            // Both 15-bit keys of a word at once: with bit 15 of each half set (the sign bits are
+                            // not part of the key), subtracting the threshold leaves that bit standing exactly
+                            // where key >= threshold, and no borrow crosses into the other half (te <= 0x8000).
+                            // ge has the low key's flag at bit 0 and the high key's at bit 16; the eight flags of
+                            // the vector are packed with three shifted adds and one fold.
+                            uint32_t ge[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                ge[j] = (((w[j] | 0x80008000u) - te2) >> 15) & 0x00010001u;
+                                w[j] &= ge[j] * 0xFFFFu;
+                            }
+                            const uint32_t sk = ge[0] + (ge[1] << 2) + (ge[2] << 4) + (ge[3] << 6);
+                            keep = (sk | (sk >> 15)) & 0xFFu;
+                            if (zeros_survive) {  // te == 0: everything is kept, the non-zero flags are key >= 1
+                                const uint32_t orig[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                                uint32_t sn = 0;
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+                                    sn += ((((orig[j] | 0x80008000u) - 0x00010001u) >> 15) & 0x00010001u) << (2 * j);
+                                nz = (sn | (sn >> 15)) & 0xFFu;
                             }
                         }
                         out[u * kTileThreads] = make_uint4(w[0], w[1], w[2], w[3]);
