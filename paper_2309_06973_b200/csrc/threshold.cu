@@ -452,7 +452,12 @@ template <int DT>
 __global__ void __launch_bounds__(kTileThreads, 4) k_ties(Tables tb, ThresholdWs ws, int n_k,
                                                           const dnns_threshold* __restrict__ thr) {
     if (*ws.any_need == 0) return;
-    __shared__ uint32_t s_bm[kBitmapWords];
+    // 31-bit keys: a bitmap of the low 15 bits of the thresholds filters the keys, survivors are compared with
+    // every threshold.  15-bit keys: a key is its own index into a byte table that names the first variant
+    // whose threshold it equals (0: none) - one lookup per key and one counter update per hit, because keys
+    // equal to a threshold are common there (thousands per threshold).
+    __shared__ uint32_t s_bm[DT == DNNS_F32 ? kBitmapWords : 1];
+    __shared__ uint8_t s_slot[DT == DNNS_BF16 ? kHistBins : 4];
     __shared__ uint32_t s_tau[kMaxVariants], s_need[kMaxVariants];
     __shared__ uint32_t s_cnt[kTileThreads / 32][kMaxVariants];  // per warp: ties of the current tile, per variant
     __shared__ uint32_t s_any, s_zero_tau;
@@ -467,9 +472,12 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_ties(Tables tb, ThresholdWs
                 __syncthreads();
                 cur_seg = d.seg;
                 if (threadIdx.x == 0) s_any = s_zero_tau = 0;
+                if (DT == DNNS_BF16)
+                    for (uint32_t i = threadIdx.x; i < kHistBins / 4; i += kTileThreads) reinterpret_cast<uint32_t*>(s_slot)[i] = 0;
                 __syncthreads();
-                for (uint32_t w = threadIdx.x; w < kBitmapWords; w += kTileThreads)
-                    s_bm[w] = ws.tie_bitmap[(size_t)cur_seg * kBitmapWords + w];
+                if (DT == DNNS_F32)
+                    for (uint32_t w = threadIdx.x; w < kBitmapWords; w += kTileThreads)
+                        s_bm[w] = ws.tie_bitmap[(size_t)cur_seg * kBitmapWords + w];
                 if ((int)threadIdx.x < n_k) {
                     const size_t idx = (size_t)threadIdx.x * S + cur_seg;
                     const uint32_t need = ws.need[idx], tau = thr[idx].tau_bits;
@@ -479,29 +487,58 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_ties(Tables tb, ThresholdWs
                     if (need && tau == 0) s_zero_tau = 1;
                 }
                 __syncthreads();
+                if (DT == DNNS_BF16 && threadIdx.x == 0) {
+                    // the first variant (in index order) that needs tie counts for a key owns the key's counter;
+                    // variants with the same threshold copy it when the tile's counts are sent
+                    for (int vv = n_k - 1; vv >= 0; --vv)
+                        if (s_need[vv] && s_tau[vv] != 0) s_slot[s_tau[vv]] = (uint8_t)(vv + 1);
+                }
+                __syncthreads();
             }
             return s_any != 0;  // no variant of this segment splits its ties: nothing to count
         },
         [&](uint32_t tile, uint32_t n_e, const uint4(&v)[kVecPerThread]) {
             uint32_t zeros = 0;
-            for_filtered_keys<DT, 0>(v, n_e, s_bm, [&](uint32_t key) {
-                if (key == 0) {
-                    ++zeros;
-                    return;
+            if (DT == DNNS_F32) {
+                for_filtered_keys<DT, 0>(v, n_e, s_bm, [&](uint32_t key) {
+                    if (key == 0) {
+                        ++zeros;
+                        return;
+                    }
+                    for (int vv = 0; vv < n_k; ++vv)
+                        if (s_need[vv] && s_tau[vv] == key) atomicAdd(&s_cnt[warp][vv], 1u);
+                });
+            } else {
+                constexpr uint32_t kTileElems = kTileBytes / Elem<DT>::kBytes;
+#pragma unroll
+                for (int u = 0; u < kVecPerThread; ++u) {
+                    const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                    const uint32_t first = (u * kTileThreads + threadIdx.x) * 8;
+                    // elements past a ragged end were loaded as zeros: they must not count as zero keys
+                    const uint32_t valid = n_e == kTileElems ? 8u : (first >= n_e ? 0u : min(8u, n_e - first));
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t key = (w[j >> 1] >> (16 * (j & 1))) & 0x7FFFu;
+                        if ((uint32_t)j >= valid) continue;
+                        if (key == 0) {
+                            ++zeros;
+                            continue;
+                        }
+                        const uint32_t slot = s_slot[key];
+                        if (slot) atomicAdd(&s_cnt[warp][slot - 1], 1u);
+                    }
                 }
-                for (int vv = 0; vv < n_k; ++vv)
-                    if (s_need[vv] && s_tau[vv] == key) atomicAdd(&s_cnt[warp][vv], 1u);
-            });
+            }
             // a warp sends its counts of the tile to the table in one atomic per variant: keys equal to
             // tau are common in 15-bit keys, and thousands of single atomics on one word would queue up
             __syncwarp();
             for (int vv = lane; vv < n_k; vv += 32) {
-                const uint32_t c = s_cnt[warp][vv];
-                if (c) {
-                    atomicAdd(&ws.tile_ties[(size_t)vv * tb.n_tiles + tile], c);
-                    s_cnt[warp][vv] = 0;
-                }
+                uint32_t c = s_cnt[warp][vv];
+                if (DT == DNNS_BF16 && s_need[vv] && s_tau[vv] != 0) c = s_cnt[warp][s_slot[s_tau[vv]] - 1];  // the owner's count
+                if (c) atomicAdd(&ws.tile_ties[(size_t)vv * tb.n_tiles + tile], c);
             }
+            __syncwarp();
+            for (int vv = lane; vv < n_k; vv += 32) s_cnt[warp][vv] = 0;
             __syncwarp();
             if (s_zero_tau) {
 #pragma unroll
