@@ -264,6 +264,18 @@ dnns_status dnns_propagate_keep(dnns_plan* plan, const uint32_t* out_nz, const u
                                 uint64_t* stats, void* stream);
 
 /*
+ * Step 4 for the n_variants (1..DNNS_MULTI_MAX) variants of a dnns_mask_and_structures_multi call in one launch:
+ * Algorithm 1 plans all layers of a model at once; the variants of a portfolio are independent models, so they
+ * are planned at once too.  out_nz, in_nz, keep_bits, keep_idx, keep_count: host arrays of n_variants device
+ * pointers (the outputs all distinct), each as in dnns_propagate_keep; stats (device, nullable): 4 words per
+ * variant, contiguous.  Outputs per variant are bit for bit those of dnns_propagate_keep.
+ */
+dnns_status dnns_propagate_keep_multi(dnns_plan* plan, int32_t n_variants, const uint32_t* const* out_nz,
+                                      const uint32_t* const* in_nz, uint32_t policy, int32_t min_keep,
+                                      uint32_t* const* keep_bits, int32_t* const* keep_idx, int32_t* const* keep_count,
+                                      uint64_t* stats, void* stream);
+
+/*
  * Step 4 applied to a fixed point.  Algorithm 1 looks at the zero channels once; once channels are
  * gone, a filter whose only non-zero 2-D kernels sit in removed input channels is a zero channel
  * too, and an input column that only removed filters read is unread.  Pass p judges every channel by

@@ -23,7 +23,7 @@ DNNS_MULTI_MAX = 4
 EXPORTS = ["dnns_status_string", "dnns_workspace_bytes", "dnns_plan_create", "dnns_plan_destroy", "dnns_plan_layout",
            "dnns_plan_launch_count", "dnns_magnitude_threshold", "dnns_apply_mask", "dnns_zero_structures",
            "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures", "dnns_fold_batchnorm", "dnns_propagate_keep_cascade",
-           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_mask_and_structures_multi", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
+           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_mask_and_structures_multi", "dnns_propagate_keep_multi", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
 
 
 class dnns_tensor(C.Structure):
@@ -103,6 +103,7 @@ def lib() -> C.CDLL:
         L.dnns_propagate_keep_cascade.argtypes = [vp, vp, u32, i32, i32, vp, vp, vp, vp, vp]
         L.dnns_magnitude_threshold_static.argtypes = [vp, i32, u64, u64, vp, vp]
         L.dnns_mask_and_structures_multi.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp, vp]
+        L.dnns_propagate_keep_multi.argtypes = [vp, i32, vp, vp, u32, i32, vp, vp, vp, vp, vp]
         L.dnns_plan_profile.argtypes = [vp, i32]
         L.dnns_plan_profile_read.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(u64)]
         for name in ("dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes"):
@@ -251,3 +252,12 @@ def dnns_mask_and_structures_multi(plan, thr_dev: int, first_variant: int, n_var
     arrays = [_ptr_array(a) for a in (masked_arenas, mask_bits, nz_map, out_nz, in_nz)]
     _check(lib().dnns_mask_and_structures_multi(plan, thr_dev, first_variant, n_variants, *arrays, stream),
            "dnns_mask_and_structures_multi")
+
+
+def dnns_propagate_keep_multi(plan, n_variants: int, out_nz, in_nz, policy: int, min_keep: int, keep_bits, keep_idx,
+                              keep_count, stats: int, stream: int = 0) -> None:
+    """out_nz ... keep_count: lists of n_variants device addresses; stats: one address (4 words per variant) or 0."""
+    arrays = [_ptr_array(a) for a in (out_nz, in_nz)]
+    outs = [_ptr_array(a) for a in (keep_bits, keep_idx, keep_count)]
+    _check(lib().dnns_propagate_keep_multi(plan, n_variants, arrays[0], arrays[1], policy, min_keep, *outs, stats or None,
+                                           stream), "dnns_propagate_keep_multi")

@@ -171,6 +171,9 @@ int launch_multi_sweep(const Tables& tb, const ThresholdWs& ws, const dnns_thres
 int launch_propagate(const Tables& tb, const uint32_t* out_nz, const uint32_t* in_nz, uint32_t policy,
                      int32_t min_keep, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count, uint64_t* stats,
                      cudaStream_t st);
+int launch_propagate_multi(const Tables& tb, int n_variants, const uint32_t* const* out_nz, const uint32_t* const* in_nz,
+                           uint32_t policy, int32_t min_keep, uint32_t* const* keep_bits, int32_t* const* keep_idx,
+                           int32_t* const* keep_count, uint64_t* stats, cudaStream_t st);
 int launch_propagate_cascade(const Tables& tb, const CascadeWs& cw, const uint32_t* nz_map, uint32_t policy,
                              int32_t min_keep, int32_t max_passes, uint32_t* keep_bits, int32_t* keep_idx,
                              int32_t* keep_count, uint64_t* stats, uint32_t n_keep_words, uint32_t n_live_words, int n_sm,

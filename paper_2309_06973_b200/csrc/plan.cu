@@ -561,6 +561,29 @@ dnns_status dnns_propagate_keep(dnns_plan* p, const uint32_t* out_nz, const uint
     return DNNS_OK;
 }
 
+dnns_status dnns_propagate_keep_multi(dnns_plan* p, int32_t n_variants, const uint32_t* const* out_nz,
+                                      const uint32_t* const* in_nz, uint32_t policy, int32_t min_keep,
+                                      uint32_t* const* keep_bits, int32_t* const* keep_idx, int32_t* const* keep_count,
+                                      uint64_t* stats, void* stream) {
+    if (!p || !out_nz || !in_nz || !keep_bits || !keep_idx || !keep_count || n_variants < 1 || n_variants > kMultiMax)
+        return DNNS_ERR_INVALID_ARG;
+    if (policy & ~(uint32_t)(DNNS_RULE_PRODUCER | DNNS_RULE_CONSUMER | DNNS_SHIFT_STRICT)) return DNNS_ERR_INVALID_ARG;
+    for (int v = 0; v < n_variants; ++v) {
+        if (!out_nz[v] || !in_nz[v] || !keep_bits[v] || !keep_idx[v] || !keep_count[v]) return DNNS_ERR_INVALID_ARG;
+        for (int u = 0; u < v; ++u)  // every variant writes buffers of its own
+            if (keep_bits[u] == keep_bits[v] || keep_idx[u] == keep_idx[v] || keep_count[u] == keep_count[v])
+                return DNNS_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (stats && cudaMemsetAsync(stats, 0, 32 * (size_t)n_variants, st) != cudaSuccess) return DNNS_ERR_CUDA;
+    ProfileScope profile_scope(p);
+    const int n = launch_propagate_multi(p->tb, n_variants, out_nz, in_nz, policy, min_keep, keep_bits, keep_idx, keep_count,
+                                         stats, st);
+    if (n < 0) return DNNS_ERR_CUDA;
+    p->launches += n;
+    return DNNS_OK;
+}
+
 dnns_status dnns_propagate_keep_cascade(dnns_plan* p, const uint32_t* nz_map, uint32_t policy, int32_t min_keep,
                                         int32_t max_passes, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count,
                                         uint64_t* stats, void* stream) {

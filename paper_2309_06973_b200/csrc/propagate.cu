@@ -166,6 +166,30 @@ __global__ void __launch_bounds__(kThreads) k_propagate(Tables tb, const uint32_
                    keep_count, stats);
 }
 
+// The same for the variants of one multi-variant sweep in one launch: blockIdx.y picks the variant's buffers.
+struct PropagateMultiArgs {
+    const uint32_t* out_nz[kMultiMax];
+    const uint32_t* in_nz[kMultiMax];
+    uint32_t* keep_bits[kMultiMax];
+    int32_t* keep_idx[kMultiMax];
+    int32_t* keep_count[kMultiMax];
+};
+
+__global__ void __launch_bounds__(kThreads) k_propagate_multi(Tables tb, PropagateMultiArgs pa, uint32_t policy,
+                                                              int32_t min_keep, unsigned long long* stats) {
+    __shared__ uint32_t s_prod[kMaxGroupWords];
+    __shared__ uint32_t s_cons[kMaxGroupWords];
+    __shared__ uint32_t s_rem[kMaxGroupWords];
+    __shared__ uint32_t s_pre[kMaxGroupWords];
+    __shared__ uint32_t scratch[33];
+    __shared__ uint32_t s_rekept;
+    const int g = blockIdx.x, v = blockIdx.y;
+    const GroupDesc gd = tb.groups[g];
+    const uint32_t removed_local = eval_group(tb, gd, pa.out_nz[v], pa.in_nz[v], policy, s_prod, s_cons, s_rem);
+    finalize_group(tb, gd, g, min_keep, removed_local, s_rem, s_prod, s_pre, scratch, &s_rekept, pa.keep_bits[v],
+                   pa.keep_idx[v], pa.keep_count[v], stats ? stats + 4 * v : nullptr);
+}
+
 // ---- fixed point: the rule applied pass after pass on kernel maps restricted to what is still kept
 //
 // Pass p: k_live recomputes the filter / input-column flags from the kernel maps, ignoring input
@@ -311,6 +335,20 @@ int launch_propagate(const Tables& tb, const uint32_t* out_nz, const uint32_t* i
     ScopedKernel timed("k_propagate", st);
     k_propagate<<<tb.n_groups, kThreads, 0, st>>>(tb, out_nz, in_nz, policy, min_keep, keep_bits, keep_idx,
                                                   keep_count, reinterpret_cast<unsigned long long*>(stats));
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_propagate_multi(const Tables& tb, int n_variants, const uint32_t* const* out_nz, const uint32_t* const* in_nz,
+                           uint32_t policy, int32_t min_keep, uint32_t* const* keep_bits, int32_t* const* keep_idx,
+                           int32_t* const* keep_count, uint64_t* stats, cudaStream_t st) {
+    PropagateMultiArgs pa{};
+    for (int v = 0; v < n_variants; ++v) {
+        pa.out_nz[v] = out_nz[v], pa.in_nz[v] = in_nz[v];
+        pa.keep_bits[v] = keep_bits[v], pa.keep_idx[v] = keep_idx[v], pa.keep_count[v] = keep_count[v];
+    }
+    ScopedKernel timed("k_propagate", st);
+    k_propagate_multi<<<dim3(tb.n_groups, n_variants), kThreads, 0, st>>>(tb, pa, policy, min_keep,
+                                                                        reinterpret_cast<unsigned long long*>(stats));
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

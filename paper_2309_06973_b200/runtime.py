@@ -118,7 +118,9 @@ class Session:
                 "masked": torch.empty(int(L.masked_arena_bytes), dtype=torch.uint8, device=dev),
                 "mask_bits": i32(L.mask_words) if want_mask_bits else None,
                 "nz_map": i32(L.nz_map_words) if want_nz_map else None,
-                "out_nz": i32(L.out_nz_words), "in_nz": i32(L.in_nz_words)})
+                "out_nz": i32(L.out_nz_words), "in_nz": i32(L.in_nz_words),
+                "keep_bits": i32(L.keep_words), "keep_idx": i32(L.keep_idx_len), "keep_count": i32(G)})
+        self.stats_multi = torch.zeros(4 * max(slots, 1), dtype=torch.int64, device=dev)
 
     def _slot(self, name: str, slot: int):
         return getattr(self, name) if slot == 0 else self.extra[slot - 1][name]
@@ -169,9 +171,21 @@ class Session:
                               self.keep_bits.data_ptr(), self.keep_idx.data_ptr(), self.keep_count.data_ptr(),
                               self.stats.data_ptr(), _stream())
 
-    def compact(self, from_model: bool = False, dst_bytes: Optional[int] = None, slot: int = 0):
-        B.dnns_compact(self.plan, 0 if from_model else self._slot("masked", slot).data_ptr(), self.keep_idx.data_ptr(),
-                       self.keep_count.data_ptr(), self.compact_arena.data_ptr(),
+    def propagate_keep_multi(self, n_variants: int, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER,
+                             min_keep: int = 1):
+        """Step 4 of the n_variants variants of the latest multi-variant sweep in one launch; slot g keeps its own
+        keep sets (slot 0: the session's), read by compact(slot=g, own_keep=True)."""
+        ptrs = lambda name: [self._slot(name, g).data_ptr() for g in range(n_variants)]
+        B.dnns_propagate_keep_multi(self.plan, n_variants, ptrs("out_nz"), ptrs("in_nz"), policy, min_keep,
+                                    ptrs("keep_bits"), ptrs("keep_idx"), ptrs("keep_count"), self.stats_multi.data_ptr(),
+                                    _stream())
+
+    def compact(self, from_model: bool = False, dst_bytes: Optional[int] = None, slot: int = 0, own_keep: bool = False):
+        """own_keep: rebuild from the keep sets of the slot itself (written by propagate_keep_multi)."""
+        keep_slot = slot if own_keep else 0
+        B.dnns_compact(self.plan, 0 if from_model else self._slot("masked", slot).data_ptr(),
+                       self._slot("keep_idx", keep_slot).data_ptr(),
+                       self._slot("keep_count", keep_slot).data_ptr(), self.compact_arena.data_ptr(),
                        self.compact_arena.numel() if dst_bytes is None else dst_bytes, self.dst_offsets.data_ptr(),
                        self.dst_shapes.data_ptr(), _stream())
 
@@ -242,16 +256,19 @@ class Session:
         return (nz, self._split_words(self._slot("out_nz", slot), self.out_nz_offset, [t.O for t in wl.tensors]),
                 self._split_words(self._slot("in_nz", slot), self.in_nz_offset, [t.I for t in wl.tensors]))
 
-    def keep_sets(self):
+    def keep_sets(self, slot: int = 0, multi_stats: bool = False):
+        """multi_stats: the statistics written by propagate_keep_multi for this slot."""
         wl = self.dm.wl
-        bits = self._split_words(self.keep_bits, self.keep_offset, [g.C for g in wl.groups])
-        cnt = self.keep_count.cpu().numpy()[: len(wl.groups)].copy()
-        idx_raw = self.keep_idx.cpu().numpy()
+        bits = self._split_words(self._slot("keep_bits", slot), self.keep_offset, [g.C for g in wl.groups])
+        cnt = self._slot("keep_count", slot).cpu().numpy()[: len(wl.groups)].copy()
+        idx_raw = self._slot("keep_idx", slot).cpu().numpy()
         idx = [idx_raw[int(o): int(o) + int(c)].copy() for o, c in zip(self.keep_idx_offset, cnt)]
-        return bits, idx, cnt, self.stats.cpu().numpy().view(np.uint64).copy()
+        st = self.stats_multi[4 * slot: 4 * slot + 4] if multi_stats else self.stats
+        return bits, idx, cnt, st.cpu().numpy().view(np.uint64).copy()
 
-    def compacted(self):
-        """(weights [(O', I', KH, KW)], bn [(g, b, m, v)], biases, shapes (T, 2), offsets)."""
+    def compacted(self, keep_slot: int = 0):
+        """(weights [(O', I', KH, KW)], bn [(g, b, m, v)], biases, shapes (T, 2), offsets) of the variant rebuilt
+        last; keep_slot: the slot whose keep sets it was rebuilt from."""
         wl, eb = self.dm.wl, self.dm.elem_bytes
         T = len(wl.tensors)
         offs = self.dst_offsets.cpu().numpy().view(np.uint64)
@@ -262,7 +279,7 @@ class Session:
             On, In = int(shapes[i, 0]), int(shapes[i, 1])
             n = On * In * t.KH * t.KW
             ws.append(raw[int(offs[i]): int(offs[i]) + n * eb].view(self._np_dtype()).reshape(On, In, t.KH, t.KW).copy())
-        cnt = self.keep_count.cpu().numpy()
+        cnt = self._slot("keep_count", keep_slot).cpu().numpy()
         bns, k = [], T
         for b in wl.bns:
             Cn = int(cnt[wl.tensors[b.tensor].out_group])

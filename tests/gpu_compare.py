@@ -28,9 +28,10 @@ def expected_offsets(sizes_bytes):
 
 
 def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCER | O.RULE_CONSUMER, min_keep=1,
-                      weights=None, check_structure_maps=True, fused=False, multi=0):
+                      weights=None, check_structure_maps=True, fused=False, multi=0, multi_plan=False):
     """Thresholds for all of wl.ks in one call, then steps 2-5 for the chosen variants.
-    multi = G > 0: steps 2 and 3 of G consecutive variants at a time through the multi-variant sweep."""
+    multi = G > 0: steps 2 and 3 of G consecutive variants at a time through the multi-variant sweep;
+    multi_plan: step 4 of those variants in one launch as well (dnns_propagate_keep_multi)."""
     om = O.OracleModel(wl, dtype, weights)
     dm = DeviceModel(wl, dtype, weights=weights)
     ses = Session(dm, wl.scope, len(wl.ks), slots=max(multi, 1))
@@ -49,8 +50,13 @@ def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCE
                 n = min(multi, len(todo) - pos)
                 assert todo[pos: pos + n] == list(range(v, v + n)), "the multi-variant sweep takes consecutive variants"
                 ses.mask_and_structures_multi(v, n)
-            ses.propagate_keep(policy, min_keep, slot=slot)
-            ses.compact(slot=slot)
+                if multi_plan:
+                    ses.propagate_keep_multi(n, policy, min_keep)
+            if multi_plan:
+                ses.compact(slot=slot, own_keep=True)
+            else:
+                ses.propagate_keep(policy, min_keep, slot=slot)
+                ses.compact(slot=slot)
         else:
             ses.variant(v, policy, min_keep, fused=fused)
         assert ses.device_status() == B.DNNS_OK
@@ -65,14 +71,14 @@ def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCE
         assert_words(out_g, out_c, f"out flags v{v}")
         assert_words(in_g, in_c, f"in flags v{v}")
         kb_c, ki_c, kc_c, st_c = O.propagate_keep(masked_cpu, out_c, in_c, policy, min_keep)
-        kb_g, ki_g, kc_g, st_g = ses.keep_sets()
+        kb_g, ki_g, kc_g, st_g = ses.keep_sets(slot if multi_plan else 0, multi_stats=multi_plan)
         assert np.array_equal(kc_g, kc_c), f"keep counts v{v}"
         assert_words(kb_g, kb_c, f"keep bits v{v}")
         for g, (a, b) in enumerate(zip(ki_g, ki_c)):
             assert np.array_equal(a, b[: kc_c[g]]), f"keep idx v{v} group {g}"
         assert st_g.tolist() == st_c.tolist(), f"stats v{v}"
         cw_c, cbn_c, cb_c, sh_c = O.compact(masked_cpu, ki_c, kc_c)
-        cw_g, cbn_g, cb_g, sh_g, offs = ses.compacted()
+        cw_g, cbn_g, cb_g, sh_g, offs = ses.compacted(slot if multi_plan else 0)
         assert np.array_equal(sh_g, sh_c), f"shapes v{v}"
         for i, (a, b) in enumerate(zip(cw_g, cw_c)):
             assert bits_eq(a, b), f"compacted weights v{v} tensor {i}"

@@ -60,6 +60,9 @@ def test_guards_survive_every_entry_point(make, dtype):
     for g in range(n_multi):
         ses.propagate_keep(slot=g)
         ses.compact(slot=g)
+    ses.propagate_keep_multi(n_multi)
+    for g in range(n_multi):
+        ses.compact(slot=g, own_keep=True)
     for v in sorted({0, len(wl.ks) - 1}):
         ses.apply_mask(v)
         ses.zero_structures()

@@ -13,12 +13,13 @@ from paper_2309_06973_b200 import workloads as W
 pytestmark = pytest.mark.gpu
 
 
-def forward_check(wl, ses, dtype, slot=0):
-    """slot: which buffer set of the session holds the masked weights of the variant rebuilt last."""
+def forward_check(wl, ses, dtype, slot=0, keep_slot=0):
+    """slot: which buffer set of the session holds the masked weights of the variant rebuilt last;
+    keep_slot: which one holds its keep sets."""
     is_bf16 = dtype == B.DNNS_BF16
     x = torch.from_numpy(np.random.default_rng(1).standard_normal((2, 3, wl.input_hw, wl.input_hw)).astype(np.float32))
-    cw, cbn, cb, _, _ = ses.compacted()
-    kb, _, _, _ = ses.keep_sets()
+    cw, cbn, cb, _, _ = ses.compacted(keep_slot)
+    kb, _, _, _ = ses.keep_sets(keep_slot)
     mw, mbn, mb = silenced_reference(wl, ses.masked_tensors(slot=slot), wl.bn_params, wl.biases, kb)
     y_ref = forward(wl, mw, mbn, mb, x, is_bf16)
     y = forward(wl, cw, cbn, cb, x, is_bf16)
@@ -48,5 +49,5 @@ def test_resnet152_portfolio(dtype):
     forward_check(wl, ses, dtype)
     # the benchmark's configuration: four (fp32) or two (bf16) variants per sweep
     G = 4 if dtype == B.DNNS_F32 else 2
-    ses = compare_portfolio(wl, dtype, variants=list(range(8 - G, 8)), multi=G)
-    forward_check(wl, ses, dtype, slot=G - 1)
+    ses = compare_portfolio(wl, dtype, variants=list(range(8 - G, 8)), multi=G, multi_plan=True)
+    forward_check(wl, ses, dtype, slot=G - 1, keep_slot=G - 1)

@@ -26,6 +26,7 @@ def test_small_configs_every_variant(make, dtype, fused):
 def test_multi_variant_sweep_every_variant(make, dtype, multi):
     """Groups of up to four variants masked and analysed in one sweep: each variant as from its own sweep."""
     compare_portfolio(make(), dtype, multi=multi)
+    compare_portfolio(make(), dtype, multi=multi, multi_plan=True)     # ... and planned in one launch
 
 
 @pytest.mark.parametrize("policy", [O.RULE_PRODUCER, O.RULE_CONSUMER, O.RULE_PRODUCER | O.RULE_CONSUMER | O.SHIFT_STRICT])
@@ -37,6 +38,7 @@ def test_policies_and_min_keep(policy, min_keep):
         mu[::2] = 0.0
     wl.ks = np.array([[W.k_fraction(wl.n_prunable, 97, 100)], [wl.n_prunable]], np.uint64)
     compare_portfolio(wl, B.DNNS_F32, policy=policy, min_keep=min_keep)
+    compare_portfolio(wl, B.DNNS_F32, policy=policy, min_keep=min_keep, multi=2, multi_plan=True)
 
 
 @pytest.mark.parametrize("dtype", [B.DNNS_F32, B.DNNS_BF16])
