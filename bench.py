@@ -205,7 +205,7 @@ def main():
     calls_per_step = {n: V for n in names}
     calls_per_step["threshold"] = 1
     if G:
-        calls_per_step["mask+structures"] = len(groups)
+        calls_per_step["mask+structures"] = calls_per_step["propagate"] = len(groups)
 
     def step(record: bool):
         def timed(name, fn, *a):
@@ -219,9 +219,9 @@ def main():
         timed("threshold", ses.magnitude_threshold, wl.ks)
         for v0, n in groups:                       # n variants per read of the dense weights
             timed("mask+structures", ses.mask_and_structures_multi, v0, n)
+            timed("propagate", ses.propagate_keep_multi, n)        # the keep sets of the n variants in one launch
             for g in range(n):
-                timed("propagate", lambda: ses.propagate_keep(slot=g))
-                timed("compact", lambda: ses.compact(slot=g))
+                timed("compact", lambda: ses.compact(slot=g, own_keep=True))
         for v in (range(V) if not G else ()):
             if args.stepwise:
                 timed("mask", ses.apply_mask, v)
@@ -449,13 +449,13 @@ def main():
             if G:
                 if v % G == 0:
                     ses.mask_and_structures_multi(v, min(G, V - v))
-                ses.propagate_keep(slot=v % G)
-                ses.compact(slot=v % G)
+                    ses.propagate_keep_multi(min(G, V - v))
+                ses.compact(slot=v % G, own_keep=True)
             else:
                 ses.variant(v, fused=not args.stepwise)
             offs = ses.dst_offsets.cpu()           # synchronises: the sizes are only known on the device
             shp = ses.dst_shapes.cpu()
-            cnt = ses.keep_count.cpu()
+            cnt = ses._slot("keep_count", v % G if G else 0).cpu()
             last_w = len(wl.tensors) - 1
             used = int(offs[-1].item()) + 4 * max(int(cnt.max().item()), 1)
             used = min((used + 255) // 256 * 256, host_out.numel())
