@@ -98,6 +98,7 @@ struct Tables {
     const ProducerDesc* producers;  // parallel to prod_list
     const ConsumerDesc* consumers;  // parallel to cons_list
     const uint32_t* flag_prefix;  // [n_tensors + 1] units of the flag kernel before each tensor
+    const uint32_t* flag_unit_tensor;  // [n_flag_units] the tensor a unit belongs to
     uint32_t* ebits;        // packed "element is non-zero" bits of the latest sweep (same packing as the mask bits)
     uint32_t* status;       // device status word (a dnns_status, 0 = ok)
     uint32_t n_tensors, n_groups, n_bn, n_segs, n_items, n_tiles, n_flag_units;

@@ -57,7 +57,7 @@ inline uint64_t align_up(uint64_t x, uint64_t a = kAlign) { return (x + a - 1) /
 
 // Byte offsets of every section of the workspace.
 struct WsMap {
-    uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, producers, consumers, flag_prefix, status;
+    uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, producers, consumers, flag_prefix, flag_unit_tensor, status;
     uint64_t tables_end;  // everything before this is uploaded once at plan creation
     uint64_t k_dev, bitmap, sel, tie_prefix, unit_prefix, item_off, item_dims, ebits;
     uint64_t casc_rem0, casc_rem1, casc_lost, casc_live, casc_changed;
@@ -68,9 +68,17 @@ struct WsMap {
 
 struct Counts {
     uint32_t T = 0, G = 0, B = 0, S = 0, items = 0, tiles = 0, n_bias = 0;
-    uint64_t mask_words = 0, keep_words = 0, out_words = 0, in_words = 0;
+    uint64_t mask_words = 0, keep_words = 0, out_words = 0, in_words = 0, flag_units = 0;
     int dtype = 0, elem_bytes = 4;
 };
+
+// Units of the flag kernel a tensor is cut into: kFlagRows filters x 32 kernel-map words when a filter is a
+// power-of-two number of map words, else 32 kernels.
+uint64_t flag_units_of(const dnns_tensor& t) {
+    const uint64_t n_kernels = (uint64_t)t.O * t.I, wpr = t.I / 32;
+    if (t.I % 32 == 0 && (wpr & (wpr - 1)) == 0) return (((uint64_t)t.O + kFlagRows - 1) / kFlagRows) * ((wpr + 31) / 32);
+    return (n_kernels + 31) / 32;
+}
 
 bool tensor_extents_ok(const dnns_tensor& t) {
     return t.O > 0 && t.I > 0 && t.KH > 0 && t.KW > 0 && t.in_spatial > 0;
@@ -107,6 +115,7 @@ dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts*
         c->mask_words += (numel + 31) / 32;
         c->out_words += ((uint64_t)t.O + 31) / 32;
         c->in_words += ((uint64_t)t.I + 31) / 32;
+        c->flag_units += flag_units_of(t);
         if (t.bias) ++c->n_bias;
         if (t.prunable) {
             n_prunable += numel;
@@ -151,6 +160,7 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.producers = take(sizeof(ProducerDesc) * c.T);
     w.consumers = take(sizeof(ConsumerDesc) * c.T);
     w.flag_prefix = take(4ull * (c.T + 1));
+    w.flag_unit_tensor = take(4ull * (c.flag_units + 1));
     w.status = take(4);
     w.tables_end = o;
     const uint64_t vs = (uint64_t)maxv * (c.S ? c.S : 1);
@@ -263,6 +273,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     auto* prod_list = reinterpret_cast<int32_t*>(host.data() + map.prod_list);
     auto* cons_list = reinterpret_cast<int32_t*>(host.data() + map.cons_list);
     auto* flag_prefix = reinterpret_cast<uint32_t*>(host.data() + map.flag_prefix);
+    auto* flag_unit_tensor = reinterpret_cast<uint32_t*>(host.data() + map.flag_unit_tensor);
     auto* producers = reinterpret_cast<ProducerDesc*>(host.data() + map.producers);
     auto* consumers = reinterpret_cast<ConsumerDesc*>(host.data() + map.consumers);
 
@@ -301,14 +312,11 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
             n_prunable += d.numel;
         }
         tile += d.n_tiles;
-        // units of the flag kernel: kFlagRows filters x 32 map words when a filter is a power-of-two number
-        // of kernel-map words, else 32 kernels
-        const uint64_t n_kernels = (uint64_t)t.O * t.I, wpr = t.I / 32;
         flag_prefix[i] = (uint32_t)flag_units;
-        if (t.I % 32 == 0 && (wpr & (wpr - 1)) == 0)
-            flag_units += (((uint64_t)t.O + kFlagRows - 1) / kFlagRows) * ((wpr + 31) / 32);
-        else
-            flag_units += (n_kernels + 31) / 32;
+        const uint64_t n_units = flag_units_of(t);
+        if (flag_units + n_units < (1ull << 32))
+            for (uint64_t k = 0; k < n_units; ++k) flag_unit_tensor[flag_units + k] = (uint32_t)i;  // unit -> its tensor
+        flag_units += n_units;
     }
     flag_prefix[c.T] = (uint32_t)flag_units;
     if (flag_units >= (1ull << 32)) {
@@ -396,6 +404,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     tb.consumers = reinterpret_cast<ConsumerDesc*>(w + map.consumers);
     tb.status = reinterpret_cast<uint32_t*>(w + map.status);
     tb.flag_prefix = reinterpret_cast<uint32_t*>(w + map.flag_prefix);
+    tb.flag_unit_tensor = reinterpret_cast<uint32_t*>(w + map.flag_unit_tensor);
     tb.ebits = reinterpret_cast<uint32_t*>(w + map.ebits);
     tb.n_flag_units = (uint32_t)flag_units;
     tb.n_tensors = c.T, tb.n_groups = c.G, tb.n_bn = c.B, tb.n_segs = c.S, tb.n_items = c.items, tb.n_tiles = c.tiles;

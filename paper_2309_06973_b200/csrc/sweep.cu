@@ -87,12 +87,7 @@ __global__ void __launch_bounds__(256) k_flags(Tables tb, const uint32_t* __rest
     const uint32_t per = (tb.n_flag_units + n_warps - 1) / n_warps;
     const uint32_t lo = min(tb.n_flag_units, warp * per), hi = min(tb.n_flag_units, lo + per);
     if (lo >= hi) return;
-    uint32_t t = 0, top = tb.n_tensors;  // tensor holding unit lo: last t with flag_prefix[t] <= lo
-    while (top - t > 1) {
-        const uint32_t mid = (t + top) >> 1;
-        if (tb.flag_prefix[mid] <= lo) t = mid;
-        else top = mid;
-    }
+    uint32_t t = tb.flag_unit_tensor[lo];  // the tensor holding unit lo
     uint32_t unit = lo;
     while (unit < hi) {
         const uint32_t t_begin = tb.flag_prefix[t], t_end = tb.flag_prefix[t + 1];
