@@ -167,3 +167,33 @@ def test_two_runs_are_bit_identical():
         outs.append(ses.masked_tensors() + ses.compacted()[0] + [ses.keep_idx.cpu().numpy(), ses.records()])
     for a, b in zip(*outs):
         assert np.array_equal(a.view(np.uint8), b.view(np.uint8))
+
+
+def test_multi_variant_calls_reject_bad_arguments():
+    """Host-side checks of the multi-variant entry points: too many variants, shared output buffers."""
+    from paper_2309_06973_b200.runtime import DeviceModel, Session
+    wl = W.resnet56()
+    ses = Session(DeviceModel(wl, B.DNNS_F32), wl.scope, len(wl.ks), slots=2)
+    ses.magnitude_threshold(wl.ks)
+    p = lambda name, g: ses._slot(name, g).data_ptr()
+    def sweep(first, n, arenas, outs, ins):
+        B.dnns_mask_and_structures_multi(ses.plan, ses.thr.data_ptr(), first, n, arenas, None, None, outs, ins)
+    good = ([p("masked", 0), p("masked", 1)], [p("out_nz", 0), p("out_nz", 1)], [p("in_nz", 0), p("in_nz", 1)])
+    sweep(0, 2, *good)                                                    # fine
+    for bad in [(0, 2, [p("masked", 0)] * 2, good[1], good[2]),           # one arena for two variants
+                (0, 2, good[0], [p("out_nz", 0)] * 2, good[2]),           # shared flags
+                (len(wl.ks) - 1, 2, *good),                               # runs past the last variant
+                (0, 5, good[0] * 3, good[1] * 3, good[2] * 3)]:           # more than DNNS_MULTI_MAX
+        with pytest.raises(B.DnnsError) as e:
+            sweep(*bad)
+        assert e.value.status == B.DNNS_ERR_INVALID_ARG
+    kb, ki, kc = ([p(n, 0), p(n, 1)] for n in ("keep_bits", "keep_idx", "keep_count"))
+    B.dnns_propagate_keep_multi(ses.plan, 2, good[1], good[2], 3, 1, kb, ki, kc, ses.stats_multi.data_ptr())
+    with pytest.raises(B.DnnsError) as e:
+        B.dnns_propagate_keep_multi(ses.plan, 2, good[1], good[2], 3, 1, kb, [p("keep_idx", 0)] * 2, kc, 0)
+    assert e.value.status == B.DNNS_ERR_INVALID_ARG
+    with pytest.raises(B.DnnsError) as e:
+        B.dnns_propagate_keep_multi(ses.plan, 2, good[1], good[2], 64, 1, kb, ki, kc, 0)    # unknown policy bit
+    assert e.value.status == B.DNNS_ERR_INVALID_ARG
+    assert ses.device_status() == B.DNNS_OK
+    ses.close()
