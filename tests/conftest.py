@@ -25,3 +25,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def built_libraries():
+    """The CUDA library and the CPU oracles are compiled in-tree on first use (no-ops when up to date)."""
+    from paper_2309_06973_b200 import build as build_mod
+    from oracle import deflate_oracle, oracle
+    build_mod.build()
+    oracle.build()
+    deflate_oracle.build()
