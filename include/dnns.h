@@ -236,7 +236,11 @@ dnns_status dnns_mask_and_structures(dnns_plan* plan, const dnns_threshold* thr_
  * model is read once per group of variants instead of once per variant.
  * masked_arenas, out_nz, in_nz: host arrays of n_variants device pointers, all distinct; mask_bits, nz_map:
  * host arrays of n_variants device pointers, or NULL (entries of mask_bits may be NULL too).  In-place
- * masking is not offered here.  Errors: INVALID_ARG, CUDA.
+ * masking is not offered here.
+ * When every entry of masked_arenas is NULL the masked weights are not written at all: the call then leaves
+ * only the mask bits (required in that case, one array per variant) and the zero structures, and
+ * dnns_compact_masked rebuilds a variant straight from the dense model - the sparse model of Section III-C,
+ * which is as large as the dense one, is never stored.  Errors: INVALID_ARG, CUDA.
  */
 #define DNNS_MULTI_MAX 4
 dnns_status dnns_mask_and_structures_multi(dnns_plan* plan, const dnns_threshold* thr_dev, int32_t first_variant,
@@ -305,6 +309,18 @@ dnns_status dnns_propagate_keep_cascade(dnns_plan* plan, const uint32_t* nz_map,
 dnns_status dnns_compact(dnns_plan* plan, const void* masked_arena, const int32_t* keep_idx,
                          const int32_t* keep_count, void* dst_arena, size_t dst_bytes, uint64_t* dst_offsets_dev,
                          int32_t* dst_shapes_dev, void* stream);
+
+/*
+ * Step 5 reading the DENSE model (the tensors of the plan's model) and applying step 2 on the way: a weight
+ * is copied when its key lies above tau of its ranking segment, or equals tau and its mask bit is set, else
+ * +0 is written.  Bit for bit the result of dnns_apply_mask followed by dnns_compact.  thr_dev / variant as in
+ * dnns_apply_mask; mask_bits: the variant's packed mask bits as written by dnns_apply_mask,
+ * dnns_mask_and_structures or dnns_mask_and_structures_multi on the same thresholds (read only where a key
+ * equals tau and the variant masks part of those weights); the remaining arguments as in dnns_compact.
+ */
+dnns_status dnns_compact_masked(dnns_plan* plan, const dnns_threshold* thr_dev, int32_t variant, const uint32_t* mask_bits,
+                                const int32_t* keep_idx, const int32_t* keep_count, void* dst_arena, size_t dst_bytes,
+                                uint64_t* dst_offsets_dev, int32_t* dst_shapes_dev, void* stream);
 
 /*
  * Module 1, Model Pre-Processor (Section III-D): fold every BatchNorm into the convolution it

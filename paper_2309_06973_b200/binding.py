@@ -23,7 +23,7 @@ DNNS_MULTI_MAX = 4
 EXPORTS = ["dnns_status_string", "dnns_workspace_bytes", "dnns_plan_create", "dnns_plan_destroy", "dnns_plan_layout",
            "dnns_plan_launch_count", "dnns_magnitude_threshold", "dnns_apply_mask", "dnns_zero_structures",
            "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures", "dnns_fold_batchnorm", "dnns_propagate_keep_cascade",
-           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_mask_and_structures_multi", "dnns_propagate_keep_multi", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
+           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_mask_and_structures_multi", "dnns_propagate_keep_multi", "dnns_compact_masked", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
 
 
 class dnns_tensor(C.Structure):
@@ -104,6 +104,7 @@ def lib() -> C.CDLL:
         L.dnns_magnitude_threshold_static.argtypes = [vp, i32, u64, u64, vp, vp]
         L.dnns_mask_and_structures_multi.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp, vp]
         L.dnns_propagate_keep_multi.argtypes = [vp, i32, vp, vp, u32, i32, vp, vp, vp, vp, vp]
+        L.dnns_compact_masked.argtypes = [vp, vp, i32, vp, vp, vp, vp, C.c_size_t, vp, vp, vp]
         L.dnns_plan_profile.argtypes = [vp, i32]
         L.dnns_plan_profile_read.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(u64)]
         for name in ("dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes"):
@@ -261,3 +262,9 @@ def dnns_propagate_keep_multi(plan, n_variants: int, out_nz, in_nz, policy: int,
     outs = [_ptr_array(a) for a in (keep_bits, keep_idx, keep_count)]
     _check(lib().dnns_propagate_keep_multi(plan, n_variants, arrays[0], arrays[1], policy, min_keep, *outs, stats or None,
                                            stream), "dnns_propagate_keep_multi")
+
+
+def dnns_compact_masked(plan, thr_dev: int, variant: int, mask_bits: int, keep_idx: int, keep_count: int, dst_arena: int,
+                        dst_bytes: int, dst_offsets_dev: int, dst_shapes_dev: int, stream: int = 0) -> None:
+    _check(lib().dnns_compact_masked(plan, thr_dev, variant, mask_bits, keep_idx, keep_count, dst_arena, dst_bytes,
+                                     dst_offsets_dev, dst_shapes_dev, stream), "dnns_compact_masked")

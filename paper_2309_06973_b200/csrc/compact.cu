@@ -64,11 +64,44 @@ __device__ __forceinline__ uint32_t load_elem(const void* base, uint32_t idx) {
     return __ldg(static_cast<const uint16_t*>(base) + idx);
 }
 
+// Masking on the fly (the rebuild reading the dense model): what steps 2 decided for one tensor and variant.
+struct MaskCtx {
+    uint32_t tau;          // threshold key of the tensor's ranking segment
+    uint32_t mode;         // 0: nothing is masked; 1: every key equal to tau is masked; 2: the mask bits decide those
+    const uint32_t* bits;  // the tensor's packed mask bits (1 = kept), consulted for key == tau in mode 2 only
+};
+
+// The element as step 2 leaves it: itself when its key lies above tau (or equals it and its mask bit is set), else +0.
+template <int BYTES>
+__device__ __forceinline__ uint32_t masked_elem(uint32_t x, const MaskCtx& m, uint32_t src_idx) {
+    const uint32_t key = x & (BYTES == 4 ? 0x7FFFFFFFu : 0x7FFFu);
+    bool keep = key > m.tau;
+    if (key == m.tau && m.mode == 2) keep = (__ldg(m.bits + (src_idx >> 5)) >> (src_idx & 31)) & 1u;
+    return (keep || m.mode == 0) ? x : 0u;
+}
+
+// The same for the VE elements of a 16-byte vector whose first element has source index src_idx.
+template <int BYTES>
+__device__ __forceinline__ uint4 masked_vec(uint4 v, const MaskCtx& m, uint32_t src_idx) {
+    if (m.mode == 0) return v;
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if (BYTES == 4) {
+            w[j] = masked_elem<4>(w[j], m, src_idx + j);
+        } else {
+            w[j] = masked_elem<2>(w[j] & 0xFFFFu, m, src_idx + 2 * j) | (masked_elem<2>(w[j] >> 16, m, src_idx + 2 * j + 1) << 16);
+        }
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 // Gather a run of consecutive units of one item whose elements are BYTES wide, starting at
 // destination element f0.  A unit is 4 x 16-byte destination vectors per thread.
-template <int BYTES>
+template <int BYTES, bool MASKED>
 __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, char* dst, const int32_t* ko,
-                                           const int32_t* ki, uint32_t On, uint32_t Cn, uint32_t f0, uint32_t n_units) {
+                                           const int32_t* ki, uint32_t On, uint32_t Cn, uint32_t f0, uint32_t n_units,
+                                           const MaskCtx& mk) {
     constexpr uint32_t VE = 16 / BYTES;  // elements per 16-byte vector
     constexpr int U = kUnitBytes / 16 / kThreads;
     constexpr uint32_t kUnitElems = kUnitBytes / BYTES;
@@ -96,12 +129,16 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
         // ko[a].  The loads of the next unit are issued before the current unit is stored.
         uint4 nxt[U];
         bool nxt_ok[U];
+        uint32_t nxt_src[MASKED ? U : 1];  // source index of the vector's first element (for the mask bits)
         auto issue = [&]() {
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 nxt_ok[u] = pos_f < total;
-                if (nxt_ok[u])
-                    nxt[u] = __ldg(reinterpret_cast<const uint4*>(src + ((size_t)(uint32_t)ko[pos_a] * L + pos_rem) * BYTES));
+                if (nxt_ok[u]) {
+                    const uint32_t s0 = (uint32_t)ko[pos_a] * L + pos_rem;
+                    nxt[u] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)s0 * BYTES));
+                    if (MASKED) nxt_src[u] = s0;
+                }
                 advance();
             }
         };
@@ -110,7 +147,10 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
             uint4 cur[U];
             bool ok[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) cur[u] = nxt[u], ok[u] = nxt_ok[u];
+            for (int u = 0; u < U; ++u) {
+                ok[u] = nxt_ok[u];
+                cur[u] = (MASKED && ok[u]) ? masked_vec<BYTES>(nxt[u], mk, nxt_src[u]) : nxt[u];
+            }
             const uint32_t fu = f0 + n * kUnitElems;
             if (n + 1 < n_units) issue();
 #pragma unroll
@@ -196,7 +236,8 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
             for (int j = 0; j < 4; ++j) w[u][j] = 0;
 #pragma unroll
             for (uint32_t e = 0; e < VE; ++e) {
-                const uint32_t x = idx[u][e] != kNone ? load_elem<BYTES>(src, idx[u][e]) : 0u;
+                uint32_t x = idx[u][e] != kNone ? load_elem<BYTES>(src, idx[u][e]) : 0u;
+                if (MASKED) x = masked_elem<BYTES>(x, mk, idx[u][e]);
                 if (BYTES == 4) w[u][e] = x;
                 else w[u][e >> 1] |= x << (16 * (e & 1));
             }
@@ -227,11 +268,14 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
 // for a separate one-block kernel; block 0 also writes the offsets and shapes the caller asked for.
 constexpr uint32_t kInlineItems = 1024;
 
-template <int WBYTES, bool INLINE_LAYOUT>  // WBYTES: element width of the weight tensors (BatchNorm, bias: 4 bytes)
+// MASKED: the source is the dense model and step 2 is applied to every element on its way (thr, variant, mask_bits).
+template <int WBYTES, bool INLINE_LAYOUT, bool MASKED>  // WBYTES: element width of the weight tensors (BatchNorm, bias: 4 bytes)
 __global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, CompactWs ws, const char* src_arena,
                                                                 const int32_t* __restrict__ keep_idx, char* dst_arena,
                                                                 const int32_t* __restrict__ keep_count, uint64_t dst_bytes,
-                                                                uint64_t* dst_offsets, int32_t* dst_shapes) {
+                                                                uint64_t* dst_offsets, int32_t* dst_shapes,
+                                                                const dnns_threshold* __restrict__ thr, int variant,
+                                                                const uint32_t* __restrict__ mask_bits) {
     __shared__ uint32_t s_unit_prefix[INLINE_LAYOUT ? kInlineItems + 1 : 1];
     __shared__ uint64_t s_item_off[INLINE_LAYOUT ? kInlineItems : 1];
     __shared__ int32_t s_item_dims[INLINE_LAYOUT ? 2 * kInlineItems : 1];
@@ -307,9 +351,16 @@ __global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, Compa
             const ItemDesc& it = tb.items[item];
             const uint32_t On = item_dims[2 * item], Cn = item_dims[2 * item + 1];
             const char* src;
+            MaskCtx mk{0u, 0u, nullptr};
             if (it.tensor >= 0) {
                 const TensorDesc& d = tb.tensors[it.tensor];
                 src = src_arena ? src_arena + d.arena_off : static_cast<const char*>(d.src);
+                if (MASKED && d.seg >= 0) {
+                    const dnns_threshold r = thr[(size_t)variant * tb.n_segs + d.seg];
+                    mk.tau = r.tau_bits;
+                    mk.mode = r.n_below + r.n_tie == 0 ? 0u : (r.n_tie >= r.n_equal ? 1u : 2u);
+                    mk.bits = mask_bits + d.off_mask;
+                }
             } else {
                 src = static_cast<const char*>(it.src);
             }
@@ -318,8 +369,8 @@ __global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, Compa
             const int32_t* ki = it.in_group >= 0 ? keep_idx + tb.groups[it.in_group].off_idx : nullptr;
             const uint32_t run_end = min(u_hi, item_end);
             const uint32_t f0 = (unit - item_begin) * (kUnitBytes / it.elem_bytes);
-            if (WBYTES == 4 || it.elem_bytes == 4) gather_run<4>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit);
-            else gather_run<2>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit);
+            if (WBYTES == 4 || it.elem_bytes == 4) gather_run<4, MASKED>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit, mk);
+            else gather_run<2, MASKED>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit, mk);
             unit = run_end;
         }
     }
@@ -329,29 +380,40 @@ __global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, Compa
 
 int launch_compact(const Tables& tb, const CompactWs& ws, const void* src_arena, const int32_t* keep_idx,
                    const int32_t* keep_count, void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets,
-                   int32_t* dst_shapes, int n_sm, cudaStream_t st) {
+                   int32_t* dst_shapes, int n_sm, cudaStream_t st, const dnns_threshold* thr, int variant,
+                   const uint32_t* mask_bits) {
     const char* src = (const char*)src_arena;
     char* dst = (char*)dst_arena;
     const int grid = n_sm * 4;
+    const bool masked = thr != nullptr;
     int launches = 1;
+#define DNNS_GATHER(W, INL, M)                                                                                        \
+    k_compact_gather<W, INL, M><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, \
+                                                           dst_shapes, thr, variant, mask_bits)
+#define DNNS_GATHER_DT(INL)                                  \
+    do {                                                     \
+        if (tb.dtype == DNNS_F32) {                          \
+            if (masked) DNNS_GATHER(4, INL, true);           \
+            else DNNS_GATHER(4, INL, false);                 \
+        } else {                                             \
+            if (masked) DNNS_GATHER(2, INL, true);           \
+            else DNNS_GATHER(2, INL, false);                 \
+        }                                                    \
+    } while (0)
     if (tb.n_items <= kInlineItems) {
-        ScopedKernel timed("k_compact_gather", st);
-        if (tb.dtype == DNNS_F32)
-            k_compact_gather<4, true><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, dst_shapes);
-        else
-            k_compact_gather<2, true><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, dst_shapes);
+        ScopedKernel timed(masked ? "k_compact_gather<masked>" : "k_compact_gather", st);
+        DNNS_GATHER_DT(true);
     } else {
         {
             ScopedKernel timed_layout("k_compact_layout", st);
             k_compact_layout<<<1, 1024, 0, st>>>(tb, ws, keep_count, dst_bytes, dst_offsets, dst_shapes);
         }
-        ScopedKernel timed("k_compact_gather", st);
-        if (tb.dtype == DNNS_F32)
-            k_compact_gather<4, false><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, dst_shapes);
-        else
-            k_compact_gather<2, false><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, dst_shapes);
+        ScopedKernel timed(masked ? "k_compact_gather<masked>" : "k_compact_gather", st);
+        DNNS_GATHER_DT(false);
         launches = 2;
     }
+#undef DNNS_GATHER_DT
+#undef DNNS_GATHER
     return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 

@@ -181,7 +181,8 @@ int launch_propagate_cascade(const Tables& tb, const CascadeWs& cw, const uint32
                              cudaStream_t st);
 int launch_compact(const Tables& tb, const CompactWs& ws, const void* src_arena, const int32_t* keep_idx,
                    const int32_t* keep_count, void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets,
-                   int32_t* dst_shapes, int n_sm, cudaStream_t st);
+                   int32_t* dst_shapes, int n_sm, cudaStream_t st, const dnns_threshold* thr = nullptr, int variant = 0,
+                   const uint32_t* mask_bits = nullptr);
 int launch_fold(const Tables& tb, void* arena, const uint64_t* offsets, const int32_t* shapes, cudaStream_t st);
 cudaError_t init_kernel_attributes();
 

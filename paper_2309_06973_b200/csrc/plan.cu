@@ -533,15 +533,26 @@ dnns_status dnns_mask_and_structures_multi(dnns_plan* p, const dnns_threshold* t
     if (!p || !thr_dev || !masked_arenas || !out_nz || !in_nz || n_variants < 1 || n_variants > kMultiMax ||
         first_variant < 0 || first_variant + n_variants > p->maxv)
         return DNNS_ERR_INVALID_ARG;
+    // masked_arenas all NULL: the masked weights are not written (see dnns_compact_masked); mask bits are then required
+    bool no_store = true;
+    for (int g = 0; g < n_variants; ++g) no_store = no_store && masked_arenas[g] == nullptr;
+    if (no_store && !mask_bits) return DNNS_ERR_INVALID_ARG;
     MultiSweepArgs ma;
     for (int g = 0; g < kMultiMax; ++g) {
         const int s = g < n_variants ? g : 0;
-        if (!masked_arenas[s] || (reinterpret_cast<uintptr_t>(masked_arenas[s]) & 15) || !out_nz[s] || !in_nz[s])
+        if (!out_nz[s] || !in_nz[s]) return DNNS_ERR_INVALID_ARG;
+        if (no_store) {
+            if (!mask_bits[s]) return DNNS_ERR_INVALID_ARG;
+        } else if (!masked_arenas[s] || (reinterpret_cast<uintptr_t>(masked_arenas[s]) & 15)) {
             return DNNS_ERR_INVALID_ARG;
-        for (int h = 0; h < s; ++h)  // every variant needs buffers of its own
-            if (masked_arenas[h] == masked_arenas[s] || out_nz[h] == out_nz[s] || in_nz[h] == in_nz[s]) return DNNS_ERR_INVALID_ARG;
+        }
+        for (int h = 0; h < s; ++h) {  // every variant needs buffers of its own
+            if ((!no_store && masked_arenas[h] == masked_arenas[s]) || out_nz[h] == out_nz[s] || in_nz[h] == in_nz[s])
+                return DNNS_ERR_INVALID_ARG;
+            if (mask_bits && mask_bits[s] && mask_bits[h] == mask_bits[s]) return DNNS_ERR_INVALID_ARG;
+        }
         ma.variant[g] = first_variant + s;
-        ma.dst[g] = static_cast<char*>(masked_arenas[s]);
+        ma.dst[g] = no_store ? nullptr : static_cast<char*>(masked_arenas[s]);
         ma.mask_bits[g] = mask_bits ? mask_bits[s] : nullptr;
         ma.ebits[g] = p->tb.ebits + (size_t)s * p->c.mask_words;
         ma.clear_a[g] = out_nz[s];
@@ -621,6 +632,21 @@ dnns_status dnns_compact(dnns_plan* p, const void* masked_arena, const int32_t* 
     ProfileScope profile_scope(p);
     const int n = launch_compact(p->tb, p->cws, masked_arena, keep_idx, keep_count, dst_arena, dst_bytes,
                                  dst_offsets_dev, dst_shapes_dev, p->n_sm, static_cast<cudaStream_t>(stream));
+    if (n < 0) return DNNS_ERR_CUDA;
+    p->launches += n;
+    return DNNS_OK;
+}
+
+dnns_status dnns_compact_masked(dnns_plan* p, const dnns_threshold* thr_dev, int32_t variant, const uint32_t* mask_bits,
+                                const int32_t* keep_idx, const int32_t* keep_count, void* dst_arena, size_t dst_bytes,
+                                uint64_t* dst_offsets_dev, int32_t* dst_shapes_dev, void* stream) {
+    if (!p || !thr_dev || !mask_bits || !keep_idx || !keep_count || !dst_arena || !dst_offsets_dev || !dst_shapes_dev ||
+        variant < 0 || variant >= p->maxv)
+        return DNNS_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) return DNNS_ERR_INVALID_ARG;
+    ProfileScope profile_scope(p);
+    const int n = launch_compact(p->tb, p->cws, nullptr, keep_idx, keep_count, dst_arena, dst_bytes, dst_offsets_dev,
+                                 dst_shapes_dev, p->n_sm, static_cast<cudaStream_t>(stream), thr_dev, variant, mask_bits);
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
     return DNNS_OK;

@@ -372,7 +372,9 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_sweep(Tables tb, ThresholdW
 // read once and masked against each variant's threshold in turn, so a variant costs one write of the
 // model plus 1/G of a read instead of a read and a write.  Same tile walk and the same two paths as
 // k_sweep<mask, structures>; the per-variant state (threshold, tie tables, destinations) is an array.
-template <int DT, int G>
+// STORE = false: the masked weights are not written at all (the rebuild then masks the dense weights on its
+// way, dnns_compact_masked); what remains are each variant's mask bits and element bits.
+template <int DT, int G, bool STORE>
 __global__ void __launch_bounds__(kTileThreads, G == 1 ? 4 : 3) k_sweep_multi(Tables tb, ThresholdWs ws, const dnns_threshold* __restrict__ thr,
                                                                  MultiSweepArgs ma, uint32_t n_clear_a, uint32_t n_clear_b) {
     constexpr int P = Elem<DT>::kPerVec;
@@ -470,7 +472,7 @@ __global__ void __launch_bounds__(kTileThreads, G == 1 ? 4 : 3) k_sweep_multi(Ta
                 // ---- lean path: a whole tile, one threshold per variant
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
-                    uint4* out = reinterpret_cast<uint4*>(ma.dst[g] + arena_off + (size_t)e0 * Elem<DT>::kBytes) + threadIdx.x;
+                    uint4* out = STORE ? reinterpret_cast<uint4*>(ma.dst[g] + arena_off + (size_t)e0 * Elem<DT>::kBytes) + threadIdx.x : nullptr;
                     uint32_t* mask_words = ma.mask_bits[g] ? ma.mask_bits[g] + off_mask : nullptr;
                     uint32_t* nz_words = ma.ebits[g] + off_mask;
                     const uint32_t te = thr_eff[g];
@@ -513,7 +515,7 @@ __global__ void __launch_bounds__(kTileThreads, G == 1 ? 4 : 3) k_sweep_multi(Ta
                                 nz = (sn | (sn >> 15)) & 0xFFu;
                             }
                         }
-                        out[u * kTileThreads] = make_uint4(w[0], w[1], w[2], w[3]);
+                        if (STORE) out[u * kTileThreads] = make_uint4(w[0], w[1], w[2], w[3]);
                         // survivors of a non-zero threshold are non-zero: their keep bits are their non-zero bits
                         const uint32_t keep_word = (mask_words || !zeros_survive) ? gather_word<P>(keep, lane) : 0u;
                         const uint32_t nz_word = zeros_survive ? gather_word<P>(nz, lane) : keep_word;
@@ -527,7 +529,7 @@ __global__ void __launch_bounds__(kTileThreads, G == 1 ? 4 : 3) k_sweep_multi(Ta
                 // ---- general path: ragged last tile of a tensor, or a tile that ranks the ties of some variant
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
-                    char* dst = ma.dst[g] + arena_off;
+                    char* dst = STORE ? ma.dst[g] + arena_off : nullptr;
                     uint32_t* mask_words = ma.mask_bits[g] ? ma.mask_bits[g] + off_mask : nullptr;
                     uint32_t* nz_words = ma.ebits[g] + off_mask;
                     const uint32_t te = thr_eff[g], tg = tau[g], qg = quota[g];
@@ -567,7 +569,7 @@ __global__ void __launch_bounds__(kTileThreads, G == 1 ? 4 : 3) k_sweep_multi(Ta
                             for (int j = 0; j < 4; ++j)
                                 w[j] &= ((keep >> (2 * j)) & 1u ? 0x0000FFFFu : 0u) | ((keep >> (2 * j + 1)) & 1u ? 0xFFFF0000u : 0u);
                         }
-                        store_vec<DT>(dst, e, numel, make_uint4(w[0], w[1], w[2], w[3]));
+                        if (STORE) store_vec<DT>(dst, e, numel, make_uint4(w[0], w[1], w[2], w[3]));
                         const uint32_t keep_word = gather_word<P>(keep, lane), nz_word = gather_word<P>(nz, lane);
                         if (word_lane && (vi / GL) * 32 < n_e) {
                             if (mask_words) mask_words[e0 / 32 + vi / GL] = keep_word;
@@ -622,9 +624,14 @@ int launch_multi_sweep(const Tables& tb, const ThresholdWs& ws, const dnns_thres
                        int n_variants, uint32_t* const* nz_map, uint32_t n_out_words, uint32_t n_in_words, int n_sm,
                        cudaStream_t st) {
     const dim3 grid(min((uint32_t)n_sm * (n_variants == 1 ? 4u : 3u), tb.n_tiles));  // resident blocks per SM
+    const bool store = ma.dst[0] != nullptr;
     {
-        ScopedKernel timed("k_sweep_multi", st);
-#define DNNS_LAUNCH_MULTI(DT, G) k_sweep_multi<DT, G><<<grid, kTileThreads, 0, st>>>(tb, ws, thr_dev, ma, n_out_words, n_in_words)
+        ScopedKernel timed(store ? "k_sweep_multi" : "k_sweep_bits", st);
+#define DNNS_LAUNCH_MULTI(DT, G)                                                                                   \
+    do {                                                                                                           \
+        if (store) k_sweep_multi<DT, G, true><<<grid, kTileThreads, 0, st>>>(tb, ws, thr_dev, ma, n_out_words, n_in_words); \
+        else k_sweep_multi<DT, G, false><<<grid, kTileThreads, 0, st>>>(tb, ws, thr_dev, ma, n_out_words, n_in_words);     \
+    } while (0)
         if (tb.dtype == DNNS_F32) {
             if (n_variants == 1) DNNS_LAUNCH_MULTI(DNNS_F32, 1);
             else if (n_variants == 2) DNNS_LAUNCH_MULTI(DNNS_F32, 2);

@@ -158,10 +158,12 @@ class Session:
                                    0 if self.nz_map is None else self.nz_map.data_ptr(), self.out_nz.data_ptr(),
                                    self.in_nz.data_ptr(), _stream())
 
-    def mask_and_structures_multi(self, first_variant: int, n_variants: int):
-        """Steps 2 and 3 of n_variants consecutive variants in one sweep; variant first_variant + g lands in slot g."""
+    def mask_and_structures_multi(self, first_variant: int, n_variants: int, store_masked: bool = True):
+        """Steps 2 and 3 of n_variants consecutive variants in one sweep; variant first_variant + g lands in slot g.
+        store_masked = False: only mask bits and zero structures are written (rebuild with compact_masked)."""
         ptrs = lambda name: [None if self._slot(name, g) is None else self._slot(name, g).data_ptr() for g in range(n_variants)]
-        B.dnns_mask_and_structures_multi(self.plan, self.thr.data_ptr(), first_variant, n_variants, ptrs("masked"),
+        B.dnns_mask_and_structures_multi(self.plan, self.thr.data_ptr(), first_variant, n_variants,
+                                         ptrs("masked") if store_masked else [None] * n_variants,
                                          None if self.mask_bits is None else ptrs("mask_bits"),
                                          None if self.nz_map is None else ptrs("nz_map"), ptrs("out_nz"), ptrs("in_nz"),
                                          _stream())
@@ -188,6 +190,14 @@ class Session:
                        self._slot("keep_count", keep_slot).data_ptr(), self.compact_arena.data_ptr(),
                        self.compact_arena.numel() if dst_bytes is None else dst_bytes, self.dst_offsets.data_ptr(),
                        self.dst_shapes.data_ptr(), _stream())
+
+    def compact_masked(self, variant: int, slot: int = 0, own_keep: bool = False):
+        """Rebuild `variant` straight from the dense model, masking on the way (mask bits of `slot`)."""
+        keep_slot = slot if own_keep else 0
+        B.dnns_compact_masked(self.plan, self.thr.data_ptr(), variant, self._slot("mask_bits", slot).data_ptr(),
+                              self._slot("keep_idx", keep_slot).data_ptr(), self._slot("keep_count", keep_slot).data_ptr(),
+                              self.compact_arena.data_ptr(), self.compact_arena.numel(), self.dst_offsets.data_ptr(),
+                              self.dst_shapes.data_ptr(), _stream())
 
     def propagate_keep_cascade(self, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1,
                                max_passes: int = 8):

@@ -28,10 +28,12 @@ def expected_offsets(sizes_bytes):
 
 
 def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCER | O.RULE_CONSUMER, min_keep=1,
-                      weights=None, check_structure_maps=True, fused=False, multi=0, multi_plan=False):
+                      weights=None, check_structure_maps=True, fused=False, multi=0, multi_plan=False, no_store=False):
     """Thresholds for all of wl.ks in one call, then steps 2-5 for the chosen variants.
     multi = G > 0: steps 2 and 3 of G consecutive variants at a time through the multi-variant sweep;
-    multi_plan: step 4 of those variants in one launch as well (dnns_propagate_keep_multi)."""
+    multi_plan: step 4 of those variants in one launch as well (dnns_propagate_keep_multi);
+    no_store: the sweep writes no masked weights and the rebuild masks the dense model on its way
+    (dnns_compact_masked) - everything but the masked weights themselves is still compared."""
     om = O.OracleModel(wl, dtype, weights)
     dm = DeviceModel(wl, dtype, weights=weights)
     ses = Session(dm, wl.scope, len(wl.ks), slots=max(multi, 1))
@@ -49,10 +51,14 @@ def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCE
             if slot == 0:
                 n = min(multi, len(todo) - pos)
                 assert todo[pos: pos + n] == list(range(v, v + n)), "the multi-variant sweep takes consecutive variants"
-                ses.mask_and_structures_multi(v, n)
+                ses.mask_and_structures_multi(v, n, store_masked=not no_store)
                 if multi_plan:
                     ses.propagate_keep_multi(n, policy, min_keep)
-            if multi_plan:
+            if no_store:
+                if not multi_plan:
+                    ses.propagate_keep(policy, min_keep, slot=slot)
+                ses.compact_masked(v, slot=slot, own_keep=multi_plan)
+            elif multi_plan:
                 ses.compact(slot=slot, own_keep=True)
             else:
                 ses.propagate_keep(policy, min_keep, slot=slot)
@@ -61,8 +67,9 @@ def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCE
             ses.variant(v, policy, min_keep, fused=fused)
         assert ses.device_status() == B.DNNS_OK
         masked_cpu, bits_cpu = O.apply_mask(om, wl.scope, rec_cpu[v])
-        for i, (a, b) in enumerate(zip(ses.masked_tensors(slot=slot), masked_cpu.weights)):
-            assert bits_eq(a, b), f"masked weights, variant {v}, tensor {i}"
+        if not no_store:
+            for i, (a, b) in enumerate(zip(ses.masked_tensors(slot=slot), masked_cpu.weights)):
+                assert bits_eq(a, b), f"masked weights, variant {v}, tensor {i}"
         assert_words(ses.mask_words(slot), bits_cpu, f"mask bits v{v}")
         nz_c, out_c, in_c = O.zero_structures(masked_cpu)
         nz_g, out_g, in_g = ses.structure_words(slot)

@@ -63,6 +63,9 @@ def test_guards_survive_every_entry_point(make, dtype):
     ses.propagate_keep_multi(n_multi)
     for g in range(n_multi):
         ses.compact(slot=g, own_keep=True)
+    ses.mask_and_structures_multi(len(wl.ks) - n_multi, n_multi, store_masked=False)
+    for g in range(n_multi):
+        ses.compact_masked(len(wl.ks) - n_multi + g, slot=g, own_keep=True)
     for v in sorted({0, len(wl.ks) - 1}):
         ses.apply_mask(v)
         ses.zero_structures()

@@ -51,3 +51,5 @@ def test_resnet152_portfolio(dtype):
     G = 4 if dtype == B.DNNS_F32 else 2
     ses = compare_portfolio(wl, dtype, variants=list(range(8 - G, 8)), multi=G, multi_plan=True)
     forward_check(wl, ses, dtype, slot=G - 1, keep_slot=G - 1)
+    # ... and without the sparse model in memory: mask bits only, the rebuild masks the dense weights on its way
+    compare_portfolio(wl, dtype, variants=list(range(8 - G, 8)), multi=G, multi_plan=True, no_store=True)

@@ -27,6 +27,7 @@ def test_multi_variant_sweep_every_variant(make, dtype, multi):
     """Groups of up to four variants masked and analysed in one sweep: each variant as from its own sweep."""
     compare_portfolio(make(), dtype, multi=multi)
     compare_portfolio(make(), dtype, multi=multi, multi_plan=True)     # ... and planned in one launch
+    compare_portfolio(make(), dtype, multi=multi, multi_plan=True, no_store=True)   # ... rebuilt from the dense model
 
 
 @pytest.mark.parametrize("policy", [O.RULE_PRODUCER, O.RULE_CONSUMER, O.RULE_PRODUCER | O.RULE_CONSUMER | O.SHIFT_STRICT])
@@ -52,6 +53,7 @@ def test_per_tensor_scope_and_odd_shapes(dtype):
     compare_portfolio(wl, dtype)
     compare_portfolio(wl, dtype, variants=[1, 3], fused=True)
     compare_portfolio(wl, dtype, multi=2)
+    compare_portfolio(wl, dtype, multi=3, no_store=True)
 
 
 def test_non_prunable_tensor_and_1x1_chain():
@@ -87,6 +89,8 @@ def test_special_values_and_heavy_ties():
     compare_portfolio(wl, B.DNNS_F32, fused=True)
     compare_portfolio(wl, B.DNNS_F32, multi=4)     # tiles that rank the ties of several variants at once
     compare_portfolio(wl, B.DNNS_BF16, multi=3)
+    compare_portfolio(wl, B.DNNS_F32, multi=4, no_store=True)      # ties decided by the mask bits during the rebuild
+    compare_portfolio(wl, B.DNNS_BF16, multi=2, multi_plan=True, no_store=True)
 
 
 def test_deep_chain_with_more_than_1024_gather_items():
@@ -195,5 +199,29 @@ def test_multi_variant_calls_reject_bad_arguments():
     with pytest.raises(B.DnnsError) as e:
         B.dnns_propagate_keep_multi(ses.plan, 2, good[1], good[2], 64, 1, kb, ki, kc, 0)    # unknown policy bit
     assert e.value.status == B.DNNS_ERR_INVALID_ARG
+    assert ses.device_status() == B.DNNS_OK
+    ses.close()
+
+
+@pytest.mark.parametrize("dtype", [B.DNNS_F32, B.DNNS_BF16])
+def test_rebuild_from_the_dense_model_equals_rebuild_from_the_masked_one(dtype):
+    """dnns_compact_masked after dnns_apply_mask gives the destination arena of dnns_compact, byte for byte."""
+    from paper_2309_06973_b200.runtime import DeviceModel, Session
+    wl = W.small_resnet(seed=11)
+    ses = Session(DeviceModel(wl, dtype), wl.scope, len(wl.ks))
+    ses.magnitude_threshold(wl.ks)
+    for v in range(len(wl.ks)):
+        ses.apply_mask(v)
+        ses.zero_structures()
+        ses.propagate_keep()
+        ses.compact_arena.fill_(0x5A)              # the gaps between items keep the fill in both runs
+        ses.compact()
+        torch.cuda.synchronize()
+        want, offs, shapes = ses.compact_arena.clone(), ses.dst_offsets.clone(), ses.dst_shapes.clone()
+        ses.compact_arena.fill_(0x5A)
+        ses.compact_masked(v)
+        torch.cuda.synchronize()
+        assert torch.equal(ses.dst_offsets, offs) and torch.equal(ses.dst_shapes, shapes)
+        assert torch.equal(ses.compact_arena, want)
     assert ses.device_status() == B.DNNS_OK
     ses.close()
