@@ -237,7 +237,7 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
 #pragma unroll
             for (uint32_t e = 0; e < VE; ++e) {
                 uint32_t x = idx[u][e] != kNone ? load_elem<BYTES>(src, idx[u][e]) : 0u;
-                if (MASKED) x = masked_elem<BYTES>(x, mk, idx[u][e]);
+                if (MASKED && idx[u][e] != kNone) x = masked_elem<BYTES>(x, mk, idx[u][e]);  // no source element: no mask bit to look at
                 if (BYTES == 4) w[u][e] = x;
                 else w[u][e >> 1] |= x << (16 * (e & 1));
             }
