@@ -8,7 +8,8 @@ import ctypes as C
 import os
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libdnns.so")
+# DNNS_LIBRARY names another build of the same library (the tests' checked build); there is still no fallback
+LIB_PATH = os.environ.get("DNNS_LIBRARY") or os.path.join(HERE, "libdnns.so")
 
 DNNS_F32, DNNS_BF16 = 0, 1
 DNNS_SCOPE_GLOBAL, DNNS_SCOPE_PER_TENSOR = 0, 1

@@ -16,6 +16,16 @@ namespace {
 constexpr int kThreads = 256;
 constexpr uint32_t kUnitBytes = 16384;
 
+// Checked build (-DDNNS_BOUNDS_CHECK, a second library used by the tests only): every index that depends on
+// data - keep lists, source elements, mask bits - is compared with its extent first; a violation is counted
+// and the access goes to element 0 instead, so nothing faults.  The normal build compiles the checks away.
+#ifdef DNNS_BOUNDS_CHECK
+__device__ unsigned int g_bounds_violations = 0;
+#define DNNS_IDX(i, n) ((uint32_t)(i) < (uint32_t)(n) ? (uint32_t)(i) : (atomicAdd(&g_bounds_violations, 1u), 0u))
+#else
+#define DNNS_IDX(i, n) (i)
+#endif
+
 __global__ void __launch_bounds__(1024) k_compact_layout(Tables tb, CompactWs ws, const int32_t* __restrict__ keep_count,
                                                          uint64_t dst_bytes, uint64_t* dst_offsets,
                                                          int32_t* dst_shapes) {
@@ -69,6 +79,7 @@ struct MaskCtx {
     uint32_t tau;          // threshold key of the tensor's ranking segment
     uint32_t mode;         // 0: nothing is masked; 1: every key equal to tau is masked; 2: the mask bits decide those
     const uint32_t* bits;  // the tensor's packed mask bits (1 = kept), consulted for key == tau in mode 2 only
+    uint32_t numel;        // elements of the tensor (extent of the bits; read by the checked build)
 };
 
 // The element as step 2 leaves it: itself when its key lies above tau (or equals it and its mask bit is set), else +0.
@@ -76,7 +87,10 @@ template <int BYTES>
 __device__ __forceinline__ uint32_t masked_elem(uint32_t x, const MaskCtx& m, uint32_t src_idx) {
     const uint32_t key = x & (BYTES == 4 ? 0x7FFFFFFFu : 0x7FFFu);
     bool keep = key > m.tau;
-    if (key == m.tau && m.mode == 2) keep = (__ldg(m.bits + (src_idx >> 5)) >> (src_idx & 31)) & 1u;
+    if (key == m.tau && m.mode == 2) {
+        const uint32_t i = DNNS_IDX(src_idx, m.numel);
+        keep = (__ldg(m.bits + (i >> 5)) >> (i & 31)) & 1u;
+    }
     return (keep || m.mode == 0) ? x : 0u;
 }
 
@@ -109,6 +123,8 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
     const uint32_t blk = it.blk, Cin = it.Cin;
     const uint32_t Ln = Cn * blk, L = Cin * blk;  // new and old row length
     const uint32_t total = On * Ln;
+    const uint32_t src_numel = (uint32_t)it.O * L;  // elements of the source item
+    (void)src_numel;
     // A thread's destination vectors are kStride elements apart, unit after unit, so its position
     // (row a, offset rem in the row) is advanced with one add and one compare instead of a division.
     constexpr uint32_t kStride = kThreads * VE;
@@ -135,8 +151,8 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
             for (int u = 0; u < U; ++u) {
                 nxt_ok[u] = pos_f < total;
                 if (nxt_ok[u]) {
-                    const uint32_t s0 = (uint32_t)ko[pos_a] * L + pos_rem;
-                    nxt[u] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)s0 * BYTES));
+                    const uint32_t s0 = (uint32_t)ko[DNNS_IDX(pos_a, On)] * L + pos_rem;
+                    nxt[u] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)DNNS_IDX(s0, src_numel - (VE - 1)) * BYTES));
                     if (MASKED) nxt_src[u] = s0;
                 }
                 advance();
@@ -177,18 +193,18 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
             if (f >= total) continue;
             if (rem + VE <= Ln && blk == 1) {
                 // 1x1 kernels, vector inside one filter: one kept-channel lookup per element
-                const uint32_t row = (uint32_t)ko[a] * Cin;
+                const uint32_t row = (uint32_t)ko[DNNS_IDX(a, On)] * Cin;
 #pragma unroll
-                for (uint32_t e = 0; e < VE; ++e) idx[u][e] = row + (ki ? (uint32_t)ki[rem + e] : rem + e);
+                for (uint32_t e = 0; e < VE; ++e) idx[u][e] = row + (ki ? (uint32_t)ki[DNNS_IDX(rem + e, Cn)] : rem + e);
                 continue;
             }
             if (rem + VE <= Ln && blk >= VE) {
                 // vector inside one filter and at most two input channels: two lookups
                 const uint32_t c0 = blk == 9 ? rem / 9u : rem / blk, r0 = rem - c0 * blk, n0 = blk - r0;
-                const uint32_t row = (uint32_t)ko[a] * Cin;
-                const uint32_t base0 = (row + (ki ? (uint32_t)ki[c0] : c0)) * blk + r0;
+                const uint32_t row = (uint32_t)ko[DNNS_IDX(a, On)] * Cin;
+                const uint32_t base0 = (row + (ki ? (uint32_t)ki[DNNS_IDX(c0, Cn)] : c0)) * blk + r0;
                 uint32_t base1 = 0;
-                if (n0 < VE) base1 = (row + (ki ? (uint32_t)ki[c0 + 1] : c0 + 1)) * blk - n0;
+                if (n0 < VE) base1 = (row + (ki ? (uint32_t)ki[DNNS_IDX(c0 + 1, Cn)] : c0 + 1)) * blk - n0;
 #pragma unroll
                 for (uint32_t e = 0; e < VE; ++e) idx[u][e] = (e < n0 ? base0 : base1) + e;
                 continue;
@@ -196,7 +212,7 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
             if (Ln >= VE) {
                 // vectors that cross into the next filter or reach the end of the item: one formula per element
                 // (element e sits at offset rem + e of row a, or past its end in row a + 1), no walk
-                const uint32_t row0 = (uint32_t)ko[a] * Cin;
+                const uint32_t row0 = (uint32_t)ko[DNNS_IDX(a, On)] * Cin;
                 const uint32_t row1 = a + 1 < On ? (uint32_t)ko[a + 1] * Cin : 0u;
 #pragma unroll
                 for (uint32_t e = 0; e < VE; ++e) {
@@ -204,14 +220,14 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
                     const bool wrap = re >= Ln;
                     re = wrap ? re - Ln : re;
                     const uint32_t c = blk == 1 ? re : (blk == 9 ? re / 9u : re / blk), r = re - c * blk;
-                    const uint32_t col = ki ? (uint32_t)ki[c] : c;
+                    const uint32_t col = ki ? (uint32_t)ki[DNNS_IDX(c, Cn)] : c;
                     if (f + e < total) idx[u][e] = ((wrap ? row1 : row0) + col) * blk + r;
                 }
                 continue;
             }
             // rows shorter than a vector: walk element by element
             uint32_t c = blk == 1 ? rem : (blk == 9 ? rem / 9u : rem / blk), r = rem - c * blk;
-            uint32_t row = (uint32_t)ko[a] * Cin, col = ki ? (uint32_t)ki[c] : c;
+            uint32_t row = (uint32_t)ko[DNNS_IDX(a, On)] * Cin, col = ki ? (uint32_t)ki[DNNS_IDX(c, Cn)] : c;
             const uint32_t nv = min(VE, total - f);
 #pragma unroll
             for (uint32_t e = 0; e < VE; ++e) {
@@ -236,7 +252,7 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
             for (int j = 0; j < 4; ++j) w[u][j] = 0;
 #pragma unroll
             for (uint32_t e = 0; e < VE; ++e) {
-                uint32_t x = idx[u][e] != kNone ? load_elem<BYTES>(src, idx[u][e]) : 0u;
+                uint32_t x = idx[u][e] != kNone ? load_elem<BYTES>(src, DNNS_IDX(idx[u][e], src_numel)) : 0u;
                 if (MASKED && idx[u][e] != kNone) x = masked_elem<BYTES>(x, mk, idx[u][e]);  // no source element: no mask bit to look at
                 if (BYTES == 4) w[u][e] = x;
                 else w[u][e >> 1] |= x << (16 * (e & 1));
@@ -351,7 +367,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, Compa
             const ItemDesc& it = tb.items[item];
             const uint32_t On = item_dims[2 * item], Cn = item_dims[2 * item + 1];
             const char* src;
-            MaskCtx mk{0u, 0u, nullptr};
+            MaskCtx mk{0u, 0u, nullptr, 0u};
             if (it.tensor >= 0) {
                 const TensorDesc& d = tb.tensors[it.tensor];
                 src = src_arena ? src_arena + d.arena_off : static_cast<const char*>(d.src);
@@ -360,6 +376,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, Compa
                     mk.tau = r.tau_bits;
                     mk.mode = r.n_below + r.n_tie == 0 ? 0u : (r.n_tie >= r.n_equal ? 1u : 2u);
                     mk.bits = mask_bits + d.off_mask;
+                    mk.numel = d.numel;
                 }
             } else {
                 src = static_cast<const char*>(it.src);
@@ -418,3 +435,14 @@ int launch_compact(const Tables& tb, const CompactWs& ws, const void* src_arena,
 }
 
 }  // namespace dnns
+
+#ifdef DNNS_BOUNDS_CHECK
+// Checked build only: violations counted so far on the current device (and the counter reset).
+extern "C" unsigned int dnns_check_bounds_violations() {
+    unsigned int n = 0, zero = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess || cudaMemcpyFromSymbol(&n, dnns::g_bounds_violations, sizeof(n)) != cudaSuccess)
+        return 0xFFFFFFFFu;
+    cudaMemcpyToSymbol(dnns::g_bounds_violations, &zero, sizeof(zero));
+    return n;
+}
+#endif
