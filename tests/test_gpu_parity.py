@@ -225,3 +225,34 @@ def test_rebuild_from_the_dense_model_equals_rebuild_from_the_masked_one(dtype):
         assert torch.equal(ses.compact_arena, want)
     assert ses.device_status() == B.DNNS_OK
     ses.close()
+
+
+@pytest.mark.parametrize("dtype", [B.DNNS_F32, B.DNNS_BF16])
+def test_two_runs_give_identical_bytes(dtype):
+    """Determinism: the same portfolio generated twice (fresh plans, atomics and all) - every mask bit, keep list
+    and rebuilt byte is the same, although histograms, tie counts and flags are accumulated with atomics."""
+    from paper_2309_06973_b200.runtime import DeviceModel, Session
+    wl = W.resnet56()
+    V = len(wl.ks)
+
+    def run():
+        ses = Session(DeviceModel(wl, dtype), wl.scope, V, slots=2)
+        ses.compact_arena.fill_(0)
+        ses.magnitude_threshold(wl.ks)
+        out = [ses.thr.clone()]
+        for v0 in range(0, V, 2):
+            ses.mask_and_structures_multi(v0, 2)
+            ses.propagate_keep_multi(2)
+            for g in range(2):
+                ses.compact(slot=g, own_keep=True)
+                torch.cuda.synchronize()
+                used = int(ses.dst_offsets[-1].item()) + 4
+                out += [ses._slot("mask_bits", g).clone(), ses._slot("out_nz", g).clone(), ses._slot("in_nz", g).clone(),
+                        ses._slot("keep_bits", g).clone(), ses._slot("keep_count", g).clone(), ses.dst_offsets.clone(),
+                        ses.dst_shapes.clone(), ses.compact_arena[:used].clone()]
+        assert ses.device_status() == B.DNNS_OK
+        ses.close()
+        return out
+
+    first, second = run(), run()
+    assert len(first) == len(second) and all(torch.equal(a, b) for a, b in zip(first, second))
