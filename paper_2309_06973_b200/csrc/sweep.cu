@@ -375,7 +375,7 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_sweep(Tables tb, ThresholdW
 // STORE = false: the masked weights are not written at all (the rebuild then masks the dense weights on its
 // way, dnns_compact_masked); what remains are each variant's mask bits and element bits.
 template <int DT, int G, bool STORE>
-__global__ void __launch_bounds__(kTileThreads, G == 1 ? 4 : 3) k_sweep_multi(Tables tb, ThresholdWs ws, const dnns_threshold* __restrict__ thr,
+__global__ void __launch_bounds__(kTileThreads, (G == 1 || DT == DNNS_BF16) ? 4 : 3) k_sweep_multi(Tables tb, ThresholdWs ws, const dnns_threshold* __restrict__ thr,
                                                                  MultiSweepArgs ma, uint32_t n_clear_a, uint32_t n_clear_b) {
     constexpr int P = Elem<DT>::kPerVec;
     constexpr int GL = 32 / P;  // lanes per bit word
@@ -623,7 +623,7 @@ int launch_tile_sweep(const Tables& tb, const ThresholdWs& ws, bool do_mask, boo
 int launch_multi_sweep(const Tables& tb, const ThresholdWs& ws, const dnns_threshold* thr_dev, const MultiSweepArgs& ma,
                        int n_variants, uint32_t* const* nz_map, uint32_t n_out_words, uint32_t n_in_words, int n_sm,
                        cudaStream_t st) {
-    const dim3 grid(min((uint32_t)n_sm * (n_variants == 1 ? 4u : 3u), tb.n_tiles));  // resident blocks per SM
+    const dim3 grid(min((uint32_t)n_sm * ((n_variants == 1 || tb.dtype == DNNS_BF16) ? 4u : 3u), tb.n_tiles));  // resident blocks per SM
     const bool store = ma.dst[0] != nullptr;
     {
         ScopedKernel timed(store ? "k_sweep_multi" : "k_sweep_bits", st);
