@@ -61,7 +61,7 @@ typedef enum {
     DNNS_ERR_WORKSPACE = 3,   /* workspace or destination arena too small                                   */
     DNNS_ERR_UNSUPPORTED = 4, /* mixed dtypes, unknown dtype, extents beyond the documented limits          */
     DNNS_ERR_CUDA = 5,        /* a CUDA runtime call failed                                                 */
-    DNNS_ERR_TIMEOUT = 6,     /* reserved for bounded device-side waits (the current kernels have none)     */
+    DNNS_ERR_TIMEOUT = 6,     /* a bounded device-side wait ran out (device status of the rebuild)          */
     DNNS_ERR_STATIC_LIMIT = 7 /* input larger than the built-in scratch of a *_static entry point allows    */
 } dnns_status;
 
@@ -176,7 +176,8 @@ uint64_t dnns_plan_launch_count(const dnns_plan* plan);
  * on while a stream is being captured); dnns_plan_profile(plan, 0) stops recording.
  * dnns_plan_profile_read synchronises the device and returns the summed device time and the number of
  * recorded launches of the kernels whose name starts with `kernel` ("k_sweep", "k_compact_gather",
- * "k_flags", "k_propagate", "k_hist1", "k_hist2", "k_ties", "k_select1", "k_select2", "k_tie_scan").
+ * "k_flags", "k_propagate", "k_rebuild_layout", "k_hist1", "k_hist2", "k_ties", "k_select1", "k_select2",
+ * "k_tie_scan", "k_tie_split").
  */
 dnns_status dnns_plan_profile(dnns_plan* plan, int32_t enable);
 dnns_status dnns_plan_profile_read(dnns_plan* plan, const char* kernel, double* total_ms, uint64_t* launches);
@@ -188,7 +189,8 @@ dnns_status dnns_plan_profile_read(dnns_plan* plan, const char* kernel, double* 
  * indexing) receives the records.  One call serves the whole portfolio: the sweeps over the
  * weights are shared by all n_k counts.  The call also leaves, in the workspace, the per-tile
  * tie tables that dnns_apply_mask needs to mask exactly k weights when several weights equal
- * tau; they belong to this call's thr_dev.
+ * tau, and the place (tensor, element) where each variant stops masking them, which
+ * dnns_compact_masked reads; both belong to this call's thr_dev.
  * Errors: INVALID_ARG (null, n_k out of range, a k above its segment), CUDA.
  */
 dnns_status dnns_magnitude_threshold(dnns_plan* plan, const uint64_t* k, int32_t n_k, dnns_threshold* thr_dev,
@@ -259,7 +261,10 @@ dnns_status dnns_mask_and_structures_multi(dnns_plan* plan, const dnns_threshold
  * Frozen groups keep everything.  If fewer than min(min_keep, C) channels stay, removed channels
  * are taken back in ascending order.  Single pass, nothing is re-evaluated after removal.
  * Outputs (device, packed per group): keep_bits, keep_idx (kept channels ascending; entries past
- * keep_count are left untouched), keep_count [n_groups].  stats (device, nullable, 4 words):
+ * keep_count are left untouched), keep_count [n_groups].  The call also prepares, in the workspace, the
+ * destination layout of step 5 for these counts (one more small kernel); dnns_compact finds it by the address
+ * of keep_count, so leave that array as this call wrote it until the rebuild has been enqueued.
+ * stats (device, nullable, 4 words):
  * [0] removed (producer, channel) pairs whose non-zero constant is dropped while some consumer
  * still reads the channel, [1] channels removed, [2] channels taken back by min_keep, [3] 0.
  */
@@ -305,6 +310,11 @@ dnns_status dnns_propagate_keep_cascade(dnns_plan* plan, const uint32_t* nz_map,
  * dst_shapes_dev [n_tensors][2] the new (O', I').  dst_bytes >= layout.compact_arena_bytes always
  * suffices; if the arena is too small for this variant nothing is copied and the device status
  * becomes DNNS_ERR_WORKSPACE.
+ * keep_idx / keep_count are normally the outputs of a dnns_propagate_keep* call on this plan, which has
+ * already laid the variant out; for any other array of counts the layout kernel is enqueued here first.
+ * Weight tensors whose filters are multiples of 16 bytes long are moved through shared memory with bulk
+ * copies that complete on barriers; every wait on such a barrier is bounded (half a second), and a wait that
+ * runs out ends the kernel and leaves DNNS_ERR_TIMEOUT in the device status instead of hanging.
  */
 dnns_status dnns_compact(dnns_plan* plan, const void* masked_arena, const int32_t* keep_idx,
                          const int32_t* keep_count, void* dst_arena, size_t dst_bytes, uint64_t* dst_offsets_dev,
@@ -312,13 +322,14 @@ dnns_status dnns_compact(dnns_plan* plan, const void* masked_arena, const int32_
 
 /*
  * Step 5 reading the DENSE model (the tensors of the plan's model) and applying step 2 on the way: a weight
- * is copied when its key lies above tau of its ranking segment, or equals tau and its mask bit is set, else
- * +0 is written.  Bit for bit the result of dnns_apply_mask followed by dnns_compact.  thr_dev / variant as in
- * dnns_apply_mask; mask_bits: the variant's packed mask bits as written by dnns_apply_mask,
- * dnns_mask_and_structures or dnns_mask_and_structures_multi on the same thresholds (read only where a key
- * equals tau and the variant masks part of those weights); the remaining arguments as in dnns_compact.
+ * is copied when its key lies above tau of its ranking segment, or equals tau and is not among the first n_tie
+ * such weights of the segment, else +0 is written.  Bit for bit the result of dnns_apply_mask followed by
+ * dnns_compact, without the sparse model ever being stored.  thr_dev / variant as in dnns_apply_mask: the
+ * thresholds of the latest dnns_magnitude_threshold call on this plan, which also left in the workspace, for
+ * every variant that masks only part of the weights equal to tau, the place where that part ends.  The
+ * remaining arguments as in dnns_compact.
  */
-dnns_status dnns_compact_masked(dnns_plan* plan, const dnns_threshold* thr_dev, int32_t variant, const uint32_t* mask_bits,
+dnns_status dnns_compact_masked(dnns_plan* plan, const dnns_threshold* thr_dev, int32_t variant,
                                 const int32_t* keep_idx, const int32_t* keep_count, void* dst_arena, size_t dst_bytes,
                                 uint64_t* dst_offsets_dev, int32_t* dst_shapes_dev, void* stream);
 

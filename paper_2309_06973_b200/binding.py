@@ -105,7 +105,7 @@ def lib() -> C.CDLL:
         L.dnns_magnitude_threshold_static.argtypes = [vp, i32, u64, u64, vp, vp]
         L.dnns_mask_and_structures_multi.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp, vp]
         L.dnns_propagate_keep_multi.argtypes = [vp, i32, vp, vp, u32, i32, vp, vp, vp, vp, vp]
-        L.dnns_compact_masked.argtypes = [vp, vp, i32, vp, vp, vp, vp, C.c_size_t, vp, vp, vp]
+        L.dnns_compact_masked.argtypes = [vp, vp, i32, vp, vp, vp, C.c_size_t, vp, vp, vp]
         L.dnns_plan_profile.argtypes = [vp, i32]
         L.dnns_plan_profile_read.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(u64)]
         for name in ("dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes"):
@@ -265,7 +265,7 @@ def dnns_propagate_keep_multi(plan, n_variants: int, out_nz, in_nz, policy: int,
                                            stream), "dnns_propagate_keep_multi")
 
 
-def dnns_compact_masked(plan, thr_dev: int, variant: int, mask_bits: int, keep_idx: int, keep_count: int, dst_arena: int,
+def dnns_compact_masked(plan, thr_dev: int, variant: int, keep_idx: int, keep_count: int, dst_arena: int,
                         dst_bytes: int, dst_offsets_dev: int, dst_shapes_dev: int, stream: int = 0) -> None:
-    _check(lib().dnns_compact_masked(plan, thr_dev, variant, mask_bits, keep_idx, keep_count, dst_arena, dst_bytes,
+    _check(lib().dnns_compact_masked(plan, thr_dev, variant, keep_idx, keep_count, dst_arena, dst_bytes,
                                      dst_offsets_dev, dst_shapes_dev, stream), "dnns_compact_masked")

@@ -3,11 +3,23 @@
 // over, all layers in one batch.  Here that is one gather over every tensor, BatchNorm vector
 // and bias of the model:
 //   layout kernel  sizes each rebuilt item from the keep counts, places it at a 256-byte aligned
-//                  offset of the destination arena and cuts it into 16 KB gather units;
-//   gather kernel  walks the units: destination element (a, c, r) of an item reads source element
-//                  (keep_out[a], keep_in[c], r).  Stores are 16-byte vectors in destination
-//                  order; rows that lose no input channel are copied with 16-byte loads too.
+//                  offset of the destination arena and cuts it into units of work (run once per set of keep
+//                  counts, right after the channels were planned);
+//   gather kernel  destination element (a, c, r) of an item reads source element
+//                  (keep_out[a], keep_in[c], r).
+//
+// Weight tensors whose filters (rows) are a multiple of 16 bytes long take the staged path: a
+// producer warp brings the kept rows of a unit - whole rows, or a range of input channels of one
+// long row - into shared memory with bulk copies (cp.async.bulk, completion on an mbarrier), a ring
+// of kStages buffers deep; eight consumer warps read the surviving elements out of the buffer, one
+// destination element per lane (a pair for 2-byte elements), so that the buffer is read without
+// bank conflicts and the stores of a warp are one contiguous run.  Every global access of that path
+// is contiguous; the only indexed reads are the kept-channel list (cached) and shared memory.
+// BatchNorm vectors and biases are copied by single warps; tensors with other row lengths take the
+// element path (gather_run): 16 KB destination units, source positions computed per element.
 #include "dnns_internal.cuh"
+
+#pragma nv_diag_suppress 186  // "pointless comparison of unsigned integer with zero": thresholds that are 0 in one instantiation
 
 namespace dnns {
 
@@ -26,71 +38,29 @@ __device__ unsigned int g_bounds_violations = 0;
 #define DNNS_IDX(i, n) (i)
 #endif
 
-__global__ void __launch_bounds__(1024) k_compact_layout(Tables tb, CompactWs ws, const int32_t* __restrict__ keep_count,
-                                                         uint64_t dst_bytes, uint64_t* dst_offsets,
-                                                         int32_t* dst_shapes) {
-    __shared__ uint64_t scratch[33];
-    uint64_t carry_bytes = 0, carry_units = 0;
-    for (uint32_t base = 0; base < tb.n_items; base += 1024) {
-        const uint32_t i = base + threadIdx.x;
-        uint64_t bytes = 0, units = 0;
-        if (i < tb.n_items) {
-            const ItemDesc& it = tb.items[i];
-            const int64_t On = keep_count[it.out_group];
-            const int64_t Cn = it.in_group >= 0 ? keep_count[it.in_group] : it.Cin;
-            const uint64_t raw = (uint64_t)(On * Cn * it.blk) * it.elem_bytes;
-            bytes = (raw + 255) & ~(uint64_t)255;
-            units = (raw + kUnitBytes - 1) / kUnitBytes;
-            ws.item_dims[2 * i] = (int32_t)On;
-            ws.item_dims[2 * i + 1] = (int32_t)Cn;
-            if (it.tensor >= 0) {
-                dst_shapes[2 * it.tensor] = (int32_t)On;
-                dst_shapes[2 * it.tensor + 1] = (int32_t)(Cn * tb.tensors[it.tensor].S);
-            }
-        }
-        uint64_t tot_b, tot_u;
-        const uint64_t ex_b = block_exclusive_scan<uint64_t>(bytes, scratch, &tot_b);
-        const uint64_t ex_u = block_exclusive_scan<uint64_t>(units, scratch, &tot_u);
-        if (i < tb.n_items) {
-            ws.item_off[i] = carry_bytes + ex_b;
-            dst_offsets[i] = carry_bytes + ex_b;
-            ws.unit_prefix[i] = (uint32_t)(carry_units + ex_u);
-        }
-        carry_bytes += tot_b;
-        carry_units += tot_u;
-    }
-    if (threadIdx.x == 0) {
-        if (carry_bytes > dst_bytes) {
-            atomicCAS(tb.status, 0u, (uint32_t)DNNS_ERR_WORKSPACE);
-            carry_units = 0;  // nothing is copied
-        }
-        ws.unit_prefix[tb.n_items] = (uint32_t)carry_units;
-    }
-}
-
 template <int BYTES>
 __device__ __forceinline__ uint32_t load_elem(const void* base, uint32_t idx) {
     if (BYTES == 4) return __ldg(static_cast<const uint32_t*>(base) + idx);
     return __ldg(static_cast<const uint16_t*>(base) + idx);
 }
 
-// Masking on the fly (the rebuild reading the dense model): what steps 2 decided for one tensor and variant.
+// Masking on the fly (the rebuild reading the dense model): what step 2 decides for one tensor and variant.
+// A weight stays when its key lies above tau, or equals tau and the weight comes at or after the place where the
+// variant stops masking such weights (threshold step: TieSplit).  Away from that place one comparison settles it.
 struct MaskCtx {
-    uint32_t tau;          // threshold key of the tensor's ranking segment
-    uint32_t mode;         // 0: nothing is masked; 1: every key equal to tau is masked; 2: the mask bits decide those
-    const uint32_t* bits;  // the tensor's packed mask bits (1 = kept), consulted for key == tau in mode 2 only
-    uint32_t numel;        // elements of the tensor (extent of the bits; read by the checked build)
+    uint32_t tau;         // threshold key of the tensor's ranking segment
+    uint32_t mode;        // 0: nothing is masked; 1: keep iff key >= thr_eff; 2: the split lies in this tensor
+    uint32_t thr_eff;     // mode 1: tau + 1 where the weights equal to tau are masked, tau where they stay
+    uint32_t split_elem;  // mode 2: weights equal to tau stay from this element of the tensor on
 };
 
-// The element as step 2 leaves it: itself when its key lies above tau (or equals it and its mask bit is set), else +0.
+// The element as step 2 leaves it (src_idx: its index in the source tensor), else +0.
 template <int BYTES>
 __device__ __forceinline__ uint32_t masked_elem(uint32_t x, const MaskCtx& m, uint32_t src_idx) {
     const uint32_t key = x & (BYTES == 4 ? 0x7FFFFFFFu : 0x7FFFu);
-    bool keep = key > m.tau;
-    if (key == m.tau && m.mode == 2) {
-        const uint32_t i = DNNS_IDX(src_idx, m.numel);
-        keep = (__ldg(m.bits + (i >> 5)) >> (i & 31)) & 1u;
-    }
+    bool keep;
+    if (m.mode == 2) keep = key > m.tau || (key == m.tau && src_idx >= m.split_elem);
+    else keep = key >= m.thr_eff;
     return (keep || m.mode == 0) ? x : 0u;
 }
 
@@ -277,161 +247,670 @@ __device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, 
     }
 }
 
-// Blocks take chunks of consecutive gather units and walk the items that own them.
-//
-// INLINE_LAYOUT (models of up to kInlineItems items): every block derives the destination layout
-// itself, in shared memory, from the keep counts - a few hundred items, one scan - instead of waiting
-// for a separate one-block kernel; block 0 also writes the offsets and shapes the caller asked for.
-constexpr uint32_t kInlineItems = 1024;
+// ---------------------------------------------------------------------------------------------
+// The staged path
+// ---------------------------------------------------------------------------------------------
+constexpr int kStages = 3;                 // ring of stage buffers per block (three blocks per SM)
+constexpr uint32_t kStageBytes = 18432;    // two 3x3 filters of 256 channels, one of 512 (fp32)
+constexpr int kConsumers = kThreads;       // threads 0..255 consume, the warp after them produces
+constexpr int kGatherThreads = kConsumers + 32;
+constexpr int kProducerWarp = kConsumers / 32;
+constexpr uint32_t kMaxRowsPerUnit = 256;  // rows of one unit (eight rounds of a row per lane of the producer)
+constexpr uint32_t kRowMapMax = 4608;      // destination row lengths (elements) that get a row map
+constexpr uint32_t kMaxChunkTab = 127;     // chunks per row whose places in the keep list are tabulated per item
+constexpr uint32_t kWaitLimitNs = 500u * 1000u * 1000u;  // a wait that lasts this long is given up (status TIMEOUT)
 
-// MASKED: the source is the dense model and step 2 is applied to every element on its way (thr, variant, mask_bits).
-template <int WBYTES, bool INLINE_LAYOUT, bool MASKED>  // WBYTES: element width of the weight tensors (BatchNorm, bias: 4 bytes)
-__global__ void __launch_bounds__(kThreads, 4) k_compact_gather(Tables tb, CompactWs ws, const char* src_arena,
-                                                                const int32_t* __restrict__ keep_idx, char* dst_arena,
-                                                                const int32_t* __restrict__ keep_count, uint64_t dst_bytes,
-                                                                uint64_t* dst_offsets, int32_t* dst_shapes,
-                                                                const dnns_threshold* __restrict__ thr, int variant,
-                                                                const uint32_t* __restrict__ mask_bits) {
-    __shared__ uint32_t s_unit_prefix[INLINE_LAYOUT ? kInlineItems + 1 : 1];
-    __shared__ uint64_t s_item_off[INLINE_LAYOUT ? kInlineItems : 1];
-    __shared__ int32_t s_item_dims[INLINE_LAYOUT ? 2 * kInlineItems : 1];
+enum : uint32_t { kUnitStop = 0, kUnitCopy = 1, kUnitGather = 2 };
+
+// What the producer tells the consumers about the unit it put into a stage buffer.
+struct UnitDesc {
+    char* dst;           // destination of the unit's first row, first kept channel of the chunk
+    const int32_t* ki;   // kept input channels, from the first one inside this chunk on
+    const int32_t* ko;   // kept filters, from the unit's first row on
+    uint32_t kind;
+    uint32_t n_r;        // rows
+    uint32_t Wd, Ws;     // elements per row at the destination / in the stage buffer
+    uint32_t Ln;         // elements of a whole destination row
+    uint32_t c_lo;       // first input channel in the stage buffer
+    uint32_t blk, magic; // elements per (row, channel); floor(2^32 / blk) + 1
+    uint32_t L;          // elements of a whole source row
+    uint32_t n_ki;       // kept input channels inside this chunk (extent of ki; read by the checked build)
+    const int32_t* ki_all;  // the item's whole list of kept input channels
+    uint32_t map_seq;    // non-zero: the unit's item has a row map; it changes from one such item to the next
+    uint32_t map_base;   // destination column of the unit's first column in a whole row
+    MaskCtx mk;
+};
+template <int BYTES>
+struct ElemWord;
+template <>
+struct ElemWord<4> {
+    typedef uint32_t type;
+};
+template <>
+struct ElemWord<2> {
+    typedef uint16_t type;
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Wait for a phase of an mbarrier, but not for ever: false when the wait was given up (or another
+// thread of the block gave up before).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63u) == 0 && (*abort_flag || global_ns() - t0 > kWaitLimitNs)) return false;
+    }
+}
+// Bulk copy global -> shared, completion counted in bytes on an mbarrier.  Addresses and size are multiples of 16.
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(smem_dst)),
+                 "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+
+// First p in [0, n) with list[p] >= c (n when none): where a range of source channels starts in the keep list.
+__device__ __forceinline__ uint32_t lower_bound_idx(const int32_t* list, uint32_t n, uint32_t c) {
+    uint32_t lo = 0, hi = n;
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if ((uint32_t)__ldg(list + mid) < c) lo = mid + 1;
+        else hi = mid;
+    }
+    return lo;
+}
+
+// The unit shape of a staged item: blocks of rows by pieces of rows when input channels are dropped, else longer
+// pieces (whole rows where they fit), which need fewer copies.
+struct Geometry {
+    uint32_t ru, ch, nch;
+};
+__device__ __forceinline__ Geometry geometry_of(const ItemDesc& it, uint32_t Cn) {
+    if (Cn == (uint32_t)it.Cin) return Geometry{(uint32_t)it.ru_c, (uint32_t)it.ch_c, (uint32_t)it.nch_c};
+    return Geometry{(uint32_t)it.ru, (uint32_t)it.ch, (uint32_t)it.nch};
+}
+
+// ---- the layout of one variant
+// From the keep counts: rows and channels every item keeps, its 256-byte aligned place in the destination arena,
+// its units of work, and where each block of the gather starts.  One block per variant; the tables stay in the
+// workspace until the keep counts change (dnns_propagate_keep* runs this right after planning the channels).
+__global__ void __launch_bounds__(1024) k_rebuild_layout(Tables tb, LayoutBatch lb, uint32_t n_blocks) {
     __shared__ uint64_t scratch[33];
-    if (INLINE_LAYOUT) {
-        constexpr uint32_t kPer = kInlineItems / kThreads;  // consecutive items per thread
-        uint64_t bytes[kPer], units[kPer], sum_b = 0, sum_u = 0;
+    const int32_t* __restrict__ keep_count = lb.keep_count[blockIdx.x];
+    const RebuildSlot slot = lb.slot[blockIdx.x];
+    uint64_t carry_bytes = 0, carry_uc = 0;  // carry_uc: cost << 32 | units (each stays below 2^32)
+    for (uint32_t base = 0; base < tb.n_items; base += 1024) {
+        const uint32_t i = base + threadIdx.x;
+        uint64_t bytes = 0, uc = 0;
+        RebuildItem r{0, 0, 0, 0, 0, 0, 0, 0};
+        if (i < tb.n_items) {
+            const ItemDesc& it = tb.items[i];
+            r.On = (uint32_t)keep_count[it.out_group];
+            r.Cn = it.in_group >= 0 ? (uint32_t)keep_count[it.in_group] : (uint32_t)it.Cin;
+            const uint64_t raw = (uint64_t)r.On * r.Cn * (uint32_t)it.blk * (uint32_t)it.elem_bytes;
+            bytes = (raw + 255) & ~(uint64_t)255;
+            if (it.kind == kItemStaged) {
+                if (r.On && r.Cn) {
+                    const Geometry g = geometry_of(it, r.Cn);
+                    const uint32_t rows = min(g.ru, r.On), chn = min(g.ch, (uint32_t)it.Cin);
+                    const uint32_t src = rows * chn * (uint32_t)it.blk * (uint32_t)it.elem_bytes;  // at most a stage buffer
+                    const uint32_t dst = (uint32_t)((uint64_t)src * r.Cn / (uint32_t)it.Cin);
+                    r.s_units = ((r.On + g.ru - 1) / g.ru) * g.nch;
+                    r.s_cost = (src + dst + 63) >> 6;
+                    uc = (uint64_t)(r.s_units * r.s_cost) << 32;
+                }
+            } else if (it.kind == kItemElement) {
+                uc = (raw + kUnitBytes - 1) / kUnitBytes;
+            }
+        }
+        uint64_t tot_b, tot_uc;
+        const uint64_t ex_b = block_exclusive_scan<uint64_t>(bytes, scratch, &tot_b);
+        const uint64_t ex_uc = block_exclusive_scan<uint64_t>(uc, scratch, &tot_uc);
+        if (i < tb.n_items) {
+            r.off256 = (uint32_t)((carry_bytes + ex_b) >> 8);
+            r.cost_pre = (uint32_t)((carry_uc + ex_uc) >> 32);
+            r.unit_pre = (uint32_t)(carry_uc + ex_uc);
+            slot.items[i] = r;
+        }
+        carry_bytes += tot_b;
+        carry_uc += tot_uc;
+    }
+    const uint32_t total_cost = (uint32_t)(carry_uc >> 32), total_units = (uint32_t)carry_uc;
+    if (threadIdx.x == 0) {
+        RebuildHeader h{};
+        h.total_bytes = carry_bytes;
+        h.total_cost = total_cost;
+        h.total_units = total_units;
+        *slot.header = h;
+    }
+    __syncthreads();  // the item table is read back below (same block: visible after the barrier)
+    // where every range of the cost axis starts: the last item whose earlier cost is <= the range's start
+    for (uint32_t r = threadIdx.x; r < rebuild_ranges(n_blocks); r += 1024) {
+        const uint32_t lo = rebuild_range_lo(r, n_blocks, total_cost);
+        uint32_t item = 0, top = tb.n_items;
+        while (top - item > 1) {
+            const uint32_t mid = (item + top) >> 1;
+            if (slot.items[mid].cost_pre <= lo) item = mid;
+            else top = mid;
+        }
+        slot.range_item[r] = item;
+    }
+    // the item of every 16 KB unit of the element path
+    for (uint32_t u = threadIdx.x; u < total_units; u += 1024) {
+        uint32_t item = 0, top = tb.n_items;
+        while (top - item > 1) {
+            const uint32_t mid = (item + top) >> 1;
+            if (slot.items[mid].unit_pre <= u) item = mid;
+            else top = mid;
+        }
+        slot.unit_item[u] = item;
+    }
+}
+
+// ---- consumers
+// The unit in a stage buffer is a matrix of n_r rows by Ws source elements (row r at r * Ws); its destination is
+// n_r rows of Wd elements, row r at dst + r * Ln.
+
+// Step 2 on the words of a 16-byte vector when every key equal to tau is treated alike: keep iff key >= thr_eff.
+template <int BYTES>
+__device__ __forceinline__ uint4 threshold_vec(uint4 v, uint32_t thr_eff) {
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    if (BYTES == 4) {
 #pragma unroll
-        for (uint32_t k = 0; k < kPer; ++k) {
-            const uint32_t i = threadIdx.x * kPer + k;
-            bytes[k] = units[k] = 0;
-            if (i < tb.n_items) {
-                const ItemDesc& it = tb.items[i];
-                const int64_t On = keep_count[it.out_group];
-                const int64_t Cn = it.in_group >= 0 ? keep_count[it.in_group] : it.Cin;
-                const uint64_t raw = (uint64_t)(On * Cn * it.blk) * it.elem_bytes;
-                bytes[k] = (raw + 255) & ~(uint64_t)255;
-                units[k] = (raw + kUnitBytes - 1) / kUnitBytes;
-                s_item_dims[2 * i] = (int32_t)On;
-                s_item_dims[2 * i + 1] = (int32_t)Cn;
-                if (blockIdx.x == 0 && it.tensor >= 0) {
-                    dst_shapes[2 * it.tensor] = (int32_t)On;
-                    dst_shapes[2 * it.tensor + 1] = (int32_t)(Cn * tb.tensors[it.tensor].S);
+        for (int j = 0; j < 4; ++j) w[j] = (w[j] & 0x7FFFFFFFu) >= thr_eff ? w[j] : 0u;
+    } else {
+        // both 15-bit keys of a word at once: with bit 15 of each half set, subtracting the threshold leaves that
+        // bit standing exactly where key >= threshold, and no borrow crosses into the other half (thr_eff <= 0x8000)
+        const uint32_t te2 = thr_eff * 0x00010001u;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) w[j] &= ((((w[j] | 0x80008000u) - te2) >> 15) & 0x00010001u) * 0xFFFFu;
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// A unit whose rows lose no channel and land on 16-byte boundaries: 16-byte vectors straight across.
+template <int BYTES, bool MASKED>
+__device__ __forceinline__ void consume_copy(const UnitDesc& desc, const unsigned char* stage, int ctid) {
+    constexpr uint32_t VE = 16 / BYTES;
+    const UnitDesc d = desc;  // in registers: the stores below could alias the descriptor as far as the compiler knows
+    const uint32_t vpr = d.Ws / VE, n_vec = d.n_r * vpr;  // vectors per row, in the unit
+    const uint32_t step_row = kConsumers / vpr, step_col = kConsumers - step_row * vpr;
+    uint32_t row = (uint32_t)ctid / vpr, col = (uint32_t)ctid - row * vpr;
+    const uint4* s = reinterpret_cast<const uint4*>(stage);
+    const size_t row_pitch = (size_t)d.Ln * BYTES;
+#pragma unroll 2
+    for (uint32_t v = ctid; v < n_vec; v += kConsumers) {
+        uint4 x = s[v];
+        if (MASKED && d.mk.mode == 1) x = threshold_vec<BYTES>(x, d.mk.thr_eff);
+        if (MASKED && d.mk.mode == 2)  // around the place where the ties split: element by element, by source position
+            x = masked_vec<BYTES>(x, d.mk, (uint32_t)__ldg(d.ko + row) * d.L + d.c_lo * d.blk + col * VE);
+        *reinterpret_cast<uint4*>(d.dst + row * row_pitch + (size_t)col * 16) = x;
+        row += step_row;
+        col += step_col;
+        if (col >= vpr) {
+            col -= vpr;
+            ++row;
+        }
+    }
+}
+
+// A unit that loses input channels.  A thread owns destination columns (column j of the unit: input channel
+// p = j / blk of the kept list, element j % blk of its 2-D kernel) and walks down the rows, so that the source
+// offset of a column is found once per unit and the loop is a shared-memory load, the mask and a store; the
+// lanes of a warp hold neighbouring columns, which keeps the shared-memory reads free of bank conflicts and a
+// warp's stores contiguous.  The source offsets come from the item's row map in shared memory (rowmap, when the
+// descriptor names one) or from the kept-channel list.  Narrow units put several rows side by side; in wide ones
+// a thread walks down several columns at once.
+template <int BYTES, bool MASKED>
+__device__ __forceinline__ void consume_gather(const UnitDesc& desc, const unsigned char* stage, const uint16_t* rowmap, int ctid) {
+    typedef typename ElemWord<BYTES>::type T;
+    constexpr int kColBatch = 4;
+    const UnitDesc d = desc;
+    const uint32_t Wd = d.Wd, Ws = d.Ws, n_r = d.n_r, blk = d.blk;
+    constexpr uint32_t key_mask = BYTES == 4 ? 0x7FFFFFFFu : 0x7FFFu;
+    // keep iff key >= thr_eff; in the unit where the weights equal to tau split, those compare their source position
+    const uint32_t thr_eff = (!MASKED || d.mk.mode == 0) ? 0u : (d.mk.mode == 1 ? d.mk.thr_eff : d.mk.tau + 1u);
+    const bool split = MASKED && d.mk.mode == 2;
+    const T* sbase = reinterpret_cast<const T*>(stage);
+    T* dbase = reinterpret_cast<T*>(d.dst);
+    // position of destination column `col` in a row of the stage buffer
+    auto source_offset = [&](uint32_t col) -> uint32_t {
+        uint32_t soff;
+        if (d.map_seq) {
+            soff = (uint32_t)rowmap[d.map_base + col] - d.c_lo * blk;
+        } else {
+            const uint32_t p = blk == 1 ? col : (blk == 9 ? col / 9u : __umulhi(col, d.magic));
+            soff = ((uint32_t)__ldg(d.ki + DNNS_IDX(p, d.n_ki)) - d.c_lo) * blk + (col - p * blk);
+        }
+#ifdef DNNS_BOUNDS_CHECK
+        if (soff >= Ws) {
+            atomicAdd(&g_bounds_violations, 1u);
+            soff = 0;
+        }
+#endif
+        return soff;
+    };
+    auto masked = [&](uint32_t x, uint32_t row, uint32_t soff) -> uint32_t {
+        if (!MASKED) return x;
+        const uint32_t key = x & key_mask;
+        bool keep = key >= thr_eff;
+        if (split && key == d.mk.tau) keep = (uint32_t)__ldg(d.ko + row) * d.L + d.c_lo * blk + soff >= d.mk.split_elem;
+        return keep ? x : 0u;
+    };
+    if (Wd > kConsumers / 2) {
+        for (uint32_t cb = ctid; cb < Wd; cb += kConsumers * kColBatch) {
+            uint32_t soff[kColBatch];
+            bool ok[kColBatch];
+#pragma unroll
+            for (int c = 0; c < kColBatch; ++c) {
+                ok[c] = cb + c * kConsumers < Wd;
+                soff[c] = ok[c] ? source_offset(cb + c * kConsumers) : 0u;
+            }
+            const T* sp = sbase;
+            T* dp = dbase + cb;
+#pragma unroll 2
+            for (uint32_t row = 0; row < n_r; ++row) {
+                uint32_t x[kColBatch];
+#pragma unroll
+                for (int c = 0; c < kColBatch; ++c) x[c] = sp[soff[c]];
+#pragma unroll
+                for (int c = 0; c < kColBatch; ++c)
+                    if (ok[c]) dp[c * kConsumers] = (T)masked(x[c], row, soff[c]);
+                sp += Ws;
+                dp += d.Ln;
+            }
+        }
+        return;
+    }
+    // columns side by side: the next power of two at or above Wd
+    const uint32_t cp = Wd <= 1 ? 1u : 1u << (32 - __clz(Wd - 1));
+    const uint32_t row_par = kConsumers / cp, rp = (uint32_t)ctid / cp, col = (uint32_t)ctid - rp * cp;
+    if (col >= Wd) return;
+    const uint32_t soff = source_offset(col);
+    const T* sp = sbase + soff + rp * Ws;
+    T* dp = dbase + col + (size_t)rp * d.Ln;
+    const uint32_t s_step = row_par * Ws;
+    const size_t d_step = (size_t)row_par * d.Ln;
+#pragma unroll 4
+    for (uint32_t row = rp; row < n_r; row += row_par) {
+        *dp = (T)masked(*sp, row, soff);
+        sp += s_step;
+        dp += d_step;
+    }
+}
+
+// ---- the kernel
+//
+// Work is dealt out statically from the variant's prepared layout: the staged units of all items lie on one
+// axis of cost (bytes read and written, a constant per unit of an item), cut into gridDim.x equal ranges, a
+// block owning the units that start in its range; vector items go to single warps, the 16 KB units of the
+// element path to blocks, round robin in pairs.
+//
+// MASKED: the source is the dense model and step 2 is applied to every element on its way (thr, variant, split).
+template <int WBYTES, bool MASKED>  // WBYTES: element width of the weight tensors (BatchNorm, bias: 4 bytes)
+__global__ void __launch_bounds__(kGatherThreads, 3) k_compact_gather(Tables tb, RebuildSlot lay, const char* src_arena,
+                                                                      const int32_t* __restrict__ keep_idx, char* dst_arena,
+                                                                      uint64_t dst_bytes, uint64_t* dst_offsets,
+                                                                      int32_t* dst_shapes,
+                                                                      const dnns_threshold* __restrict__ thr, int variant,
+                                                                      const TieSplit* __restrict__ split) {
+    extern __shared__ uint4 s_stage_mem[];  // kStages buffers of kStageBytes
+    __shared__ __align__(8) uint64_t s_full[kStages], s_empty[kStages];
+    __shared__ UnitDesc s_desc[kStages];
+    __shared__ uint32_t s_abort;
+    __shared__ uint32_t s_chunk_start[kMaxChunkTab + 1];  // the producer's: first kept channel at or above every chunk start
+    // The consumers' row map of the item they are working on: position in a source row of every element of a
+    // destination row (ki[j / blk] * blk + j % blk), built once per item and block.
+    __shared__ uint16_t s_rowmap[kRowMapMax];
+    unsigned char* const stage_mem = reinterpret_cast<unsigned char*>(s_stage_mem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const RebuildHeader* header = lay.header;
+    const RebuildItem* __restrict__ ritems = lay.items;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&s_full[s], 1);                // the producer's arrive; the bytes of its copies
+            mbar_init(&s_empty[s], kConsumers / 32);  // one arrive per consumer warp
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    const uint64_t total_bytes = header->total_bytes;
+    const uint32_t total_cost = header->total_cost, total_units = header->total_units;
+    __syncthreads();
+    if (total_bytes > dst_bytes) {  // too small an arena: nothing is copied
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicCAS(tb.status, 0u, (uint32_t)DNNS_ERR_WORKSPACE);
+        return;
+    }
+    volatile uint32_t* abort_flag = &s_abort;
+    auto give_up = [&]() {
+        *abort_flag = 1;
+        atomicCAS(tb.status, 0u, (uint32_t)DNNS_ERR_TIMEOUT);
+    };
+    auto mask_ctx = [&](const ItemDesc& it) {
+        MaskCtx mk{0u, 0u, 0u, 0u};
+        if (MASKED && it.tensor >= 0 && it.seg >= 0) {
+            const size_t idx = (size_t)variant * tb.n_segs + it.seg;
+            const dnns_threshold r = thr[idx];
+            const TieSplit sp = split[idx];
+            mk.tau = r.tau_bits;
+            if (r.n_below + r.n_tie == 0) {
+                mk.mode = 0;
+            } else if ((uint32_t)it.tensor == sp.tensor) {
+                mk.mode = 2, mk.split_elem = sp.elem;
+            } else {  // tensors before the split have their weights equal to tau masked, tensors after it keep them
+                mk.mode = 1, mk.thr_eff = (uint32_t)it.tensor < sp.tensor ? r.tau_bits + 1u : r.tau_bits;
+            }
+        }
+        return mk;
+    };
+
+    if (warp == kProducerWarp) {
+        // ================= producer: takes ranges of the cost axis, walks their units, fills the ring =================
+        const uint32_t n_ranges = rebuild_ranges(gridDim.x);
+        auto next_range = [&]() {  // the counter's value k stands for range gridDim.x + k
+            uint32_t r = 0;
+            if (lane == 0) r = atomicAdd(&lay.header->next_range, 1u);
+            return gridDim.x + __shfl_sync(0xffffffffu, r, 0);
+        };
+        uint32_t issued = 0, map_seq = 0;
+        bool alive = true;
+        uint32_t range = blockIdx.x, range_after = total_cost ? next_range() : n_ranges;
+        for (; alive && total_cost && range < n_ranges; range = range_after, range_after = range < n_ranges ? next_range() : n_ranges) {
+            const uint32_t lo = rebuild_range_lo(range, gridDim.x, total_cost), hi = rebuild_range_lo(range + 1, gridDim.x, total_cost);
+            if (lo >= hi) continue;
+            for (uint32_t item = lay.range_item[range]; alive && item < tb.n_items; ++item) {
+                const RebuildItem z = ritems[item];
+                if (z.cost_pre >= hi) break;
+                if (z.s_units == 0) continue;
+                const uint32_t pre = z.cost_pre;
+                const uint32_t j_lo = lo > pre ? (lo - pre + z.s_cost - 1) / z.s_cost : 0u;
+                const uint32_t j_hi = min(z.s_units, (hi - pre + z.s_cost - 1) / z.s_cost);
+                if (j_lo >= j_hi) continue;
+                const ItemDesc it = tb.items[item];
+                const char* src = src_arena ? src_arena + it.arena_off : static_cast<const char*>(it.src);
+                char* dst = dst_arena + ((uint64_t)z.off256 << 8);
+                const int32_t* ko = keep_idx + it.ko_off;
+                const int32_t* ki = keep_idx + it.ki_off;
+                const uint32_t blk = it.blk, Cin = it.Cin, L = Cin * blk, Ln = z.Cn * blk;
+                const MaskCtx mk = mask_ctx(it);
+                const Geometry g = geometry_of(it, z.Cn);
+                const uint32_t nch = g.nch, ru = g.ru, ch = g.ch;
+                const bool identity = z.Cn == Cin;  // no input channel is dropped: kept channel p is channel p
+                const bool use_map = !identity && Ln <= kRowMapMax && L <= 65536u;
+                if (use_map) ++map_seq;
+                // where every chunk of channels starts in the keep list (the same for all rows of the item)
+                const bool bounds_tab = nch > 1 && !identity && nch <= kMaxChunkTab;
+                if (bounds_tab) {
+                    __syncwarp();
+                    for (uint32_t c = lane; c <= nch; c += 32) s_chunk_start[c] = c == nch ? z.Cn : lower_bound_idx(ki, z.Cn, c * ch);
+                    __syncwarp();
+                }
+                uint32_t rg = j_lo / nch, cc = j_lo - rg * nch;
+                int32_t rows[kMaxRowsPerUnit / 32];  // this lane's source rows of the current row group (-2: none)
+                for (uint32_t j = j_lo; alive && j < j_hi; ++j) {
+                    const uint32_t a0 = rg * ru, n_r = min(ru, z.On - a0);
+                    if (cc == 0 || j == j_lo) {
+#pragma unroll
+                        for (uint32_t k = 0; k < kMaxRowsPerUnit / 32; ++k) {
+                            const uint32_t r = k * 32 + lane;
+                            rows[k] = r < n_r ? __ldg(ko + DNNS_IDX(a0 + r, z.On)) : -2;
+                        }
+                    }
+                    const uint32_t c_lo = cc * ch, c_hi = min(Cin, c_lo + ch);
+                    uint32_t p_lo = 0, p_hi = z.Cn;
+                    if (identity) {
+                        p_lo = c_lo, p_hi = c_hi;
+                    } else if (bounds_tab) {
+                        p_lo = s_chunk_start[cc], p_hi = s_chunk_start[cc + 1];
+                    } else if (nch > 1) {
+                        p_lo = lower_bound_idx(ki, z.Cn, c_lo);
+                        p_hi = c_hi == Cin ? z.Cn : lower_bound_idx(ki, z.Cn, c_hi);
+                    }
+                    if (++cc == nch) cc = 0, ++rg;
+                    if (p_hi == p_lo) continue;  // every channel of this chunk is dropped: nothing to bring in
+                    const uint32_t Ws = (c_hi - c_lo) * blk, Wd = (p_hi - p_lo) * blk;
+                    const uint32_t row_bytes = Ws * WBYTES;
+                    char* const unit_dst = dst + ((size_t)a0 * Ln + (size_t)p_lo * blk) * WBYTES;
+                    // rows that lose nothing and start on 16-byte boundaries are copied as they are
+                    const bool image = Wd == Ws && (reinterpret_cast<uintptr_t>(unit_dst) & 15) == 0 &&
+                                       (n_r == 1 || ((size_t)Ln * WBYTES & 15) == 0);
+                    // the tensor where the weights equal to tau split: rows wholly before the split mask them, rows wholly
+                    // after it keep them, and only a unit with a row across the split looks at positions
+                    MaskCtx unit_mk = mk;
+                    if (MASKED && mk.mode == 2) {
+                        const uint32_t first_row = (uint32_t)__shfl_sync(0xffffffffu, rows[0], 0);
+                        uint32_t last_row = 0;
+#pragma unroll
+                        for (uint32_t k = 0; k < kMaxRowsPerUnit / 32; ++k)
+                            if ((n_r - 1) / 32 == k) last_row = (uint32_t)__shfl_sync(0xffffffffu, rows[k], (n_r - 1) & 31);
+                        if ((uint64_t)(last_row + 1) * L <= mk.split_elem) unit_mk.mode = 1, unit_mk.thr_eff = mk.tau + 1u;
+                        else if ((uint64_t)first_row * L >= mk.split_elem) unit_mk.mode = 1, unit_mk.thr_eff = mk.tau;
+                    }
+                    const uint32_t s = issued % kStages, use = issued / kStages;
+                    if (!mbar_wait(&s_empty[s], (use & 1u) ^ 1u, abort_flag)) {
+                        give_up();
+                        alive = false;
+                        break;
+                    }
+                    if (lane == 0) {
+                        UnitDesc& d = s_desc[s];
+                        d.dst = unit_dst;
+                        d.ki = ki + p_lo;
+                        d.ko = ko + a0;
+                        d.n_r = n_r;
+                        d.Wd = Wd, d.Ws = Ws, d.Ln = Ln, d.c_lo = c_lo, d.blk = blk, d.magic = it.magic, d.L = L;
+                        d.n_ki = p_hi - p_lo;
+                        d.ki_all = ki;
+                        d.map_seq = use_map ? map_seq : 0u;
+                        d.map_base = p_lo * blk;
+                        d.mk = unit_mk;
+                        d.kind = image ? kUnitCopy : kUnitGather;
+                        mbar_arrive_expect_tx(&s_full[s], n_r * row_bytes);
+                    }
+                    __syncwarp();
+                    // one bulk copy per run of consecutive source rows (whole rows only), 32 rows per round
+                    unsigned char* const stage = stage_mem + (size_t)s * kStageBytes;
+                    const char* const src_col = src + (size_t)c_lo * blk * WBYTES;
+#pragma unroll
+                    for (uint32_t k = 0; k < kMaxRowsPerUnit / 32; ++k) {
+                        if (k * 32 < n_r) {
+                            const uint32_t r = k * 32 + lane;
+                            const int32_t row = rows[k];
+                            const bool valid = row >= 0;
+                            const int32_t prev = __shfl_up_sync(0xffffffffu, row, 1);
+                            const bool head = valid && (lane == 0 || row != prev + 1 || nch > 1);
+                            const uint32_t heads = __ballot_sync(0xffffffffu, head);
+                            const uint32_t n_valid = __popc(__ballot_sync(0xffffffffu, valid));
+                            if (head) {
+                                const uint32_t later = lane == 31 ? 0u : (heads >> (lane + 1));
+                                const uint32_t len = later ? (uint32_t)__ffs(later) : n_valid - lane;
+                                bulk_load(stage + (size_t)r * row_bytes, src_col + (size_t)DNNS_IDX(row, it.O) * L * WBYTES,
+                                          len * row_bytes, &s_full[s]);
+                            }
+                        }
+                    }
+                    ++issued;
                 }
             }
-            sum_b += bytes[k];
-            sum_u += units[k];
         }
-        uint64_t tot_b, tot_u;
-        uint64_t ex_b = block_exclusive_scan<uint64_t>(sum_b, scratch, &tot_b);
-        uint64_t ex_u = block_exclusive_scan<uint64_t>(sum_u, scratch, &tot_u);
-        const bool fits = tot_b <= dst_bytes;
-#pragma unroll
-        for (uint32_t k = 0; k < kPer; ++k) {
-            const uint32_t i = threadIdx.x * kPer + k;
-            if (i < tb.n_items) {
-                s_item_off[i] = ex_b;
-                s_unit_prefix[i] = (uint32_t)ex_u;
-                if (blockIdx.x == 0) dst_offsets[i] = ex_b;
-            }
-            ex_b += bytes[k];
-            ex_u += units[k];
+        if (total_cost && lane == 0 && atomicAdd(&lay.header->done_blocks, 1u) == gridDim.x - 1) {
+            // every block has taken its last range: the counters are ready for the next launch on this layout
+            lay.header->next_range = 0;
+            lay.header->done_blocks = 0;
         }
-        if (threadIdx.x == 0) {
-            s_unit_prefix[tb.n_items] = fits ? (uint32_t)tot_u : 0u;  // too small an arena: nothing is copied
-            if (!fits && blockIdx.x == 0) atomicCAS(tb.status, 0u, (uint32_t)DNNS_ERR_WORKSPACE);
-        }
-        __syncthreads();
-    }
-    const uint32_t* unit_prefix = INLINE_LAYOUT ? s_unit_prefix : ws.unit_prefix;
-    const uint64_t* item_off = INLINE_LAYOUT ? s_item_off : ws.item_off;
-    const int32_t* item_dims = INLINE_LAYOUT ? s_item_dims : ws.item_dims;
-    const uint32_t total_units = unit_prefix[tb.n_items];
-    // Units are dealt to the blocks in chunks, round robin: items differ a lot in cost per unit (plain
-    // row copies against element gathers), and interleaving evens that out without any shared counter.
-    constexpr uint32_t kChunkUnits = 2;
-    for (uint32_t u_lo = blockIdx.x * kChunkUnits; u_lo < total_units; u_lo += gridDim.x * kChunkUnits) {
-        const uint32_t u_hi = min(total_units, u_lo + kChunkUnits);
-        // the item holding the first unit: last i with unit_prefix[i] <= u_lo
-        uint32_t item = 0, hi = tb.n_items;
-        while (hi - item > 1) {
-            const uint32_t mid = (item + hi) >> 1;
-            if (unit_prefix[mid] <= u_lo) item = mid;
-            else hi = mid;
-        }
-        uint32_t unit = u_lo;
-        while (unit < u_hi) {
-            const uint32_t item_begin = unit_prefix[item], item_end = unit_prefix[item + 1];
-            if (unit >= item_end) {  // items that shrank to nothing own no units
-                ++item;
-                continue;
-            }
-            const ItemDesc& it = tb.items[item];
-            const uint32_t On = item_dims[2 * item], Cn = item_dims[2 * item + 1];
-            const char* src;
-            MaskCtx mk{0u, 0u, nullptr, 0u};
-            if (it.tensor >= 0) {
-                const TensorDesc& d = tb.tensors[it.tensor];
-                src = src_arena ? src_arena + d.arena_off : static_cast<const char*>(d.src);
-                if (MASKED && d.seg >= 0) {
-                    const dnns_threshold r = thr[(size_t)variant * tb.n_segs + d.seg];
-                    mk.tau = r.tau_bits;
-                    mk.mode = r.n_below + r.n_tie == 0 ? 0u : (r.n_tie >= r.n_equal ? 1u : 2u);
-                    mk.bits = mask_bits + d.off_mask;
-                    mk.numel = d.numel;
+        if (alive) {  // tell the consumers that this was all
+            const uint32_t s = issued % kStages, use = issued / kStages;
+            if (mbar_wait(&s_empty[s], (use & 1u) ^ 1u, abort_flag)) {
+                if (lane == 0) {
+                    s_desc[s].kind = kUnitStop;
+                    mbar_arrive(&s_full[s]);
                 }
             } else {
-                src = static_cast<const char*>(it.src);
+                give_up();
+                alive = false;
             }
-            char* dst = dst_arena + item_off[item];
-            const int32_t* ko = keep_idx + tb.groups[it.out_group].off_idx;
-            const int32_t* ki = it.in_group >= 0 ? keep_idx + tb.groups[it.in_group].off_idx : nullptr;
-            const uint32_t run_end = min(u_hi, item_end);
-            const uint32_t f0 = (unit - item_begin) * (kUnitBytes / it.elem_bytes);
-            if (WBYTES == 4 || it.elem_bytes == 4) gather_run<4, MASKED>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit, mk);
-            else gather_run<2, MASKED>(it, src, dst, ko, ki, On, Cn, f0, run_end - unit, mk);
-            unit = run_end;
         }
+        if (!alive) {
+            // given up: the copies still in flight must land before the block's shared memory is released
+            const uint32_t first = issued > (uint32_t)kStages ? issued - kStages : 0u;
+            for (uint32_t u = first; u < issued; ++u) {
+                const uint64_t t0 = global_ns();
+                while (!mbar_try_wait(&s_full[u % kStages], (u / kStages) & 1u) && global_ns() - t0 < kWaitLimitNs) {
+                }
+            }
+        }
+        return;
+    }
+
+    // ================= consumers =================
+    // what the caller asked for beside the arena: the offset of every item, the new shape of every tensor
+    for (uint32_t i = blockIdx.x * kConsumers + threadIdx.x; i < tb.n_items; i += gridDim.x * kConsumers) {
+        const RebuildItem z = ritems[i];
+        dst_offsets[i] = (uint64_t)z.off256 << 8;
+        const ItemDesc& it = tb.items[i];
+        if (it.tensor >= 0) {
+            dst_shapes[2 * it.tensor] = (int32_t)z.On;
+            dst_shapes[2 * it.tensor + 1] = (int32_t)(z.Cn * (uint32_t)it.S);
+        }
+    }
+    // vector items (BatchNorm vectors, biases): one warp each, v'[a] = v[keep[a]]
+    {
+        const uint32_t n_warps = gridDim.x * (kConsumers / 32), gwarp = blockIdx.x + gridDim.x * warp;  // neighbours in different blocks
+        for (uint32_t r = gwarp; r < tb.n_vec_items; r += n_warps) {
+            const uint32_t i = tb.vec_items[r];
+            const ItemDesc& it = tb.items[i];
+            const RebuildItem z = ritems[i];
+            const uint32_t* src = static_cast<const uint32_t*>(it.src);
+            uint32_t* dst = reinterpret_cast<uint32_t*>(dst_arena + ((uint64_t)z.off256 << 8));
+            const int32_t* ko = keep_idx + it.ko_off;
+            for (uint32_t a = lane; a < z.On; a += 32) dst[a] = __ldg(src + DNNS_IDX(__ldg(ko + a), it.O));
+        }
+    }
+    // the element path (rows that are not multiples of 16 bytes): 16 KB destination units, a block per pair
+    {
+        constexpr uint32_t kChunkUnits = 2;
+        for (uint32_t u_lo = blockIdx.x * kChunkUnits; u_lo < total_units; u_lo += gridDim.x * kChunkUnits) {
+            const uint32_t u_hi = min(total_units, u_lo + kChunkUnits);
+            uint32_t unit = u_lo;
+            while (unit < u_hi) {
+                const uint32_t item = lay.unit_item[unit];
+                const RebuildItem z = ritems[item];
+                const ItemDesc& it = tb.items[item];
+                const uint32_t item_begin = z.unit_pre;
+                const uint32_t item_end = item_begin + (uint32_t)(((uint64_t)z.On * z.Cn * (uint32_t)it.blk * (uint32_t)it.elem_bytes + kUnitBytes - 1) / kUnitBytes);
+                const char* src = (it.tensor >= 0 && src_arena) ? src_arena + it.arena_off : static_cast<const char*>(it.src);
+                const MaskCtx mk = mask_ctx(it);
+                char* dst = dst_arena + ((uint64_t)z.off256 << 8);
+                const int32_t* ko = keep_idx + it.ko_off;
+                const int32_t* ki = it.in_group >= 0 ? keep_idx + it.ki_off : nullptr;
+                const uint32_t run_end = min(u_hi, item_end);
+                const uint32_t f0 = (unit - item_begin) * (kUnitBytes / it.elem_bytes);
+                if (WBYTES == 4 || it.elem_bytes == 4) gather_run<4, MASKED>(it, src, dst, ko, ki, z.On, z.Cn, f0, run_end - unit, mk);
+                else gather_run<2, MASKED>(it, src, dst, ko, ki, z.On, z.Cn, f0, run_end - unit, mk);
+                unit = run_end;
+            }
+        }
+    }
+    // then the ring
+    uint32_t cur_map = 0;
+    for (uint32_t taken = 0;; ++taken) {
+        const uint32_t s = taken % kStages, use = taken / kStages;
+        if (!mbar_wait(&s_full[s], use & 1u, abort_flag)) {
+            give_up();
+            break;
+        }
+        const UnitDesc& d = s_desc[s];
+        const uint32_t kind = d.kind;
+        if (kind == kUnitStop) break;
+        const unsigned char* stage = stage_mem + (size_t)s * kStageBytes;
+        if (kind == kUnitGather && d.map_seq != 0 && d.map_seq != cur_map) {
+            // a new item: all consumers are done with the old map once they meet here, then build the new one
+            asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+            const uint32_t blk = d.blk, Ln = d.Ln, magic = d.magic;
+            const int32_t* __restrict__ ki_all = d.ki_all;
+            for (uint32_t j = threadIdx.x; j < Ln; j += kConsumers) {
+                const uint32_t p = blk == 1 ? j : (blk == 9 ? j / 9u : __umulhi(j, magic));
+                s_rowmap[j] = (uint16_t)((uint32_t)__ldg(ki_all + DNNS_IDX(p, Ln / blk)) * blk + (j - p * blk));
+            }
+            cur_map = d.map_seq;
+            asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+        }
+        if (kind == kUnitCopy) consume_copy<WBYTES, MASKED>(d, stage, threadIdx.x);
+        else consume_gather<WBYTES, MASKED>(d, stage, s_rowmap, threadIdx.x);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_empty[s]);
     }
 }
 
 }  // namespace
 
-int launch_compact(const Tables& tb, const CompactWs& ws, const void* src_arena, const int32_t* keep_idx,
-                   const int32_t* keep_count, void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets,
-                   int32_t* dst_shapes, int n_sm, cudaStream_t st, const dnns_threshold* thr, int variant,
-                   const uint32_t* mask_bits) {
+cudaError_t init_compact_attributes() {
+    cudaError_t e = cudaSuccess;
+#define DNNS_SET(W, M)                                                                                          \
+    if (e == cudaSuccess)                                                                                       \
+        e = cudaFuncSetAttribute(k_compact_gather<W, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kStages * kStageBytes));
+    DNNS_SET(4, true) DNNS_SET(4, false) DNNS_SET(2, true) DNNS_SET(2, false)
+#undef DNNS_SET
+    return e;
+}
+
+int gather_grid(int n_sm) { return n_sm * 3 < 1024 ? n_sm * 3 : 1024; }  // three resident blocks per SM
+
+int launch_rebuild_layout(const Tables& tb, const LayoutBatch& lb, int n_layouts, int n_sm, cudaStream_t st) {
+    ScopedKernel timed("k_rebuild_layout", st);
+    k_rebuild_layout<<<n_layouts, 1024, 0, st>>>(tb, lb, (uint32_t)gather_grid(n_sm));
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_compact(const Tables& tb, const RebuildSlot& slot, const void* src_arena, const int32_t* keep_idx,
+                   void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets, int32_t* dst_shapes, int n_sm,
+                   cudaStream_t st, const dnns_threshold* thr, int variant, const TieSplit* split) {
     const char* src = (const char*)src_arena;
     char* dst = (char*)dst_arena;
-    const int grid = n_sm * 4;
+    const int grid = gather_grid(n_sm);
+    const size_t smem = (size_t)kStages * kStageBytes;
     const bool masked = thr != nullptr;
-    int launches = 1;
-#define DNNS_GATHER(W, INL, M)                                                                                        \
-    k_compact_gather<W, INL, M><<<grid, kThreads, 0, st>>>(tb, ws, src, keep_idx, dst, keep_count, dst_bytes, dst_offsets, \
-                                                           dst_shapes, thr, variant, mask_bits)
-#define DNNS_GATHER_DT(INL)                                  \
-    do {                                                     \
-        if (tb.dtype == DNNS_F32) {                          \
-            if (masked) DNNS_GATHER(4, INL, true);           \
-            else DNNS_GATHER(4, INL, false);                 \
-        } else {                                             \
-            if (masked) DNNS_GATHER(2, INL, true);           \
-            else DNNS_GATHER(2, INL, false);                 \
-        }                                                    \
-    } while (0)
-    if (tb.n_items <= kInlineItems) {
-        ScopedKernel timed(masked ? "k_compact_gather<masked>" : "k_compact_gather", st);
-        DNNS_GATHER_DT(true);
+    ScopedKernel timed(masked ? "k_compact_gather<masked>" : "k_compact_gather", st);
+#define DNNS_GATHER(W, M)                                                                                          \
+    k_compact_gather<W, M><<<grid, kGatherThreads, smem, st>>>(tb, slot, src, keep_idx, dst, dst_bytes, dst_offsets, \
+                                                               dst_shapes, thr, variant, split)
+    if (tb.dtype == DNNS_F32) {
+        if (masked) DNNS_GATHER(4, true);
+        else DNNS_GATHER(4, false);
     } else {
-        {
-            ScopedKernel timed_layout("k_compact_layout", st);
-            k_compact_layout<<<1, 1024, 0, st>>>(tb, ws, keep_count, dst_bytes, dst_offsets, dst_shapes);
-        }
-        ScopedKernel timed(masked ? "k_compact_gather<masked>" : "k_compact_gather", st);
-        DNNS_GATHER_DT(false);
-        launches = 2;
+        if (masked) DNNS_GATHER(2, true);
+        else DNNS_GATHER(2, false);
     }
-#undef DNNS_GATHER_DT
 #undef DNNS_GATHER
-    return cudaGetLastError() == cudaSuccess ? launches : -1;
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace dnns

@@ -68,12 +68,69 @@ struct SegDesc {
 };
 
 // One gather job of the rebuild: a weight tensor, a BatchNorm vector or a bias.
+enum : int32_t { kItemElement = 0, kItemStaged = 1, kItemVector = 2 };
 struct ItemDesc {
-    const void* src;        // absolute source, or NULL when the source is tensor `tensor` of the arena/model
+    const void* src;        // the vector, or the model's own weight tensor
+    uint64_t arena_off;     // weight tensors: byte offset in a masked arena
     int32_t tensor;         // tensor index for weight items, -1 otherwise
     int32_t O, Cin, blk;    // rows, input channels, elements per (row, input channel)
     int32_t out_group, in_group;  // in_group -1: columns are kept as they are
     int32_t elem_bytes;
+    uint32_t ko_off, ki_off;      // element offsets of the two groups' keep index lists
+    int32_t seg;                  // ranking segment of a weight tensor, -1 when not prunable (or no tensor)
+    uint32_t off_mask, numel;     // weight tensors: word offset of the packed mask bits, elements
+    int32_t S;                    // weight tensors: columns per input channel (shapes are reported in columns)
+    // How the rebuild handles the item:
+    //   kItemStaged   rows brought into shared memory by bulk copies (weight tensors whose rows are multiples of 16 bytes)
+    //   kItemVector   one value per row (BatchNorm vectors, biases): a warp copies v'[a] = v[keep[a]]
+    //   kItemElement  source position computed per destination element, 16 KB destination units, a block per unit
+    int32_t kind;
+    int32_t ru;      // staged: rows per unit
+    int32_t ch;      // input channels per chunk of a row (a multiple of 8 when a row is cut, else Cin)
+    int32_t nch;     // chunks per row
+    int32_t ru_c, ch_c, nch_c;  // the same for a variant that drops none of the item's input channels: longer pieces
+    uint32_t magic;  // floor(2^32 / blk) + 1 for blk > 1: j / blk = umulhi(j, magic) for the j that occur
+    int32_t vec_rank;  // vector items: index among the vector items
+};
+
+// What the keep counts of one variant make of an item (written by the layout kernel, read by the gather).
+struct RebuildItem {
+    uint32_t On, Cn;     // rows and input channels that stay
+    uint32_t off256;     // offset in the destination arena, in units of 256 bytes
+    uint32_t s_units;    // staged units
+    uint32_t s_cost;     // bytes a staged unit reads and writes, in 64-byte granules
+    uint32_t cost_pre;   // cost of the staged units of all earlier items
+    uint32_t unit_pre;   // 16 KB destination units (element path) of all earlier items
+    uint32_t pad;
+};
+struct RebuildHeader {
+    uint64_t total_bytes;  // destination bytes the variant needs
+    uint32_t total_cost, total_units;
+    uint32_t next_range;   // ranges of the cost axis handed out beyond every block's first one (see kSmallRanges)
+    uint32_t done_blocks;  // blocks of the running gather that took their last range; the last one clears both counters
+    uint32_t pad[10];
+};
+// The cost axis of the staged units is cut into ranges: one large range per block of the gather over the first
+// half (taken by block index), then kSmallRanges small ones per block over the second half, handed out through a
+// counter as blocks come free - units differ in cost per byte, and the small ranges even that out.
+constexpr uint32_t kSmallRanges = 4;
+__host__ __device__ inline uint32_t rebuild_ranges(uint32_t n_blocks) { return n_blocks * (1 + kSmallRanges); }
+__host__ __device__ inline uint32_t rebuild_range_lo(uint32_t r, uint32_t n_blocks, uint32_t total_cost) {
+    const uint64_t half = total_cost / 2;
+    if (r <= n_blocks) return (uint32_t)(half * r / n_blocks);
+    return (uint32_t)(half + (uint64_t)(total_cost - half) * (r - n_blocks) / ((uint64_t)kSmallRanges * n_blocks));
+}
+// One prepared layout in the workspace.
+struct RebuildSlot {
+    RebuildHeader* header;
+    RebuildItem* items;        // [n_items]
+    uint32_t* range_item;      // [rebuild_ranges(n_blocks)] the item in which each range of the cost axis starts
+    uint32_t* unit_item;       // [max_units] the item of every unit of the element path
+};
+constexpr int kLayoutBatch = 8;  // layouts one launch of the layout kernel prepares
+struct LayoutBatch {
+    const int32_t* keep_count[kLayoutBatch];
+    RebuildSlot slot[kLayoutBatch];
 };
 
 // Per (variant, segment) state of the radix select between its two passes.
@@ -101,9 +158,16 @@ struct Tables {
     const uint32_t* flag_unit_tensor;  // [n_flag_units] the tensor a unit belongs to
     uint32_t* ebits;        // packed "element is non-zero" bits of the latest sweep (same packing as the mask bits)
     uint32_t* status;       // device status word (a dnns_status, 0 = ok)
-    uint32_t n_tensors, n_groups, n_bn, n_segs, n_items, n_tiles, n_flag_units;
+    const uint32_t* vec_items;  // [n_vec_items] the vector items (BatchNorm vectors, biases) of the rebuild
+    uint32_t n_tensors, n_groups, n_bn, n_segs, n_items, n_tiles, n_flag_units, n_vec_items;
     uint32_t tile_elems;    // 4096 (fp32) or 8192 (bf16)
     int32_t dtype;
+};
+
+// Where a variant stops masking the weights equal to tau, in the ranking order of its segment (tensors in descriptor
+// order, row-major inside): the first such weight that stays.  tensor = 0xFFFFFFFF: none of them stays.
+struct TieSplit {
+    uint32_t tensor, elem;
 };
 
 struct ThresholdWs {
@@ -117,6 +181,7 @@ struct ThresholdWs {
     uint32_t* any_need;     // [1]
     uint32_t* tile_ties;    // [max_variants][n_tiles]: weights equal to tau_v in the tile
     uint32_t* tie_prefix;   // [max_variants][n_tiles]: those in earlier tiles of the segment
+    TieSplit* split;        // [n_k][S]
 };
 
 constexpr int kMultiMax = DNNS_MULTI_MAX;  // variants one multi-variant sweep can produce
@@ -140,12 +205,6 @@ struct CascadeWs {
     uint32_t* live;          // filter flags, then (at live_in_offset words) input-column flags of the current pass
     uint32_t live_in_offset;
     uint32_t* changed;       // [kMaxCascadePasses + 1] pass p removed something
-};
-
-struct CompactWs {
-    uint32_t* unit_prefix;  // [n_items + 1] gather units before each item
-    uint64_t* item_off;     // [n_items] byte offset in the destination arena
-    int32_t* item_dims;     // [n_items][2] rows', input channels' of the rebuilt item
 };
 
 // ---- optional per-kernel timing (dnns_plan_profile): while a plan's profile is on, every kernel launch
@@ -179,12 +238,17 @@ int launch_propagate_cascade(const Tables& tb, const CascadeWs& cw, const uint32
                              int32_t min_keep, int32_t max_passes, uint32_t* keep_bits, int32_t* keep_idx,
                              int32_t* keep_count, uint64_t* stats, uint32_t n_keep_words, uint32_t n_live_words, int n_sm,
                              cudaStream_t st);
-int launch_compact(const Tables& tb, const CompactWs& ws, const void* src_arena, const int32_t* keep_idx,
-                   const int32_t* keep_count, void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets,
-                   int32_t* dst_shapes, int n_sm, cudaStream_t st, const dnns_threshold* thr = nullptr, int variant = 0,
-                   const uint32_t* mask_bits = nullptr);
+int launch_rebuild_layout(const Tables& tb, const LayoutBatch& lb, int n_layouts, int n_sm, cudaStream_t st);
+int launch_compact(const Tables& tb, const RebuildSlot& slot, const void* src_arena, const int32_t* keep_idx,
+                   void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets, int32_t* dst_shapes, int n_sm,
+                   cudaStream_t st, const dnns_threshold* thr = nullptr, int variant = 0,
+                   const TieSplit* split = nullptr);
+int gather_grid(int n_sm);  // blocks of the gather kernel (the layout is cut for this many)
 int launch_fold(const Tables& tb, void* arena, const uint64_t* offsets, const int32_t* shapes, cudaStream_t st);
 cudaError_t init_kernel_attributes();
+cudaError_t init_compact_attributes();
+constexpr uint32_t kGatherStageBytes = 18432;  // one stage buffer of the staged rebuild
+constexpr uint32_t kGatherPieceBytes = 2304;   // longest piece of a row in a unit (64 channels of a 3x3 fp32 filter)
 
 // ---- small device helpers ----
 template <int DT>

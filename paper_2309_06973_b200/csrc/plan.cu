@@ -1,5 +1,6 @@
 // Host side of libdnns: model validation, table construction, workspace map and the C entry
 // points.  Every entry point checks its arguments on the host, enqueues kernels and returns.
+#include <algorithm>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -59,7 +60,8 @@ inline uint64_t align_up(uint64_t x, uint64_t a = kAlign) { return (x + a - 1) /
 struct WsMap {
     uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, producers, consumers, flag_prefix, flag_unit_tensor, status;
     uint64_t tables_end;  // everything before this is uploaded once at plan creation
-    uint64_t k_dev, bitmap, sel, tie_prefix, unit_prefix, item_off, item_dims, ebits;
+    uint64_t k_dev, bitmap, sel, tie_prefix, tie_split, layouts, ebits;
+    uint64_t vec_items;
     uint64_t casc_rem0, casc_rem1, casc_lost, casc_live, casc_changed;
     uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
     uint64_t any_need, need, tie_bitmap, tile_ties, hist1, hist2;
@@ -69,6 +71,7 @@ struct WsMap {
 struct Counts {
     uint32_t T = 0, G = 0, B = 0, S = 0, items = 0, tiles = 0, n_bias = 0;
     uint64_t mask_words = 0, keep_words = 0, out_words = 0, in_words = 0, flag_units = 0;
+    uint32_t n_vec = 0, element_units = 0;   // vector items of the rebuild; 16 KB units its element path can need at most
     int dtype = 0, elem_bytes = 4;
 };
 
@@ -78,6 +81,35 @@ uint64_t flag_units_of(const dnns_tensor& t) {
     const uint64_t n_kernels = (uint64_t)t.O * t.I, wpr = t.I / 32;
     if (t.I % 32 == 0 && (wpr & (wpr - 1)) == 0) return (((uint64_t)t.O + kFlagRows - 1) / kFlagRows) * ((wpr + 31) / 32);
     return (n_kernels + 31) / 32;
+}
+
+// How the rebuild stages a weight tensor in shared memory: a unit is a block of rows (filters) by a range of input
+// channels that fits one stage buffer.  Row pieces are kept at or below kGatherPieceBytes so that a unit has at
+// least eight rows for a thread to walk down; a row is cut at multiples of 8 channels, which is a multiple of 16
+// bytes for either element width (bulk copies).  ru stays 0 when the tensor cannot be staged: rows that are not
+// multiples of 16 bytes, 2-D kernels so large that eight of them exceed a stage buffer.
+void stage_plan(ItemDesc* it) {
+    const uint64_t cell = (uint64_t)it->blk * it->elem_bytes, row_bytes = cell * it->Cin;
+    if (row_bytes % 16 != 0 || (uint64_t)it->Cin * it->blk >= (1ull << 31)) return;
+    auto shape = [&](uint64_t longest_piece, int32_t* ru, int32_t* ch, int32_t* nch) {
+        uint64_t piece = row_bytes;
+        if (row_bytes <= longest_piece) {
+            *ch = it->Cin, *nch = 1;
+        } else {
+            uint64_t c = (longest_piece / cell) & ~7ull;
+            if (c == 0) c = 8;
+            piece = c * cell;
+            if (piece > kGatherStageBytes) return false;
+            *ch = (int32_t)c, *nch = (int32_t)((it->Cin + c - 1) / c);
+        }
+        *ru = (int32_t)std::min<uint64_t>(256, kGatherStageBytes / piece);
+        return true;
+    };
+    int32_t ru, ch, nch;
+    if (!shape(kGatherPieceBytes, &ru, &ch, &nch) || !shape(kGatherStageBytes, &it->ru_c, &it->ch_c, &it->nch_c)) return;
+    it->ru = ru, it->ch = ch, it->nch = nch;
+    it->kind = kItemStaged;
+    it->magic = it->blk > 1 ? (uint32_t)((1ull << 32) / (uint32_t)it->blk) + 1u : 0u;
 }
 
 bool tensor_extents_ok(const dnns_tensor& t) {
@@ -117,6 +149,12 @@ dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts*
         c->in_words += ((uint64_t)t.I + 31) / 32;
         c->flag_units += flag_units_of(t);
         if (t.bias) ++c->n_bias;
+        {   // tensors the rebuild cannot stage take its element path: 16 KB units, at most the whole tensor
+            ItemDesc probe{};
+            probe.Cin = t.I / t.in_spatial, probe.blk = t.KH * t.KW * t.in_spatial, probe.elem_bytes = c->elem_bytes;
+            stage_plan(&probe);
+            if (probe.kind != kItemStaged) c->element_units += (uint32_t)((numel * c->elem_bytes + 16383) / 16384);
+        }
         if (t.prunable) {
             n_prunable += numel;
             ++seg_count;
@@ -138,8 +176,17 @@ dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts*
         has_bn[bn.tensor] = 1;
     }
     c->items = c->T + 4 * c->B + c->n_bias;
+    c->n_vec = 4 * c->B + c->n_bias;
     return DNNS_OK;
 }
+
+// Prepared layouts of the rebuild (one per set of keep counts in use): header, item table, block starts, unit -> item.
+constexpr uint32_t kMaxGatherBlocks = 1024;
+uint64_t layout_slot_bytes(const Counts& c) {
+    return align_up(sizeof(RebuildHeader)) + align_up(sizeof(RebuildItem) * (uint64_t)c.items) + align_up(4ull * rebuild_ranges(kMaxGatherBlocks)) +
+           align_up(4ull * (c.element_units + 1));
+}
+uint32_t layout_slots(int32_t maxv) { return (uint32_t)std::max(maxv, (int32_t)DNNS_MULTI_MAX) + 1; }
 
 WsMap map_workspace(const Counts& c, int32_t maxv) {
     WsMap w{};
@@ -161,6 +208,7 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.consumers = take(sizeof(ConsumerDesc) * c.T);
     w.flag_prefix = take(4ull * (c.T + 1));
     w.flag_unit_tensor = take(4ull * (c.flag_units + 1));
+    w.vec_items = take(4ull * (c.n_vec + 1));
     w.status = take(4);
     w.tables_end = o;
     const uint64_t vs = (uint64_t)maxv * (c.S ? c.S : 1);
@@ -168,9 +216,8 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.bitmap = take(4ull * kBitmapWords * (c.S ? c.S : 1));
     w.sel = take(sizeof(SelectState) * vs);
     w.tie_prefix = take(4ull * maxv * c.tiles);
-    w.unit_prefix = take(4ull * (c.items + 1));
-    w.item_off = take(8ull * c.items);
-    w.item_dims = take(8ull * c.items);
+    w.tie_split = take(sizeof(TieSplit) * vs);
+    w.layouts = take(layout_slot_bytes(c) * layout_slots(maxv));
     w.ebits = take(4ull * c.mask_words * kMultiMax);  // one buffer per slot of the multi-variant sweep
     w.casc_rem0 = take(4ull * c.keep_words);
     w.casc_rem1 = take(4ull * c.keep_words);
@@ -199,7 +246,10 @@ struct dnns_plan {
     char* ws;
     Tables tb;
     ThresholdWs tws;
-    CompactWs cws;
+    // Layouts of the rebuild prepared for sets of keep counts: the device array a dnns_propagate_keep* call wrote
+    // its counts to names the slot its layout went to; dnns_compact looks its keep_count argument up here.
+    std::vector<const int32_t*> layout_owner;
+    uint32_t layout_next;
     CascadeWs kws;
     uint64_t launches;
     int last_n_k;
@@ -215,6 +265,58 @@ struct ProfileScope {  // makes the plan's profile the active one for the launch
     explicit ProfileScope(dnns_plan* p) { dnns::g_timer = p ? &p->timer : nullptr; }
     ~ProfileScope() { dnns::g_timer = nullptr; }
 };
+}  // namespace
+
+namespace {
+
+RebuildSlot layout_slot(const dnns_plan* p, uint32_t index) {
+    char* base = p->ws + p->map.layouts + (uint64_t)index * layout_slot_bytes(p->c);
+    RebuildSlot r;
+    r.header = reinterpret_cast<RebuildHeader*>(base);
+    base += align_up(sizeof(RebuildHeader));
+    r.items = reinterpret_cast<RebuildItem*>(base);
+    base += align_up(sizeof(RebuildItem) * (uint64_t)p->c.items);
+    r.range_item = reinterpret_cast<uint32_t*>(base);
+    base += align_up(4ull * rebuild_ranges(kMaxGatherBlocks));
+    r.unit_item = reinterpret_cast<uint32_t*>(base);
+    return r;
+}
+
+int find_layout(const dnns_plan* p, const int32_t* keep_count) {
+    for (size_t s = 0; s < p->layout_owner.size(); ++s)
+        if (p->layout_owner[s] == keep_count) return (int)s;
+    return -1;
+}
+
+// Enqueue the layout kernel for n arrays of keep counts (device) and remember which slot belongs to which array.
+// Returns the number of launches, -1 on a CUDA error.
+int prepare_layouts(dnns_plan* p, const int32_t* const* keep_count, int n, cudaStream_t st) {
+    int launches = 0;
+    for (int first = 0; first < n; first += kLayoutBatch) {
+        const int nb = std::min(kLayoutBatch, n - first);
+        LayoutBatch lb{};
+        std::vector<int> used;
+        for (int i = 0; i < nb; ++i) {
+            const int32_t* kc = keep_count[first + i];
+            int s = find_layout(p, kc);
+            if (s >= 0 && std::find(used.begin(), used.end(), s) != used.end()) s = -1;  // the same array twice in one batch
+            while (s < 0) {   // the next slot in turn that this batch has not taken yet
+                const int cand = (int)(p->layout_next++ % p->layout_owner.size());
+                if (std::find(used.begin(), used.end(), cand) == used.end()) s = cand;
+            }
+            for (auto& o : p->layout_owner)
+                if (o == kc) o = nullptr;
+            p->layout_owner[s] = kc;
+            used.push_back(s);
+            lb.keep_count[i] = kc;
+            lb.slot[i] = layout_slot(p, (uint32_t)s);
+        }
+        if (launch_rebuild_layout(p->tb, lb, nb, p->n_sm, st) < 0) return -1;
+        ++launches;
+    }
+    return launches;
+}
+
 }  // namespace
 
 extern "C" {
@@ -257,7 +359,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
 
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&p->n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        init_kernel_attributes() != cudaSuccess) {
+        init_kernel_attributes() != cudaSuccess || init_compact_attributes() != cudaSuccess) {
         delete p;
         return DNNS_ERR_CUDA;
     }
@@ -361,26 +463,38 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     }
     for (int i = 0; i < nc; ++i) consumers[i] = ConsumerDesc{td[cons_list[i]].off_innz, td[cons_list[i]].S};
     // gather items: weights, then BN vectors, then biases
-    uint32_t n_it = 0;
+    auto* vec_items = reinterpret_cast<uint32_t*>(host.data() + map.vec_items);
+    uint32_t n_it = 0, n_vec = 0;
     for (uint32_t i = 0; i < c.T; ++i) {
         const dnns_tensor& t = m->tensors[i];
-        id[n_it++] = ItemDesc{nullptr, (int32_t)i, t.O, t.I / t.in_spatial, t.KH * t.KW * t.in_spatial,
-                              t.out_group, t.in_group, c.elem_bytes};
+        ItemDesc w_it{};
+        w_it.src = t.data, w_it.arena_off = td[i].arena_off, w_it.tensor = (int32_t)i;
+        w_it.O = t.O, w_it.Cin = t.I / t.in_spatial, w_it.blk = t.KH * t.KW * t.in_spatial;
+        w_it.out_group = t.out_group, w_it.in_group = t.in_group, w_it.elem_bytes = c.elem_bytes;
+        w_it.ko_off = gd[t.out_group].off_idx, w_it.ki_off = gd[t.in_group].off_idx;
+        w_it.seg = td[i].seg, w_it.off_mask = td[i].off_mask, w_it.numel = td[i].numel, w_it.S = t.in_spatial;
+        w_it.kind = kItemElement, w_it.vec_rank = -1;
+        stage_plan(&w_it);
+        id[n_it++] = w_it;
         compact_bytes += align_up((uint64_t)td[i].numel * c.elem_bytes);
     }
+    auto vector_item = [&](const float* v, int32_t C, int32_t group) {
+        ItemDesc it{};
+        it.src = v, it.tensor = -1, it.O = C, it.Cin = 1, it.blk = 1, it.out_group = group, it.in_group = -1, it.elem_bytes = 4;
+        it.ko_off = gd[group].off_idx, it.seg = -1, it.S = 1, it.kind = kItemVector, it.vec_rank = (int32_t)n_vec;
+        vec_items[n_vec++] = n_it;
+        id[n_it++] = it;
+        compact_bytes += align_up(4ull * C);
+    };
     for (uint32_t b = 0; b < c.B; ++b) {
         const dnns_bn& bn = m->bns[b];
         const float* vec[4] = {bn.gamma, bn.beta, bn.mean, bn.var};
-        for (int k = 0; k < 4; ++k) {
-            id[n_it++] = ItemDesc{vec[k], -1, bn.C, 1, 1, m->tensors[bn.tensor].out_group, -1, 4};
-            compact_bytes += align_up(4ull * bn.C);
-        }
+        for (int k = 0; k < 4; ++k) vector_item(vec[k], bn.C, m->tensors[bn.tensor].out_group);
     }
     for (uint32_t i = 0; i < c.T; ++i)
         if (m->tensors[i].bias) {
             if (td[i].bn >= 0) bd[td[i].bn].bias_item = (int32_t)n_it;
-            id[n_it++] = ItemDesc{m->tensors[i].bias, -1, m->tensors[i].O, 1, 1, m->tensors[i].out_group, -1, 4};
-            compact_bytes += align_up(4ull * m->tensors[i].O);
+            vector_item(m->tensors[i].bias, m->tensors[i].O, m->tensors[i].out_group);
         }
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -421,9 +535,11 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     t.any_need = reinterpret_cast<uint32_t*>(w + map.any_need);
     t.tile_ties = reinterpret_cast<uint32_t*>(w + map.tile_ties);
     t.tie_prefix = reinterpret_cast<uint32_t*>(w + map.tie_prefix);
-    p->cws.unit_prefix = reinterpret_cast<uint32_t*>(w + map.unit_prefix);
-    p->cws.item_off = reinterpret_cast<uint64_t*>(w + map.item_off);
-    p->cws.item_dims = reinterpret_cast<int32_t*>(w + map.item_dims);
+    t.split = reinterpret_cast<TieSplit*>(w + map.tie_split);
+    tb.vec_items = reinterpret_cast<uint32_t*>(w + map.vec_items);
+    tb.n_vec_items = c.n_vec;
+    p->layout_owner.assign(layout_slots(maxv), nullptr);
+    p->layout_next = 0;
     p->kws.rem[0] = reinterpret_cast<uint32_t*>(w + map.casc_rem0);
     p->kws.rem[1] = reinterpret_cast<uint32_t*>(w + map.casc_rem1);
     p->kws.lost = reinterpret_cast<uint32_t*>(w + map.casc_lost);
@@ -577,7 +693,10 @@ dnns_status dnns_propagate_keep(dnns_plan* p, const uint32_t* out_nz, const uint
     ProfileScope profile_scope(p);
     const int n = launch_propagate(p->tb, out_nz, in_nz, policy, min_keep, keep_bits, keep_idx, keep_count, stats, st);
     if (n < 0) return DNNS_ERR_CUDA;
-    p->launches += n;
+    const int32_t* kc[1] = {keep_count};
+    const int nl = prepare_layouts(p, kc, 1, st);  // the rebuild's layout for these counts, while they are hot
+    if (nl < 0) return DNNS_ERR_CUDA;
+    p->launches += n + nl;
     return DNNS_OK;
 }
 
@@ -600,7 +719,9 @@ dnns_status dnns_propagate_keep_multi(dnns_plan* p, int32_t n_variants, const ui
     const int n = launch_propagate_multi(p->tb, n_variants, out_nz, in_nz, policy, min_keep, keep_bits, keep_idx, keep_count,
                                          stats, st);
     if (n < 0) return DNNS_ERR_CUDA;
-    p->launches += n;
+    const int nl = prepare_layouts(p, keep_count, n_variants, st);
+    if (nl < 0) return DNNS_ERR_CUDA;
+    p->launches += n + nl;
     return DNNS_OK;
 }
 
@@ -618,7 +739,10 @@ dnns_status dnns_propagate_keep_cascade(dnns_plan* p, const uint32_t* nz_map, ui
                                            keep_count, stats, (uint32_t)L.keep_words,
                                            (uint32_t)(L.out_nz_words + L.in_nz_words), p->n_sm, st);
     if (n < 0) return DNNS_ERR_CUDA;
-    p->launches += n;
+    const int32_t* kc[1] = {keep_count};
+    const int nl = prepare_layouts(p, kc, 1, st);
+    if (nl < 0) return DNNS_ERR_CUDA;
+    p->launches += n + nl;
     return DNNS_OK;
 }
 
@@ -630,25 +754,39 @@ dnns_status dnns_compact(dnns_plan* p, const void* masked_arena, const int32_t* 
         (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)))
         return DNNS_ERR_INVALID_ARG;
     ProfileScope profile_scope(p);
-    const int n = launch_compact(p->tb, p->cws, masked_arena, keep_idx, keep_count, dst_arena, dst_bytes,
-                                 dst_offsets_dev, dst_shapes_dev, p->n_sm, static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int nl = 0, slot = find_layout(p, keep_count);
+    if (slot < 0) {  // counts that no dnns_propagate_keep* call of this plan wrote: lay them out now
+        const int32_t* kc[1] = {keep_count};
+        if ((nl = prepare_layouts(p, kc, 1, st)) < 0) return DNNS_ERR_CUDA;
+        slot = find_layout(p, keep_count);
+    }
+    const int n = launch_compact(p->tb, layout_slot(p, (uint32_t)slot), masked_arena, keep_idx, dst_arena, dst_bytes,
+                                 dst_offsets_dev, dst_shapes_dev, p->n_sm, st);
     if (n < 0) return DNNS_ERR_CUDA;
-    p->launches += n;
+    p->launches += n + nl;
     return DNNS_OK;
 }
 
-dnns_status dnns_compact_masked(dnns_plan* p, const dnns_threshold* thr_dev, int32_t variant, const uint32_t* mask_bits,
+dnns_status dnns_compact_masked(dnns_plan* p, const dnns_threshold* thr_dev, int32_t variant,
                                 const int32_t* keep_idx, const int32_t* keep_count, void* dst_arena, size_t dst_bytes,
                                 uint64_t* dst_offsets_dev, int32_t* dst_shapes_dev, void* stream) {
-    if (!p || !thr_dev || !mask_bits || !keep_idx || !keep_count || !dst_arena || !dst_offsets_dev || !dst_shapes_dev ||
+    if (!p || !thr_dev || !keep_idx || !keep_count || !dst_arena || !dst_offsets_dev || !dst_shapes_dev ||
         variant < 0 || variant >= p->maxv)
         return DNNS_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) return DNNS_ERR_INVALID_ARG;
     ProfileScope profile_scope(p);
-    const int n = launch_compact(p->tb, p->cws, nullptr, keep_idx, keep_count, dst_arena, dst_bytes, dst_offsets_dev,
-                                 dst_shapes_dev, p->n_sm, static_cast<cudaStream_t>(stream), thr_dev, variant, mask_bits);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int nl = 0, slot = find_layout(p, keep_count);
+    if (slot < 0) {
+        const int32_t* kc[1] = {keep_count};
+        if ((nl = prepare_layouts(p, kc, 1, st)) < 0) return DNNS_ERR_CUDA;
+        slot = find_layout(p, keep_count);
+    }
+    const int n = launch_compact(p->tb, layout_slot(p, (uint32_t)slot), nullptr, keep_idx, dst_arena, dst_bytes,
+                                 dst_offsets_dev, dst_shapes_dev, p->n_sm, st, thr_dev, variant, p->tws.split);
     if (n < 0) return DNNS_ERR_CUDA;
-    p->launches += n;
+    p->launches += n + nl;
     return DNNS_OK;
 }
 

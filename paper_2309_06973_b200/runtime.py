@@ -192,9 +192,9 @@ class Session:
                        self.dst_shapes.data_ptr(), _stream())
 
     def compact_masked(self, variant: int, slot: int = 0, own_keep: bool = False):
-        """Rebuild `variant` straight from the dense model, masking on the way (mask bits of `slot`)."""
+        """Rebuild `variant` straight from the dense model, masking on the way (keep sets of `slot` with own_keep)."""
         keep_slot = slot if own_keep else 0
-        B.dnns_compact_masked(self.plan, self.thr.data_ptr(), variant, self._slot("mask_bits", slot).data_ptr(),
+        B.dnns_compact_masked(self.plan, self.thr.data_ptr(), variant,
                               self._slot("keep_idx", keep_slot).data_ptr(), self._slot("keep_count", keep_slot).data_ptr(),
                               self.compact_arena.data_ptr(), self.compact_arena.numel(), self.dst_offsets.data_ptr(),
                               self.dst_shapes.data_ptr(), _stream())
