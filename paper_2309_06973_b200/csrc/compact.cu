@@ -83,7 +83,7 @@ __device__ __forceinline__ uint4 masked_vec(uint4 v, const MaskCtx& m, uint32_t 
 // Gather a run of consecutive units of one item whose elements are BYTES wide, starting at
 // destination element f0.  A unit is 4 x 16-byte destination vectors per thread.
 template <int BYTES, bool MASKED>
-__device__ __forceinline__ void gather_run(const ItemDesc& it, const char* src, char* dst, const int32_t* ko,
+__device__ __noinline__ void gather_run(const ItemDesc& it, const char* src, char* dst, const int32_t* ko,
                                            const int32_t* ki, uint32_t On, uint32_t Cn, uint32_t f0, uint32_t n_units,
                                            const MaskCtx& mk) {
     constexpr uint32_t VE = 16 / BYTES;  // elements per 16-byte vector
@@ -461,22 +461,36 @@ __device__ __forceinline__ void consume_copy(const UnitDesc& desc, const unsigne
     constexpr uint32_t VE = 16 / BYTES;
     const UnitDesc d = desc;  // in registers: the stores below could alias the descriptor as far as the compiler knows
     const uint32_t vpr = d.Ws / VE, n_vec = d.n_r * vpr;  // vectors per row, in the unit
-    const uint32_t step_row = kConsumers / vpr, step_col = kConsumers - step_row * vpr;
-    uint32_t row = (uint32_t)ctid / vpr, col = (uint32_t)ctid - row * vpr;
     const uint4* s = reinterpret_cast<const uint4*>(stage);
-    const size_t row_pitch = (size_t)d.Ln * BYTES;
+    const uint32_t row_pitch = d.Ln * BYTES;  // a unit spans less than 2^32 destination bytes
+    if (MASKED && d.mk.mode == 2) {
+        // around the place where the weights equal to tau split: element by element, by source position
+        for (uint32_t v = ctid; v < n_vec; v += kConsumers) {
+            const uint32_t row = v / vpr, col = v - row * vpr;
+            const uint4 x = masked_vec<BYTES>(s[v], d.mk, (uint32_t)__ldg(d.ko + row) * d.L + d.c_lo * d.blk + col * VE);
+            *reinterpret_cast<uint4*>(d.dst + (size_t)row * row_pitch + (size_t)col * 16) = x;
+        }
+        return;
+    }
+    const bool mask = MASKED && d.mk.mode == 1;
+    if (row_pitch == vpr * 16) {  // whole rows: the destination is one run as well
+        uint4* g = reinterpret_cast<uint4*>(d.dst);
+#pragma unroll 4
+        for (uint32_t v = ctid; v < n_vec; v += kConsumers) g[v] = mask ? threshold_vec<BYTES>(s[v], d.mk.thr_eff) : s[v];
+        return;
+    }
+    const uint32_t step_row = kConsumers / vpr, step_col = kConsumers - step_row * vpr;
+    const uint32_t step_off = step_row * row_pitch + step_col * 16, wrap_off = row_pitch - vpr * 16;
+    uint32_t row = (uint32_t)ctid / vpr, col = (uint32_t)ctid - row * vpr;
+    uint32_t off = row * row_pitch + col * 16;
 #pragma unroll 2
     for (uint32_t v = ctid; v < n_vec; v += kConsumers) {
-        uint4 x = s[v];
-        if (MASKED && d.mk.mode == 1) x = threshold_vec<BYTES>(x, d.mk.thr_eff);
-        if (MASKED && d.mk.mode == 2)  // around the place where the ties split: element by element, by source position
-            x = masked_vec<BYTES>(x, d.mk, (uint32_t)__ldg(d.ko + row) * d.L + d.c_lo * d.blk + col * VE);
-        *reinterpret_cast<uint4*>(d.dst + row * row_pitch + (size_t)col * 16) = x;
-        row += step_row;
+        *reinterpret_cast<uint4*>(d.dst + off) = mask ? threshold_vec<BYTES>(s[v], d.mk.thr_eff) : s[v];
         col += step_col;
+        off += step_off;
         if (col >= vpr) {
             col -= vpr;
-            ++row;
+            off += wrap_off;
         }
     }
 }
@@ -487,17 +501,17 @@ __device__ __forceinline__ void consume_copy(const UnitDesc& desc, const unsigne
 // lanes of a warp hold neighbouring columns, which keeps the shared-memory reads free of bank conflicts and a
 // warp's stores contiguous.  The source offsets come from the item's row map in shared memory (rowmap, when the
 // descriptor names one) or from the kept-channel list.  Narrow units put several rows side by side; in wide ones
-// a thread walks down several columns at once.
-template <int BYTES, bool MASKED>
+// a thread walks down several columns at once.  CAREFUL: the unit holds the place where the weights equal to
+// tau split (one row of one tensor per variant), and those weights compare their source position.
+template <int BYTES, bool MASKED, bool CAREFUL>
 __device__ __forceinline__ void consume_gather(const UnitDesc& desc, const unsigned char* stage, const uint16_t* rowmap, int ctid) {
     typedef typename ElemWord<BYTES>::type T;
     constexpr int kColBatch = 4;
     const UnitDesc d = desc;
-    const uint32_t Wd = d.Wd, Ws = d.Ws, n_r = d.n_r, blk = d.blk;
+    const uint32_t Wd = d.Wd, Ws = d.Ws, n_r = d.n_r, blk = d.blk, Ln = d.Ln;
     constexpr uint32_t key_mask = BYTES == 4 ? 0x7FFFFFFFu : 0x7FFFu;
-    // keep iff key >= thr_eff; in the unit where the weights equal to tau split, those compare their source position
+    // keep iff key >= thr_eff (0: everything stays)
     const uint32_t thr_eff = (!MASKED || d.mk.mode == 0) ? 0u : (d.mk.mode == 1 ? d.mk.thr_eff : d.mk.tau + 1u);
-    const bool split = MASKED && d.mk.mode == 2;
     const T* sbase = reinterpret_cast<const T*>(stage);
     T* dbase = reinterpret_cast<T*>(d.dst);
     // position of destination column `col` in a row of the stage buffer
@@ -521,7 +535,7 @@ __device__ __forceinline__ void consume_gather(const UnitDesc& desc, const unsig
         if (!MASKED) return x;
         const uint32_t key = x & key_mask;
         bool keep = key >= thr_eff;
-        if (split && key == d.mk.tau) keep = (uint32_t)__ldg(d.ko + row) * d.L + d.c_lo * blk + soff >= d.mk.split_elem;
+        if (CAREFUL && key == d.mk.tau) keep = (uint32_t)__ldg(d.ko + row) * d.L + d.c_lo * blk + soff >= d.mk.split_elem;
         return keep ? x : 0u;
     };
     if (Wd > kConsumers / 2) {
@@ -544,7 +558,7 @@ __device__ __forceinline__ void consume_gather(const UnitDesc& desc, const unsig
                 for (int c = 0; c < kColBatch; ++c)
                     if (ok[c]) dp[c * kConsumers] = (T)masked(x[c], row, soff[c]);
                 sp += Ws;
-                dp += d.Ln;
+                dp += Ln;
             }
         }
         return;
@@ -555,9 +569,9 @@ __device__ __forceinline__ void consume_gather(const UnitDesc& desc, const unsig
     if (col >= Wd) return;
     const uint32_t soff = source_offset(col);
     const T* sp = sbase + soff + rp * Ws;
-    T* dp = dbase + col + (size_t)rp * d.Ln;
+    T* dp = dbase + col + (size_t)rp * Ln;
     const uint32_t s_step = row_par * Ws;
-    const size_t d_step = (size_t)row_par * d.Ln;
+    const uint32_t d_step = row_par * Ln;
 #pragma unroll 4
     for (uint32_t row = rp; row < n_r; row += row_par) {
         *dp = (T)masked(*sp, row, soff);
@@ -864,7 +878,8 @@ __global__ void __launch_bounds__(kGatherThreads, 3) k_compact_gather(Tables tb,
             asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
         }
         if (kind == kUnitCopy) consume_copy<WBYTES, MASKED>(d, stage, threadIdx.x);
-        else consume_gather<WBYTES, MASKED>(d, stage, s_rowmap, threadIdx.x);
+        else if (MASKED && d.mk.mode == 2) consume_gather<WBYTES, MASKED, true>(d, stage, s_rowmap, threadIdx.x);
+        else consume_gather<WBYTES, MASKED, false>(d, stage, s_rowmap, threadIdx.x);
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_empty[s]);
     }
