@@ -203,7 +203,8 @@ dnns_status dnns_magnitude_threshold(dnns_plan* plan, const uint64_t* k, int32_t
  * descriptor order, row-major inside): exactly k weights per segment.  Masked weights become
  * +0, the others are copied bit for bit; tensors that are not prunable are copied.
  * masked_arena (device): destination in arena layout, or NULL to mask the model's tensors in
- * place (only meaningful for the weights the thresholds were computed on).
+ * place (only meaningful for the weights the thresholds were computed on).  variant must be one of
+ * the latest threshold call's (INVALID_ARG otherwise; the same holds for every call that takes one).
  * mask_bits (device, nullable): packed mask bits, 1 = kept; padding bits are written as 0.
  */
 dnns_status dnns_apply_mask(dnns_plan* plan, const dnns_threshold* thr_dev, int32_t variant, void* masked_arena,
@@ -251,6 +252,24 @@ dnns_status dnns_mask_and_structures_multi(dnns_plan* plan, const dnns_threshold
                                            void* stream);
 
 /*
+ * Step 3 for up to DNNS_PORTFOLIO_MAX variants of the latest threshold call from ONE sweep over the dense
+ * weights, without forming any sparse model.  Step 2 keeps a weight of variant v when its key lies above tau_v
+ * (or equals it and is not among the first n_tie such weights), so a filter or an input column still holds a
+ * non-zero weight for v exactly when the largest key in it does: the sweep records the largest key of every
+ * filter and every input column (in the workspace), and each variant's flags follow from comparing those with
+ * its threshold; where a maximum equals tau in the tensor in which the variant's equal weights split, that one
+ * filter or column is read again.  out_nz, in_nz: host arrays of n_variants device pointers, all distinct, each
+ * as in dnns_zero_structures and bit for bit what dnns_apply_mask + dnns_zero_structures give for variant
+ * first_variant + i.  Kernel maps and mask bits are not produced here.  Follow with dnns_propagate_keep_multi
+ * and, per variant, dnns_compact_masked: the sparse model of Section III-C is never stored.
+ * Errors: INVALID_ARG (null, count or range outside the latest threshold call, repeated buffers), CUDA.
+ */
+#define DNNS_PORTFOLIO_MAX 16
+dnns_status dnns_zero_structures_portfolio(dnns_plan* plan, const dnns_threshold* thr_dev, int32_t first_variant,
+                                           int32_t n_variants, uint32_t* const* out_nz, uint32_t* const* in_nz,
+                                           void* stream);
+
+/*
  * Step 4 - keep sets per channel group (Algorithm 1 generalised from a chain to groups).
  * Channel j of a group is removed when
  *   (policy & RULE_PRODUCER) and every producer's filter j is all zero [the paper's rule], and,
@@ -273,7 +292,8 @@ dnns_status dnns_propagate_keep(dnns_plan* plan, const uint32_t* out_nz, const u
                                 uint64_t* stats, void* stream);
 
 /*
- * Step 4 for the n_variants (1..DNNS_MULTI_MAX) variants of a dnns_mask_and_structures_multi call in one launch:
+ * Step 4 for n_variants (1..DNNS_PORTFOLIO_MAX) variants - those of a dnns_mask_and_structures_multi or
+ * dnns_zero_structures_portfolio call - in one launch:
  * Algorithm 1 plans all layers of a model at once; the variants of a portfolio are independent models, so they
  * are planned at once too.  out_nz, in_nz, keep_bits, keep_idx, keep_count: host arrays of n_variants device
  * pointers (the outputs all distinct), each as in dnns_propagate_keep; stats (device, nullable): 4 words per

@@ -20,11 +20,12 @@ DNNS_GROUP_FROZEN = 1
 DNNS_STATIC_MAX_NUMEL = 1 << 26
 DNNS_DEFLATE_CHUNK, DNNS_DEFLATE_SUB = 16384, 512
 DNNS_MULTI_MAX = 4
+DNNS_PORTFOLIO_MAX = 16
 
 EXPORTS = ["dnns_status_string", "dnns_workspace_bytes", "dnns_plan_create", "dnns_plan_destroy", "dnns_plan_layout",
            "dnns_plan_launch_count", "dnns_magnitude_threshold", "dnns_apply_mask", "dnns_zero_structures",
            "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures", "dnns_fold_batchnorm", "dnns_propagate_keep_cascade",
-           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_mask_and_structures_multi", "dnns_propagate_keep_multi", "dnns_compact_masked", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
+           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_mask_and_structures_multi", "dnns_propagate_keep_multi", "dnns_compact_masked", "dnns_zero_structures_portfolio", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
 
 
 class dnns_tensor(C.Structure):
@@ -106,6 +107,7 @@ def lib() -> C.CDLL:
         L.dnns_mask_and_structures_multi.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp, vp]
         L.dnns_propagate_keep_multi.argtypes = [vp, i32, vp, vp, u32, i32, vp, vp, vp, vp, vp]
         L.dnns_compact_masked.argtypes = [vp, vp, i32, vp, vp, vp, C.c_size_t, vp, vp, vp]
+        L.dnns_zero_structures_portfolio.argtypes = [vp, vp, i32, i32, vp, vp, vp]
         L.dnns_plan_profile.argtypes = [vp, i32]
         L.dnns_plan_profile_read.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(u64)]
         for name in ("dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes"):
@@ -263,6 +265,13 @@ def dnns_propagate_keep_multi(plan, n_variants: int, out_nz, in_nz, policy: int,
     outs = [_ptr_array(a) for a in (keep_bits, keep_idx, keep_count)]
     _check(lib().dnns_propagate_keep_multi(plan, n_variants, arrays[0], arrays[1], policy, min_keep, *outs, stats or None,
                                            stream), "dnns_propagate_keep_multi")
+
+
+def dnns_zero_structures_portfolio(plan, thr_dev: int, first_variant: int, n_variants: int, out_nz, in_nz,
+                                   stream: int = 0) -> None:
+    """out_nz, in_nz: lists of n_variants device addresses."""
+    _check(lib().dnns_zero_structures_portfolio(plan, thr_dev, first_variant, n_variants, _ptr_array(out_nz),
+                                                _ptr_array(in_nz), stream), "dnns_zero_structures_portfolio")
 
 
 def dnns_compact_masked(plan, thr_dev: int, variant: int, keep_idx: int, keep_count: int, dst_arena: int,

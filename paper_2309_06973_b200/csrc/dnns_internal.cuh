@@ -32,6 +32,7 @@ struct TensorDesc {
     int32_t bn;             // BatchNorm that follows it, -1 when none
     uint32_t tile0, n_tiles;
     uint32_t off_mask, off_nzmap, off_outnz, off_innz;  // word offsets into the packed bit arrays
+    uint32_t off_row, off_col;  // element offsets of the tensor's filters / input columns in the per-row / per-column tables
 };
 
 struct GroupDesc {
@@ -185,6 +186,7 @@ struct ThresholdWs {
 };
 
 constexpr int kMultiMax = DNNS_MULTI_MAX;  // variants one multi-variant sweep can produce
+constexpr int kPortfolioMax = DNNS_PORTFOLIO_MAX;  // variants one portfolio-wide call (zero structures, keep sets) can take
 
 // Per-variant arguments of the multi-variant sweep (unused slots repeat slot 0).
 struct MultiSweepArgs {
@@ -244,6 +246,10 @@ int launch_compact(const Tables& tb, const RebuildSlot& slot, const void* src_ar
                    cudaStream_t st, const dnns_threshold* thr = nullptr, int variant = 0,
                    const TieSplit* split = nullptr);
 int gather_grid(int n_sm);  // blocks of the gather kernel (the layout is cut for this many)
+int launch_extrema(const Tables& tb, uint32_t* rowmax, uint32_t* colmax, int n_sm, cudaStream_t st);
+int launch_extrema_flags(const Tables& tb, const uint32_t* rowmax, const uint32_t* colmax, const dnns_threshold* thr,
+                         const TieSplit* split, int first_variant, int n_variants, uint32_t* const* out_nz,
+                         uint32_t* const* in_nz, cudaStream_t st);
 int launch_fold(const Tables& tb, void* arena, const uint64_t* offsets, const int32_t* shapes, cudaStream_t st);
 cudaError_t init_kernel_attributes();
 cudaError_t init_compact_attributes();

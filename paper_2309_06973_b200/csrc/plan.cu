@@ -60,7 +60,7 @@ inline uint64_t align_up(uint64_t x, uint64_t a = kAlign) { return (x + a - 1) /
 struct WsMap {
     uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, producers, consumers, flag_prefix, flag_unit_tensor, status;
     uint64_t tables_end;  // everything before this is uploaded once at plan creation
-    uint64_t k_dev, bitmap, sel, tie_prefix, tie_split, layouts, ebits;
+    uint64_t k_dev, bitmap, sel, tie_prefix, tie_split, layouts, ebits, rowmax, colmax;
     uint64_t vec_items;
     uint64_t casc_rem0, casc_rem1, casc_lost, casc_live, casc_changed;
     uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
@@ -71,6 +71,7 @@ struct WsMap {
 struct Counts {
     uint32_t T = 0, G = 0, B = 0, S = 0, items = 0, tiles = 0, n_bias = 0;
     uint64_t mask_words = 0, keep_words = 0, out_words = 0, in_words = 0, flag_units = 0;
+    uint64_t sum_O = 0, sum_I = 0;           // filters / input columns of all tensors
     uint32_t n_vec = 0, element_units = 0;   // vector items of the rebuild; 16 KB units its element path can need at most
     int dtype = 0, elem_bytes = 4;
 };
@@ -146,6 +147,7 @@ dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts*
         c->tiles += (uint32_t)((numel * c->elem_bytes + kTileBytes - 1) / kTileBytes);
         c->mask_words += (numel + 31) / 32;
         c->out_words += ((uint64_t)t.O + 31) / 32;
+        c->sum_O += t.O, c->sum_I += t.I;
         c->in_words += ((uint64_t)t.I + 31) / 32;
         c->flag_units += flag_units_of(t);
         if (t.bias) ++c->n_bias;
@@ -219,6 +221,8 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.tie_split = take(sizeof(TieSplit) * vs);
     w.layouts = take(layout_slot_bytes(c) * layout_slots(maxv));
     w.ebits = take(4ull * c.mask_words * kMultiMax);  // one buffer per slot of the multi-variant sweep
+    w.rowmax = take(4ull * c.sum_O);   // largest key per filter and per input column (portfolio-wide zero structures);
+    w.colmax = take(4ull * c.sum_I);   // contiguous, cleared together
     w.casc_rem0 = take(4ull * c.keep_words);
     w.casc_rem1 = take(4ull * c.keep_words);
     w.casc_lost = take(4ull * c.keep_words);
@@ -383,6 +387,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     p->innz_off.resize(c.T), p->seg_of_tensor.assign(c.T, -1), p->keep_off.resize(c.G), p->keepidx_off.resize(c.G);
     p->seg_size.assign(c.S ? c.S : 1, 0);
     uint64_t arena = 0, mask_w = 0, map_w = 0, out_w = 0, in_w = 0, compact_bytes = 0, n_prunable = 0, flag_units = 0;
+    uint64_t row_e = 0, col_e = 0;
     uint32_t tile = 0, seg = 0;
     for (uint32_t S = 0; S < c.S; ++S) sd[S] = SegDesc{0xFFFFFFFFu, 0, 0};
     for (uint32_t i = 0; i < c.T; ++i) {
@@ -402,6 +407,8 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
         d.off_nzmap = (uint32_t)map_w, p->nzmap_off[i] = map_w, map_w += ((uint64_t)t.O * t.I + 31) / 32;
         d.off_outnz = (uint32_t)out_w, p->outnz_off[i] = out_w, out_w += ((uint64_t)t.O + 31) / 32;
         d.off_innz = (uint32_t)in_w, p->innz_off[i] = in_w, in_w += ((uint64_t)t.I + 31) / 32;
+        d.off_row = (uint32_t)row_e, row_e += t.O;
+        d.off_col = (uint32_t)col_e, col_e += t.I;
         d.seg = -1;
         if (t.prunable) {
             const uint32_t sgi = scope == DNNS_SCOPE_GLOBAL ? 0 : seg++;
@@ -425,7 +432,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
         delete p;
         return DNNS_ERR_UNSUPPORTED;
     }
-    if (mask_w >= (1ull << 32) || map_w >= (1ull << 32)) {
+    if (mask_w >= (1ull << 32) || map_w >= (1ull << 32) || row_e >= (1ull << 32) || col_e >= (1ull << 32)) {
         delete p;
         return DNNS_ERR_UNSUPPORTED;
     }
@@ -601,7 +608,7 @@ dnns_status dnns_magnitude_threshold(dnns_plan* p, const uint64_t* k, int32_t n_
 
 dnns_status dnns_apply_mask(dnns_plan* p, const dnns_threshold* thr_dev, int32_t variant, void* masked_arena,
                             uint32_t* mask_bits, void* stream) {
-    if (!p || !thr_dev || variant < 0 || variant >= p->maxv) return DNNS_ERR_INVALID_ARG;
+    if (!p || !thr_dev || variant < 0 || variant >= p->last_n_k) return DNNS_ERR_INVALID_ARG;  // a variant of the latest threshold call
     if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
     ProfileScope profile_scope(p);
     const int n = launch_tile_sweep(p->tb, p->tws, true, false, thr_dev, variant, nullptr, masked_arena, mask_bits,
@@ -629,7 +636,7 @@ dnns_status dnns_zero_structures(dnns_plan* p, const void* masked_arena, uint32_
 dnns_status dnns_mask_and_structures(dnns_plan* p, const dnns_threshold* thr_dev, int32_t variant, void* masked_arena,
                                      uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz,
                                      void* stream) {
-    if (!p || !thr_dev || !out_nz || !in_nz || variant < 0 || variant >= p->maxv) return DNNS_ERR_INVALID_ARG;
+    if (!p || !thr_dev || !out_nz || !in_nz || variant < 0 || variant >= p->last_n_k) return DNNS_ERR_INVALID_ARG;
     if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const dnns_layout& L = p->layout;
@@ -647,7 +654,7 @@ dnns_status dnns_mask_and_structures_multi(dnns_plan* p, const dnns_threshold* t
                                            uint32_t* const* nz_map, uint32_t* const* out_nz, uint32_t* const* in_nz,
                                            void* stream) {
     if (!p || !thr_dev || !masked_arenas || !out_nz || !in_nz || n_variants < 1 || n_variants > kMultiMax ||
-        first_variant < 0 || first_variant + n_variants > p->maxv)
+        first_variant < 0 || first_variant + n_variants > p->last_n_k)
         return DNNS_ERR_INVALID_ARG;
     // masked_arenas all NULL: the masked weights are not written (see dnns_compact_masked); mask bits are then required
     bool no_store = true;
@@ -683,6 +690,32 @@ dnns_status dnns_mask_and_structures_multi(dnns_plan* p, const dnns_threshold* t
     return DNNS_OK;
 }
 
+dnns_status dnns_zero_structures_portfolio(dnns_plan* p, const dnns_threshold* thr_dev, int32_t first_variant,
+                                           int32_t n_variants, uint32_t* const* out_nz, uint32_t* const* in_nz,
+                                           void* stream) {
+    if (!p || !thr_dev || !out_nz || !in_nz || n_variants < 1 || n_variants > kPortfolioMax || first_variant < 0 ||
+        first_variant + n_variants > p->last_n_k)
+        return DNNS_ERR_INVALID_ARG;
+    for (int v = 0; v < n_variants; ++v) {
+        if (!out_nz[v] || !in_nz[v]) return DNNS_ERR_INVALID_ARG;
+        for (int u = 0; u < v; ++u)  // every variant writes flags of its own
+            if (out_nz[u] == out_nz[v] || in_nz[u] == in_nz[v]) return DNNS_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t* rowmax = reinterpret_cast<uint32_t*>(p->ws + p->map.rowmax);
+    uint32_t* colmax = reinterpret_cast<uint32_t*>(p->ws + p->map.colmax);
+    const uint64_t clear_bytes = p->map.colmax + 4ull * p->c.sum_I - p->map.rowmax;  // both tables: the maxima start at zero
+    if (cudaMemsetAsync(rowmax, 0, clear_bytes, st) != cudaSuccess) return DNNS_ERR_CUDA;
+    ProfileScope profile_scope(p);
+    const int n1 = launch_extrema(p->tb, rowmax, colmax, p->n_sm, st);
+    if (n1 < 0) return DNNS_ERR_CUDA;
+    const int n2 = launch_extrema_flags(p->tb, rowmax, colmax, thr_dev, p->tws.split, first_variant, n_variants, out_nz,
+                                        in_nz, st);
+    if (n2 < 0) return DNNS_ERR_CUDA;
+    p->launches += n1 + n2;
+    return DNNS_OK;
+}
+
 dnns_status dnns_propagate_keep(dnns_plan* p, const uint32_t* out_nz, const uint32_t* in_nz, uint32_t policy,
                                 int32_t min_keep, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count,
                                 uint64_t* stats, void* stream) {
@@ -704,7 +737,7 @@ dnns_status dnns_propagate_keep_multi(dnns_plan* p, int32_t n_variants, const ui
                                       const uint32_t* const* in_nz, uint32_t policy, int32_t min_keep,
                                       uint32_t* const* keep_bits, int32_t* const* keep_idx, int32_t* const* keep_count,
                                       uint64_t* stats, void* stream) {
-    if (!p || !out_nz || !in_nz || !keep_bits || !keep_idx || !keep_count || n_variants < 1 || n_variants > kMultiMax)
+    if (!p || !out_nz || !in_nz || !keep_bits || !keep_idx || !keep_count || n_variants < 1 || n_variants > kPortfolioMax)
         return DNNS_ERR_INVALID_ARG;
     if (policy & ~(uint32_t)(DNNS_RULE_PRODUCER | DNNS_RULE_CONSUMER | DNNS_SHIFT_STRICT)) return DNNS_ERR_INVALID_ARG;
     for (int v = 0; v < n_variants; ++v) {
@@ -772,7 +805,7 @@ dnns_status dnns_compact_masked(dnns_plan* p, const dnns_threshold* thr_dev, int
                                 const int32_t* keep_idx, const int32_t* keep_count, void* dst_arena, size_t dst_bytes,
                                 uint64_t* dst_offsets_dev, int32_t* dst_shapes_dev, void* stream) {
     if (!p || !thr_dev || !keep_idx || !keep_count || !dst_arena || !dst_offsets_dev || !dst_shapes_dev ||
-        variant < 0 || variant >= p->maxv)
+        variant < 0 || variant >= p->last_n_k)
         return DNNS_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) return DNNS_ERR_INVALID_ARG;
     ProfileScope profile_scope(p);

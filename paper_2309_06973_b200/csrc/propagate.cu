@@ -168,11 +168,11 @@ __global__ void __launch_bounds__(kThreads) k_propagate(Tables tb, const uint32_
 
 // The same for the variants of one multi-variant sweep in one launch: blockIdx.y picks the variant's buffers.
 struct PropagateMultiArgs {
-    const uint32_t* out_nz[kMultiMax];
-    const uint32_t* in_nz[kMultiMax];
-    uint32_t* keep_bits[kMultiMax];
-    int32_t* keep_idx[kMultiMax];
-    int32_t* keep_count[kMultiMax];
+    const uint32_t* out_nz[kPortfolioMax];
+    const uint32_t* in_nz[kPortfolioMax];
+    uint32_t* keep_bits[kPortfolioMax];
+    int32_t* keep_idx[kPortfolioMax];
+    int32_t* keep_count[kPortfolioMax];
 };
 
 __global__ void __launch_bounds__(kThreads) k_propagate_multi(Tables tb, PropagateMultiArgs pa, uint32_t policy,

@@ -77,8 +77,9 @@ class Session:
     """A plan with its workspace and one set of output buffers for one variant at a time."""
 
     def __init__(self, dm: DeviceModel, scope: int, max_variants: int, want_mask_bits: bool = True,
-                 want_nz_map: bool = True, slots: int = 1):
-        """slots > 1 adds that many more sets of per-variant buffers for the multi-variant sweep."""
+                 want_nz_map: bool = True, slots: int = 1, portfolio_slots: int = 0):
+        """slots > 1 adds that many more sets of per-variant buffers for the multi-variant sweep;
+        portfolio_slots adds sets of flags and keep sets only (no sparse model) for the portfolio-wide calls."""
         self.dm, self.scope, self.max_variants, self.slots = dm, scope, max_variants, slots
         dev = dm.device
         nbytes = B.dnns_workspace_bytes(dm.c, scope, max_variants)
@@ -120,7 +121,9 @@ class Session:
                 "nz_map": i32(L.nz_map_words) if want_nz_map else None,
                 "out_nz": i32(L.out_nz_words), "in_nz": i32(L.in_nz_words),
                 "keep_bits": i32(L.keep_words), "keep_idx": i32(L.keep_idx_len), "keep_count": i32(G)})
-        self.stats_multi = torch.zeros(4 * max(slots, 1), dtype=torch.int64, device=dev)
+        self.stats_multi = torch.zeros(4 * max(slots, portfolio_slots, 1), dtype=torch.int64, device=dev)
+        self.pf = [{"out_nz": i32(L.out_nz_words), "in_nz": i32(L.in_nz_words), "keep_bits": i32(L.keep_words),
+                    "keep_idx": i32(L.keep_idx_len), "keep_count": i32(G)} for _ in range(portfolio_slots)]
 
     def _slot(self, name: str, slot: int):
         return getattr(self, name) if slot == 0 else self.extra[slot - 1][name]
@@ -199,6 +202,26 @@ class Session:
                               self.compact_arena.data_ptr(), self.compact_arena.numel(), self.dst_offsets.data_ptr(),
                               self.dst_shapes.data_ptr(), _stream())
 
+    # ---- the whole portfolio without a sparse model: flags of all variants from one sweep, keep sets in one launch,
+    # then a masking rebuild per variant (slot i holds variant first_variant + i)
+    def zero_structures_portfolio(self, first_variant: int, n_variants: int):
+        B.dnns_zero_structures_portfolio(self.plan, self.thr.data_ptr(), first_variant, n_variants,
+                                         [self.pf[i]["out_nz"].data_ptr() for i in range(n_variants)],
+                                         [self.pf[i]["in_nz"].data_ptr() for i in range(n_variants)], _stream())
+
+    def propagate_keep_portfolio(self, n_variants: int, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER,
+                                 min_keep: int = 1):
+        ptrs = lambda name: [self.pf[i][name].data_ptr() for i in range(n_variants)]
+        B.dnns_propagate_keep_multi(self.plan, n_variants, ptrs("out_nz"), ptrs("in_nz"), policy, min_keep,
+                                    ptrs("keep_bits"), ptrs("keep_idx"), ptrs("keep_count"), self.stats_multi.data_ptr(),
+                                    _stream())
+
+    def compact_portfolio(self, variant: int, slot: int):
+        """Rebuild `variant` from the dense model with the keep sets of portfolio slot `slot`."""
+        B.dnns_compact_masked(self.plan, self.thr.data_ptr(), variant, self.pf[slot]["keep_idx"].data_ptr(),
+                              self.pf[slot]["keep_count"].data_ptr(), self.compact_arena.data_ptr(),
+                              self.compact_arena.numel(), self.dst_offsets.data_ptr(), self.dst_shapes.data_ptr(), _stream())
+
     def propagate_keep_cascade(self, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1,
                                max_passes: int = 8):
         B.dnns_propagate_keep_cascade(self.plan, self.nz_map.data_ptr(), policy, min_keep, max_passes,
@@ -259,24 +282,26 @@ class Session:
     def mask_words(self, slot: int = 0):
         return self._split_words(self._slot("mask_bits", slot), self.mask_offset, [t.numel for t in self.dm.wl.tensors])
 
-    def structure_words(self, slot: int = 0):
+    def structure_words(self, slot: int = 0, portfolio: bool = False):
         wl = self.dm.wl
-        nz = None if self.nz_map is None else self._split_words(self._slot("nz_map", slot), self.nz_map_offset,
-                                                                 [t.O * t.I for t in wl.tensors])
-        return (nz, self._split_words(self._slot("out_nz", slot), self.out_nz_offset, [t.O for t in wl.tensors]),
-                self._split_words(self._slot("in_nz", slot), self.in_nz_offset, [t.I for t in wl.tensors]))
+        get = (lambda n: self.pf[slot][n]) if portfolio else (lambda n: self._slot(n, slot))
+        nz = None if self.nz_map is None or portfolio else self._split_words(get("nz_map"), self.nz_map_offset,
+                                                                              [t.O * t.I for t in wl.tensors])
+        return (nz, self._split_words(get("out_nz"), self.out_nz_offset, [t.O for t in wl.tensors]),
+                self._split_words(get("in_nz"), self.in_nz_offset, [t.I for t in wl.tensors]))
 
-    def keep_sets(self, slot: int = 0, multi_stats: bool = False):
+    def keep_sets(self, slot: int = 0, multi_stats: bool = False, portfolio: bool = False):
         """multi_stats: the statistics written by propagate_keep_multi for this slot."""
         wl = self.dm.wl
-        bits = self._split_words(self._slot("keep_bits", slot), self.keep_offset, [g.C for g in wl.groups])
-        cnt = self._slot("keep_count", slot).cpu().numpy()[: len(wl.groups)].copy()
-        idx_raw = self._slot("keep_idx", slot).cpu().numpy()
+        get = (lambda n: self.pf[slot][n]) if portfolio else (lambda n: self._slot(n, slot))
+        bits = self._split_words(get("keep_bits"), self.keep_offset, [g.C for g in wl.groups])
+        cnt = get("keep_count").cpu().numpy()[: len(wl.groups)].copy()
+        idx_raw = get("keep_idx").cpu().numpy()
         idx = [idx_raw[int(o): int(o) + int(c)].copy() for o, c in zip(self.keep_idx_offset, cnt)]
         st = self.stats_multi[4 * slot: 4 * slot + 4] if multi_stats else self.stats
         return bits, idx, cnt, st.cpu().numpy().view(np.uint64).copy()
 
-    def compacted(self, keep_slot: int = 0):
+    def compacted(self, keep_slot: int = 0, portfolio: bool = False):
         """(weights [(O', I', KH, KW)], bn [(g, b, m, v)], biases, shapes (T, 2), offsets) of the variant rebuilt
         last; keep_slot: the slot whose keep sets it was rebuilt from."""
         wl, eb = self.dm.wl, self.dm.elem_bytes
@@ -289,7 +314,7 @@ class Session:
             On, In = int(shapes[i, 0]), int(shapes[i, 1])
             n = On * In * t.KH * t.KW
             ws.append(raw[int(offs[i]): int(offs[i]) + n * eb].view(self._np_dtype()).reshape(On, In, t.KH, t.KW).copy())
-        cnt = self._slot("keep_count", keep_slot).cpu().numpy()
+        cnt = (self.pf[keep_slot]["keep_count"] if portfolio else self._slot("keep_count", keep_slot)).cpu().numpy()
         bns, k = [], T
         for b in wl.bns:
             Cn = int(cnt[wl.tensors[b.tensor].out_group])

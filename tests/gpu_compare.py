@@ -98,3 +98,55 @@ def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCE
                 [4 * len(b) for b in cb_c if b is not None]
         assert offs.tolist() == expected_offsets(sizes), f"arena offsets v{v}"
     return ses
+
+
+def compare_sparse_free(wl, dtype=B.DNNS_F32, policy=O.RULE_PRODUCER | O.RULE_CONSUMER, min_keep=1, weights=None):
+    """The portfolio without any sparse model: thresholds once, the zero structures of every variant from one sweep
+    over the dense weights (dnns_zero_structures_portfolio), keep sets of all variants in one launch, then a masking
+    rebuild per variant (dnns_compact_masked).  Flags, keep sets, statistics and every rebuilt item are compared
+    with the oracle's step-by-step result (mask, zero structures, keep propagation, compaction)."""
+    om = O.OracleModel(wl, dtype, weights)
+    dm = DeviceModel(wl, dtype, weights=weights)
+    V = len(wl.ks)
+    per_call = min(V, B.DNNS_PORTFOLIO_MAX)
+    ses = Session(dm, wl.scope, V, want_mask_bits=False, want_nz_map=False, portfolio_slots=per_call)
+    ses.magnitude_threshold(wl.ks)
+    rec_gpu, rec_cpu = ses.records(), O.threshold(om, wl.scope, wl.ks)
+    for f in ("tau_bits", "n_below", "n_tie", "n_equal"):
+        assert np.array_equal(rec_gpu[f], rec_cpu[f]), f
+    eb = 4 if dtype == B.DNNS_F32 else 2
+    for v0 in range(0, V, per_call):
+        n = min(per_call, V - v0)
+        ses.zero_structures_portfolio(v0, n)
+        ses.propagate_keep_portfolio(n, policy, min_keep)
+        for s in range(n):
+            v = v0 + s
+            ses.compact_portfolio(v, s)
+            assert ses.device_status() == B.DNNS_OK
+            masked_cpu, _ = O.apply_mask(om, wl.scope, rec_cpu[v])
+            _, out_c, in_c = O.zero_structures(masked_cpu)
+            _, out_g, in_g = ses.structure_words(s, portfolio=True)
+            assert_words(out_g, out_c, f"out flags v{v}")
+            assert_words(in_g, in_c, f"in flags v{v}")
+            kb_c, ki_c, kc_c, st_c = O.propagate_keep(masked_cpu, out_c, in_c, policy, min_keep)
+            kb_g, ki_g, kc_g, st_g = ses.keep_sets(s, multi_stats=True, portfolio=True)
+            assert np.array_equal(kc_g, kc_c), f"keep counts v{v}"
+            assert_words(kb_g, kb_c, f"keep bits v{v}")
+            for g, (a, b) in enumerate(zip(ki_g, ki_c)):
+                assert np.array_equal(a, b[: kc_c[g]]), f"keep idx v{v} group {g}"
+            assert st_g.tolist() == st_c.tolist(), f"stats v{v}"
+            cw_c, cbn_c, cb_c, sh_c = O.compact(masked_cpu, ki_c, kc_c)
+            cw_g, cbn_g, cb_g, sh_g, offs = ses.compacted(s, portfolio=True)
+            assert np.array_equal(sh_g, sh_c), f"shapes v{v}"
+            for i, (a, b) in enumerate(zip(cw_g, cw_c)):
+                assert bits_eq(a, b), f"compacted weights v{v} tensor {i}"
+            for i, (a, b) in enumerate(zip(cbn_g, cbn_c)):
+                for x, y in zip(a, b):
+                    assert bits_eq(x, y), f"compacted bn v{v} {i}"
+            for a, b in zip(cb_g, cb_c):
+                assert (a is None and b is None) or bits_eq(a, b)
+            sizes = [w.size * eb for w in cw_c] + [4 * len(x) for p in cbn_c for x in p] + \
+                    [4 * len(b) for b in cb_c if b is not None]
+            assert offs.tolist() == expected_offsets(sizes), f"arena offsets v{v}"
+            ses.last_masked, ses.last_slot = masked_cpu.weights, s   # the oracle's sparse model of the variant rebuilt last
+    return ses
