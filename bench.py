@@ -4,8 +4,12 @@ detection, keep propagation and compaction for every variant.
 
 One "step" is one whole portfolio on one model.  Prints ONE JSON line (rank 0).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet152] [--dtype f32|bf16]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet152] [--dtype f32|bf16] [--path sparse_free]
   python bench.py --impl reference ...     # the CPU oracle, as it stands, on the host cores
+
+The default path stores no sparse model: thresholds of all variants from one ranking, the zero structures of all
+variants from one sweep over the dense weights, keep sets of all variants in one launch, then one masking rebuild
+per variant.  --path multi / fused / stepwise time the paths that write the sparse model of every variant.
 """
 from __future__ import annotations
 
@@ -110,104 +114,94 @@ def oracle_portfolio(wl, dtype, variants):
     return time.perf_counter() - t0
 
 
+def dtype_label(dtype):
+    return "u32 keys / fp32 words" if dtype == 0 else "u16 keys / bf16 words"
+
+
+def config_of(wl, dtype):
+    return {"workload": f"{wl.name} ({'fp32' if dtype == 0 else 'bf16'}), {wl.n_prunable} prunable weights, "
+                        f"{len(wl.ks)} variants, {'global' if wl.scope == 0 else 'per-tensor'} ranking, seed {wl.seed}",
+            "variants": len(wl.ks), "prunable_weights": wl.n_prunable,
+            "l2": f"L2 flushed before every timed step ({FLUSH_BYTES >> 20} MiB scratch write, outside the timed region)"}
+
+
 def run_reference(args, wl, dtype):
+    """The whole workload (every variant) per step, as the cpu_baseline leg of the main arm times it."""
     V = len(wl.ks)
-    variants = sorted({0, V - 1})
+    variants = list(range(V))
     for _ in range(args.warmup):
         oracle_portfolio(wl, dtype, variants)
     times = [oracle_portfolio(wl, dtype, variants) for _ in range(args.steps)]
-    total = sum(times)
-    ms_per_variant = 1e3 * total / (args.steps * len(variants))
-    sample = f"variants {variants} of {V} (threshold sort shared by {len(variants)} instead of {V}), full weights"
+    ms = [1e3 * t / V for t in times]
+    sample = f"the whole workload per step: all {V} variants, full weights"
     line = {
-        "impl": "reference", "metric": METRIC, "value": ms_per_variant, "unit": "ms", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
-        "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-        "dtype": "u32 keys / fp32 words" if dtype == 0 else "u16 keys / bf16 words", "data": "synthetic",
-        "config": config_of(args, wl, dtype),
-        "cpu_baseline": {"value": ms_per_variant, "unit": "ms", "cores": 1, "kind": "oracle", "sample": sample},
-        "e2e": {"value": ms_per_variant, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "impl": "reference", "metric": METRIC, "value": statistics.median(ms), "unit": "ms", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * statistics.median(times),
+        "ms_per_variant_min": min(ms), "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": dtype_label(dtype), "data": "synthetic", "config": config_of(wl, dtype),
+        "cpu_baseline": {"value": statistics.median(ms), "unit": "ms", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": statistics.median(ms), "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
 
 
-def config_of(args, wl, dtype):
-    return {"workload": f"{wl.name} ({'fp32' if dtype == 0 else 'bf16'}), {wl.n_prunable} prunable weights, "
-                        f"{len(wl.ks)} variants, {'global' if wl.scope == 0 else 'per-tensor'} ranking, seed {wl.seed}",
-            "variants": len(wl.ks), "prunable_weights": wl.n_prunable,
-            "l2": "weights larger than L2 (no flush)" if wl.n_prunable * (4 if dtype == 0 else 2) > 126e6
-                  else "L2 flushed between steps (256 MiB scratch write)"}
+FLUSH_BYTES = 512 << 20
+KERNELS = ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_ties", "k_tie_scan", "k_tie_split", "k_extrema_sweep", "k_extrema_flags",
+           "k_sweep<", "k_sweep_multi", "k_flags", "k_propagate", "k_rebuild_layout", "k_compact_gather"]
 
 
-# --------------------------------------------------------------------------------------------
-# the CUDA arm
-# --------------------------------------------------------------------------------------------
+def item_sizes(wl, keep_count, eb):
+    """Bytes of every rebuilt item (weights, BatchNorm vectors, biases) for one array of keep counts, R and N'."""
+    R = Nn = 0
+    sizes = []
+    for t in wl.tensors:
+        On, Cn = int(keep_count[t.out_group]), int(keep_count[t.in_group])
+        R += On * t.I * t.KH * t.KW
+        Nn += On * Cn * t.in_spatial * t.KH * t.KW
+        sizes.append(On * Cn * t.in_spatial * t.KH * t.KW * eb)
+    for b in wl.bns:
+        sizes += [4 * int(keep_count[wl.tensors[b.tensor].out_group])] * 4
+    for t in wl.tensors:
+        if t.has_bias:
+            sizes.append(4 * int(keep_count[t.out_group]))
+    used = 0
+    for s in sizes:                      # items in order, each at the next multiple of 256 bytes
+        used = (used + 255) // 256 * 256 + s
+    return R, Nn, (used + 255) // 256 * 256
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="dnns", choices=["dnns", "reference"])
-    ap.add_argument("--workload", default="resnet152", choices=["toy", "vgg16", "resnet56", "resnet50", "resnet152"])
-    ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--stepwise", action="store_true", help="mask and zero-structure detection as two sweeps")
-    ap.add_argument("--multi", type=int, default=-1,
-                    help="variants per sweep over the dense weights (1..4; 0: one fused call per variant; default 4 for f32, 2 for bf16)")
-    ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph replay")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 0)
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+class Config:
+    """One (workload, dtype) on the GPU: buffers, the step of the chosen path, timing."""
 
-    from paper_2309_06973_b200 import workloads as W
-    dtype = 0 if args.dtype == "f32" else 1
+    def __init__(self, args, name, dtype, device, pinned_host=False, freeze=False):
+        import torch
+        from paper_2309_06973_b200 import workloads as W
+        from paper_2309_06973_b200.runtime import DeviceModel, Session
+        self.torch, self.args, self.dtype = torch, args, dtype
+        wl = W.BY_NAME[name]()
+        if freeze:
+            W.freeze_streams(wl)
+        self.wl, self.V, self.eb, self.N = wl, len(wl.ks), 4 if dtype == 0 else 2, wl.n_prunable
+        V = self.V
+        self.path = args.path
+        self.dm = DeviceModel(wl, dtype, device=device, pinned_host=pinned_host)
+        G = args.multi if args.multi >= 0 else (4 if dtype == 0 else 2)
+        self.G = min(G, 4, V) if self.path == "multi" else 0
+        self.groups = [(v0, min(self.G, V - v0)) for v0 in range(0, V, self.G)] if self.G else []
+        sparse_free = self.path == "sparse_free"
+        self.ses = Session(self.dm, wl.scope, V, want_mask_bits=not sparse_free, want_nz_map=False,
+                           slots=max(self.G, 1), portfolio_slots=V if sparse_free else 0)
+        self.flush_buf = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=self.dm.device)
+        self.call_names = {"sparse_free": ["threshold", "structures(portfolio)", "propagate", "compact"],
+                           "multi": ["threshold", "mask+structures", "propagate", "compact"],
+                           "fused": ["threshold", "mask+structures", "propagate", "compact"],
+                           "stepwise": ["threshold", "mask", "structures", "propagate", "compact"]}[self.path]
+        self.spans = {n: [] for n in self.call_names}
 
-    if args.impl == "reference":
-        if rank != 0:
-            return
-        wl = W.BY_NAME[args.workload]()
-        run_reference(args, wl, dtype)
-        return
+    def step(self, record=False):
+        torch, ses, wl, V = self.torch, self.ses, self.wl, self.V
 
-    import torch
-    import torch.distributed as dist
-    from paper_2309_06973_b200 import binding as B
-    from paper_2309_06973_b200.runtime import Deflater, DeviceModel, Session
-    from paper_2309_06973_b200.dist_util import max_over_ranks, ms_per_variant as whole_job_ms_per_variant
-
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
-    B.lib()  # fail loudly if the extension is missing
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-
-    wl = W.BY_NAME[args.workload]()
-    V = len(wl.ks)
-    eb = 4 if dtype == 0 else 2
-    N = wl.n_prunable
-    dm = DeviceModel(wl, dtype, device=f"cuda:{local_rank}", pinned_host=True)
-    G = args.multi if args.multi >= 0 else (4 if dtype == 0 else 2)
-    G = 0 if args.stepwise else min(G, 4, V)
-    groups = [(v0, min(G, V - v0)) for v0 in range(0, V, G)] if G else []
-    ses = Session(dm, wl.scope, V, want_mask_bits=True, want_nz_map=False, slots=max(G, 1))
-    need_flush = N * eb <= 126e6
-    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dm.device) if need_flush else None
-
-    names = (["threshold", "mask", "structures", "propagate", "compact"] if args.stepwise
-             else ["threshold", "mask+structures", "propagate", "compact"])
-    spans = {n: [] for n in names}
-    calls_per_step = {n: V for n in names}
-    calls_per_step["threshold"] = 1
-    if G:
-        calls_per_step["mask+structures"] = calls_per_step["propagate"] = len(groups)
-
-    def step(record: bool):
         def timed(name, fn, *a):
             if not record:
                 return fn(*a)
@@ -215,15 +209,23 @@ def main():
             e0.record()
             fn(*a)
             e1.record()
-            spans[name].append((e0, e1))
+            self.spans[name].append((e0, e1))
         timed("threshold", ses.magnitude_threshold, wl.ks)
-        for v0, n in groups:                       # n variants per read of the dense weights
+        if self.path == "sparse_free":
+            for v0 in range(0, V, 16):                        # the portfolio-wide calls take up to 16 variants
+                n = min(16, V - v0)
+                timed("structures(portfolio)", ses.zero_structures_portfolio, v0, n)
+                timed("propagate", ses.propagate_keep_portfolio, n)
+                for s in range(n):
+                    timed("compact", ses.compact_portfolio, v0 + s, s)
+            return
+        for v0, n in self.groups:                             # n variants per read of the dense weights
             timed("mask+structures", ses.mask_and_structures_multi, v0, n)
-            timed("propagate", ses.propagate_keep_multi, n)        # the keep sets of the n variants in one launch
+            timed("propagate", ses.propagate_keep_multi, n)
             for g in range(n):
                 timed("compact", lambda: ses.compact(slot=g, own_keep=True))
-        for v in (range(V) if not G else ()):
-            if args.stepwise:
+        for v in (range(V) if not self.G else ()):
+            if self.path == "stepwise":
                 timed("mask", ses.apply_mask, v)
                 timed("structures", ses.zero_structures)
             else:
@@ -231,36 +233,68 @@ def main():
             timed("propagate", ses.propagate_keep)
             timed("compact", ses.compact)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
+    def timed_steps(self, run, steps):
+        """`steps` runs, the L2 flushed before each, one event pair per run. Returns the list of ms."""
+        torch = self.torch
+        pairs = []
+        for _ in range(steps):
+            self.flush_buf.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            run()
+            b.record()
+            pairs.append((a, b))
         torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in pairs]
 
-    # ---- device-resident timing --------------------------------------------------------------
-    for _ in range(max(args.warmup, 3)):
-        step(False)
+    def variant_sizes(self):
+        """Per variant: R (weights in kept filter rows), N' (rebuilt weights), used arena bytes, keep counts, stats."""
+        ses, wl, V = self.ses, self.wl, self.V
+        out = []
+        if self.path == "sparse_free":
+            assert V <= 16
+            ses.magnitude_threshold(wl.ks)
+            ses.zero_structures_portfolio(0, V)
+            ses.propagate_keep_portfolio(V)
+            self.torch.cuda.synchronize()
+            st = ses.stats_multi.cpu().numpy().view(np.uint64)
+            for v in range(V):
+                kc = ses.pf[v]["keep_count"].cpu().numpy()
+                out.append((kc, st[4 * v: 4 * v + 4].copy()))
+        else:
+            ses.magnitude_threshold(wl.ks)
+            for v in range(V):
+                ses.variant(v, fused=self.path != "stepwise")
+                self.torch.cuda.synchronize()
+                out.append((ses.keep_count.cpu().numpy().copy(), ses.stats.cpu().numpy().view(np.uint64).copy()))
+        res = []
+        for kc, st in out:
+            R, Nn, used = item_sizes(wl, kc, self.eb)
+            res.append({"R": R, "Nn": Nn, "used": used, "keep_count": kc, "stats": st})
+        return res
+
+
+def measure(cfg, steps, warmup, barrier, max_over_ranks, ms_per_variant_of, peak, peak_kind, workload_key):
+    """Device-resident timing of one configuration: whole-portfolio steps (CUDA graph replay), per-call and
+    per-kernel durations (plain launches), bytes moved, roofline of the dominant kernel."""
+    import torch
+    from paper_2309_06973_b200 import binding as B
+    ses, wl, V, N, eb, args = cfg.ses, cfg.wl, cfg.V, cfg.N, cfg.eb, cfg.args
+    for _ in range(max(warmup, 3)):
+        cfg.step()
     torch.cuda.synchronize()
     assert ses.device_status() == B.DNNS_OK
-    # data-dependent sizes of every variant (outside the timed region): R = kept filter rows, N' = rebuilt size
-    R, Nn = [], []
-    for v in range(V):
-        ses.variant(v, fused=not args.stepwise)
-        torch.cuda.synchronize()
-        sh = ses.dst_shapes.cpu().numpy()[: 2 * len(wl.tensors)].reshape(-1, 2)
-        R.append(sum(int(sh[i, 0]) * t.I * t.KH * t.KW for i, t in enumerate(wl.tensors)))
-        Nn.append(sum(int(sh[i, 0]) * int(sh[i, 1]) * t.KH * t.KW for i, t in enumerate(wl.tensors)))
+    sizes = cfg.variant_sizes()
+    rec = ses.records()
+    ties_swept = bool((rec["n_tie"] < rec["n_equal"]).any())     # the tie sweep only reads the weights when some variant splits its ties
 
-    # One portfolio captured once as a CUDA graph (the calls are plain stream work: no allocation, no
-    # synchronisation), replayed for the timed steps.  A second, plain pass with an event pair around
-    # every call gives the per-call durations; its total is reported as ms_per_step_plain.
-    graph = None
-    launches_per_step = None
+    graph, launches_per_step = None, None
     if not args.no_graph:
         try:
             l0 = ses.launch_count()
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph):
-                step(False)
+                cfg.step()
             launches_per_step = ses.launch_count() - l0
             graph.replay()
             torch.cuda.synchronize()
@@ -268,97 +302,196 @@ def main():
             print(f"bench: CUDA graph capture failed ({e}); timing plain launches", file=sys.stderr)
             graph = None
 
-    def timed_steps(run_step):
-        """K steps; returns total ms.  Models that fit in L2 get a flush before every step."""
-        if need_flush:
-            pairs = []
-            for _ in range(args.steps):
-                flush_buf.fill_(1)
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record()
-                run_step()
-                b.record()
-                pairs.append((a, b))
-            torch.cuda.synchronize()
-            return sum(a.elapsed_time(b) for a, b in pairs)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(args.steps):
-            run_step()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b)
-
-    sampler = ClockSampler(local_rank)
     barrier()
-    sampler.start()
     launches0 = ses.launch_count()
-    plain_ms = timed_steps(lambda: step(True))
+    plain = cfg.timed_steps(lambda: cfg.step(True), steps)
     launches_plain = ses.launch_count() - launches0
-    # the same steps once more with an event pair around every single kernel (dnns_plan_profile)
-    kernel_names = ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_ties", "k_tie_scan", "k_sweep<", "k_sweep_multi", "k_flags",
-                    "k_propagate", "k_compact_layout", "k_compact_gather"]
-    ses.profile(True)
-    timed_steps(lambda: step(False))
+    ses.profile(True)                                 # the same steps with an event pair around every single kernel
+    cfg.timed_steps(cfg.step, steps)
     ses.profile(False)
     kernel_ms = {}
-    for kn in kernel_names:
+    for kn in KERNELS:
         ms, n = ses.kernel_time(kn)
         if n:
-            kernel_ms[kn] = {"avg_ms": ms / n, "launches_per_step": n / args.steps, "ms_per_step": ms / args.steps}
+            kernel_ms[kn] = {"avg_ms": ms / n, "launches_per_step": n / steps, "ms_per_step": ms / steps}
     if graph is not None:
         barrier()
-        total_ms = timed_steps(graph.replay)
-        launches = launches_per_step * args.steps
+        timed = cfg.timed_steps(graph.replay, steps)
+        launches = launches_per_step * steps
     else:
-        total_ms = plain_ms
-        launches = launches_plain
-    clocks = sampler.stop()
+        timed, launches = plain, launches_plain
     barrier()
-    total_ms, plain_ms = max_over_ranks([total_ms, plain_ms], dm.device)
+    med, mn, mean, plain_med = max_over_ranks([statistics.median(timed), min(timed), statistics.mean(timed),
+                                               statistics.median(plain)])
     assert ses.device_status() == B.DNNS_OK
 
-    ms_per_step = total_ms / args.steps
-    ms_per_variant = whole_job_ms_per_variant(ms_per_step, V, world)
-    per_call = {n: statistics.mean(a.elapsed_time(b) for a, b in spans[n]) for n in names}
-    plain_per_step = plain_ms / args.steps
-    share = {n: per_call[n] * calls_per_step[n] / plain_per_step for n in names}
+    # ---- bytes: what the kernels of this path really read and write, and the step-by-step accounting
+    thr_sweeps = (2 if cfg.dtype == 0 else 1) + (1 if ties_swept else 0)
+    rebuild = [(s["R"] + s["Nn"]) * eb for s in sizes]
+    if cfg.path == "sparse_free":
+        moved = (thr_sweeps + 1) * N * eb + sum(rebuild)
+        sweeps = (f"no sparse model: {thr_sweeps} ranking sweeps and one sweep for the zero structures of all {V} variants, "
+                  "then one masking rebuild per variant")
+    elif cfg.path == "multi":
+        moved = thr_sweeps * N * eb + sum(N * eb + n * (N * eb + N / 4) for _, n in cfg.groups) + sum(rebuild)
+        sweeps = f"fused mask+structures, {cfg.G} variants per read of the dense weights; {thr_sweeps} ranking sweeps"
+    elif cfg.path == "fused":
+        moved = thr_sweeps * N * eb + V * (2 * N * eb + N / 4) + sum(rebuild)
+        sweeps = f"fused mask+structures, one variant per sweep; {thr_sweeps} ranking sweeps"
+    else:
+        moved = thr_sweeps * N * eb + V * (3 * N * eb + N / 4) + sum(rebuild)
+        sweeps = f"stepwise: mask sweep and structure sweep per variant; {thr_sweeps} ranking sweeps"
+    stepwise_bytes = N * eb * (1 + 3 * V) + V * N / 8 + sum(rebuild)   # one read per input, one write per output of every step
 
-    # algorithmic bytes: one read of every input a step consumes, one write of every output
-    # (the fused sweep moves 2*N*b + N/8 per launch; the stepwise accounting B_v charges the path 3*N*b + N/8)
-    alg = {"threshold": N * eb, "mask": 2 * N * eb + N / 8, "structures": N * eb, "mask+structures": 2 * N * eb + N / 8,
-           "propagate": 0, "compact": statistics.mean((r + n) * eb for r, n in zip(R, Nn))}
-    portfolio_bytes = alg["threshold"] + V * (alg["mask"] + alg["structures"]) + sum((r + n) * eb for r, n in zip(R, Nn))
-    moved_bytes = alg["threshold"] + V * (alg["mask"] + (alg["structures"] if args.stepwise else 0)) + \
-        sum((r + n) * eb for r, n in zip(R, Nn))
-    if G:   # one read of the dense weights per group, one write (+ mask bits) per variant
-        multi_bytes = sum(N * eb + n * (N * eb + N / 8) for _, n in groups)
-        alg["mask+structures"] = multi_bytes / len(groups)
-        moved_bytes = alg["threshold"] + multi_bytes + sum((r + n) * eb for r, n in zip(R, Nn))
-    peak, peak_kind = load_peaks()
-    # the dominant kernel: largest share of the summed kernel time; its algorithmic bytes per launch
-    kernel_alg = {"k_hist1": N * eb, "k_hist2": N * eb, "k_ties": N * eb,
-                  "k_sweep<": 2 * N * eb + N / 4,          # weights in and out, mask bits, the element bits it packs
-                  "k_compact_gather": alg["compact"]}
-    if args.stepwise:
-        kernel_alg["k_sweep<"] = (alg["mask"] + alg["structures"] + N / 8) / 2   # two sweeps per variant, averaged
-    if G:   # per launch: one read, n writes with their mask and element bits
-        kernel_alg["k_sweep_multi"] = sum(N * eb + n * (N * eb + N / 4) for _, n in groups) / len(groups)
-    kernel_total = sum(k["ms_per_step"] for k in kernel_ms.values())
-    for k in kernel_ms.values():
-        k["share"] = k["ms_per_step"] / kernel_total
-    dominant = max((kn for kn in kernel_ms if kn in kernel_alg), key=lambda kn: kernel_ms[kn]["ms_per_step"])
-    achieved = kernel_alg[dominant] / (kernel_ms[dominant]["avg_ms"] * 1e-3) / 1e9
+    kernel_alg = {"k_hist1": N * eb, "k_hist2": N * eb, "k_ties": N * eb if ties_swept else 0, "k_extrema_sweep": N * eb,
+                  "k_compact_gather": statistics.mean(rebuild),
+                  "k_sweep<": (3 * N * eb + N / 4) / 2 if cfg.path == "stepwise" else 2 * N * eb + N / 4}
+    if cfg.groups:
+        kernel_alg["k_sweep_multi"] = sum(N * eb + n * (N * eb + N / 4) for _, n in cfg.groups) / len(cfg.groups)
+    total_k = sum(k["ms_per_step"] for k in kernel_ms.values())
     for kn, k in kernel_ms.items():
-        if kn in kernel_alg:
+        k["share"] = k["ms_per_step"] / total_k
+        if kernel_alg.get(kn):
             k["gbs"] = kernel_alg[kn] / (k["avg_ms"] * 1e-3) / 1e9
-    kernel_label = {"k_sweep<": "k_sweep<mask>+<structures>" if args.stepwise else "k_sweep<mask+structures>",
-                    "k_sweep_multi": f"k_sweep_multi<{G}>"}
+            k["frac_of_peak"] = k["gbs"] / peak
+    dominant = max((kn for kn in kernel_ms if kernel_alg.get(kn)), key=lambda kn: kernel_ms[kn]["ms_per_step"])
+    label = {"k_sweep<": "k_sweep", "k_sweep_multi": f"k_sweep_multi<{cfg.G}>"}.get(dominant, dominant)
+    traffic = measured_traffic(workload_key, "f32" if cfg.dtype == 0 else "bf16", label)
+    roof = {"bound": "hbm", "kernel": label, "achieved": kernel_ms[dominant]["gbs"], "peak": peak,
+            "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": kernel_ms[dominant]["gbs"] / peak,
+            "algorithmic_bytes": kernel_alg[dominant], "avg_launch_ms": kernel_ms[dominant]["avg_ms"],
+            "timed_by": f"CUDA event pair around every launch of the kernel on its stream, {steps} steps of plain launches, "
+                        "L2 flushed before every step",
+            "traffic": traffic,
+            "frac_measured": (traffic / (kernel_ms[dominant]["avg_ms"] * 1e-3) / 1e9 / peak) if traffic else None}
+    per_call = {n: statistics.mean(a.elapsed_time(b) for a, b in cfg.spans[n]) for n in cfg.call_names if cfg.spans[n]}
+    variants = []
+    total_params = wl.n_params
+    for v, s in enumerate(sizes):
+        kept_params = s["Nn"] + sum(2 * int(s["keep_count"][wl.tensors[b.tensor].out_group]) for b in wl.bns) + \
+            sum(int(s["keep_count"][t.out_group]) for t in wl.tensors if t.has_bias)
+        variants.append({"k": [int(x) for x in wl.ks[v]], "tau_bits": [int(x) for x in rec["tau_bits"][v]],
+                         "n_tie": [int(x) for x in rec["n_tie"][v]], "rebuilt_weights": s["Nn"], "kept_filter_row_weights": s["R"],
+                         "channels_removed": int(s["stats"][1]), "dropped_nonzero_shift": int(s["stats"][0]),
+                         "spatial_compression": total_params / max(kept_params, 1)})
+    return {
+        "ms_per_variant": ms_per_variant_of(med, V), "ms_per_variant_min": ms_per_variant_of(mn, V),
+        "ms_per_step": med, "ms_per_step_min": mn, "ms_per_step_mean": mean, "ms_per_step_plain": plain_med,
+        "steps": steps, "launch": "cuda graph replay" if graph is not None else "plain stream launches",
+        "gpu_launches": launches, "sweeps": sweeps,
+        "moved_bytes_per_step": moved, "moved_gbs": moved / (med * 1e-3) / 1e9, "moved_frac_of_peak": moved / (med * 1e-3) / 1e9 / peak,
+        "stepwise_equivalent_gbs": stepwise_bytes / (med * 1e-3) / 1e9,
+        "stepwise_equivalent_frac_of_peak": stepwise_bytes / (med * 1e-3) / 1e9 / peak,
+        "stepwise_equivalent_note": "bytes a step-by-step run would move (one read per input and one write per output of "
+                                    "every step) over the time of this path: not achieved bandwidth, can exceed the roofline",
+        "per_call_ms": per_call, "kernel_ms": kernel_ms, "roofline": roof, "variants": variants, "_sizes": sizes,
+    }
 
-    # ---- Module 1 on a rebuilt variant (not part of the portfolio step): conv + BatchNorm fusion in place
+
+def end_to_end(cfg, steps, barrier, max_over_ranks, ms_per_variant_of):
+    """The same portfolio through host buffers: every step copies the dense weights host -> device and every rebuilt
+    variant (arena, offsets, shapes, keep counts) device -> host.  With the default path the rebuild of variant v+1
+    runs while variant v travels back: two destination arenas, a copy stream, one host synchronisation per
+    portfolio (for the keep counts, from which the host knows how many bytes every variant has)."""
+    import torch
+    ses, wl, V, dm = cfg.ses, cfg.wl, cfg.V, cfg.dm
+    n_arena = ses.compact_arena.numel()
+    host_out = [torch.empty(n_arena, dtype=torch.uint8).pin_memory() for _ in range(2)]
+    host_small = [torch.empty(ses.dst_offsets.numel() * 8 + ses.dst_shapes.numel() * 4, dtype=torch.uint8).pin_memory()
+                  for _ in range(V)]
+    arenas = [ses.compact_arena, torch.empty_like(ses.compact_arena)]
+    copy_stream = torch.cuda.Stream(device=dm.device)
+    counters = {"h2d": 0, "d2h": 0}
+
+    def step_overlapped():
+        dm.upload_weights()
+        counters["h2d"] += dm.weight_bytes
+        ses.magnitude_threshold(wl.ks)
+        ses.zero_structures_portfolio(0, V)
+        ses.propagate_keep_portfolio(V)
+        kcs = [ses.pf[v]["keep_count"].cpu().numpy() for v in range(V)]      # synchronises once: sizes are data
+        counters["d2h"] += sum(k.nbytes for k in kcs)
+        main = torch.cuda.current_stream()
+        free = [None, None]
+        for v in range(V):
+            b = v & 1
+            used = min(item_sizes(wl, kcs[v], cfg.eb)[2], n_arena)
+            if free[b] is not None:
+                main.wait_event(free[b])                  # the arena's previous variant has left the device
+            ses.compact_portfolio(v, v, arenas[b])
+            no, ns = ses.dst_offsets.numel() * 8, ses.dst_shapes.numel() * 4
+            host_small[v][:no].copy_(ses.dst_offsets.view(torch.uint8), non_blocking=True)
+            host_small[v][no:no + ns].copy_(ses.dst_shapes.view(torch.uint8), non_blocking=True)
+            done = torch.cuda.Event()
+            done.record(main)
+            with torch.cuda.stream(copy_stream):
+                copy_stream.wait_event(done)
+                host_out[b][:used].copy_(arenas[b][:used], non_blocking=True)
+                free[b] = torch.cuda.Event()
+                free[b].record(copy_stream)
+            counters["d2h"] += used + no + ns
+        copy_stream.synchronize()
+        torch.cuda.synchronize()
+
+    def step_sequential():
+        dm.upload_weights()
+        counters["h2d"] += dm.weight_bytes
+        ses.magnitude_threshold(wl.ks)
+        for v in range(V):
+            if cfg.G:
+                if v % cfg.G == 0:
+                    ses.mask_and_structures_multi(v, min(cfg.G, V - v))
+                    ses.propagate_keep_multi(min(cfg.G, V - v))
+                ses.compact(slot=v % cfg.G, own_keep=True)
+                cnt = ses._slot("keep_count", v % cfg.G).cpu()
+            else:
+                ses.variant(v, fused=cfg.path != "stepwise")
+                cnt = ses.keep_count.cpu()
+            offs, shp = ses.dst_offsets.cpu(), ses.dst_shapes.cpu()
+            used = min(item_sizes(wl, cnt.numpy(), cfg.eb)[2], n_arena)
+            host_out[0][:used].copy_(ses.compact_arena[:used], non_blocking=True)
+            counters["d2h"] += used + offs.numel() * 8 + shp.numel() * 4 + cnt.numel() * 4
+        torch.cuda.synchronize()
+
+    run = step_overlapped if cfg.path == "sparse_free" and V <= 16 else step_sequential
+    for _ in range(2):
+        run()
+    counters["h2d"] = counters["d2h"] = 0
+    times = []
+    for _ in range(steps):
+        barrier()
+        t0 = time.perf_counter()
+        run()
+        times.append((time.perf_counter() - t0) * 1e3)
+    barrier()
+    med, mn = max_over_ranks([statistics.median(times), min(times)])
+    return {"value": ms_per_variant_of(med, V), "min": ms_per_variant_of(mn, V), "unit": "ms",
+            "h2d_bytes_per_step": counters["h2d"] // steps, "d2h_bytes_per_step": counters["d2h"] // steps,
+            "how": "host wall clock around a whole portfolio through the C ABI with pinned host buffers: weights up, "
+                   "every rebuilt variant down" + (" (rebuild of the next variant overlaps the copy of the last)" if run is step_overlapped else "")}
+
+
+def extras(cfg, sizes):
+    """Rows beyond the five steps, on the rebuilt variants (not part of the timed portfolio step): conv+BN fusion,
+    fixed-point keep propagation, deflation / inflation."""
+    import torch
+    from paper_2309_06973_b200 import binding as B
+    from paper_2309_06973_b200.runtime import Deflater, Session
+    ses, wl, V, eb, dm = cfg.ses, cfg.wl, cfg.V, cfg.eb, cfg.dm
+
+    def rebuild(v):
+        if cfg.path == "sparse_free":
+            ses.compact_portfolio(v, v)
+        else:
+            ses.variant(v, fused=cfg.path != "stepwise")
+    if cfg.path == "sparse_free":
+        ses.magnitude_threshold(wl.ks)
+        ses.zero_structures_portfolio(0, V)
+        ses.propagate_keep_portfolio(V)
+
     fold_ms = []
     for _ in range(5):
-        ses.compact()                      # a fresh rebuilt variant (the last one of the portfolio)
+        rebuild(V - 1)                      # a fresh rebuilt variant (the last one of the portfolio)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         ses.fold_batchnorm()
@@ -366,12 +499,12 @@ def main():
         torch.cuda.synchronize()
         fold_ms.append(a.elapsed_time(b))
     fold_ms = statistics.median(fold_ms)
+    fold = {"ms": fold_ms, "gbs": 2 * sizes[-1]["Nn"] * eb / (fold_ms * 1e-3) / 1e9,
+            "what": "conv + BatchNorm fusion of the last variant in place (read + write of its weights)"}
 
-    # ---- fixed-point keep propagation on the last variant (not part of the portfolio step)
     def params_of(session):
         sh = session.dst_shapes.cpu().numpy()[: 2 * len(wl.tensors)].reshape(-1, 2)
         return sum(int(sh[i, 0]) * int(sh[i, 1]) * t.KH * t.KW for i, t in enumerate(wl.tensors))
-
     ses2 = Session(dm, wl.scope, V, want_mask_bits=False, want_nz_map=True)
     ses2.magnitude_threshold(wl.ks)
     ses2.mask_and_structures(V - 1)
@@ -395,19 +528,14 @@ def main():
                "what": "last variant: rule of Algorithm 1 applied to a fixed point on the kernel maps"}
     ses2.close()
 
-    # ---- Module 7 / 8 on the rebuilt variants (not part of the portfolio step): every variant deflated into
-    # one package, smallest first; timings for the last variant (deflate) and its inflation
     deflater = Deflater(ses.compact_arena.numel(), dm.device)
     raw_sizes, packed_sizes, codec_ms = [], [], {"deflate": [], "inflate": []}
     restored = torch.empty_like(ses.compact_arena)
     for v in range(V):
-        ses.variant(v, fused=not args.stepwise)
+        rebuild(v)
         torch.cuda.synchronize()
-        offs = ses.dst_offsets.cpu().numpy().view(np.uint64)
-        cnt = ses.keep_count.cpu().numpy()
-        used = min((int(offs[-1]) + 4 * max(int(cnt.max()), 1) + 255) // 256 * 256, ses.compact_arena.numel())
-        reps = 5 if v == V - 1 else 1
-        for _ in range(reps):
+        used = min(sizes[v]["used"], ses.compact_arena.numel())
+        for _ in range(5 if v == V - 1 else 1):
             ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
             ev[0].record()
             deflater.deflate(ses.compact_arena, used)
@@ -425,88 +553,128 @@ def main():
         packed_sizes.append(size + 8 * (B.dnns_deflate_chunks(used) + 1) + 4 * 32 * B.dnns_deflate_chunks(used))
     order = sorted(range(V), key=lambda v: raw_sizes[v])           # Module 7 sorts the portfolio by model size
     dms, ims = statistics.median(codec_ms["deflate"]), statistics.median(codec_ms["inflate"])
-    deflate_info = {"package_order": order, "raw_bytes": [raw_sizes[v] for v in order],
-                    "packed_bytes_with_index": [packed_sizes[v] for v in order],
-                    "package_ratio": sum(packed_sizes) / sum(raw_sizes),
-                    "last_variant": {"deflate_ms": dms, "inflate_ms": ims,
-                                     "deflate_gbs": (raw_sizes[-1] + packed_sizes[-1]) / (dms * 1e-3) / 1e9,
-                                     "inflate_gbs": (raw_sizes[-1] + packed_sizes[-1]) / (ims * 1e-3) / 1e9},
-                    "what": "RFC 1951 streams (fixed Huffman / stored blocks, runs as distance-1 matches) plus chunk and "
-                            "sub-block index; paper context: 43 ms to switch a VGG-16 variant in (Table V)"}
-    del restored
+    deflate = {"package_order": order, "raw_bytes": [raw_sizes[v] for v in order],
+               "packed_bytes_with_index": [packed_sizes[v] for v in order],
+               "package_ratio": sum(packed_sizes) / sum(raw_sizes),
+               "last_variant": {"deflate_ms": dms, "inflate_ms": ims,
+                                "deflate_gbs": (raw_sizes[-1] + packed_sizes[-1]) / (dms * 1e-3) / 1e9,
+                                "inflate_gbs": (raw_sizes[-1] + packed_sizes[-1]) / (ims * 1e-3) / 1e9},
+               "what": "RFC 1951 streams (fixed Huffman / stored blocks, runs as distance-1 matches) plus chunk and "
+                       "sub-block index; paper context: 43 ms to switch a VGG-16 variant in (Table V)"}
+    return fold, cascade, deflate
 
-    # ---- end to end through the C ABI with host buffers -----------------------------------------
-    small = torch.empty(1 << 16, dtype=torch.uint8).pin_memory()
-    host_out = torch.empty(ses.compact_arena.numel(), dtype=torch.uint8).pin_memory()
-    h2d = d2h = 0
 
-    def e2e_step():
-        nonlocal h2d, d2h
-        dm.upload_weights()
-        h2d += dm.weight_bytes
-        ses.magnitude_threshold(wl.ks)
-        for v in range(V):
-            if G:
-                if v % G == 0:
-                    ses.mask_and_structures_multi(v, min(G, V - v))
-                    ses.propagate_keep_multi(min(G, V - v))
-                ses.compact(slot=v % G, own_keep=True)
-            else:
-                ses.variant(v, fused=not args.stepwise)
-            offs = ses.dst_offsets.cpu()           # synchronises: the sizes are only known on the device
-            shp = ses.dst_shapes.cpu()
-            cnt = ses._slot("keep_count", v % G if G else 0).cpu()
-            last_w = len(wl.tensors) - 1
-            used = int(offs[-1].item()) + 4 * max(int(cnt.max().item()), 1)
-            used = min((used + 255) // 256 * 256, host_out.numel())
-            host_out[:used].copy_(ses.compact_arena[:used], non_blocking=True)
-            d2h += used + offs.numel() * 8 + shp.numel() * 4 + cnt.numel() * 4
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="dnns", choices=["dnns", "reference"])
+    ap.add_argument("--workload", default="resnet152", choices=["toy", "vgg16", "resnet56", "resnet50", "resnet152"])
+    ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
+    ap.add_argument("--path", default="sparse_free", choices=["sparse_free", "multi", "fused", "stepwise"],
+                    help="sparse_free: no sparse model is stored (default); multi: several variants per sweep, sparse models "
+                         "written; fused: one fused sweep per variant; stepwise: the five calls one by one")
+    ap.add_argument("--stepwise", action="store_true", help="same as --path stepwise")
+    ap.add_argument("--multi", type=int, default=-1, help="--path multi: variants per sweep (1..4; default 4 for f32, 2 for bf16)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph replay")
+    ap.add_argument("--no-also", action="store_true", help="skip the other target configurations (resnet152 bf16, resnet50 f32)")
+    ap.add_argument("--no-extras", action="store_true", help="skip fold / cascade / deflate / frozen-streams figures")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    if args.stepwise:
+        args.path = "stepwise"
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2309_06973_b200 import workloads as W
+    dtype = 0 if args.dtype == "f32" else 1
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        run_reference(args, W.BY_NAME[args.workload](), dtype)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2309_06973_b200 import binding as B
+    from paper_2309_06973_b200.dist_util import max_over_ranks as _max_over_ranks, ms_per_variant as whole_job_ms_per_variant
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    B.lib()  # fail loudly if the extension is missing
+    torch.cuda.set_device(local_rank)
+    device = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(2):
-        e2e_step()
-    h2d = d2h = 0
+    max_over_ranks = lambda xs: _max_over_ranks(xs, torch.device(device))
+    ms_per_variant_of = lambda ms_per_step, V: whole_job_ms_per_variant(ms_per_step, V, world)
+    peak, peak_kind = load_peaks()
+
+    cfg = Config(args, args.workload, dtype, device, pinned_host=True)
+    wl, V = cfg.wl, cfg.V
+    sampler = ClockSampler(local_rank)
     barrier()
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        e2e_step()
-    barrier()
-    e2e_ms = (time.perf_counter() - t0) * 1e3
-    e2e_ms = max_over_ranks([e2e_ms], dm.device)[0]
-    e2e_per_variant = whole_job_ms_per_variant(e2e_ms / args.steps, V, world)
+    sampler.start()
+    m = measure(cfg, args.steps, args.warmup, barrier, max_over_ranks, ms_per_variant_of, peak, peak_kind, args.workload)
+    clocks = sampler.stop()
+    sizes = m.pop("_sizes")
+    e2e = end_to_end(cfg, max(3, min(args.steps, 10)), barrier, max_over_ranks, ms_per_variant_of)
 
     line = {
-        "metric": METRIC, "value": ms_per_variant, "unit": "ms", "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
-        "vs_baseline": None, "dtype": "u32 keys / fp32 words" if dtype == 0 else "u16 keys / bf16 words",
-        "data": "synthetic", "config": config_of(args, wl, dtype),
-        "effective_gbs": portfolio_bytes / (ms_per_step * 1e-3) / 1e9,
-        "effective_frac_of_peak": portfolio_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
-        "algorithmic_bytes_per_variant": portfolio_bytes / V,
-        "moved_gbs": moved_bytes / (ms_per_step * 1e-3) / 1e9,
-        "sweeps": "stepwise" if args.stepwise else (f"fused mask+structures, {G} variants per read of the dense weights" if G
-                                                    else "fused mask+structures"),
-        "launch": "cuda graph replay" if graph is not None else "plain stream launches", "ms_per_step_plain": plain_per_step,
-        "per_call_ms": per_call, "share": share,
-        "per_call_gbs": {n: (alg[n] / (per_call[n] * 1e-3) / 1e9 if alg[n] else None) for n in names},
-        "kernel_ms": kernel_ms,
-        "roofline": {"bound": "hbm", "kernel": kernel_label.get(dominant, dominant), "achieved": achieved, "peak": peak,
-                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                     "algorithmic_bytes": kernel_alg[dominant],
-                     "avg_launch_ms": kernel_ms[dominant]["avg_ms"],
-                     "timed_by": "CUDA event pair around every launch of the kernel on its stream, "
-                                 f"{args.steps} steps of plain launches",
-                     "traffic": measured_traffic(args.workload, args.dtype, kernel_label.get(dominant, dominant))},
-        "e2e": {"value": e2e_per_variant, "unit": "ms", "h2d_bytes_per_step": h2d // args.steps,
-                "d2h_bytes_per_step": d2h // args.steps},
-        "gpu_launches": launches,
-        "cascade": cascade,
-        "fold_batchnorm": {"ms": fold_ms, "gbs": 2 * Nn[-1] * eb / (fold_ms * 1e-3) / 1e9,
-                           "what": "conv + BatchNorm fusion of the last variant in place (read + write of its weights)"},
-        "deflate": deflate_info,
-        "clocks": clocks,
-        "context": {"paper_pruning_time_ms": 120, "paper_hardware": "not stated for that figure"},
+        "metric": METRIC, "value": m["ms_per_variant"], "unit": "ms", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": m["ms_per_step"], "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": dtype_label(dtype), "data": "synthetic", "config": config_of(wl, dtype),
+        "value_is": "median over the timed steps (one CUDA event pair per step, L2 flushed before each); ms_per_variant_min beside it",
     }
+    line.update({k: v for k, v in m.items() if k not in ("ms_per_variant", "ms_per_step", "steps")})
+    line["e2e"] = e2e
+    line["clocks"] = clocks
+    line["context"] = {"paper_pruning_time_ms": 120, "paper_hardware": "not stated for that figure"}
+
+    if not args.no_extras:
+        fold, cascade, deflate = extras(cfg, sizes)
+        line["fold_batchnorm"], line["cascade"], line["deflate"] = fold, cascade, deflate
+    del cfg
+    torch.cuda.empty_cache()
+
+    if not args.no_extras and any(sum(1 for t in wl.tensors if t.out_group == g) > 1 for g in range(len(wl.groups))):
+        # the paper's own setting: residual streams (skip connections, downsampling layers) are left alone
+        fz = Config(args, args.workload, dtype, device, freeze=True)
+        mf = measure(fz, max(5, args.steps // 2), 3, barrier, max_over_ranks, ms_per_variant_of, peak, peak_kind, args.workload)
+        line["frozen_streams_vs_coupled"] = {
+            "what": "groups written by several layers (residual streams) frozen, as the paper leaves skip and downsampling "
+                    "layers unpruned (Section IV-B-2), against the coupled keep sets of the headline run",
+            "coupled": {"ms_per_variant": m["ms_per_variant"], "rebuilt_weights": [v["rebuilt_weights"] for v in m["variants"]]},
+            "frozen": {"ms_per_variant": mf["ms_per_variant"], "rebuilt_weights": [v["rebuilt_weights"] for v in mf["variants"]]}}
+        del fz
+        torch.cuda.empty_cache()
+
+    if not args.no_also and args.workload == "resnet152" and args.dtype == "f32":
+        # the other configurations the target names, in the same record (device-resident timing only)
+        also = {}
+        for name, dt in (("resnet152", 1), ("resnet50", 0)):
+            c2 = Config(args, name, dt, device)
+            m2 = measure(c2, args.steps, 3, barrier, max_over_ranks, ms_per_variant_of, peak, peak_kind, name)
+            m2.pop("_sizes")
+            also[f"{name}_{'f32' if dt == 0 else 'bf16'}"] = {
+                "config": config_of(c2.wl, dt), "dtype": dtype_label(dt),
+                **{k: m2[k] for k in ("ms_per_variant", "ms_per_variant_min", "ms_per_step", "moved_gbs", "moved_frac_of_peak",
+                                      "stepwise_equivalent_frac_of_peak", "sweeps", "launch", "kernel_ms", "roofline")},
+                "spatial_compression": [v["spatial_compression"] for v in m2["variants"]]}
+            del c2
+            torch.cuda.empty_cache()
+        line["also"] = also
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         t = oracle_portfolio(wl, dtype, list(range(V)))

@@ -815,17 +815,31 @@ __global__ void __launch_bounds__(kGatherThreads, 3) k_compact_gather(Tables tb,
             dst_shapes[2 * it.tensor + 1] = (int32_t)(z.Cn * (uint32_t)it.S);
         }
     }
-    // vector items (BatchNorm vectors, biases): one warp each, v'[a] = v[keep[a]]
+    // vector items (BatchNorm vectors, biases): v'[a] = v[keep[a]], a warp per piece of kVecPiece rows; all index
+    // loads of a piece are issued before the first value is fetched
     {
         const uint32_t n_warps = gridDim.x * (kConsumers / 32), gwarp = blockIdx.x + gridDim.x * warp;  // neighbours in different blocks
         for (uint32_t r = gwarp; r < tb.n_vec_items; r += n_warps) {
-            const uint32_t i = tb.vec_items[r];
+            const uint32_t i = tb.vec_items[2 * r], a0 = tb.vec_items[2 * r + 1] * kVecPiece;
             const ItemDesc& it = tb.items[i];
             const RebuildItem z = ritems[i];
+            if (a0 >= z.On) continue;
             const uint32_t* src = static_cast<const uint32_t*>(it.src);
             uint32_t* dst = reinterpret_cast<uint32_t*>(dst_arena + ((uint64_t)z.off256 << 8));
             const int32_t* ko = keep_idx + it.ko_off;
-            for (uint32_t a = lane; a < z.On; a += 32) dst[a] = __ldg(src + DNNS_IDX(__ldg(ko + a), it.O));
+            constexpr int kPer = kVecPiece / 32;
+            int32_t row[kPer];
+            uint32_t val[kPer];
+#pragma unroll
+            for (int k = 0; k < kPer; ++k) {
+                const uint32_t a = a0 + k * 32 + lane;
+                row[k] = a < z.On ? __ldg(ko + a) : -1;
+            }
+#pragma unroll
+            for (int k = 0; k < kPer; ++k) val[k] = row[k] >= 0 ? __ldg(src + DNNS_IDX(row[k], it.O)) : 0u;
+#pragma unroll
+            for (int k = 0; k < kPer; ++k)
+                if (row[k] >= 0) dst[a0 + k * 32 + lane] = val[k];
         }
     }
     // the element path (rows that are not multiples of 16 bytes): 16 KB destination units, a block per pair

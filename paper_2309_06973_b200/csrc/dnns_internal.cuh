@@ -128,6 +128,7 @@ struct RebuildSlot {
     uint32_t* range_item;      // [rebuild_ranges(n_blocks)] the item in which each range of the cost axis starts
     uint32_t* unit_item;       // [max_units] the item of every unit of the element path
 };
+constexpr uint32_t kVecPiece = 256;  // rows of a vector item that one warp of the gather copies
 constexpr int kLayoutBatch = 8;  // layouts one launch of the layout kernel prepares
 struct LayoutBatch {
     const int32_t* keep_count[kLayoutBatch];
@@ -159,7 +160,7 @@ struct Tables {
     const uint32_t* flag_unit_tensor;  // [n_flag_units] the tensor a unit belongs to
     uint32_t* ebits;        // packed "element is non-zero" bits of the latest sweep (same packing as the mask bits)
     uint32_t* status;       // device status word (a dnns_status, 0 = ok)
-    const uint32_t* vec_items;  // [n_vec_items] the vector items (BatchNorm vectors, biases) of the rebuild
+    const uint32_t* vec_items;  // [n_vec_items][2] pieces of the vector items (BatchNorm vectors, biases) of the rebuild: item, piece
     uint32_t n_tensors, n_groups, n_bn, n_segs, n_items, n_tiles, n_flag_units, n_vec_items;
     uint32_t tile_elems;    // 4096 (fp32) or 8192 (bf16)
     int32_t dtype;

@@ -256,7 +256,7 @@ __global__ void __launch_bounds__(256) k_extrema_flags(Tables tb, const uint32_t
 
 int launch_extrema(const Tables& tb, uint32_t* rowmax, uint32_t* colmax, int n_sm, cudaStream_t st) {
     const dim3 grid(min((uint32_t)n_sm * 4u, tb.n_tiles));
-    ScopedKernel timed("k_extrema", st);
+    ScopedKernel timed("k_extrema_sweep", st);
     if (tb.dtype == DNNS_F32) k_extrema<DNNS_F32><<<grid, kTileThreads, 0, st>>>(tb, rowmax, colmax);
     else k_extrema<DNNS_BF16><<<grid, kTileThreads, 0, st>>>(tb, rowmax, colmax);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;

@@ -8,6 +8,8 @@
 
 #include <string>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "dnns_internal.cuh"
 
 using namespace dnns;
@@ -178,7 +180,11 @@ dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts*
         has_bn[bn.tensor] = 1;
     }
     c->items = c->T + 4 * c->B + c->n_bias;
-    c->n_vec = 4 * c->B + c->n_bias;
+    // vector items are dealt out in pieces of kVecPiece rows
+    c->n_vec = 0;
+    for (int b = 0; b < m->n_bn; ++b) c->n_vec += 4 * (((uint32_t)m->bns[b].C + kVecPiece - 1) / kVecPiece);
+    for (int i = 0; i < m->n_tensors; ++i)
+        if (m->tensors[i].bias) c->n_vec += ((uint32_t)m->tensors[i].O + kVecPiece - 1) / kVecPiece;
     return DNNS_OK;
 }
 
@@ -210,7 +216,7 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.consumers = take(sizeof(ConsumerDesc) * c.T);
     w.flag_prefix = take(4ull * (c.T + 1));
     w.flag_unit_tensor = take(4ull * (c.flag_units + 1));
-    w.vec_items = take(4ull * (c.n_vec + 1));
+    w.vec_items = take(8ull * (c.n_vec + 1));
     w.status = take(4);
     w.tables_end = o;
     const uint64_t vs = (uint64_t)maxv * (c.S ? c.S : 1);
@@ -268,6 +274,10 @@ namespace {
 struct ProfileScope {  // makes the plan's profile the active one for the launches of one call
     explicit ProfileScope(dnns_plan* p) { dnns::g_timer = p ? &p->timer : nullptr; }
     ~ProfileScope() { dnns::g_timer = nullptr; }
+};
+struct Range {  // an NVTX range around the host side of one entry point, named after the step it enqueues
+    explicit Range(const char* name) { nvtxRangePushA(name); }
+    ~Range() { nvtxRangePop(); }
 };
 }  // namespace
 
@@ -488,8 +498,8 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     auto vector_item = [&](const float* v, int32_t C, int32_t group) {
         ItemDesc it{};
         it.src = v, it.tensor = -1, it.O = C, it.Cin = 1, it.blk = 1, it.out_group = group, it.in_group = -1, it.elem_bytes = 4;
-        it.ko_off = gd[group].off_idx, it.seg = -1, it.S = 1, it.kind = kItemVector, it.vec_rank = (int32_t)n_vec;
-        vec_items[n_vec++] = n_it;
+        it.ko_off = gd[group].off_idx, it.seg = -1, it.S = 1, it.kind = kItemVector, it.vec_rank = (int32_t)n_vec;  // (rank of its first piece)
+        for (uint32_t piece = 0; piece * kVecPiece < (uint32_t)C; ++piece) vec_items[2 * n_vec] = n_it, vec_items[2 * n_vec + 1] = piece, ++n_vec;
         id[n_it++] = it;
         compact_bytes += align_up(4ull * C);
     };
@@ -588,6 +598,7 @@ uint64_t dnns_plan_launch_count(const dnns_plan* plan) { return plan ? plan->lau
 
 dnns_status dnns_magnitude_threshold(dnns_plan* p, const uint64_t* k, int32_t n_k, dnns_threshold* thr_dev,
                                      void* stream) {
+    Range nvtx_range("dnns: step 1 threshold");
     if (!p || !k || !thr_dev || n_k < 1 || n_k > p->maxv) return DNNS_ERR_INVALID_ARG;
     const uint32_t S = p->c.S;
     if (S == 0) return DNNS_OK;
@@ -608,6 +619,7 @@ dnns_status dnns_magnitude_threshold(dnns_plan* p, const uint64_t* k, int32_t n_
 
 dnns_status dnns_apply_mask(dnns_plan* p, const dnns_threshold* thr_dev, int32_t variant, void* masked_arena,
                             uint32_t* mask_bits, void* stream) {
+    Range nvtx_range("dnns: step 2 mask");
     if (!p || !thr_dev || variant < 0 || variant >= p->last_n_k) return DNNS_ERR_INVALID_ARG;  // a variant of the latest threshold call
     if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
     ProfileScope profile_scope(p);
@@ -620,6 +632,7 @@ dnns_status dnns_apply_mask(dnns_plan* p, const dnns_threshold* thr_dev, int32_t
 
 dnns_status dnns_zero_structures(dnns_plan* p, const void* masked_arena, uint32_t* nz_map, uint32_t* out_nz,
                                  uint32_t* in_nz, void* stream) {
+    Range nvtx_range("dnns: step 3 zero structures");
     if (!p || !out_nz || !in_nz) return DNNS_ERR_INVALID_ARG;
     if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -636,6 +649,7 @@ dnns_status dnns_zero_structures(dnns_plan* p, const void* masked_arena, uint32_
 dnns_status dnns_mask_and_structures(dnns_plan* p, const dnns_threshold* thr_dev, int32_t variant, void* masked_arena,
                                      uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz,
                                      void* stream) {
+    Range nvtx_range("dnns: steps 2+3");
     if (!p || !thr_dev || !out_nz || !in_nz || variant < 0 || variant >= p->last_n_k) return DNNS_ERR_INVALID_ARG;
     if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -653,6 +667,7 @@ dnns_status dnns_mask_and_structures_multi(dnns_plan* p, const dnns_threshold* t
                                            int32_t n_variants, void* const* masked_arenas, uint32_t* const* mask_bits,
                                            uint32_t* const* nz_map, uint32_t* const* out_nz, uint32_t* const* in_nz,
                                            void* stream) {
+    Range nvtx_range("dnns: steps 2+3, several variants");
     if (!p || !thr_dev || !masked_arenas || !out_nz || !in_nz || n_variants < 1 || n_variants > kMultiMax ||
         first_variant < 0 || first_variant + n_variants > p->last_n_k)
         return DNNS_ERR_INVALID_ARG;
@@ -693,6 +708,7 @@ dnns_status dnns_mask_and_structures_multi(dnns_plan* p, const dnns_threshold* t
 dnns_status dnns_zero_structures_portfolio(dnns_plan* p, const dnns_threshold* thr_dev, int32_t first_variant,
                                            int32_t n_variants, uint32_t* const* out_nz, uint32_t* const* in_nz,
                                            void* stream) {
+    Range nvtx_range("dnns: step 3, portfolio");
     if (!p || !thr_dev || !out_nz || !in_nz || n_variants < 1 || n_variants > kPortfolioMax || first_variant < 0 ||
         first_variant + n_variants > p->last_n_k)
         return DNNS_ERR_INVALID_ARG;
@@ -719,6 +735,7 @@ dnns_status dnns_zero_structures_portfolio(dnns_plan* p, const dnns_threshold* t
 dnns_status dnns_propagate_keep(dnns_plan* p, const uint32_t* out_nz, const uint32_t* in_nz, uint32_t policy,
                                 int32_t min_keep, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count,
                                 uint64_t* stats, void* stream) {
+    Range nvtx_range("dnns: step 4 keep sets");
     if (!p || !out_nz || !in_nz || !keep_bits || !keep_idx || !keep_count) return DNNS_ERR_INVALID_ARG;
     if (policy & ~(uint32_t)(DNNS_RULE_PRODUCER | DNNS_RULE_CONSUMER | DNNS_SHIFT_STRICT)) return DNNS_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -737,6 +754,7 @@ dnns_status dnns_propagate_keep_multi(dnns_plan* p, int32_t n_variants, const ui
                                       const uint32_t* const* in_nz, uint32_t policy, int32_t min_keep,
                                       uint32_t* const* keep_bits, int32_t* const* keep_idx, int32_t* const* keep_count,
                                       uint64_t* stats, void* stream) {
+    Range nvtx_range("dnns: step 4, several variants");
     if (!p || !out_nz || !in_nz || !keep_bits || !keep_idx || !keep_count || n_variants < 1 || n_variants > kPortfolioMax)
         return DNNS_ERR_INVALID_ARG;
     if (policy & ~(uint32_t)(DNNS_RULE_PRODUCER | DNNS_RULE_CONSUMER | DNNS_SHIFT_STRICT)) return DNNS_ERR_INVALID_ARG;
@@ -761,6 +779,7 @@ dnns_status dnns_propagate_keep_multi(dnns_plan* p, int32_t n_variants, const ui
 dnns_status dnns_propagate_keep_cascade(dnns_plan* p, const uint32_t* nz_map, uint32_t policy, int32_t min_keep,
                                         int32_t max_passes, uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count,
                                         uint64_t* stats, void* stream) {
+    Range nvtx_range("dnns: step 4 to a fixed point");
     if (!p || !nz_map || !keep_bits || !keep_idx || !keep_count) return DNNS_ERR_INVALID_ARG;
     if (policy & ~(uint32_t)(DNNS_RULE_PRODUCER | DNNS_RULE_CONSUMER | DNNS_SHIFT_STRICT)) return DNNS_ERR_INVALID_ARG;
     if (max_passes < 1 || max_passes > kMaxCascadePasses) return DNNS_ERR_INVALID_ARG;
@@ -782,6 +801,7 @@ dnns_status dnns_propagate_keep_cascade(dnns_plan* p, const uint32_t* nz_map, ui
 dnns_status dnns_compact(dnns_plan* p, const void* masked_arena, const int32_t* keep_idx, const int32_t* keep_count,
                          void* dst_arena, size_t dst_bytes, uint64_t* dst_offsets_dev, int32_t* dst_shapes_dev,
                          void* stream) {
+    Range nvtx_range("dnns: step 5 rebuild");
     if (!p || !keep_idx || !keep_count || !dst_arena || !dst_offsets_dev || !dst_shapes_dev) return DNNS_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) ||
         (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)))
@@ -804,6 +824,7 @@ dnns_status dnns_compact(dnns_plan* p, const void* masked_arena, const int32_t* 
 dnns_status dnns_compact_masked(dnns_plan* p, const dnns_threshold* thr_dev, int32_t variant,
                                 const int32_t* keep_idx, const int32_t* keep_count, void* dst_arena, size_t dst_bytes,
                                 uint64_t* dst_offsets_dev, int32_t* dst_shapes_dev, void* stream) {
+    Range nvtx_range("dnns: steps 2+5 rebuild from the dense model");
     if (!p || !thr_dev || !keep_idx || !keep_count || !dst_arena || !dst_offsets_dev || !dst_shapes_dev ||
         variant < 0 || variant >= p->last_n_k)
         return DNNS_ERR_INVALID_ARG;
@@ -825,6 +846,7 @@ dnns_status dnns_compact_masked(dnns_plan* p, const dnns_threshold* thr_dev, int
 
 dnns_status dnns_fold_batchnorm(dnns_plan* p, void* dst_arena, const uint64_t* dst_offsets_dev,
                                 const int32_t* dst_shapes_dev, void* stream) {
+    Range nvtx_range("dnns: conv+BN fusion");
     if (!p || !dst_arena || !dst_offsets_dev || !dst_shapes_dev) return DNNS_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) return DNNS_ERR_INVALID_ARG;
     ProfileScope profile_scope(p);

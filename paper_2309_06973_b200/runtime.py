@@ -216,11 +216,13 @@ class Session:
                                     ptrs("keep_bits"), ptrs("keep_idx"), ptrs("keep_count"), self.stats_multi.data_ptr(),
                                     _stream())
 
-    def compact_portfolio(self, variant: int, slot: int):
-        """Rebuild `variant` from the dense model with the keep sets of portfolio slot `slot`."""
+    def compact_portfolio(self, variant: int, slot: int, arena: Optional[torch.Tensor] = None):
+        """Rebuild `variant` from the dense model with the keep sets of portfolio slot `slot` (arena: another
+        destination than the session's own)."""
+        arena = self.compact_arena if arena is None else arena
         B.dnns_compact_masked(self.plan, self.thr.data_ptr(), variant, self.pf[slot]["keep_idx"].data_ptr(),
-                              self.pf[slot]["keep_count"].data_ptr(), self.compact_arena.data_ptr(),
-                              self.compact_arena.numel(), self.dst_offsets.data_ptr(), self.dst_shapes.data_ptr(), _stream())
+                              self.pf[slot]["keep_count"].data_ptr(), arena.data_ptr(), arena.numel(),
+                              self.dst_offsets.data_ptr(), self.dst_shapes.data_ptr(), _stream())
 
     def propagate_keep_cascade(self, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1,
                                max_passes: int = 8):

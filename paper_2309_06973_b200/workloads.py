@@ -412,4 +412,17 @@ def _shrink(wl: Workload, f: int) -> Workload:
     return wl
 
 
+def freeze_streams(wl: Workload) -> Workload:
+    """Mark every channel group that more than one layer writes (a residual stream: the stem or a projection plus
+    the last conv of every block on it) as frozen, so that only plain layer-to-layer connections are pruned -
+    the paper's own setting, which leaves skip connections and downsampling layers alone (Section IV-B-2)."""
+    writers = [0] * len(wl.groups)
+    for t in wl.tensors:
+        writers[t.out_group] += 1
+    for g, n in zip(wl.groups, writers):
+        if n > 1:
+            g.flags |= GROUP_FROZEN
+    return wl
+
+
 BY_NAME = {"toy": toy, "vgg16": vgg16, "resnet56": resnet56, "resnet50": resnet50, "resnet152": resnet152}
