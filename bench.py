@@ -191,7 +191,8 @@ class Config:
         self.groups = [(v0, min(self.G, V - v0)) for v0 in range(0, V, self.G)] if self.G else []
         sparse_free = self.path == "sparse_free"
         self.ses = Session(self.dm, wl.scope, V, want_mask_bits=not sparse_free, want_nz_map=False,
-                           slots=max(self.G, 1), portfolio_slots=V if sparse_free else 0)
+                           slots=max(self.G, 1), portfolio_slots=V if sparse_free else 0,
+                           portfolio_arenas=sparse_free and not args.rebuild_per_variant)
         self.flush_buf = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=self.dm.device)
         self.call_names = {"sparse_free": ["threshold", "structures(portfolio)", "propagate", "compact"],
                            "multi": ["threshold", "mask+structures", "propagate", "compact"],
@@ -216,8 +217,11 @@ class Config:
                 n = min(16, V - v0)
                 timed("structures(portfolio)", ses.zero_structures_portfolio, v0, n)
                 timed("propagate", ses.propagate_keep_portfolio, n)
-                for s in range(n):
-                    timed("compact", ses.compact_portfolio, v0 + s, s)
+                if self.args.rebuild_per_variant:
+                    for s in range(n):
+                        timed("compact", ses.compact_portfolio, v0 + s, s)
+                else:                                         # the n rebuilds in one launch, each into its own arena
+                    timed("compact", ses.compact_portfolio_multi, v0, n)
             return
         for v0, n in self.groups:                             # n variants per read of the dense weights
             timed("mask+structures", ses.mask_and_structures_multi, v0, n)
@@ -331,7 +335,7 @@ def measure(cfg, steps, warmup, barrier, max_over_ranks, ms_per_variant_of, peak
     if cfg.path == "sparse_free":
         moved = (thr_sweeps + 1) * N * eb + sum(rebuild)
         sweeps = (f"no sparse model: {thr_sweeps} ranking sweeps and one sweep for the zero structures of all {V} variants, "
-                  "then one masking rebuild per variant")
+                  + ("then one masking rebuild per variant" if args.rebuild_per_variant else "then the masking rebuilds of all variants in one launch"))
     elif cfg.path == "multi":
         moved = thr_sweeps * N * eb + sum(N * eb + n * (N * eb + N / 4) for _, n in cfg.groups) + sum(rebuild)
         sweeps = f"fused mask+structures, {cfg.G} variants per read of the dense weights; {thr_sweeps} ranking sweeps"
@@ -344,7 +348,8 @@ def measure(cfg, steps, warmup, barrier, max_over_ranks, ms_per_variant_of, peak
     stepwise_bytes = N * eb * (1 + 3 * V) + V * N / 8 + sum(rebuild)   # one read per input, one write per output of every step
 
     kernel_alg = {"k_hist1": N * eb, "k_hist2": N * eb, "k_ties": N * eb if ties_swept else 0, "k_extrema_sweep": N * eb,
-                  "k_compact_gather": statistics.mean(rebuild),
+                  "k_compact_gather": statistics.mean(rebuild) if (cfg.path != "sparse_free" or args.rebuild_per_variant)
+                  else sum(rebuild) / ((V + 15) // 16),      # one launch rebuilds up to 16 variants
                   "k_sweep<": (3 * N * eb + N / 4) / 2 if cfg.path == "stepwise" else 2 * N * eb + N / 4}
     if cfg.groups:
         kernel_alg["k_sweep_multi"] = sum(N * eb + n * (N * eb + N / 4) for _, n in cfg.groups) / len(cfg.groups)
@@ -577,6 +582,8 @@ def main():
                          "written; fused: one fused sweep per variant; stepwise: the five calls one by one")
     ap.add_argument("--stepwise", action="store_true", help="same as --path stepwise")
     ap.add_argument("--multi", type=int, default=-1, help="--path multi: variants per sweep (1..4; default 4 for f32, 2 for bf16)")
+    ap.add_argument("--rebuild-per-variant", action="store_true",
+                    help="--path sparse_free: one rebuild launch per variant instead of one for all variants")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph replay")
     ap.add_argument("--no-also", action="store_true", help="skip the other target configurations (resnet152 bf16, resnet50 f32)")

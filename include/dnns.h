@@ -354,6 +354,19 @@ dnns_status dnns_compact_masked(dnns_plan* plan, const dnns_threshold* thr_dev, 
                                 uint64_t* dst_offsets_dev, int32_t* dst_shapes_dev, void* stream);
 
 /*
+ * dnns_compact_masked for n_variants (1..DNNS_PORTFOLIO_MAX) variants first_variant .. first_variant + n_variants - 1
+ * in ONE launch: the variants of a portfolio are rebuilt from the same dense model and are independent of one
+ * another, so their gathers share one grid, and a block that has finished its share of one variant goes on with
+ * the next.  keep_idx, keep_count, dst_arenas, dst_offsets_dev, dst_shapes_dev: host arrays of n_variants device
+ * pointers, entry i for variant first_variant + i, each as in dnns_compact_masked; the destinations (and the
+ * arrays of counts) all distinct, every arena of dst_bytes.  Bit for bit n_variants calls of dnns_compact_masked.
+ */
+dnns_status dnns_compact_masked_multi(dnns_plan* plan, const dnns_threshold* thr_dev, int32_t first_variant,
+                                      int32_t n_variants, const int32_t* const* keep_idx,
+                                      const int32_t* const* keep_count, void* const* dst_arenas, size_t dst_bytes,
+                                      uint64_t* const* dst_offsets_dev, int32_t* const* dst_shapes_dev, void* stream);
+
+/*
  * Module 1, Model Pre-Processor (Section III-D): fold every BatchNorm into the convolution it
  * follows, on a rebuilt variant as dnns_compact left it (same dst_arena, dst_offsets_dev,
  * dst_shapes_dev).  In place, fp32 arithmetic (bf16 weights are widened, scaled, rounded to nearest

@@ -25,7 +25,7 @@ DNNS_PORTFOLIO_MAX = 16
 EXPORTS = ["dnns_status_string", "dnns_workspace_bytes", "dnns_plan_create", "dnns_plan_destroy", "dnns_plan_layout",
            "dnns_plan_launch_count", "dnns_magnitude_threshold", "dnns_apply_mask", "dnns_zero_structures",
            "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures", "dnns_fold_batchnorm", "dnns_propagate_keep_cascade",
-           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_mask_and_structures_multi", "dnns_propagate_keep_multi", "dnns_compact_masked", "dnns_zero_structures_portfolio", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
+           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_mask_and_structures_multi", "dnns_propagate_keep_multi", "dnns_compact_masked", "dnns_zero_structures_portfolio", "dnns_compact_masked_multi", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
 
 
 class dnns_tensor(C.Structure):
@@ -108,6 +108,7 @@ def lib() -> C.CDLL:
         L.dnns_propagate_keep_multi.argtypes = [vp, i32, vp, vp, u32, i32, vp, vp, vp, vp, vp]
         L.dnns_compact_masked.argtypes = [vp, vp, i32, vp, vp, vp, C.c_size_t, vp, vp, vp]
         L.dnns_zero_structures_portfolio.argtypes = [vp, vp, i32, i32, vp, vp, vp]
+        L.dnns_compact_masked_multi.argtypes = [vp, vp, i32, i32, vp, vp, vp, C.c_size_t, vp, vp, vp]
         L.dnns_plan_profile.argtypes = [vp, i32]
         L.dnns_plan_profile_read.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(u64)]
         for name in ("dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes"):
@@ -272,6 +273,15 @@ def dnns_zero_structures_portfolio(plan, thr_dev: int, first_variant: int, n_var
     """out_nz, in_nz: lists of n_variants device addresses."""
     _check(lib().dnns_zero_structures_portfolio(plan, thr_dev, first_variant, n_variants, _ptr_array(out_nz),
                                                 _ptr_array(in_nz), stream), "dnns_zero_structures_portfolio")
+
+
+def dnns_compact_masked_multi(plan, thr_dev: int, first_variant: int, n_variants: int, keep_idx, keep_count, dst_arenas,
+                              dst_bytes: int, dst_offsets_dev, dst_shapes_dev, stream: int = 0) -> None:
+    """keep_idx ... dst_shapes_dev: lists of n_variants device addresses (dst_bytes: size of every arena)."""
+    a = [_ptr_array(x) for x in (keep_idx, keep_count, dst_arenas)]
+    b = [_ptr_array(x) for x in (dst_offsets_dev, dst_shapes_dev)]
+    _check(lib().dnns_compact_masked_multi(plan, thr_dev, first_variant, n_variants, a[0], a[1], a[2], dst_bytes, b[0], b[1],
+                                           stream), "dnns_compact_masked_multi")
 
 
 def dnns_compact_masked(plan, thr_dev: int, variant: int, keep_idx: int, keep_count: int, dst_arena: int,

@@ -306,10 +306,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"  // may sleep up to the hint (ns) before it answers
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done)
-        : "r"(smem_addr(bar)), "r"(parity)
+        : "r"(smem_addr(bar)), "r"(parity), "r"(20000u)
         : "memory");
     return done != 0;
 }
@@ -459,24 +459,29 @@ __device__ __forceinline__ uint4 threshold_vec(uint4 v, uint32_t thr_eff) {
 template <int BYTES, bool MASKED>
 __device__ __forceinline__ void consume_copy(const UnitDesc& desc, const unsigned char* stage, int ctid) {
     constexpr uint32_t VE = 16 / BYTES;
-    const UnitDesc d = desc;  // in registers: the stores below could alias the descriptor as far as the compiler knows
-    const uint32_t vpr = d.Ws / VE, n_vec = d.n_r * vpr;  // vectors per row, in the unit
+    // (fields read once into registers: the stores below could alias the descriptor as far as the compiler knows)
+    char* const dst = desc.dst;
+    const uint32_t vpr = desc.Ws / VE, n_vec = desc.n_r * vpr;  // vectors per row, in the unit
     const uint4* s = reinterpret_cast<const uint4*>(stage);
-    const uint32_t row_pitch = d.Ln * BYTES;  // a unit spans less than 2^32 destination bytes
-    if (MASKED && d.mk.mode == 2) {
+    const uint32_t row_pitch = desc.Ln * BYTES;  // a unit spans less than 2^32 destination bytes
+    const uint32_t mode = MASKED ? desc.mk.mode : 0u, thr_eff = desc.mk.thr_eff;
+    if (MASKED && mode == 2) {
         // around the place where the weights equal to tau split: element by element, by source position
+        const MaskCtx mk = desc.mk;
+        const int32_t* ko = desc.ko;
+        const uint32_t L = desc.L, first = desc.c_lo * desc.blk;
         for (uint32_t v = ctid; v < n_vec; v += kConsumers) {
             const uint32_t row = v / vpr, col = v - row * vpr;
-            const uint4 x = masked_vec<BYTES>(s[v], d.mk, (uint32_t)__ldg(d.ko + row) * d.L + d.c_lo * d.blk + col * VE);
-            *reinterpret_cast<uint4*>(d.dst + (size_t)row * row_pitch + (size_t)col * 16) = x;
+            const uint4 x = masked_vec<BYTES>(s[v], mk, (uint32_t)__ldg(ko + row) * L + first + col * VE);
+            *reinterpret_cast<uint4*>(dst + (size_t)row * row_pitch + (size_t)col * 16) = x;
         }
         return;
     }
-    const bool mask = MASKED && d.mk.mode == 1;
+    const bool mask = mode == 1;
     if (row_pitch == vpr * 16) {  // whole rows: the destination is one run as well
-        uint4* g = reinterpret_cast<uint4*>(d.dst);
+        uint4* g = reinterpret_cast<uint4*>(dst);
 #pragma unroll 4
-        for (uint32_t v = ctid; v < n_vec; v += kConsumers) g[v] = mask ? threshold_vec<BYTES>(s[v], d.mk.thr_eff) : s[v];
+        for (uint32_t v = ctid; v < n_vec; v += kConsumers) g[v] = mask ? threshold_vec<BYTES>(s[v], thr_eff) : s[v];
         return;
     }
     const uint32_t step_row = kConsumers / vpr, step_col = kConsumers - step_row * vpr;
@@ -485,7 +490,7 @@ __device__ __forceinline__ void consume_copy(const UnitDesc& desc, const unsigne
     uint32_t off = row * row_pitch + col * 16;
 #pragma unroll 2
     for (uint32_t v = ctid; v < n_vec; v += kConsumers) {
-        *reinterpret_cast<uint4*>(d.dst + off) = mask ? threshold_vec<BYTES>(s[v], d.mk.thr_eff) : s[v];
+        *reinterpret_cast<uint4*>(dst + off) = mask ? threshold_vec<BYTES>(s[v], thr_eff) : s[v];
         col += step_col;
         off += step_off;
         if (col >= vpr) {
@@ -507,21 +512,27 @@ template <int BYTES, bool MASKED, bool CAREFUL>
 __device__ __forceinline__ void consume_gather(const UnitDesc& desc, const unsigned char* stage, const uint16_t* rowmap, int ctid) {
     typedef typename ElemWord<BYTES>::type T;
     constexpr int kColBatch = 4;
-    const UnitDesc d = desc;
-    const uint32_t Wd = d.Wd, Ws = d.Ws, n_r = d.n_r, blk = d.blk, Ln = d.Ln;
+    // (fields read once into registers: the stores below could alias the descriptor as far as the compiler knows)
+    const uint32_t Wd = desc.Wd, Ws = desc.Ws, n_r = desc.n_r, blk = desc.blk, Ln = desc.Ln;
+    const uint32_t map_seq = desc.map_seq, map_base = desc.map_base, first = desc.c_lo * blk, c_lo = desc.c_lo;
+    const uint32_t magic = desc.magic, n_ki = desc.n_ki, L = desc.L;
+    const int32_t* const ki = desc.ki;
+    const int32_t* const ko = desc.ko;
+    const uint32_t mode = MASKED ? desc.mk.mode : 0u, tau = desc.mk.tau, split_elem = desc.mk.split_elem;
+    (void)n_ki;
     constexpr uint32_t key_mask = BYTES == 4 ? 0x7FFFFFFFu : 0x7FFFu;
     // keep iff key >= thr_eff (0: everything stays)
-    const uint32_t thr_eff = (!MASKED || d.mk.mode == 0) ? 0u : (d.mk.mode == 1 ? d.mk.thr_eff : d.mk.tau + 1u);
+    const uint32_t thr_eff = mode == 0 ? 0u : (mode == 1 ? desc.mk.thr_eff : tau + 1u);
     const T* sbase = reinterpret_cast<const T*>(stage);
-    T* dbase = reinterpret_cast<T*>(d.dst);
+    T* dbase = reinterpret_cast<T*>(desc.dst);
     // position of destination column `col` in a row of the stage buffer
     auto source_offset = [&](uint32_t col) -> uint32_t {
         uint32_t soff;
-        if (d.map_seq) {
-            soff = (uint32_t)rowmap[d.map_base + col] - d.c_lo * blk;
+        if (map_seq) {
+            soff = (uint32_t)rowmap[map_base + col] - first;
         } else {
-            const uint32_t p = blk == 1 ? col : (blk == 9 ? col / 9u : __umulhi(col, d.magic));
-            soff = ((uint32_t)__ldg(d.ki + DNNS_IDX(p, d.n_ki)) - d.c_lo) * blk + (col - p * blk);
+            const uint32_t p = blk == 1 ? col : (blk == 9 ? col / 9u : __umulhi(col, magic));
+            soff = ((uint32_t)__ldg(ki + DNNS_IDX(p, n_ki)) - c_lo) * blk + (col - p * blk);
         }
 #ifdef DNNS_BOUNDS_CHECK
         if (soff >= Ws) {
@@ -535,7 +546,7 @@ __device__ __forceinline__ void consume_gather(const UnitDesc& desc, const unsig
         if (!MASKED) return x;
         const uint32_t key = x & key_mask;
         bool keep = key >= thr_eff;
-        if (CAREFUL && key == d.mk.tau) keep = (uint32_t)__ldg(d.ko + row) * d.L + d.c_lo * blk + soff >= d.mk.split_elem;
+        if (CAREFUL && key == tau) keep = (uint32_t)__ldg(ko + row) * L + first + soff >= split_elem;
         return keep ? x : 0u;
     };
     if (Wd > kConsumers / 2) {
@@ -589,11 +600,8 @@ __device__ __forceinline__ void consume_gather(const UnitDesc& desc, const unsig
 //
 // MASKED: the source is the dense model and step 2 is applied to every element on its way (thr, variant, split).
 template <int WBYTES, bool MASKED>  // WBYTES: element width of the weight tensors (BatchNorm, bias: 4 bytes)
-__global__ void __launch_bounds__(kGatherThreads, 3) k_compact_gather(Tables tb, RebuildSlot lay, const char* src_arena,
-                                                                      const int32_t* __restrict__ keep_idx, char* dst_arena,
-                                                                      uint64_t dst_bytes, uint64_t* dst_offsets,
-                                                                      int32_t* dst_shapes,
-                                                                      const dnns_threshold* __restrict__ thr, int variant,
+__global__ void __launch_bounds__(kGatherThreads, 3) k_compact_gather(Tables tb, GatherBatch gb,
+                                                                      const dnns_threshold* __restrict__ thr,
                                                                       const TieSplit* __restrict__ split) {
     extern __shared__ uint4 s_stage_mem[];  // kStages buffers of kStageBytes
     __shared__ __align__(8) uint64_t s_full[kStages], s_empty[kStages];
@@ -605,8 +613,6 @@ __global__ void __launch_bounds__(kGatherThreads, 3) k_compact_gather(Tables tb,
     __shared__ uint16_t s_rowmap[kRowMapMax];
     unsigned char* const stage_mem = reinterpret_cast<unsigned char*>(s_stage_mem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const RebuildHeader* header = lay.header;
-    const RebuildItem* __restrict__ ritems = lay.items;
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -616,19 +622,15 @@ __global__ void __launch_bounds__(kGatherThreads, 3) k_compact_gather(Tables tb,
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    const uint64_t total_bytes = header->total_bytes;
-    const uint32_t total_cost = header->total_cost, total_units = header->total_units;
     __syncthreads();
-    if (total_bytes > dst_bytes) {  // too small an arena: nothing is copied
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicCAS(tb.status, 0u, (uint32_t)DNNS_ERR_WORKSPACE);
-        return;
-    }
+    // a job whose arena is too small for its variant copies nothing
+    auto job_fits = [&](int j) { return gb.job[j].lay.header->total_bytes <= gb.job[j].dst_bytes; };
     volatile uint32_t* abort_flag = &s_abort;
     auto give_up = [&]() {
         *abort_flag = 1;
         atomicCAS(tb.status, 0u, (uint32_t)DNNS_ERR_TIMEOUT);
     };
-    auto mask_ctx = [&](const ItemDesc& it) {
+    auto mask_ctx = [&](const ItemDesc& it, int variant) {
         MaskCtx mk{0u, 0u, 0u, 0u};
         if (MASKED && it.tensor >= 0 && it.seg >= 0) {
             const size_t idx = (size_t)variant * tb.n_segs + it.seg;
@@ -647,20 +649,32 @@ __global__ void __launch_bounds__(kGatherThreads, 3) k_compact_gather(Tables tb,
     };
 
     if (warp == kProducerWarp) {
-        // ================= producer: takes ranges of the cost axis, walks their units, fills the ring =================
-        const uint32_t n_ranges = rebuild_ranges(gridDim.x);
+        // ================= producer: takes ranges of the cost axes of the jobs, walks their units, fills the ring =====
+        const uint32_t per_job = rebuild_ranges(gridDim.x), n_ranges = per_job * (uint32_t)gb.n;
+        RebuildHeader* const counters = gb.job[0].lay.header;
         auto next_range = [&]() {  // the counter's value k stands for range gridDim.x + k
             uint32_t r = 0;
-            if (lane == 0) r = atomicAdd(&lay.header->next_range, 1u);
+            if (lane == 0) r = atomicAdd(&counters->next_range, 1u);
             return gridDim.x + __shfl_sync(0xffffffffu, r, 0);
         };
         uint32_t issued = 0, map_seq = 0;
         bool alive = true;
-        uint32_t range = blockIdx.x, range_after = total_cost ? next_range() : n_ranges;
-        for (; alive && total_cost && range < n_ranges; range = range_after, range_after = range < n_ranges ? next_range() : n_ranges) {
-            const uint32_t lo = rebuild_range_lo(range, gridDim.x, total_cost), hi = rebuild_range_lo(range + 1, gridDim.x, total_cost);
+        int cur_job = -1;
+        uint32_t total_cost = 0;
+        uint32_t range = blockIdx.x, range_after = next_range();
+        for (; alive && range < n_ranges; range = range_after, range_after = range < n_ranges ? next_range() : n_ranges) {
+            const int jb = (int)(range / per_job);
+            const uint32_t rj = range - (uint32_t)jb * per_job;
+            if (jb != cur_job) {
+                cur_job = jb;
+                total_cost = job_fits(jb) ? gb.job[jb].lay.header->total_cost : 0u;
+            }
+            const GatherJob& job = gb.job[jb];
+            const RebuildItem* __restrict__ ritems = job.lay.items;
+            const int32_t* __restrict__ keep_idx = job.keep_idx;
+            const uint32_t lo = rebuild_range_lo(rj, gridDim.x, total_cost), hi = rebuild_range_lo(rj + 1, gridDim.x, total_cost);
             if (lo >= hi) continue;
-            for (uint32_t item = lay.range_item[range]; alive && item < tb.n_items; ++item) {
+            for (uint32_t item = job.lay.range_item[rj]; alive && item < tb.n_items; ++item) {
                 const RebuildItem z = ritems[item];
                 if (z.cost_pre >= hi) break;
                 if (z.s_units == 0) continue;
@@ -669,12 +683,12 @@ __global__ void __launch_bounds__(kGatherThreads, 3) k_compact_gather(Tables tb,
                 const uint32_t j_hi = min(z.s_units, (hi - pre + z.s_cost - 1) / z.s_cost);
                 if (j_lo >= j_hi) continue;
                 const ItemDesc it = tb.items[item];
-                const char* src = src_arena ? src_arena + it.arena_off : static_cast<const char*>(it.src);
-                char* dst = dst_arena + ((uint64_t)z.off256 << 8);
+                const char* src = job.src_arena ? job.src_arena + it.arena_off : static_cast<const char*>(it.src);
+                char* dst = job.dst_arena + ((uint64_t)z.off256 << 8);
                 const int32_t* ko = keep_idx + it.ko_off;
                 const int32_t* ki = keep_idx + it.ki_off;
                 const uint32_t blk = it.blk, Cin = it.Cin, L = Cin * blk, Ln = z.Cn * blk;
-                const MaskCtx mk = mask_ctx(it);
+                const MaskCtx mk = mask_ctx(it, job.variant);
                 const Geometry g = geometry_of(it, z.Cn);
                 const uint32_t nch = g.nch, ru = g.ru, ch = g.ch;
                 const bool identity = z.Cn == Cin;  // no input channel is dropped: kept channel p is channel p
@@ -775,10 +789,10 @@ __global__ void __launch_bounds__(kGatherThreads, 3) k_compact_gather(Tables tb,
                 }
             }
         }
-        if (total_cost && lane == 0 && atomicAdd(&lay.header->done_blocks, 1u) == gridDim.x - 1) {
+        if (lane == 0 && atomicAdd(&counters->done_blocks, 1u) == gridDim.x - 1) {
             // every block has taken its last range: the counters are ready for the next launch on this layout
-            lay.header->next_range = 0;
-            lay.header->done_blocks = 0;
+            counters->next_range = 0;
+            counters->done_blocks = 0;
         }
         if (alive) {  // tell the consumers that this was all
             const uint32_t s = issued % kStages, use = issued / kStages;
@@ -805,65 +819,75 @@ __global__ void __launch_bounds__(kGatherThreads, 3) k_compact_gather(Tables tb,
     }
 
     // ================= consumers =================
-    // what the caller asked for beside the arena: the offset of every item, the new shape of every tensor
-    for (uint32_t i = blockIdx.x * kConsumers + threadIdx.x; i < tb.n_items; i += gridDim.x * kConsumers) {
-        const RebuildItem z = ritems[i];
-        dst_offsets[i] = (uint64_t)z.off256 << 8;
-        const ItemDesc& it = tb.items[i];
-        if (it.tensor >= 0) {
-            dst_shapes[2 * it.tensor] = (int32_t)z.On;
-            dst_shapes[2 * it.tensor + 1] = (int32_t)(z.Cn * (uint32_t)it.S);
+    for (int jb = 0; jb < gb.n; ++jb) {
+        const GatherJob& job = gb.job[jb];
+        const RebuildItem* __restrict__ ritems = job.lay.items;
+        const int32_t* __restrict__ keep_idx = job.keep_idx;
+        if (!job_fits(jb)) {
+            if (blockIdx.x == 0 && threadIdx.x == 0) atomicCAS(tb.status, 0u, (uint32_t)DNNS_ERR_WORKSPACE);
+            continue;
         }
-    }
-    // vector items (BatchNorm vectors, biases): v'[a] = v[keep[a]], a warp per piece of kVecPiece rows; all index
-    // loads of a piece are issued before the first value is fetched
-    {
-        const uint32_t n_warps = gridDim.x * (kConsumers / 32), gwarp = blockIdx.x + gridDim.x * warp;  // neighbours in different blocks
-        for (uint32_t r = gwarp; r < tb.n_vec_items; r += n_warps) {
-            const uint32_t i = tb.vec_items[2 * r], a0 = tb.vec_items[2 * r + 1] * kVecPiece;
-            const ItemDesc& it = tb.items[i];
+        // what the caller asked for beside the arena: the offset of every item, the new shape of every tensor
+        for (uint32_t i = blockIdx.x * kConsumers + threadIdx.x; i < tb.n_items; i += gridDim.x * kConsumers) {
             const RebuildItem z = ritems[i];
-            if (a0 >= z.On) continue;
-            const uint32_t* src = static_cast<const uint32_t*>(it.src);
-            uint32_t* dst = reinterpret_cast<uint32_t*>(dst_arena + ((uint64_t)z.off256 << 8));
-            const int32_t* ko = keep_idx + it.ko_off;
-            constexpr int kPer = kVecPiece / 32;
-            int32_t row[kPer];
-            uint32_t val[kPer];
-#pragma unroll
-            for (int k = 0; k < kPer; ++k) {
-                const uint32_t a = a0 + k * 32 + lane;
-                row[k] = a < z.On ? __ldg(ko + a) : -1;
+            job.dst_offsets[i] = (uint64_t)z.off256 << 8;
+            const ItemDesc& it = tb.items[i];
+            if (it.tensor >= 0) {
+                job.dst_shapes[2 * it.tensor] = (int32_t)z.On;
+                job.dst_shapes[2 * it.tensor + 1] = (int32_t)(z.Cn * (uint32_t)it.S);
             }
-#pragma unroll
-            for (int k = 0; k < kPer; ++k) val[k] = row[k] >= 0 ? __ldg(src + DNNS_IDX(row[k], it.O)) : 0u;
-#pragma unroll
-            for (int k = 0; k < kPer; ++k)
-                if (row[k] >= 0) dst[a0 + k * 32 + lane] = val[k];
         }
-    }
-    // the element path (rows that are not multiples of 16 bytes): 16 KB destination units, a block per pair
-    {
-        constexpr uint32_t kChunkUnits = 2;
-        for (uint32_t u_lo = blockIdx.x * kChunkUnits; u_lo < total_units; u_lo += gridDim.x * kChunkUnits) {
-            const uint32_t u_hi = min(total_units, u_lo + kChunkUnits);
-            uint32_t unit = u_lo;
-            while (unit < u_hi) {
-                const uint32_t item = lay.unit_item[unit];
-                const RebuildItem z = ritems[item];
-                const ItemDesc& it = tb.items[item];
-                const uint32_t item_begin = z.unit_pre;
-                const uint32_t item_end = item_begin + (uint32_t)(((uint64_t)z.On * z.Cn * (uint32_t)it.blk * (uint32_t)it.elem_bytes + kUnitBytes - 1) / kUnitBytes);
-                const char* src = (it.tensor >= 0 && src_arena) ? src_arena + it.arena_off : static_cast<const char*>(it.src);
-                const MaskCtx mk = mask_ctx(it);
-                char* dst = dst_arena + ((uint64_t)z.off256 << 8);
+        // vector items (BatchNorm vectors, biases): v'[a] = v[keep[a]], a warp per piece of kVecPiece rows; all index
+        // loads of a piece are issued before the first value is fetched
+        {
+            const uint32_t n_warps = gridDim.x * (kConsumers / 32), gwarp = blockIdx.x + gridDim.x * warp;  // neighbours in different blocks
+            for (uint32_t r = gwarp; r < tb.n_vec_items; r += n_warps) {
+                const uint32_t i = tb.vec_items[2 * r], a0 = tb.vec_items[2 * r + 1] * kVecPiece;
+                const ItemDesc& it = tb.items[i];
+                const RebuildItem z = ritems[i];
+                if (a0 >= z.On) continue;
+                const uint32_t* src = static_cast<const uint32_t*>(it.src);
+                uint32_t* dst = reinterpret_cast<uint32_t*>(job.dst_arena + ((uint64_t)z.off256 << 8));
                 const int32_t* ko = keep_idx + it.ko_off;
-                const int32_t* ki = it.in_group >= 0 ? keep_idx + it.ki_off : nullptr;
-                const uint32_t run_end = min(u_hi, item_end);
-                const uint32_t f0 = (unit - item_begin) * (kUnitBytes / it.elem_bytes);
-                if (WBYTES == 4 || it.elem_bytes == 4) gather_run<4, MASKED>(it, src, dst, ko, ki, z.On, z.Cn, f0, run_end - unit, mk);
-                else gather_run<2, MASKED>(it, src, dst, ko, ki, z.On, z.Cn, f0, run_end - unit, mk);
-                unit = run_end;
+                constexpr int kPer = kVecPiece / 32;
+                int32_t row[kPer];
+                uint32_t val[kPer];
+#pragma unroll
+                for (int k = 0; k < kPer; ++k) {
+                    const uint32_t a = a0 + k * 32 + lane;
+                    row[k] = a < z.On ? __ldg(ko + a) : -1;
+                }
+#pragma unroll
+                for (int k = 0; k < kPer; ++k) val[k] = row[k] >= 0 ? __ldg(src + DNNS_IDX(row[k], it.O)) : 0u;
+#pragma unroll
+                for (int k = 0; k < kPer; ++k)
+                    if (row[k] >= 0) dst[a0 + k * 32 + lane] = val[k];
+            }
+        }
+        // the element path (rows that are not multiples of 16 bytes): 16 KB destination units, a block per pair
+        {
+            const uint32_t total_units = job.lay.header->total_units;
+            constexpr uint32_t kChunkUnits = 2;
+            for (uint32_t u_lo = blockIdx.x * kChunkUnits; u_lo < total_units; u_lo += gridDim.x * kChunkUnits) {
+                const uint32_t u_hi = min(total_units, u_lo + kChunkUnits);
+                uint32_t unit = u_lo;
+                while (unit < u_hi) {
+                    const uint32_t item = job.lay.unit_item[unit];
+                    const RebuildItem z = ritems[item];
+                    const ItemDesc& it = tb.items[item];
+                    const uint32_t item_begin = z.unit_pre;
+                    const uint32_t item_end = item_begin + (uint32_t)(((uint64_t)z.On * z.Cn * (uint32_t)it.blk * (uint32_t)it.elem_bytes + kUnitBytes - 1) / kUnitBytes);
+                    const char* src = (it.tensor >= 0 && job.src_arena) ? job.src_arena + it.arena_off : static_cast<const char*>(it.src);
+                    const MaskCtx mk = mask_ctx(it, job.variant);
+                    char* dst = job.dst_arena + ((uint64_t)z.off256 << 8);
+                    const int32_t* ko = keep_idx + it.ko_off;
+                    const int32_t* ki = it.in_group >= 0 ? keep_idx + it.ki_off : nullptr;
+                    const uint32_t run_end = min(u_hi, item_end);
+                    const uint32_t f0 = (unit - item_begin) * (kUnitBytes / it.elem_bytes);
+                    if (WBYTES == 4 || it.elem_bytes == 4) gather_run<4, MASKED>(it, src, dst, ko, ki, z.On, z.Cn, f0, run_end - unit, mk);
+                    else gather_run<2, MASKED>(it, src, dst, ko, ki, z.On, z.Cn, f0, run_end - unit, mk);
+                    unit = run_end;
+                }
             }
         }
     }
@@ -919,18 +943,13 @@ int launch_rebuild_layout(const Tables& tb, const LayoutBatch& lb, int n_layouts
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
-int launch_compact(const Tables& tb, const RebuildSlot& slot, const void* src_arena, const int32_t* keep_idx,
-                   void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets, int32_t* dst_shapes, int n_sm,
-                   cudaStream_t st, const dnns_threshold* thr, int variant, const TieSplit* split) {
-    const char* src = (const char*)src_arena;
-    char* dst = (char*)dst_arena;
+int launch_compact(const Tables& tb, const GatherBatch& gb, int n_sm, cudaStream_t st, const dnns_threshold* thr,
+                   const TieSplit* split) {
     const int grid = gather_grid(n_sm);
     const size_t smem = (size_t)kStages * kStageBytes;
     const bool masked = thr != nullptr;
     ScopedKernel timed(masked ? "k_compact_gather<masked>" : "k_compact_gather", st);
-#define DNNS_GATHER(W, M)                                                                                          \
-    k_compact_gather<W, M><<<grid, kGatherThreads, smem, st>>>(tb, slot, src, keep_idx, dst, dst_bytes, dst_offsets, \
-                                                               dst_shapes, thr, variant, split)
+#define DNNS_GATHER(W, M) k_compact_gather<W, M><<<grid, kGatherThreads, smem, st>>>(tb, gb, thr, split)
     if (tb.dtype == DNNS_F32) {
         if (masked) DNNS_GATHER(4, true);
         else DNNS_GATHER(4, false);

@@ -107,19 +107,18 @@ struct RebuildItem {
 struct RebuildHeader {
     uint64_t total_bytes;  // destination bytes the variant needs
     uint32_t total_cost, total_units;
-    uint32_t next_range;   // ranges of the cost axis handed out beyond every block's first one (see kSmallRanges)
+    uint32_t next_range;   // ranges handed out beyond every block's first one (the first job's header counts for a launch)
     uint32_t done_blocks;  // blocks of the running gather that took their last range; the last one clears both counters
     uint32_t pad[10];
 };
-// The cost axis of the staged units is cut into ranges: one large range per block of the gather over the first
-// half (taken by block index), then kSmallRanges small ones per block over the second half, handed out through a
-// counter as blocks come free - units differ in cost per byte, and the small ranges even that out.
-constexpr uint32_t kSmallRanges = 4;
-__host__ __device__ inline uint32_t rebuild_ranges(uint32_t n_blocks) { return n_blocks * (1 + kSmallRanges); }
+// The cost axis of the staged units of a variant is cut into kRangesPerBlock equal ranges per block of the gather.
+// A launch rebuilds one or several variants; their ranges form one sequence, of which every block takes the one
+// with its own index first and then whatever a counter hands out as blocks come free - units differ in cost per
+// byte, and the small ranges even that out.
+constexpr uint32_t kRangesPerBlock = 6;
+__host__ __device__ inline uint32_t rebuild_ranges(uint32_t n_blocks) { return n_blocks * kRangesPerBlock; }
 __host__ __device__ inline uint32_t rebuild_range_lo(uint32_t r, uint32_t n_blocks, uint32_t total_cost) {
-    const uint64_t half = total_cost / 2;
-    if (r <= n_blocks) return (uint32_t)(half * r / n_blocks);
-    return (uint32_t)(half + (uint64_t)(total_cost - half) * (r - n_blocks) / ((uint64_t)kSmallRanges * n_blocks));
+    return (uint32_t)((uint64_t)total_cost * r / rebuild_ranges(n_blocks));
 }
 // One prepared layout in the workspace.
 struct RebuildSlot {
@@ -129,6 +128,22 @@ struct RebuildSlot {
     uint32_t* unit_item;       // [max_units] the item of every unit of the element path
 };
 constexpr uint32_t kVecPiece = 256;  // rows of a vector item that one warp of the gather copies
+// One variant of a gather launch.
+struct GatherJob {
+    RebuildSlot lay;
+    const char* src_arena;   // masked arena to read, NULL: the model's own tensors
+    const int32_t* keep_idx;
+    char* dst_arena;
+    uint64_t dst_bytes;
+    uint64_t* dst_offsets;
+    int32_t* dst_shapes;
+    int32_t variant;         // masking rebuild: variant of the threshold call
+    int32_t pad;
+};
+struct GatherBatch {
+    int32_t n, pad;
+    GatherJob job[DNNS_PORTFOLIO_MAX];
+};
 constexpr int kLayoutBatch = 8;  // layouts one launch of the layout kernel prepares
 struct LayoutBatch {
     const int32_t* keep_count[kLayoutBatch];
@@ -242,9 +257,7 @@ int launch_propagate_cascade(const Tables& tb, const CascadeWs& cw, const uint32
                              int32_t* keep_count, uint64_t* stats, uint32_t n_keep_words, uint32_t n_live_words, int n_sm,
                              cudaStream_t st);
 int launch_rebuild_layout(const Tables& tb, const LayoutBatch& lb, int n_layouts, int n_sm, cudaStream_t st);
-int launch_compact(const Tables& tb, const RebuildSlot& slot, const void* src_arena, const int32_t* keep_idx,
-                   void* dst_arena, uint64_t dst_bytes, uint64_t* dst_offsets, int32_t* dst_shapes, int n_sm,
-                   cudaStream_t st, const dnns_threshold* thr = nullptr, int variant = 0,
+int launch_compact(const Tables& tb, const GatherBatch& gb, int n_sm, cudaStream_t st, const dnns_threshold* thr = nullptr,
                    const TieSplit* split = nullptr);
 int gather_grid(int n_sm);  // blocks of the gather kernel (the layout is cut for this many)
 int launch_extrema(const Tables& tb, uint32_t* rowmax, uint32_t* colmax, int n_sm, cudaStream_t st);

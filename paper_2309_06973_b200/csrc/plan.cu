@@ -798,27 +798,57 @@ dnns_status dnns_propagate_keep_cascade(dnns_plan* p, const uint32_t* nz_map, ui
     return DNNS_OK;
 }
 
+// The rebuild of n variants in one launch.  masked_arenas NULL: from the dense model, masking on the way (thr_dev set).
+static dnns_status rebuild_variants(dnns_plan* p, int n, const void* const* masked_arenas, const dnns_threshold* thr_dev,
+                                    int32_t first_variant, const int32_t* const* keep_idx, const int32_t* const* keep_count,
+                                    void* const* dst_arena, size_t dst_bytes, uint64_t* const* dst_offsets,
+                                    int32_t* const* dst_shapes, void* stream) {
+    for (int i = 0; i < n; ++i) {
+        if (!keep_idx[i] || !keep_count[i] || !dst_arena[i] || !dst_offsets[i] || !dst_shapes[i]) return DNNS_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(dst_arena[i]) & (kAlign - 1)) return DNNS_ERR_INVALID_ARG;
+        if (masked_arenas && masked_arenas[i] && (reinterpret_cast<uintptr_t>(masked_arenas[i]) & 15)) return DNNS_ERR_INVALID_ARG;
+        for (int j = 0; j < i; ++j)  // every variant has outputs of its own
+            if (dst_arena[j] == dst_arena[i] || dst_offsets[j] == dst_offsets[i] || dst_shapes[j] == dst_shapes[i] ||
+                keep_count[j] == keep_count[i])
+                return DNNS_ERR_INVALID_ARG;
+    }
+    ProfileScope profile_scope(p);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // counts that no dnns_propagate_keep* call of this plan wrote are laid out now
+    std::vector<const int32_t*> missing;
+    for (int i = 0; i < n; ++i)
+        if (find_layout(p, keep_count[i]) < 0) missing.push_back(keep_count[i]);
+    int nl = 0;
+    if (!missing.empty() && (nl = prepare_layouts(p, missing.data(), (int)missing.size(), st)) < 0) return DNNS_ERR_CUDA;
+    GatherBatch gb{};
+    gb.n = n;
+    for (int i = 0; i < n; ++i) {
+        const int slot = find_layout(p, keep_count[i]);
+        if (slot < 0) return DNNS_ERR_INVALID_ARG;  // more distinct count arrays in one call than layouts can be held
+        GatherJob& job = gb.job[i];
+        job.lay = layout_slot(p, (uint32_t)slot);
+        job.src_arena = masked_arenas ? static_cast<const char*>(masked_arenas[i]) : nullptr;
+        job.keep_idx = keep_idx[i];
+        job.dst_arena = static_cast<char*>(dst_arena[i]);
+        job.dst_bytes = dst_bytes;
+        job.dst_offsets = dst_offsets[i];
+        job.dst_shapes = dst_shapes[i];
+        job.variant = first_variant + i;
+    }
+    const int k = launch_compact(p->tb, gb, p->n_sm, st, thr_dev, thr_dev ? p->tws.split : nullptr);
+    if (k < 0) return DNNS_ERR_CUDA;
+    p->launches += k + nl;
+    return DNNS_OK;
+}
+
 dnns_status dnns_compact(dnns_plan* p, const void* masked_arena, const int32_t* keep_idx, const int32_t* keep_count,
                          void* dst_arena, size_t dst_bytes, uint64_t* dst_offsets_dev, int32_t* dst_shapes_dev,
                          void* stream) {
     Range nvtx_range("dnns: step 5 rebuild");
     if (!p || !keep_idx || !keep_count || !dst_arena || !dst_offsets_dev || !dst_shapes_dev) return DNNS_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) ||
-        (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)))
-        return DNNS_ERR_INVALID_ARG;
-    ProfileScope profile_scope(p);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int nl = 0, slot = find_layout(p, keep_count);
-    if (slot < 0) {  // counts that no dnns_propagate_keep* call of this plan wrote: lay them out now
-        const int32_t* kc[1] = {keep_count};
-        if ((nl = prepare_layouts(p, kc, 1, st)) < 0) return DNNS_ERR_CUDA;
-        slot = find_layout(p, keep_count);
-    }
-    const int n = launch_compact(p->tb, layout_slot(p, (uint32_t)slot), masked_arena, keep_idx, dst_arena, dst_bytes,
-                                 dst_offsets_dev, dst_shapes_dev, p->n_sm, st);
-    if (n < 0) return DNNS_ERR_CUDA;
-    p->launches += n + nl;
-    return DNNS_OK;
+    const void* arenas[1] = {masked_arena};
+    return rebuild_variants(p, 1, arenas, nullptr, 0, &keep_idx, &keep_count, &dst_arena, dst_bytes, &dst_offsets_dev,
+                            &dst_shapes_dev, stream);
 }
 
 dnns_status dnns_compact_masked(dnns_plan* p, const dnns_threshold* thr_dev, int32_t variant,
@@ -828,20 +858,20 @@ dnns_status dnns_compact_masked(dnns_plan* p, const dnns_threshold* thr_dev, int
     if (!p || !thr_dev || !keep_idx || !keep_count || !dst_arena || !dst_offsets_dev || !dst_shapes_dev ||
         variant < 0 || variant >= p->last_n_k)
         return DNNS_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) return DNNS_ERR_INVALID_ARG;
-    ProfileScope profile_scope(p);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int nl = 0, slot = find_layout(p, keep_count);
-    if (slot < 0) {
-        const int32_t* kc[1] = {keep_count};
-        if ((nl = prepare_layouts(p, kc, 1, st)) < 0) return DNNS_ERR_CUDA;
-        slot = find_layout(p, keep_count);
-    }
-    const int n = launch_compact(p->tb, layout_slot(p, (uint32_t)slot), nullptr, keep_idx, dst_arena, dst_bytes,
-                                 dst_offsets_dev, dst_shapes_dev, p->n_sm, st, thr_dev, variant, p->tws.split);
-    if (n < 0) return DNNS_ERR_CUDA;
-    p->launches += n + nl;
-    return DNNS_OK;
+    return rebuild_variants(p, 1, nullptr, thr_dev, variant, &keep_idx, &keep_count, &dst_arena, dst_bytes,
+                            &dst_offsets_dev, &dst_shapes_dev, stream);
+}
+
+dnns_status dnns_compact_masked_multi(dnns_plan* p, const dnns_threshold* thr_dev, int32_t first_variant,
+                                      int32_t n_variants, const int32_t* const* keep_idx,
+                                      const int32_t* const* keep_count, void* const* dst_arenas, size_t dst_bytes,
+                                      uint64_t* const* dst_offsets_dev, int32_t* const* dst_shapes_dev, void* stream) {
+    Range nvtx_range("dnns: steps 2+5 rebuild from the dense model, several variants");
+    if (!p || !thr_dev || !keep_idx || !keep_count || !dst_arenas || !dst_offsets_dev || !dst_shapes_dev || n_variants < 1 ||
+        n_variants > kPortfolioMax || first_variant < 0 || first_variant + n_variants > p->last_n_k)
+        return DNNS_ERR_INVALID_ARG;
+    return rebuild_variants(p, n_variants, nullptr, thr_dev, first_variant, keep_idx, keep_count, dst_arenas, dst_bytes,
+                            dst_offsets_dev, dst_shapes_dev, stream);
 }
 
 dnns_status dnns_fold_batchnorm(dnns_plan* p, void* dst_arena, const uint64_t* dst_offsets_dev,

@@ -77,9 +77,10 @@ class Session:
     """A plan with its workspace and one set of output buffers for one variant at a time."""
 
     def __init__(self, dm: DeviceModel, scope: int, max_variants: int, want_mask_bits: bool = True,
-                 want_nz_map: bool = True, slots: int = 1, portfolio_slots: int = 0):
+                 want_nz_map: bool = True, slots: int = 1, portfolio_slots: int = 0, portfolio_arenas: bool = False):
         """slots > 1 adds that many more sets of per-variant buffers for the multi-variant sweep;
-        portfolio_slots adds sets of flags and keep sets only (no sparse model) for the portfolio-wide calls."""
+        portfolio_slots adds sets of flags and keep sets only (no sparse model) for the portfolio-wide calls;
+        portfolio_arenas gives each of those a destination arena of its own (rebuild of all variants in one launch)."""
         self.dm, self.scope, self.max_variants, self.slots = dm, scope, max_variants, slots
         dev = dm.device
         nbytes = B.dnns_workspace_bytes(dm.c, scope, max_variants)
@@ -124,6 +125,11 @@ class Session:
         self.stats_multi = torch.zeros(4 * max(slots, portfolio_slots, 1), dtype=torch.int64, device=dev)
         self.pf = [{"out_nz": i32(L.out_nz_words), "in_nz": i32(L.in_nz_words), "keep_bits": i32(L.keep_words),
                     "keep_idx": i32(L.keep_idx_len), "keep_count": i32(G)} for _ in range(portfolio_slots)]
+        if portfolio_arenas:
+            for slot in self.pf:
+                slot["arena"] = torch.empty(int(L.compact_arena_bytes), dtype=torch.uint8, device=dev)
+                slot["dst_offsets"] = torch.zeros(L.n_compact_items, dtype=torch.int64, device=dev)
+                slot["dst_shapes"] = i32(2 * T)
 
     def _slot(self, name: str, slot: int):
         return getattr(self, name) if slot == 0 else self.extra[slot - 1][name]
@@ -224,6 +230,13 @@ class Session:
                               self.pf[slot]["keep_count"].data_ptr(), arena.data_ptr(), arena.numel(),
                               self.dst_offsets.data_ptr(), self.dst_shapes.data_ptr(), _stream())
 
+    def compact_portfolio_multi(self, first_variant: int, n_variants: int):
+        """Rebuild variants first_variant .. from the dense model in one launch, slot i into its own arena."""
+        ptrs = lambda name: [self.pf[i][name].data_ptr() for i in range(n_variants)]
+        B.dnns_compact_masked_multi(self.plan, self.thr.data_ptr(), first_variant, n_variants, ptrs("keep_idx"),
+                                    ptrs("keep_count"), ptrs("arena"), self.pf[0]["arena"].numel(), ptrs("dst_offsets"),
+                                    ptrs("dst_shapes"), _stream())
+
     def propagate_keep_cascade(self, policy: int = B.DNNS_RULE_PRODUCER | B.DNNS_RULE_CONSUMER, min_keep: int = 1,
                                max_passes: int = 8):
         B.dnns_propagate_keep_cascade(self.plan, self.nz_map.data_ptr(), policy, min_keep, max_passes,
@@ -303,14 +316,16 @@ class Session:
         st = self.stats_multi[4 * slot: 4 * slot + 4] if multi_stats else self.stats
         return bits, idx, cnt, st.cpu().numpy().view(np.uint64).copy()
 
-    def compacted(self, keep_slot: int = 0, portfolio: bool = False):
+    def compacted(self, keep_slot: int = 0, portfolio: bool = False, own_arena: bool = False):
         """(weights [(O', I', KH, KW)], bn [(g, b, m, v)], biases, shapes (T, 2), offsets) of the variant rebuilt
         last; keep_slot: the slot whose keep sets it was rebuilt from."""
         wl, eb = self.dm.wl, self.dm.elem_bytes
         T = len(wl.tensors)
-        offs = self.dst_offsets.cpu().numpy().view(np.uint64)
-        shapes = self.dst_shapes.cpu().numpy()[: 2 * T].reshape(T, 2).copy()
-        raw = self.compact_arena.cpu().numpy()
+        src = self.pf[keep_slot] if own_arena else {"dst_offsets": self.dst_offsets, "dst_shapes": self.dst_shapes,
+                                                      "arena": self.compact_arena}
+        offs = src["dst_offsets"].cpu().numpy().view(np.uint64)
+        shapes = src["dst_shapes"].cpu().numpy()[: 2 * T].reshape(T, 2).copy()
+        raw = src["arena"].cpu().numpy()
         ws = []
         for i, t in enumerate(wl.tensors):
             On, In = int(shapes[i, 0]), int(shapes[i, 1])

@@ -100,16 +100,19 @@ def compare_portfolio(wl, dtype=B.DNNS_F32, variants=None, policy=O.RULE_PRODUCE
     return ses
 
 
-def compare_sparse_free(wl, dtype=B.DNNS_F32, policy=O.RULE_PRODUCER | O.RULE_CONSUMER, min_keep=1, weights=None):
+def compare_sparse_free(wl, dtype=B.DNNS_F32, policy=O.RULE_PRODUCER | O.RULE_CONSUMER, min_keep=1, weights=None,
+                        one_launch=False):
     """The portfolio without any sparse model: thresholds once, the zero structures of every variant from one sweep
     over the dense weights (dnns_zero_structures_portfolio), keep sets of all variants in one launch, then a masking
-    rebuild per variant (dnns_compact_masked).  Flags, keep sets, statistics and every rebuilt item are compared
+    rebuild per variant (dnns_compact_masked; one_launch: of all variants of a call at once, each into an arena of
+    its own, dnns_compact_masked_multi).  Flags, keep sets, statistics and every rebuilt item are compared
     with the oracle's step-by-step result (mask, zero structures, keep propagation, compaction)."""
     om = O.OracleModel(wl, dtype, weights)
     dm = DeviceModel(wl, dtype, weights=weights)
     V = len(wl.ks)
     per_call = min(V, B.DNNS_PORTFOLIO_MAX)
-    ses = Session(dm, wl.scope, V, want_mask_bits=False, want_nz_map=False, portfolio_slots=per_call)
+    ses = Session(dm, wl.scope, V, want_mask_bits=False, want_nz_map=False, portfolio_slots=per_call,
+                  portfolio_arenas=one_launch)
     ses.magnitude_threshold(wl.ks)
     rec_gpu, rec_cpu = ses.records(), O.threshold(om, wl.scope, wl.ks)
     for f in ("tau_bits", "n_below", "n_tie", "n_equal"):
@@ -119,9 +122,12 @@ def compare_sparse_free(wl, dtype=B.DNNS_F32, policy=O.RULE_PRODUCER | O.RULE_CO
         n = min(per_call, V - v0)
         ses.zero_structures_portfolio(v0, n)
         ses.propagate_keep_portfolio(n, policy, min_keep)
+        if one_launch:
+            ses.compact_portfolio_multi(v0, n)
         for s in range(n):
             v = v0 + s
-            ses.compact_portfolio(v, s)
+            if not one_launch:
+                ses.compact_portfolio(v, s)
             assert ses.device_status() == B.DNNS_OK
             masked_cpu, _ = O.apply_mask(om, wl.scope, rec_cpu[v])
             _, out_c, in_c = O.zero_structures(masked_cpu)
@@ -136,7 +142,7 @@ def compare_sparse_free(wl, dtype=B.DNNS_F32, policy=O.RULE_PRODUCER | O.RULE_CO
                 assert np.array_equal(a, b[: kc_c[g]]), f"keep idx v{v} group {g}"
             assert st_g.tolist() == st_c.tolist(), f"stats v{v}"
             cw_c, cbn_c, cb_c, sh_c = O.compact(masked_cpu, ki_c, kc_c)
-            cw_g, cbn_g, cb_g, sh_g, offs = ses.compacted(s, portfolio=True)
+            cw_g, cbn_g, cb_g, sh_g, offs = ses.compacted(s, portfolio=True, own_arena=one_launch)
             assert np.array_equal(sh_g, sh_c), f"shapes v{v}"
             for i, (a, b) in enumerate(zip(cw_g, cw_c)):
                 assert bits_eq(a, b), f"compacted weights v{v} tensor {i}"

@@ -32,7 +32,7 @@ def forward_check_sparse_free(wl, ses, dtype):
     removed channels silenced."""
     is_bf16 = dtype == B.DNNS_BF16
     x = torch.from_numpy(np.random.default_rng(1).standard_normal((2, 3, wl.input_hw, wl.input_hw)).astype(np.float32))
-    cw, cbn, cb, _, _ = ses.compacted(ses.last_slot, portfolio=True)
+    cw, cbn, cb, _, _ = ses.compacted(ses.last_slot, portfolio=True, own_arena="arena" in ses.pf[ses.last_slot])
     kb, _, _, _ = ses.keep_sets(ses.last_slot, portfolio=True)
     mw, mbn, mb = silenced_reference(wl, ses.last_masked, wl.bn_params, wl.biases, kb)
     y_ref = forward(wl, mw, mbn, mb, x, is_bf16)
@@ -82,5 +82,6 @@ def test_resnet152_portfolio_sparse_free(dtype):
     """The benchmark's own configuration: all eight variants, zero structures from one sweep, keep sets in one
     launch, masking rebuild per variant."""
     wl = W.resnet152()
-    ses = compare_sparse_free(wl, dtype)
+    ses = compare_sparse_free(wl, dtype, one_launch=True)      # the eight rebuilds in one launch, as the benchmark runs them
     forward_check_sparse_free(wl, ses, dtype)
+    compare_sparse_free(wl, dtype)                             # ... and one launch per variant

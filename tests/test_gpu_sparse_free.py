@@ -18,6 +18,7 @@ pytestmark = pytest.mark.gpu
                                   W.resnet56])
 def test_small_configs_every_variant(make, dtype):
     compare_sparse_free(make(), dtype)
+    compare_sparse_free(make(), dtype, one_launch=True)     # all variants rebuilt by one launch
 
 
 @pytest.mark.parametrize("policy", [O.RULE_PRODUCER, O.RULE_CONSUMER, O.RULE_PRODUCER | O.RULE_CONSUMER | O.SHIFT_STRICT])
@@ -40,6 +41,7 @@ def test_per_tensor_scope_and_odd_shapes(dtype):
     wl.ks = np.array([[0] * len(sizes), [n // 2 for n in sizes], [n * 9 // 10 for n in sizes],
                       [n - 1 for n in sizes], sizes], np.uint64)
     compare_sparse_free(wl, dtype)
+    compare_sparse_free(wl, dtype, one_launch=True)
 
 
 def test_non_prunable_tensor_and_1x1_chain():
@@ -73,6 +75,7 @@ def test_special_values_and_heavy_ties():
     rec = ses.records()
     assert (rec["n_tie"] < rec["n_equal"]).any()                   # the equal weights really split
     compare_sparse_free(wl, B.DNNS_BF16)
+    compare_sparse_free(wl, B.DNNS_BF16, one_launch=True)
 
 
 def test_filters_whose_largest_weight_equals_the_threshold():
@@ -96,6 +99,7 @@ def test_more_variants_than_one_call_takes():
     n = wl.n_prunable
     wl.ks = np.array([[n * (i + 1) // 21] for i in range(20)], np.uint64)
     compare_sparse_free(wl, B.DNNS_F32)
+    compare_sparse_free(wl, B.DNNS_F32, one_launch=True)
 
 
 def test_fc_with_spatial_columns():
