@@ -429,7 +429,10 @@ const char* dnns_status_string(dnns_status s);
  * whose device memory was fully handed out at start-up.  Such callers own the weights and the
  * result record but cannot supply the workspace a plan needs, so the histograms and tables live
  * in a fixed array inside the library (about 0.6 MB, held by every GPU that loads the library
- * until the process exits).  The call makes no allocation of any kind, on device or host.
+ * until the process exits).  Apart from the first call on a device (below), a call makes no allocation of any
+ * kind, on device or host: it enqueues one memset, one one-thread kernel that stores the call's descriptors
+ * (they travel as kernel arguments, so a captured call replays with the arguments it was captured with) and the
+ * kernels of the threshold step.
  *
  * weights_dev: device, 16-byte aligned, numel elements of dtype (DNNS_F32 / DNNS_BF16), treated as
  * one ranking segment in index order.  k: how many weights to mask, 0 <= k <= numel.  thr_dev:
@@ -437,8 +440,10 @@ const char* dnns_status_string(dnns_status s);
  * Limits and errors: numel > DNNS_STATIC_MAX_NUMEL returns DNNS_ERR_STATIC_LIMIT and launches
  * nothing; INVALID_ARG (null or misaligned pointer, numel == 0, k > numel), UNSUPPORTED (dtype,
  * device ordinal above 63), CUDA.
- * The first call on each device resolves the array's device address and clears it; make that
- * first call outside any stream capture.  All calls on a device share the one array and each call
+ * The first call on each device resolves the array's device address; it is also the moment at which the CUDA
+ * runtime loads this library's device code and places the array, so make that call at start-up, before the
+ * allocator is locked (k = 0 on any small buffer will do), and outside any stream capture: a first call on a
+ * capturing stream returns DNNS_ERR_UNSUPPORTED and enqueues nothing.  All calls on a device share the one array and each call
  * clears the parts it needs at its start: calls that overlap on the GPU (different streams
  * without ordering between them) race on it and give wrong results; order them on one stream.
  */

@@ -28,15 +28,7 @@ namespace {
 constexpr int kThreads = 256;
 constexpr uint32_t kUnitBytes = 16384;
 
-// Checked build (-DDNNS_BOUNDS_CHECK, a second library used by the tests only): every index that depends on
-// data - keep lists, source elements, mask bits - is compared with its extent first; a violation is counted
-// and the access goes to element 0 instead, so nothing faults.  The normal build compiles the checks away.
-#ifdef DNNS_BOUNDS_CHECK
-__device__ unsigned int g_bounds_violations = 0;
-#define DNNS_IDX(i, n) ((uint32_t)(i) < (uint32_t)(n) ? (uint32_t)(i) : (atomicAdd(&g_bounds_violations, 1u), 0u))
-#else
-#define DNNS_IDX(i, n) (i)
-#endif
+DNNS_BOUNDS_COUNTER  // (checked build: index violations counted in this file)
 
 template <int BYTES>
 __device__ __forceinline__ uint32_t load_elem(const void* base, uint32_t idx) {
@@ -970,6 +962,6 @@ extern "C" unsigned int dnns_check_bounds_violations() {
     if (cudaDeviceSynchronize() != cudaSuccess || cudaMemcpyFromSymbol(&n, dnns::g_bounds_violations, sizeof(n)) != cudaSuccess)
         return 0xFFFFFFFFu;
     cudaMemcpyToSymbol(dnns::g_bounds_violations, &zero, sizeof(zero));
-    return n;
+    return n + dnns::bounds_violations_sweep(true) + dnns::bounds_violations_propagate(true);
 }
 #endif

@@ -270,6 +270,20 @@ cudaError_t init_compact_attributes();
 constexpr uint32_t kGatherStageBytes = 18432;  // one stage buffer of the staged rebuild
 constexpr uint32_t kGatherPieceBytes = 2304;   // longest piece of a row in a unit (64 channels of a 3x3 fp32 filter)
 
+// ---- checked build (-DDNNS_BOUNDS_CHECK, a second library used by the tests only): indices into keep lists, source
+// elements, bit arrays and flag words are compared with their extent first; a violation is counted (one counter per
+// source file, summed by dnns_check_bounds_violations) and the access goes to element 0 instead, so nothing faults.
+// The normal build compiles the checks away.
+#ifdef DNNS_BOUNDS_CHECK
+#define DNNS_BOUNDS_COUNTER __device__ unsigned int g_bounds_violations = 0;
+#define DNNS_IDX(i, n) ((uint32_t)(i) < (uint32_t)(n) ? (uint32_t)(i) : (atomicAdd(&g_bounds_violations, 1u), 0u))
+unsigned int bounds_violations_sweep(bool reset);      // counters of the other source files (compact.cu holds its own)
+unsigned int bounds_violations_propagate(bool reset);
+#else
+#define DNNS_BOUNDS_COUNTER
+#define DNNS_IDX(i, n) (i)
+#endif
+
 // ---- small device helpers ----
 template <int DT>
 struct Elem;

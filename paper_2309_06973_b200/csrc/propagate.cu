@@ -13,6 +13,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kMaxGroupWords = 65536 / 32;
+DNNS_BOUNDS_COUNTER  // (checked build: index violations counted in this file)
 
 __device__ __forceinline__ bool get_bit(const uint32_t* w, uint32_t b) { return (w[b >> 5] >> (b & 31)) & 1u; }
 
@@ -231,7 +232,7 @@ __global__ void __launch_bounds__(256) k_live(Tables tb, const uint32_t* __restr
             for (; unit < run_end; ++unit) {
                 const uint32_t local = unit - t_begin, rb = local / n_chunks, cc = local - rb * n_chunks;
                 const uint32_t row0 = rb * kFlagRows, iw = cc * 32 + (lane & (cw - 1));
-                const uint32_t kept_cols = ~rem_in[iw];
+                const uint32_t kept_cols = ~rem_in[DNNS_IDX(iw, (I / S + 31) / 32)];
                 uint32_t acc = 0, rows = 0;
                 const uint32_t n_steps = (kFlagRows * cw + 31) / 32;
                 const uint32_t group_mask = cw == 32 ? 0xffffffffu : ((1u << cw) - 1u);
@@ -262,7 +263,7 @@ __global__ void __launch_bounds__(256) k_live(Tables tb, const uint32_t* __restr
                 const uint32_t q_begin = (unit - t_begin) * per_unit, q_end = min(n_kernels, q_begin + per_unit);
                 for (uint32_t qb = q_begin; qb < q_end; qb += 32) {
                     const uint32_t q = qb + lane;
-                    if (q < q_end && ((map[q >> 5] >> (q & 31)) & 1u)) {
+                    if (q < q_end && ((map[DNNS_IDX(q >> 5, (n_kernels + 31) / 32)] >> (q & 31)) & 1u)) {
                         const uint32_t o = q / I, i = q - o * I, c = i / S;
                         if (!((rem_in[c >> 5] >> (c & 31)) & 1u)) atomicOr(&g_out[o >> 5], 1u << (o & 31));
                         if (!((rem_out[o >> 5] >> (o & 31)) & 1u)) atomicOr(&g_in[i >> 5], 1u << (i & 31));
@@ -371,5 +372,14 @@ int launch_propagate_cascade(const Tables& tb, const CascadeWs& cw, const uint32
                                                        reinterpret_cast<unsigned long long*>(stats));
     return cudaGetLastError() == cudaSuccess ? launches + 1 : -1;
 }
+
+#ifdef DNNS_BOUNDS_CHECK
+unsigned int bounds_violations_propagate(bool reset) {
+    unsigned int n = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&n, g_bounds_violations, sizeof(n)) != cudaSuccess) return 0xFFFFFFFFu;
+    if (reset) cudaMemcpyToSymbol(g_bounds_violations, &zero, sizeof(zero));
+    return n;
+}
+#endif
 
 }  // namespace dnns

@@ -21,6 +21,7 @@ namespace dnns {
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
+DNNS_BOUNDS_COUNTER  // (checked build: index violations counted in this file)
 
 // OR the per-lane bit groups (P bits each, lane order = element order) of 32/P neighbouring
 // lanes into one word; every lane of the group gets the word.
@@ -98,6 +99,8 @@ __global__ void __launch_bounds__(256) k_flags(Tables tb, const uint32_t* __rest
         const TensorDesc& d = tb.tensors[t];
         const uint32_t KK = d.KK, I = d.I, O = d.O, n_kernels = O * I;
         const uint32_t* ebits = ebits_all + d.off_mask;
+        const uint32_t n_ewords = (d.numel + 31) / 32, n_mwords = (n_kernels + 31) / 32;  // extents (checked build)
+        (void)n_ewords, (void)n_mwords;
         uint32_t* g_in = in_nz + d.off_innz;
         uint32_t* g_out = out_nz + d.off_outnz;
         uint32_t* g_map = nz_map ? nz_map + d.off_nzmap : nullptr;
@@ -123,15 +126,15 @@ __global__ void __launch_bounds__(256) k_flags(Tables tb, const uint32_t* __rest
                         const uint32_t gw = o * wpr + iw;  // this lane's word of the kernel map
                         uint32_t word = 0;
                         if (KK == 1) {
-                            word = __ldg(ebits + gw);
+                            word = __ldg(ebits + DNNS_IDX(gw, n_ewords));
                         } else if (KK == 9) {
-                            word = kernel_word_3x3(ebits + (size_t)gw * 9);
+                            word = kernel_word_3x3(ebits + (DNNS_IDX(gw * 9 + 8, n_ewords) == gw * 9 + 8 ? (size_t)gw * 9 : (size_t)0));
                         } else {
                             const uint32_t q0 = gw * 32;
                             for (uint32_t j = 0; j < 32; ++j)
                                 word |= (uint32_t)any_bits(ebits, (q0 + j) * KK, (q0 + j + 1) * KK) << j;
                         }
-                        if (g_map) g_map[gw] = word;
+                        if (g_map) g_map[DNNS_IDX(gw, n_mwords)] = word;
                         words[step] = word;
                     }
                     acc |= words[step];
@@ -147,9 +150,9 @@ __global__ void __launch_bounds__(256) k_flags(Tables tb, const uint32_t* __rest
                         if ((nzl >> (g << cw_shift)) & group_mask) rows |= 1u << (((step * 32) >> cw_shift) + g);
                 }
                 // kFlagRows divides 32, so the filters of a unit share one flag word
-                if (lane == 0 && rows) or_if_missing(&g_out[row0 >> 5], rows << (row0 & 31));
+                if (lane == 0 && rows) or_if_missing(&g_out[DNNS_IDX(row0 >> 5, (O + 31) / 32)], rows << (row0 & 31));
                 for (uint32_t sft = cw; sft < 32; sft <<= 1) acc |= __shfl_xor_sync(kFull, acc, sft);
-                if ((uint32_t)lane < cw && acc) or_if_missing(&g_in[iw], acc);
+                if ((uint32_t)lane < cw && acc) or_if_missing(&g_in[DNNS_IDX(iw, (I + 31) / 32)], acc);
             }
         } else {
             // one kernel per lane, every kernel sets its own two flags
@@ -157,11 +160,11 @@ __global__ void __launch_bounds__(256) k_flags(Tables tb, const uint32_t* __rest
                 const uint32_t q = (unit - t_begin) * 32 + lane;
                 const bool bit = q < n_kernels && any_bits(ebits, q * KK, (q + 1) * KK);
                 const uint32_t word = __ballot_sync(kFull, bit);
-                if (lane == 0 && g_map) g_map[unit - t_begin] = word;
+                if (lane == 0 && g_map) g_map[DNNS_IDX(unit - t_begin, n_mwords)] = word;
                 if (bit) {
                     const uint32_t o = q / I, i = q - o * I;
-                    or_if_missing(&g_in[i >> 5], 1u << (i & 31));
-                    or_if_missing(&g_out[o >> 5], 1u << (o & 31));
+                    or_if_missing(&g_in[DNNS_IDX(i >> 5, (I + 31) / 32)], 1u << (i & 31));
+                    or_if_missing(&g_out[DNNS_IDX(o >> 5, (O + 31) / 32)], 1u << (o & 31));
                 }
             }
         }
@@ -652,5 +655,14 @@ int launch_multi_sweep(const Tables& tb, const ThresholdWs& ws, const dnns_thres
     }
     return cudaGetLastError() == cudaSuccess ? 1 + n_variants : -1;
 }
+
+#ifdef DNNS_BOUNDS_CHECK
+unsigned int bounds_violations_sweep(bool reset) {
+    unsigned int n = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&n, g_bounds_violations, sizeof(n)) != cudaSuccess) return 0xFFFFFFFFu;
+    if (reset) cudaMemcpyToSymbol(g_bounds_violations, &zero, sizeof(zero));
+    return n;
+}
+#endif
 
 }  // namespace dnns

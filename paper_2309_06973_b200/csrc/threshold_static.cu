@@ -12,6 +12,7 @@
 // loads the library holds these ~0.6 MB until the process exits.  Host code must not pass the
 // array's name to a kernel (on the host that name is only a stand-in for the symbol); the device
 // address is obtained once per device with cudaGetSymbolAddress and handed to the kernels.
+#include <atomic>
 #include <mutex>
 
 #include "dnns_internal.cuh"
@@ -28,6 +29,7 @@ constexpr size_t kOffTensor = 0;                                  // TensorDesc[
 constexpr size_t kOffSeg = 256;                                   // SegDesc[1]
 constexpr size_t kOffK = 512;                                     // uint64 k
 constexpr size_t kOffSel = 768;                                   // SelectState[1]
+constexpr size_t kOffSplit = 896;                                 // TieSplit[1]
 constexpr size_t kOffBitmap = 1024;                               // kBitmapWords words
 constexpr size_t kOffTileTensor = kOffBitmap + 4 * kBitmapWords;  // kMaxTiles words, always zero (tensor 0)
 constexpr size_t kOffTiePrefix = kOffTileTensor + 4 * (size_t)kMaxTiles;
@@ -45,23 +47,32 @@ static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 64;
 std::mutex g_mutex;
-unsigned char* g_scratch_ptr[kMaxDevices] = {};  // device address of the array, per device ordinal
-int g_n_sm[kMaxDevices] = {};
+std::atomic<unsigned char*> g_scratch_ptr[kMaxDevices];  // device address of the array, per device ordinal
+int g_n_sm[kMaxDevices] = {};                            // written before the pointer is published
 
-// One-time set-up on the current device: resolve the device address of the scratch array, zero
-// the part that stays constant, raise the shared-memory limit of the histogram kernel.
-dnns_status setup_device(int dev, cudaStream_t st) {
+// One-time set-up on the current device: resolve the device address of the scratch array and raise the
+// shared-memory limit of the histogram kernel.  (A __device__ array without an initialiser starts as zeros, which
+// is what the constant sections of the scratch - the tile -> tensor table - rely on.)  Loading the library's
+// device code, which the first CUDA call of a process into this library triggers, happens here too.
+dnns_status setup_device(int dev) {
+    if (g_scratch_ptr[dev].load(std::memory_order_acquire)) return DNNS_OK;
     std::lock_guard<std::mutex> lock(g_mutex);
-    if (g_scratch_ptr[dev]) return DNNS_OK;
+    if (g_scratch_ptr[dev].load(std::memory_order_relaxed)) return DNNS_OK;
     unsigned char* p = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_scratch) != cudaSuccess || !p) return DNNS_ERR_CUDA;
     int n_sm = 0;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DNNS_ERR_CUDA;
     if (init_kernel_attributes() != cudaSuccess) return DNNS_ERR_CUDA;
-    if (cudaMemsetAsync(p, 0, kScratchBytes, st) != cudaSuccess) return DNNS_ERR_CUDA;
     g_n_sm[dev] = n_sm;
-    g_scratch_ptr[dev] = p;
+    g_scratch_ptr[dev].store(p, std::memory_order_release);
     return DNNS_OK;
+}
+
+// The descriptors of the call travel as kernel arguments (copied when the launch is enqueued - or captured - not
+// when it runs) and are stored into the scratch by one thread.
+__global__ void k_static_descriptors(TensorDesc td, SegDesc sd, TensorDesc* td_out, SegDesc* sd_out) {
+    *td_out = td;
+    *sd_out = sd;
 }
 
 }  // namespace
@@ -77,9 +88,15 @@ extern "C" dnns_status dnns_magnitude_threshold_static(const void* weights_dev, 
     if (cudaGetDevice(&dev) != cudaSuccess) return DNNS_ERR_CUDA;
     if (dev < 0 || dev >= kMaxDevices) return DNNS_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const dnns_status s = setup_device(dev, st);
+    if (!g_scratch_ptr[dev].load(std::memory_order_acquire)) {
+        // the first call on a device resolves the array's address: not something a stream capture can record
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) return DNNS_ERR_CUDA;
+        if (cap != cudaStreamCaptureStatusNone) return DNNS_ERR_UNSUPPORTED;
+    }
+    const dnns_status s = setup_device(dev);
     if (s != DNNS_OK) return s;
-    unsigned char* base = g_scratch_ptr[dev];
+    unsigned char* base = g_scratch_ptr[dev].load(std::memory_order_acquire);
 
     const uint32_t elem_bytes = dtype == DNNS_F32 ? 4 : 2;
     const uint32_t n_tiles = (uint32_t)((numel * elem_bytes + kTileBytes - 1) / kTileBytes);
@@ -95,10 +112,10 @@ extern "C" dnns_status dnns_magnitude_threshold_static(const void* weights_dev, 
     const SegDesc sd{0, n_tiles, numel};
 
     // what must start at zero: histograms, tie tables and flags of the previous call
-    if (cudaMemsetAsync(base + kOffClear, 0, kScratchBytes - kOffClear, st) != cudaSuccess ||
-        cudaMemcpyAsync(base + kOffTensor, &td, sizeof(td), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(base + kOffSeg, &sd, sizeof(sd), cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return DNNS_ERR_CUDA;
+    if (cudaMemsetAsync(base + kOffClear, 0, kScratchBytes - kOffClear, st) != cudaSuccess) return DNNS_ERR_CUDA;
+    k_static_descriptors<<<1, 1, 0, st>>>(td, sd, reinterpret_cast<TensorDesc*>(base + kOffTensor),
+                                          reinterpret_cast<SegDesc*>(base + kOffSeg));
+    if (cudaGetLastError() != cudaSuccess) return DNNS_ERR_CUDA;
 
     Tables tb{};
     tb.tensors = reinterpret_cast<const TensorDesc*>(base + kOffTensor);
@@ -118,5 +135,6 @@ extern "C" dnns_status dnns_magnitude_threshold_static(const void* weights_dev, 
     ws.any_need = reinterpret_cast<uint32_t*>(base + kOffAnyNeed);
     ws.tile_ties = reinterpret_cast<uint32_t*>(base + kOffTileTies);
     ws.tie_prefix = reinterpret_cast<uint32_t*>(base + kOffTiePrefix);
+    ws.split = reinterpret_cast<TieSplit*>(base + kOffSplit);
     return launch_threshold(tb, ws, 1, &k, thr_dev, g_n_sm[dev], st) < 0 ? DNNS_ERR_CUDA : DNNS_OK;
 }

@@ -9,7 +9,9 @@ import numpy as np
 sys.path.insert(0, __file__.rsplit("/", 2)[0])
 sys.path.insert(0, __file__.rsplit("/", 1)[0])
 
-from gpu_compare import compare_portfolio          # noqa: E402
+from gpu_compare import compare_portfolio, compare_sparse_free          # noqa: E402
+from oracle import oracle as O                     # noqa: E402
+from test_gpu_cascade import run_case              # noqa: E402
 from paper_2309_06973_b200 import binding as B     # noqa: E402
 from paper_2309_06973_b200 import workloads as W   # noqa: E402
 
@@ -28,6 +30,9 @@ def main():
             compare_portfolio(wl, dtype)
             compare_portfolio(wl, dtype, multi=2, multi_plan=True)
             compare_portfolio(wl, dtype, multi=3, no_store=True)
+            compare_sparse_free(wl, dtype)                          # no sparse model: flags from the maxima, masking rebuild
+            compare_sparse_free(wl, dtype, one_launch=True)
+            run_case(wl, dtype, len(wl.ks) - 1, O.RULE_PRODUCER | O.RULE_CONSUMER, 1, 8)   # fixed-point propagation
     print("violations", L.dnns_check_bounds_violations())
 
 

@@ -114,6 +114,8 @@ def test_null_plan_calls_return_invalid_arg():
     assert L.dnns_zero_structures(None, None, None, None, None, None) == B.DNNS_ERR_INVALID_ARG
     assert L.dnns_propagate_keep(None, None, None, 3, 1, None, None, None, None, None) == B.DNNS_ERR_INVALID_ARG
     assert L.dnns_compact(None, None, None, None, None, 0, None, None, None) == B.DNNS_ERR_INVALID_ARG
+    assert L.dnns_zero_structures_portfolio(None, None, 0, 1, None, None, None) == B.DNNS_ERR_INVALID_ARG
+    assert L.dnns_compact_masked_multi(None, None, 0, 1, None, None, None, 0, None, None, None) == B.DNNS_ERR_INVALID_ARG
     assert L.dnns_last_device_status(None, None) == B.DNNS_ERR_INVALID_ARG
     assert B.dnns_plan_launch_count(None) == 0
     assert B.dnns_status_string(B.DNNS_ERR_BAD_GRAPH) == "inconsistent model graph"

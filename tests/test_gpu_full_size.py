@@ -59,6 +59,13 @@ def test_resnet50_three_variants():
     forward_check_sparse_free(wl, ses, B.DNNS_F32)
 
 
+def test_resnet50_frozen_residual_streams():
+    """ResNet-50 as the paper prunes it: residual streams frozen (Section IV-B-2)."""
+    wl = W.freeze_streams(W.resnet50())
+    ses = compare_sparse_free(wl, B.DNNS_F32, one_launch=True)
+    forward_check_sparse_free(wl, ses, B.DNNS_F32)
+
+
 def test_resnet50_bf16_sparse_free():
     compare_sparse_free(W.resnet50(), B.DNNS_BF16)
 

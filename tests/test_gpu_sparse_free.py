@@ -114,3 +114,40 @@ def test_fc_with_spatial_columns():
     wl.biases[1][:] = np.arange(7)
     W._set_ks(wl, lambda n: [n // 2, n * 9 // 10])
     compare_sparse_free(wl, B.DNNS_F32)
+
+
+@pytest.mark.parametrize("make", [W.resnet56, lambda: W.small_resnet(seed=3)])
+def test_frozen_residual_streams(make):
+    """The paper's own setting (Section IV-B-2): skip connections and downsampling layers are left alone - every
+    group that several layers write is frozen, only plain layer-to-layer channels are pruned."""
+    from gpu_compare import compare_portfolio
+    wl = W.freeze_streams(make())
+    ses = compare_sparse_free(wl, B.DNNS_F32)
+    _, _, kc, _ = ses.keep_sets(ses.last_slot, portfolio=True)
+    for g, c in zip(wl.groups, kc):
+        if g.flags & W.GROUP_FROZEN:
+            assert c == g.C
+    compare_sparse_free(W.freeze_streams(make()), B.DNNS_BF16, one_launch=True)
+    compare_portfolio(W.freeze_streams(make()), B.DNNS_F32, multi=2, multi_plan=True)
+
+
+def test_variants_outside_the_latest_threshold_call_are_rejected():
+    from paper_2309_06973_b200.runtime import DeviceModel, Session
+    wl = W.toy()
+    dm = DeviceModel(wl, B.DNNS_F32)
+    ses = Session(dm, wl.scope, 4, portfolio_slots=4)
+    n = wl.n_prunable
+    ses.magnitude_threshold(np.array([[n // 2], [n // 3]], np.uint64))      # two of at most four variants
+    L = B.lib()
+    thr, s = ses.thr.data_ptr(), 0
+    assert L.dnns_apply_mask(ses.plan, thr, 2, ses.masked.data_ptr(), None, s) == B.DNNS_ERR_INVALID_ARG
+    assert L.dnns_mask_and_structures(ses.plan, thr, 3, ses.masked.data_ptr(), None, None, ses.out_nz.data_ptr(),
+                                      ses.in_nz.data_ptr(), s) == B.DNNS_ERR_INVALID_ARG
+    with pytest.raises(B.DnnsError):
+        ses.zero_structures_portfolio(1, 2)
+    with pytest.raises(B.DnnsError):
+        ses.compact_portfolio(2, 0)
+    ses.zero_structures_portfolio(0, 2)                                      # inside the call: fine
+    ses.propagate_keep_portfolio(2)
+    ses.compact_portfolio(1, 1)
+    assert ses.device_status() == B.DNNS_OK
