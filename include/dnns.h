@@ -189,8 +189,13 @@ dnns_status dnns_plan_profile_read(dnns_plan* plan, const char* kernel, double* 
  * indexing) receives the records.  One call serves the whole portfolio: the sweeps over the
  * weights are shared by all n_k counts.  The call also leaves, in the workspace, the per-tile
  * tie tables that dnns_apply_mask needs to mask exactly k weights when several weights equal
- * tau, and the place (tensor, element) where each variant stops masking them, which
- * dnns_compact_masked reads; both belong to this call's thr_dev.
+ * tau, the place (tensor, element) where each variant stops masking them, which
+ * dnns_compact_masked reads, and the largest key of every filter and every input column of every
+ * tensor, which dnns_zero_structures_portfolio reads (one more sweep over the weights, enqueued on a
+ * stream of the plan's own that forks from `stream` at the start of the call and joins it again at
+ * the end, so that it runs beside the ranking kernels; a call inside a stream capture records that
+ * fork and join as well).  All of these belong to this call's thr_dev and to the weights as they
+ * were during the call.
  * Errors: INVALID_ARG (null, n_k out of range, a k above its segment), CUDA.
  */
 dnns_status dnns_magnitude_threshold(dnns_plan* plan, const uint64_t* k, int32_t n_k, dnns_threshold* thr_dev,
@@ -252,11 +257,11 @@ dnns_status dnns_mask_and_structures_multi(dnns_plan* plan, const dnns_threshold
                                            void* stream);
 
 /*
- * Step 3 for up to DNNS_PORTFOLIO_MAX variants of the latest threshold call from ONE sweep over the dense
- * weights, without forming any sparse model.  Step 2 keeps a weight of variant v when its key lies above tau_v
+ * Step 3 for up to DNNS_PORTFOLIO_MAX variants of the latest threshold call without a sweep of its own and
+ * without forming any sparse model.  Step 2 keeps a weight of variant v when its key lies above tau_v
  * (or equals it and is not among the first n_tie such weights), so a filter or an input column still holds a
- * non-zero weight for v exactly when the largest key in it does: the sweep records the largest key of every
- * filter and every input column (in the workspace), and each variant's flags follow from comparing those with
+ * non-zero weight for v exactly when the largest key in it does: the threshold call recorded the largest key of
+ * every filter and every input column (in the workspace), and each variant's flags follow from comparing those with
  * its threshold; where a maximum equals tau in the tensor in which the variant's equal weights split, that one
  * filter or column is read again.  out_nz, in_nz: host arrays of n_variants device pointers, all distinct, each
  * as in dnns_zero_structures and bit for bit what dnns_apply_mask + dnns_zero_structures give for variant

@@ -1,5 +1,6 @@
 // Zero structures of a whole portfolio from ONE sweep over the dense weights (Module 2, the Sparsity
-// Analyser, for every variant at once).
+// Analyser, for every variant at once).  The sweep does not depend on the thresholds and is enqueued by the
+// threshold call, beside its ranking kernels; the flag kernel runs once the thresholds are known.
 //
 // Step 2 keeps a weight of variant v when its magnitude key lies above tau_v, or equals tau_v and the
 // weight comes at or after the place where v stops masking such weights.  A filter (row) of a tensor
@@ -24,20 +25,8 @@ namespace {
 constexpr unsigned kFull = 0xffffffffu;
 constexpr uint32_t kColTab = 8192;  // input columns of a tensor that fit the shared-memory table
 
-// Largest key among the elements of a vector (keys of elements past `n` are ignored).
 template <int DT>
-__device__ __forceinline__ uint32_t vec_max_key(const uint4& v, int n) {
-    constexpr int P = Elem<DT>::kPerVec;
-    uint32_t key[P];
-    vec_keys<DT>(v, key);
-    uint32_t m = 0;
-#pragma unroll
-    for (int j = 0; j < P; ++j) m = max(m, j < n ? key[j] : 0u);
-    return m;
-}
-
-template <int DT>
-__global__ void __launch_bounds__(kTileThreads, 4) k_extrema(Tables tb, uint32_t* __restrict__ rowmax, uint32_t* __restrict__ colmax) {
+__global__ void __launch_bounds__(kTileThreads, 3) k_extrema(Tables tb, uint32_t* __restrict__ rowmax, uint32_t* __restrict__ colmax) {
     constexpr int P = Elem<DT>::kPerVec;
     constexpr uint32_t kTileElems = kTileBytes / Elem<DT>::kBytes;
     constexpr uint32_t kKeyMask = DT == DNNS_F32 ? 0x7FFFFFFFu : 0x7FFF7FFFu;
@@ -46,8 +35,8 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_extrema(Tables tb, uint32_t
     for (uint32_t i = threadIdx.x; i < kColTab; i += kTileThreads) s_col[i] = 0;
     __syncthreads();
 
-    const uint32_t per = (tb.n_tiles + gridDim.x - 1) / gridDim.x;
-    const uint32_t lo = min(tb.n_tiles, blockIdx.x * per), hi = min(tb.n_tiles, lo + per);
+    // contiguous tile ranges of about equal cost (tiles of tensors whose column maxima stay in registers are cheaper)
+    const uint32_t lo = tb.extrema_bounds[blockIdx.x], hi = tb.extrema_bounds[blockIdx.x + 1];
     uint32_t tile = lo;
     while (tile < hi) {
         // ---- per-tensor context: constant over the run of tiles [tile, span_end)
@@ -59,6 +48,10 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_extrema(Tables tb, uint32_t
         uint32_t* g_col = colmax + d.off_col;
         const bool tab = I <= kColTab;                                      // column maxima through the shared table
         const bool fixed_cols = kTileElems % L == 0 && L % P == 0 && tab;  // a thread meets the same columns in every tile
+        const bool warp_in_row = L % (32u * P) == 0;                       // the 32 vectors a warp holds never straddle rows
+        const uint64_t inv_L = ~0ull / L + 1;  // e / L = umul64hi(e, inv_L) for e, L < 2^32 (L a power of two: wraps to the exact quotient)
+        const bool lean = L % P == 0 && L >= 32u * P;  // whole tiles of such tensors take the short path below
+        const uint32_t step_row = (kTileThreads * P) / L, step_pos = (kTileThreads * P) - step_row * L;
         auto col_max = [&](uint32_t col, uint32_t m) {
             if (tab) atomicMax(&s_col[col], m);
             else atomicMax(&g_col[col], m);
@@ -89,39 +82,108 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_extrema(Tables tb, uint32_t
             for (int u = 0; u < kVecPerThread; ++u) v[u] = nxt[u];
             if (tile + 1 < span_end) issue(tile + 1);
             const uint32_t e0 = (tile - tile0) * kTileElems;
+            if (lean && e0 + kTileElems <= numel) {
+                // ---- a whole tile of a tensor whose rows are multiples of a vector and at least a warp's span long:
+                // every vector lies in one row, a warp's 32 vectors in at most two neighbouring rows
+                uint32_t r0 = (uint32_t)__umul64hi((uint64_t)(e0 + threadIdx.x * P), inv_L), pos0 = e0 + threadIdx.x * P - r0 * L;
+#pragma unroll
+                for (int u = 0; u < kVecPerThread; ++u) {
+                    uint32_t key[P];
+                    vec_keys<DT>(v[u], key);
+                    uint32_t m = key[0];
+#pragma unroll
+                    for (int j = 1; j < P; ++j) m = max(m, key[j]);
+                    const uint32_t ra = __shfl_sync(kFull, r0, 0);
+                    const uint32_t ma = __reduce_max_sync(kFull, r0 == ra ? m : 0u), mb = __reduce_max_sync(kFull, r0 == ra ? 0u : m);
+                    if (lane == 0) {
+                        if (ma) atomicMax(&g_row[ra], ma);
+                        if (mb) atomicMax(&g_row[ra + 1], mb);
+                    }
+                    if (fixed_cols) {
+                        const uint32_t w[4] = {v[u].x & kKeyMask, v[u].y & kKeyMask, v[u].z & kKeyMask, v[u].w & kKeyMask};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) acc[u][k] = DT == DNNS_F32 ? max(acc[u][k], w[k]) : __vmaxu2(acc[u][k], w[k]);
+                    } else if (KK == 9) {
+                        const uint32_t col = pos0 / 9u, first = 9u - (pos0 - col * 9u);  // elements of the vector in column `col`
+                        uint32_t ca = 0, cb = 0;
+#pragma unroll
+                        for (int j = 0; j < P; ++j) {
+                            ca = max(ca, (uint32_t)j < first ? key[j] : 0u);
+                            cb = max(cb, (uint32_t)j < first ? 0u : key[j]);
+                        }
+                        if (ca) col_max(col, ca);
+                        if (cb) col_max(col + 1, cb);
+                    } else {
+                        uint32_t col = KK == 1 ? pos0 : pos0 / KK, rem = pos0 - col * KK, cur = 0;
+#pragma unroll
+                        for (int j = 0; j < P; ++j) {
+                            if (rem == KK) {
+                                if (cur) col_max(col, cur);
+                                ++col, rem = 0, cur = 0;
+                            }
+                            cur = max(cur, key[j]);
+                            ++rem;
+                        }
+                        if (cur) col_max(col, cur);
+                    }
+                    // the thread's next vector lies kTileThreads * P elements further on
+                    r0 += step_row;
+                    pos0 += step_pos;
+                    if (pos0 >= L) pos0 -= L, ++r0;
+                }
+                continue;
+            }
 #pragma unroll
             for (int u = 0; u < kVecPerThread; ++u) {
                 const uint32_t e = e0 + (u * kTileThreads + threadIdx.x) * P;
                 const int n = e >= numel ? 0 : (int)min((uint32_t)P, numel - e);  // valid elements
-                const uint32_t r0 = e / L, pos0 = e - r0 * L;
+                const uint32_t r0 = L == 1 ? e : (uint32_t)__umul64hi((uint64_t)e, inv_L), pos0 = e - r0 * L;  // e / L, e % L
                 const bool whole = n > 0 && pos0 + (uint32_t)n <= L;  // the vector lies in one row
-                const uint32_t m = vec_max_key<DT>(v[u], n);
+                uint32_t key[P];
+                vec_keys<DT>(v[u], key);
+                uint32_t m = 0;
+#pragma unroll
+                for (int j = 0; j < P; ++j) m = max(m, j < n ? key[j] : 0u);
                 // ---- row maxima: one atomic per row that the warp's 32 vectors touch
-                const bool has = whole && m != 0;
-                unsigned todo = __ballot_sync(kFull, has);
-                while (todo) {
-                    const int leader = __ffs(todo) - 1;
-                    const uint32_t rr = __shfl_sync(kFull, r0, leader);
-                    const bool mine = has && r0 == rr;
-                    const unsigned grp = __ballot_sync(kFull, mine);
-                    if (mine) {
-                        const uint32_t mm = __reduce_max_sync(grp, m);
-                        if (lane == leader) atomicMax(&g_row[rr], mm);
+                if (warp_in_row) {  // the 32 vectors of the warp lie in one row (a ragged end holds zeros)
+                    const uint32_t mm = __reduce_max_sync(kFull, m);
+                    if (lane == 0 && mm) atomicMax(&g_row[r0], mm);
+                } else {
+                    const bool has = whole && m != 0;
+                    unsigned todo = __ballot_sync(kFull, has);
+                    while (todo) {
+                        const int leader = __ffs(todo) - 1;
+                        const uint32_t rr = __shfl_sync(kFull, r0, leader);
+                        const bool mine = has && r0 == rr;
+                        const unsigned grp = __ballot_sync(kFull, mine);
+                        if (mine) {
+                            const uint32_t mm = __reduce_max_sync(grp, m);
+                            if (lane == leader) atomicMax(&g_row[rr], mm);
+                        }
+                        todo &= ~grp;
                     }
-                    todo &= ~grp;
                 }
                 // ---- column maxima
-                const uint32_t w[4] = {v[u].x & kKeyMask, v[u].y & kKeyMask, v[u].z & kKeyMask, v[u].w & kKeyMask};
                 if (fixed_cols) {
                     // (a ragged vector holds zeros past the end of the tensor: harmless)
+                    const uint32_t w[4] = {v[u].x & kKeyMask, v[u].y & kKeyMask, v[u].z & kKeyMask, v[u].w & kKeyMask};
 #pragma unroll
                     for (int k = 0; k < 4; ++k) acc[u][k] = DT == DNNS_F32 ? max(acc[u][k], w[k]) : __vmaxu2(acc[u][k], w[k]);
+                } else if (whole && n == P && KK == 9) {
+                    // 3x3 kernels: the P <= 9 elements of the vector belong to one column or to two neighbours
+                    const uint32_t col = pos0 / 9u, first = 9u - (pos0 - col * 9u);  // elements of the vector in column `col`
+                    uint32_t ma = 0, mb = 0;
+#pragma unroll
+                    for (int j = 0; j < P; ++j) {
+                        ma = max(ma, (uint32_t)j < first ? key[j] : 0u);
+                        mb = max(mb, (uint32_t)j < first ? 0u : key[j]);
+                    }
+                    if (ma) col_max(col, ma);
+                    if (mb) col_max(col + 1, mb);
                 } else if (n > 0) {
-                    uint32_t key[P];
-                    vec_keys<DT>(v[u], key);
                     if (whole) {
                         // runs of elements of one column: one table update per run
-                        uint32_t col = KK == 1 ? pos0 : (KK == 9 ? pos0 / 9u : pos0 / KK), rem = pos0 - col * KK, cur = 0;
+                        uint32_t col = KK == 1 ? pos0 : pos0 / KK, rem = pos0 - col * KK, cur = 0;
 #pragma unroll
                         for (int j = 0; j < P; ++j) {
                             if (j < n) {
@@ -136,9 +198,10 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_extrema(Tables tb, uint32_t
                         if (cur) col_max(col, cur);
                     } else {
                         // the vector crosses into the next row: element by element, rows included
-                        for (int j = 0; j < n; ++j) {
-                            const uint32_t ee = e + j, r = ee / L, pos = ee - r * L;
-                            if (key[j]) {
+#pragma unroll
+                        for (int j = 0; j < P; ++j) {  // (unrolled: the keys stay in registers)
+                            if (j < n && key[j]) {
+                                const uint32_t ee = e + j, r = ee / L, pos = ee - r * L;
                                 atomicMax(&g_row[r], key[j]);
                                 col_max(pos / KK, key[j]);
                             }
@@ -255,7 +318,7 @@ __global__ void __launch_bounds__(256) k_extrema_flags(Tables tb, const uint32_t
 }  // namespace
 
 int launch_extrema(const Tables& tb, uint32_t* rowmax, uint32_t* colmax, int n_sm, cudaStream_t st) {
-    const dim3 grid(min((uint32_t)n_sm * 4u, tb.n_tiles));
+    const dim3 grid(min((uint32_t)n_sm * 3u, tb.n_tiles));  // three resident blocks per SM
     ScopedKernel timed("k_extrema_sweep", st);
     if (tb.dtype == DNNS_F32) k_extrema<DNNS_F32><<<grid, kTileThreads, 0, st>>>(tb, rowmax, colmax);
     else k_extrema<DNNS_BF16><<<grid, kTileThreads, 0, st>>>(tb, rowmax, colmax);

@@ -63,7 +63,7 @@ struct WsMap {
     uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, producers, consumers, flag_prefix, flag_unit_tensor, status;
     uint64_t tables_end;  // everything before this is uploaded once at plan creation
     uint64_t k_dev, bitmap, sel, tie_prefix, tie_split, layouts, ebits, rowmax, colmax;
-    uint64_t vec_items;
+    uint64_t vec_items, extrema_bounds;
     uint64_t casc_rem0, casc_rem1, casc_lost, casc_live, casc_changed;
     uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
     uint64_t any_need, need, tie_bitmap, tile_ties, hist1, hist2;
@@ -190,6 +190,7 @@ dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts*
 
 // Prepared layouts of the rebuild (one per set of keep counts in use): header, item table, block starts, unit -> item.
 constexpr uint32_t kMaxGatherBlocks = 1024;
+constexpr uint32_t kMaxSweepBlocks = 4096;  // blocks of the extrema sweep (three per SM)
 uint64_t layout_slot_bytes(const Counts& c) {
     return align_up(sizeof(RebuildHeader)) + align_up(sizeof(RebuildItem) * (uint64_t)c.items) + align_up(4ull * rebuild_ranges(kMaxGatherBlocks)) +
            align_up(4ull * (c.element_units + 1));
@@ -217,6 +218,7 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.flag_prefix = take(4ull * (c.T + 1));
     w.flag_unit_tensor = take(4ull * (c.flag_units + 1));
     w.vec_items = take(8ull * (c.n_vec + 1));
+    w.extrema_bounds = take(4ull * (kMaxSweepBlocks + 1));
     w.status = take(4);
     w.tables_end = o;
     const uint64_t vs = (uint64_t)maxv * (c.S ? c.S : 1);
@@ -260,6 +262,10 @@ struct dnns_plan {
     // its counts to names the slot its layout went to; dnns_compact looks its keep_count argument up here.
     std::vector<const int32_t*> layout_owner;
     uint32_t layout_next;
+    // The sweep for the per-filter / per-column maxima runs beside the ranking kernels of a threshold call: a second
+    // stream forked from the caller's and joined again before the call returns (host objects, no device memory).
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     CascadeWs kws;
     uint64_t launches;
     int last_n_k;
@@ -398,6 +404,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     p->seg_size.assign(c.S ? c.S : 1, 0);
     uint64_t arena = 0, mask_w = 0, map_w = 0, out_w = 0, in_w = 0, compact_bytes = 0, n_prunable = 0, flag_units = 0;
     uint64_t row_e = 0, col_e = 0;
+    uint32_t tb_extrema_blocks = 1;
     uint32_t tile = 0, seg = 0;
     for (uint32_t S = 0; S < c.S; ++S) sd[S] = SegDesc{0xFFFFFFFFu, 0, 0};
     for (uint32_t i = 0; i < c.T; ++i) {
@@ -479,6 +486,26 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
         producers[i] = pd;
     }
     for (int i = 0; i < nc; ++i) consumers[i] = ConsumerDesc{td[cons_list[i]].off_innz, td[cons_list[i]].S};
+    {   // tile ranges of the extrema sweep: about equal cost per block; a tile whose column maxima stay in registers
+        // (rows that divide the tile) counts 2, any other tile 3
+        auto* bounds = reinterpret_cast<uint32_t*>(host.data() + map.extrema_bounds);
+        const uint32_t blocks = std::max(1u, std::min({(uint32_t)p->n_sm * 3u, kMaxSweepBlocks, c.tiles}));
+        const uint32_t tile_elems = kTileBytes / c.elem_bytes, vec = 16 / c.elem_bytes;
+        std::vector<uint64_t> cost_before(c.tiles + 1, 0);
+        for (uint32_t i = 0; i < c.T; ++i) {
+            const uint64_t L = (uint64_t)td[i].I * td[i].KK;
+            const bool cheap = L <= tile_elems && tile_elems % L == 0 && L % vec == 0 && (uint32_t)td[i].I <= 8192u;
+            for (uint32_t k = 0; k < td[i].n_tiles; ++k) cost_before[td[i].tile0 + k + 1] = cheap ? 2 : 3;
+        }
+        for (uint32_t t = 0; t < c.tiles; ++t) cost_before[t + 1] += cost_before[t];
+        uint32_t t = 0;
+        for (uint32_t b = 0; b <= blocks; ++b) {
+            const uint64_t want = cost_before[c.tiles] * b / blocks;
+            while (t < c.tiles && cost_before[t] < want) ++t;
+            bounds[b] = b == blocks ? c.tiles : t;
+        }
+        tb_extrema_blocks = blocks;
+    }
     // gather items: weights, then BN vectors, then biases
     auto* vec_items = reinterpret_cast<uint32_t*>(host.data() + map.vec_items);
     uint32_t n_it = 0, n_vec = 0;
@@ -555,8 +582,16 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     t.split = reinterpret_cast<TieSplit*>(w + map.tie_split);
     tb.vec_items = reinterpret_cast<uint32_t*>(w + map.vec_items);
     tb.n_vec_items = c.n_vec;
+    tb.extrema_bounds = reinterpret_cast<uint32_t*>(w + map.extrema_bounds);
+    tb.extrema_blocks = tb_extrema_blocks;
     p->layout_owner.assign(layout_slots(maxv), nullptr);
     p->layout_next = 0;
+    if (cudaStreamCreateWithFlags(&p->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        dnns_plan_destroy(p);
+        return DNNS_ERR_CUDA;
+    }
     p->kws.rem[0] = reinterpret_cast<uint32_t*>(w + map.casc_rem0);
     p->kws.rem[1] = reinterpret_cast<uint32_t*>(w + map.casc_rem1);
     p->kws.lost = reinterpret_cast<uint32_t*>(w + map.casc_lost);
@@ -585,6 +620,9 @@ void dnns_plan_destroy(dnns_plan* plan) {
     if (!plan) return;
     cudaDeviceSynchronize();
     plan->timer.clear();
+    if (plan->ev_fork) cudaEventDestroy(plan->ev_fork);
+    if (plan->ev_join) cudaEventDestroy(plan->ev_join);
+    if (plan->side) cudaStreamDestroy(plan->side);
     delete plan;
 }
 
@@ -610,9 +648,17 @@ dnns_status dnns_magnitude_threshold(dnns_plan* p, const uint64_t* k, int32_t n_
     if (cudaMemsetAsync(p->ws + p->map.clear_begin, 0, clear_end - p->map.clear_begin, st) != cudaSuccess)
         return DNNS_ERR_CUDA;
     ProfileScope profile_scope(p);
+    // beside the ranking: the largest key of every filter and every input column, for dnns_zero_structures_portfolio
+    uint32_t* rowmax = reinterpret_cast<uint32_t*>(p->ws + p->map.rowmax);
+    const uint64_t clear_bytes = p->map.colmax + 4ull * p->c.sum_I - p->map.rowmax;  // both tables: the maxima start at zero
+    if (cudaEventRecord(p->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(p->side, p->ev_fork, 0) != cudaSuccess ||
+        cudaMemsetAsync(rowmax, 0, clear_bytes, p->side) != cudaSuccess)
+        return DNNS_ERR_CUDA;
+    const int n_side = launch_extrema(p->tb, rowmax, reinterpret_cast<uint32_t*>(p->ws + p->map.colmax), p->n_sm, p->side);
+    const bool joined = cudaEventRecord(p->ev_join, p->side) == cudaSuccess;
     const int n = launch_threshold(p->tb, p->tws, n_k, k, thr_dev, p->n_sm, st);
-    if (n < 0) return DNNS_ERR_CUDA;
-    p->launches += n;
+    if (!joined || cudaStreamWaitEvent(st, p->ev_join, 0) != cudaSuccess || n < 0 || n_side < 0) return DNNS_ERR_CUDA;
+    p->launches += n + n_side;
     p->last_n_k = n_k;
     return DNNS_OK;
 }
@@ -718,16 +764,12 @@ dnns_status dnns_zero_structures_portfolio(dnns_plan* p, const dnns_threshold* t
             if (out_nz[u] == out_nz[v] || in_nz[u] == in_nz[v]) return DNNS_ERR_INVALID_ARG;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    uint32_t* rowmax = reinterpret_cast<uint32_t*>(p->ws + p->map.rowmax);
-    uint32_t* colmax = reinterpret_cast<uint32_t*>(p->ws + p->map.colmax);
-    const uint64_t clear_bytes = p->map.colmax + 4ull * p->c.sum_I - p->map.rowmax;  // both tables: the maxima start at zero
-    if (cudaMemsetAsync(rowmax, 0, clear_bytes, st) != cudaSuccess) return DNNS_ERR_CUDA;
     ProfileScope profile_scope(p);
-    const int n1 = launch_extrema(p->tb, rowmax, colmax, p->n_sm, st);
-    if (n1 < 0) return DNNS_ERR_CUDA;
-    const int n2 = launch_extrema_flags(p->tb, rowmax, colmax, thr_dev, p->tws.split, first_variant, n_variants, out_nz,
-                                        in_nz, st);
+    const int n2 = launch_extrema_flags(p->tb, reinterpret_cast<uint32_t*>(p->ws + p->map.rowmax),
+                                        reinterpret_cast<uint32_t*>(p->ws + p->map.colmax), thr_dev, p->tws.split,
+                                        first_variant, n_variants, out_nz, in_nz, st);
     if (n2 < 0) return DNNS_ERR_CUDA;
+    const int n1 = 0;
     p->launches += n1 + n2;
     return DNNS_OK;
 }
