@@ -353,8 +353,11 @@ __device__ __forceinline__ Geometry geometry_of(const ItemDesc& it, uint32_t Cn)
 // From the keep counts: rows and channels every item keeps, its 256-byte aligned place in the destination arena,
 // its units of work, and where each block of the gather starts.  One block per variant; the tables stay in the
 // workspace until the keep counts change (dnns_propagate_keep* runs this right after planning the channels).
+constexpr uint32_t kLayoutTab = 4096;  // items whose prefix sums the layout kernel also keeps in shared memory
 __global__ void __launch_bounds__(1024) k_rebuild_layout(Tables tb, LayoutBatch lb, uint32_t n_blocks) {
     __shared__ uint64_t scratch[33];
+    __shared__ uint32_t s_cost_pre[kLayoutTab], s_unit_pre[kLayoutTab];  // searched below: thousands of probes, none to global memory
+    const bool in_smem = tb.n_items <= kLayoutTab;
     const int32_t* __restrict__ keep_count = lb.keep_count[blockIdx.x];
     const RebuildSlot slot = lb.slot[blockIdx.x];
     uint64_t carry_bytes = 0, carry_uc = 0;  // carry_uc: cost << 32 | units (each stays below 2^32)
@@ -390,6 +393,7 @@ __global__ void __launch_bounds__(1024) k_rebuild_layout(Tables tb, LayoutBatch 
             r.cost_pre = (uint32_t)((carry_uc + ex_uc) >> 32);
             r.unit_pre = (uint32_t)(carry_uc + ex_uc);
             slot.items[i] = r;
+            if (in_smem) s_cost_pre[i] = r.cost_pre, s_unit_pre[i] = r.unit_pre;
         }
         carry_bytes += tot_b;
         carry_uc += tot_uc;
@@ -409,7 +413,7 @@ __global__ void __launch_bounds__(1024) k_rebuild_layout(Tables tb, LayoutBatch 
         uint32_t item = 0, top = tb.n_items;
         while (top - item > 1) {
             const uint32_t mid = (item + top) >> 1;
-            if (slot.items[mid].cost_pre <= lo) item = mid;
+            if ((in_smem ? s_cost_pre[mid] : slot.items[mid].cost_pre) <= lo) item = mid;
             else top = mid;
         }
         slot.range_item[r] = item;
@@ -419,7 +423,7 @@ __global__ void __launch_bounds__(1024) k_rebuild_layout(Tables tb, LayoutBatch 
         uint32_t item = 0, top = tb.n_items;
         while (top - item > 1) {
             const uint32_t mid = (item + top) >> 1;
-            if (slot.items[mid].unit_pre <= u) item = mid;
+            if ((in_smem ? s_unit_pre[mid] : slot.items[mid].unit_pre) <= u) item = mid;
             else top = mid;
         }
         slot.unit_item[u] = item;

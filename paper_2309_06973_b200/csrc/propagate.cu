@@ -42,25 +42,47 @@ __device__ __forceinline__ uint32_t eval_group(const Tables& tb, const GroupDesc
         // One (tensor, word) pair per thread and step, producers first, then consumers: all flag
         // words of the group are requested in one go.  Producers OR their filter flags; consumers OR
         // their input-column flags (with S columns per channel the S bits are folded).
-        const int n_pw = n_prod * n_words;
-        for (int it = threadIdx.x; it < n_pw + n_cons * n_words; it += kThreads) {
-            if (it < n_pw) {
-                const int p = it / n_words, w = it - p * n_words;
-                const uint32_t x = out_nz[tb.producers[gd.prod_begin + p].off_outnz + w];
-                if (x) atomicOr(&s_prod[w], x);
-                continue;
+        const int n_pw = n_prod * n_words, n_all = n_pw + n_cons * n_words;
+        constexpr int kBatch = 4;  // pairs per thread and round: their loads are all issued before the first one is used
+        for (int base = threadIdx.x; base < n_all; base += kThreads * kBatch) {
+            uint32_t off[kBatch], x[kBatch];
+            int S[kBatch], w[kBatch];
+            bool prod[kBatch], ok[kBatch];
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+                const int it = base + b * kThreads;
+                ok[b] = it < n_all;
+                prod[b] = it < n_pw;
+                off[b] = 0, S[b] = 1, w[b] = 0;
+                if (!ok[b]) continue;
+                if (prod[b]) {
+                    const int p = it / n_words;
+                    w[b] = it - p * n_words;
+                    off[b] = tb.producers[gd.prod_begin + p].off_outnz;
+                } else {
+                    const int q = (it - n_pw) / n_words;
+                    w[b] = (it - n_pw) - q * n_words;
+                    const ConsumerDesc d = tb.consumers[gd.cons_begin + q];
+                    off[b] = d.off_innz, S[b] = d.S;
+                }
             }
-            const int q = (it - n_pw) / n_words, w = (it - n_pw) - q * n_words;
-            const ConsumerDesc d = tb.consumers[gd.cons_begin + q];
-            uint32_t x = 0;
-            if (d.S == 1) {
-                x = in_nz[d.off_innz + w];
-            } else {
-                for (int b = 0; b < 32 && w * 32 + b < C; ++b)
-                    for (int s = 0; s < d.S; ++s)
-                        if (get_bit(in_nz + d.off_innz, (uint32_t)(w * 32 + b) * d.S + s)) x |= 1u << b;
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+                x[b] = 0;
+                if (!ok[b]) continue;
+                if (prod[b]) {
+                    x[b] = out_nz[off[b] + w[b]];
+                } else if (S[b] == 1) {
+                    x[b] = in_nz[off[b] + w[b]];
+                } else {  // S columns per channel: the S bits of a channel are folded
+                    for (int bit = 0; bit < 32 && w[b] * 32 + bit < C; ++bit)
+                        for (int sc = 0; sc < S[b]; ++sc)
+                            if (get_bit(in_nz + off[b], (uint32_t)(w[b] * 32 + bit) * S[b] + sc)) x[b] |= 1u << bit;
+                }
             }
-            if (x) atomicOr(&s_cons[w], x);
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b)
+                if (ok[b] && x[b]) atomicOr(prod[b] ? &s_prod[w[b]] : &s_cons[w[b]], x[b]);
         }
     }
     __syncthreads();

@@ -11,9 +11,9 @@
 //   ties    a sweep that counts, per 16 KB tile, the keys equal to tau_v - only run when some
 //           variant must mask part of the weights equal to tau (n_tie < n_equal); followed by
 //           an exclusive scan per (variant, segment).  The mask kernel then needs no ordering
-//           between tiles to mask exactly k weights;
-//   split   for such a variant, the position (tensor, element) of the first weight equal to tau
-//           that stays: every equal weight before it is masked, every one from it on is kept.
+//           between tiles to mask exactly k weights.  The scan kernel also finds, for such a
+//           variant, the position (tensor, element) of the first weight equal to tau that stays:
+//           every equal weight before it is masked, every one from it on is kept.
 #include "dnns_internal.cuh"
 
 namespace dnns {
@@ -552,14 +552,27 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_ties(Tables tb, ThresholdWs
         });
 }
 
-// Exclusive scan of the tile counts over the tiles of a segment, one block per (variant, segment).
-// Every thread owns a contiguous run of tiles: one pass of independent loads, one block scan.
-__global__ void __launch_bounds__(1024) k_tie_scan(Tables tb, ThresholdWs ws) {
-    if (*ws.any_need == 0) return;
+// Exclusive scan of the tile counts over the tiles of a segment, one block per (variant, segment); every thread
+// owns a contiguous run of tiles: one pass of independent loads, one block scan.  The mask kernel then needs no
+// ordering between tiles.
+//
+// The same block then finds where the variant's ties split.  Weights equal to tau are masked in index order until
+// n_tie of them are gone; the first one that stays is the tie of rank n_tie.  Its tile follows from the scanned
+// counts (the last tile whose exclusive prefix is <= n_tie), its place in the tile from one ranking of that tile's
+// ties (a 16 KB tile is one 16-byte vector per thread).
+template <int DT>
+__global__ void __launch_bounds__(1024) k_tie_scan(Tables tb, ThresholdWs ws, const dnns_threshold* __restrict__ thr) {
+    constexpr int P = Elem<DT>::kPerVec;
+    constexpr uint32_t kTileElems = kTileBytes / Elem<DT>::kBytes;
+    static_assert(kTileBytes / 16 == 1024, "one vector of the tile per thread");
     __shared__ uint32_t scratch[33];
     const uint32_t S = tb.n_segs;
     const uint32_t v = blockIdx.x / S, seg = blockIdx.x % S;
-    if (!ws.need[(size_t)v * S + seg]) return;
+    const size_t idx = (size_t)v * S + seg;
+    if (*ws.any_need == 0 || !ws.need[idx]) {
+        if (threadIdx.x == 0) ws.split[idx] = TieSplit{0xFFFFFFFFu, 0u};  // no weight equal to tau stays
+        return;
+    }
     const SegDesc sd = tb.segs[seg];
     const uint32_t* cnt = ws.tile_ties + (size_t)v * tb.n_tiles;
     uint32_t* pre = ws.tie_prefix + (size_t)v * tb.n_tiles;
@@ -569,64 +582,37 @@ __global__ void __launch_bounds__(1024) k_tie_scan(Tables tb, ThresholdWs ws) {
     uint32_t sum = 0;
     for (uint32_t t = t0; t < t1; ++t) sum += cnt[t];
     uint32_t total;
-    uint32_t ex = block_exclusive_scan<uint32_t>(sum, scratch, &total);
-    for (uint32_t t = t0; t < t1; ++t) {
-        pre[t] = ex;
-        ex += cnt[t];
-    }
-}
-
-// ---------------------------------------------------------------- where the ties split
-// One block per (variant, segment).  Weights equal to tau are masked in index order until n_tie of them are
-// gone; the first one that stays is the tie of rank n_tie.  Its tile follows from the scanned tile counts
-// (the last tile whose exclusive prefix is <= n_tie), its place in the tile from one ranking of that tile's ties.
-template <int DT>
-__global__ void __launch_bounds__(kTileThreads) k_tie_split(Tables tb, ThresholdWs ws, const dnns_threshold* __restrict__ thr) {
-    constexpr int P = Elem<DT>::kPerVec;
-    constexpr uint32_t kTileElems = kTileBytes / Elem<DT>::kBytes;
-    __shared__ uint32_t scratch[33];
-    const uint32_t S = tb.n_segs;
-    const uint32_t v = blockIdx.x / S, seg = blockIdx.x % S;
-    const size_t idx = (size_t)v * S + seg;
-    if (*ws.any_need == 0 || !ws.need[idx]) {
-        if (threadIdx.x == 0) ws.split[idx] = TieSplit{0xFFFFFFFFu, 0u};  // no weight equal to tau stays
-        return;
-    }
+    const uint32_t ex0 = block_exclusive_scan<uint32_t>(sum, scratch, &total);
     const dnns_threshold r = thr[idx];
     const uint32_t n_tie = (uint32_t)r.n_tie;  // below n_equal, which fits 32 bits
-    const SegDesc sd = tb.segs[seg];
-    const uint32_t* pre = ws.tie_prefix + (size_t)v * tb.n_tiles;
-    uint32_t lo = sd.tile_begin, hi = sd.tile_end;  // the last tile in [lo, hi) with pre[tile] <= n_tie
-    while (hi - lo > 1) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (pre[mid] <= n_tie) lo = mid;
-        else hi = mid;
+    // the tile that holds the tie of rank n_tie lies in the run of exactly one thread
+    __shared__ uint32_t s_tile, s_want;
+    uint32_t ex = ex0;
+    for (uint32_t t = t0; t < t1; ++t) {
+        pre[t] = ex;
+        const uint32_t c = cnt[t];
+        if (ex <= n_tie && n_tie < ex + c) s_tile = t, s_want = n_tie - ex;
+        ex += c;
     }
-    const uint32_t tile = lo, want = n_tie - pre[tile];  // rank, inside the tile, of the tie that stays
+    __syncthreads();
+    const uint32_t tile = s_tile, want = s_want;  // rank, inside the tile, of the tie that stays
     const uint32_t t = tb.tile_tensor[tile];
     const TensorDesc& d = tb.tensors[t];
-    const uint32_t e0 = (tile - d.tile0) * kTileElems;
-    uint32_t carry = 0;
-#pragma unroll 1
-    for (int u = 0; u < kVecPerThread; ++u) {
-        const uint32_t e = e0 + (u * kTileThreads + threadIdx.x) * P;
-        uint4 vec;
-        const int n = load_vec<DT>(d.src, e, d.numel, vec);
-        uint32_t key[P];
-        vec_keys<DT>(vec, key);
-        uint32_t c = 0;
+    const uint32_t e = (tile - d.tile0) * kTileElems + threadIdx.x * P;
+    uint4 vec;
+    const int nv = load_vec<DT>(d.src, e, d.numel, vec);
+    uint32_t key[P];
+    vec_keys<DT>(vec, key);
+    uint32_t c = 0;
 #pragma unroll
-        for (int j = 0; j < P; ++j) c += (j < n && key[j] == r.tau_bits);
-        uint32_t total;
-        uint32_t rank = carry + block_exclusive_scan<uint32_t>(c, scratch, &total);
-        carry += total;
-        if (rank <= want && want < rank + c) {
+    for (int j = 0; j < P; ++j) c += (j < nv && key[j] == r.tau_bits);
+    uint32_t rank = block_exclusive_scan<uint32_t>(c, scratch, &total);
+    if (rank <= want && want < rank + c) {
 #pragma unroll
-            for (int j = 0; j < P; ++j) {
-                if (j < n && key[j] == r.tau_bits) {
-                    if (rank == want) ws.split[idx] = TieSplit{t, e + j};
-                    ++rank;
-                }
+        for (int j = 0; j < P; ++j) {
+            if (j < nv && key[j] == r.tau_bits) {
+                if (rank == want) ws.split[idx] = TieSplit{t, e + j};
+                ++rank;
             }
         }
     }
@@ -668,13 +654,12 @@ int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, const uin
         { ScopedKernel t("k_ties", st); k_ties<DNNS_BF16><<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k, thr_dev); }
         launches = 3;
     }
-    { ScopedKernel t("k_tie_scan", st); k_tie_scan<<<S * n_k, 1024, 0, st>>>(tb, ws); }
     {
-        ScopedKernel t("k_tie_split", st);
-        if (tb.dtype == DNNS_F32) k_tie_split<DNNS_F32><<<S * n_k, kTileThreads, 0, st>>>(tb, ws, thr_dev);
-        else k_tie_split<DNNS_BF16><<<S * n_k, kTileThreads, 0, st>>>(tb, ws, thr_dev);
+        ScopedKernel t("k_tie_scan", st);
+        if (tb.dtype == DNNS_F32) k_tie_scan<DNNS_F32><<<S * n_k, 1024, 0, st>>>(tb, ws, thr_dev);
+        else k_tie_scan<DNNS_BF16><<<S * n_k, 1024, 0, st>>>(tb, ws, thr_dev);
     }
-    launches += 2;
+    ++launches;
     return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
