@@ -265,7 +265,15 @@ int launch_extrema(const Tables& tb, uint32_t* rowmax, uint32_t* colmax, int n_s
 int launch_extrema_flags(const Tables& tb, const uint32_t* rowmax, const uint32_t* colmax, const dnns_threshold* thr,
                          const TieSplit* split, int first_variant, int n_variants, uint32_t* const* out_nz,
                          uint32_t* const* in_nz, cudaStream_t st);
-int launch_fold(const Tables& tb, void* arena, const uint64_t* offsets, const int32_t* shapes, cudaStream_t st);
+// One 16 KB tile of a rebuilt tensor that the conv+BN fusion scales (listed by its first kernel, read by its second).
+struct FoldJob {
+    char* w;             // the rebuilt tensor
+    const float* scale;  // per-filter factors
+    uint32_t Ln, total;  // elements per filter, elements of the tensor
+    uint32_t e0, pad;    // first element of the tile
+};
+int launch_fold(const Tables& tb, void* arena, const uint64_t* offsets, const int32_t* shapes, uint32_t* job_count,
+                FoldJob* jobs, int n_sm, cudaStream_t st);
 cudaError_t init_kernel_attributes();
 cudaError_t init_compact_attributes();
 constexpr uint32_t kGatherStageBytes = 18432;  // one stage buffer of the staged rebuild

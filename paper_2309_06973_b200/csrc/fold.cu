@@ -3,10 +3,12 @@
 //   s_o   = gamma_o / sqrt(var_o + eps)
 //   W_f[o] = W[o] * s_o                       (in place)
 //   b_f[o] = beta_o + (bias_o - mean_o) * s_o  (bias_o = 0 without a bias)
-// Two launches: k_fold_prepare writes s into the arena slot of gamma and b_f into the slot of
-// beta (the BatchNorm vectors have no further use once folded); k_fold_scale multiplies the
-// weights, 16 bytes per thread and step.  Arithmetic is fp32; bf16 weights are widened, scaled and
+// Two launches: k_fold_prepare (a block per BatchNorm) writes s into the arena slot of gamma and b_f into the
+// slot of beta (the BatchNorm vectors have no further use once folded) and lists the 16 KB tiles of the rebuilt
+// tensor in front of it; k_fold_scale multiplies the weights of the listed tiles, four 16-byte vectors per thread.  Arithmetic is fp32; bf16 weights are widened, scaled and
 // rounded to nearest even.
+#include <algorithm>
+
 #include "dnns_internal.cuh"
 
 namespace dnns {
@@ -21,22 +23,47 @@ struct FoldArgs {
     const int32_t* shapes;    // [n_tensors][2] rebuilt (O', I')
 };
 
-__global__ void __launch_bounds__(kThreads) k_fold_prepare(Tables tb, FoldArgs fa) {
+template <int DT>
+__global__ void __launch_bounds__(kThreads) k_fold_prepare(Tables tb, FoldArgs fa, uint32_t* __restrict__ job_count,
+                                                           FoldJob* __restrict__ jobs) {
+    constexpr uint32_t kTileElems = kTileBytes / Elem<DT>::kBytes;
+    constexpr int kBatch = 4;  // channels per thread whose loads are issued together
+    __shared__ uint32_t s_first;
     const uint32_t b = blockIdx.x;
     const BnDesc bn = tb.bns[b];
     const int32_t On = fa.shapes[2 * bn.tensor];
+    const uint32_t Ln = (uint32_t)fa.shapes[2 * bn.tensor + 1] * tb.tensors[bn.tensor].KK;
     const uint32_t base = tb.n_tensors + 4 * b;
     float* gamma = reinterpret_cast<float*>(fa.arena + fa.offsets[base]);
     float* beta = reinterpret_cast<float*>(fa.arena + fa.offsets[base + 1]);
     const float* mean = reinterpret_cast<const float*>(fa.arena + fa.offsets[base + 2]);
     const float* var = reinterpret_cast<const float*>(fa.arena + fa.offsets[base + 3]);
     const float* bias = bn.bias_item >= 0 ? reinterpret_cast<const float*>(fa.arena + fa.offsets[bn.bias_item]) : nullptr;
-    for (int a = threadIdx.x; a < On; a += kThreads) {
-        const float s = gamma[a] / sqrtf(var[a] + bn.eps);
-        const float shift = (bias ? bias[a] : 0.0f) - mean[a];
-        gamma[a] = s;
-        beta[a] = fmaf(shift, s, beta[a]);
+    char* w = fa.arena + fa.offsets[bn.tensor];
+    // the tiles of the rebuilt tensor join the list the second kernel works through
+    const uint32_t total = (uint32_t)On * Ln, n_tiles = (total + kTileElems - 1) / kTileElems;
+    if (threadIdx.x == 0) s_first = n_tiles ? atomicAdd(job_count, n_tiles) : 0u;
+    for (int a0 = threadIdx.x; a0 < On; a0 += kThreads * kBatch) {
+        float g[kBatch], vr[kBatch], mn[kBatch], be[kBatch], bi[kBatch];
+#pragma unroll
+        for (int t = 0; t < kBatch; ++t) {
+            const int a = a0 + t * kThreads;
+            const bool in = a < On;
+            g[t] = in ? gamma[a] : 0.0f, vr[t] = in ? var[a] : 1.0f, mn[t] = in ? mean[a] : 0.0f, be[t] = in ? beta[a] : 0.0f;
+            bi[t] = in && bias ? bias[a] : 0.0f;
+        }
+#pragma unroll
+        for (int t = 0; t < kBatch; ++t) {
+            const int a = a0 + t * kThreads;
+            if (a >= On) continue;
+            const float s = g[t] / sqrtf(vr[t] + bn.eps);
+            gamma[a] = s;
+            beta[a] = fmaf(bi[t] - mn[t], s, be[t]);
+        }
     }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < n_tiles; i += kThreads)
+        jobs[s_first + i] = FoldJob{w, gamma, Ln, total, i * kTileElems, 0u};
 }
 
 __device__ __forceinline__ uint32_t bf16_round(float x) {
@@ -45,52 +72,69 @@ __device__ __forceinline__ uint32_t bf16_round(float x) {
     return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
 }
 
+// W[o] *= s_o over the rebuilt tensors, a block per listed 16 KB tile and round.  A thread holds four 16-byte
+// vectors of a tile; the row of a vector is one division, and a vector inside one row (nearly all of them) is
+// scaled by one factor.
 template <int DT>
-__global__ void __launch_bounds__(kThreads) k_fold_scale(Tables tb, FoldArgs fa) {
+__device__ __forceinline__ uint32_t scaled_word(uint32_t x, float s_lo, float s_hi) {
+    if (DT == DNNS_F32) return __float_as_uint(__uint_as_float(x) * s_lo);
+    const float a = __uint_as_float(x << 16) * s_lo, b = __uint_as_float(x & 0xFFFF0000u) * s_hi;
+    return bf16_round(a) | (bf16_round(b) << 16);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kTileThreads, 4) k_fold_scale(const uint32_t* __restrict__ job_count, const FoldJob* __restrict__ jobs) {
     constexpr uint32_t VE = Elem<DT>::kPerVec;
-    const uint32_t b = blockIdx.y;
-    const BnDesc bn = tb.bns[b];
-    const TensorDesc& d = tb.tensors[bn.tensor];
-    const uint32_t On = fa.shapes[2 * bn.tensor], Ln = (uint32_t)fa.shapes[2 * bn.tensor + 1] * d.KK;
-    const uint32_t total = On * Ln;
-    if (total == 0) return;
-    char* w = fa.arena + fa.offsets[bn.tensor];
-    const float* scale = reinterpret_cast<const float*>(fa.arena + fa.offsets[tb.n_tensors + 4 * b]);
-    for (uint32_t f = (blockIdx.x * kThreads + threadIdx.x) * VE; f < total; f += gridDim.x * kThreads * VE) {
-        uint32_t a = f / Ln, rem = f - a * Ln;
-        float s = scale[a];
-        if (f + VE <= total) {
-            uint4 v = *reinterpret_cast<uint4*>(w + (size_t)f * Elem<DT>::kBytes);
-            uint32_t x[4] = {v.x, v.y, v.z, v.w};
+    const uint32_t n_jobs = *job_count;
+    for (uint32_t i = blockIdx.x; i < n_jobs; i += gridDim.x) {
+        const FoldJob job = jobs[i];
+        const uint32_t Ln = job.Ln, total = job.total, e0 = job.e0, On = total / Ln;
+        char* w = job.w;
+        const float* __restrict__ scale = job.scale;
+        uint4 v[kVecPerThread];
+        uint32_t f[kVecPerThread];
 #pragma unroll
-            for (uint32_t e = 0; e < VE; ++e) {
-                if (DT == DNNS_F32) {
-                    x[e] = __float_as_uint(__uint_as_float(x[e]) * s);
+        for (int u = 0; u < kVecPerThread; ++u) {
+            f[u] = e0 + (u * kTileThreads + threadIdx.x) * VE;
+            if (f[u] + VE <= total) v[u] = *reinterpret_cast<const uint4*>(w + (size_t)f[u] * Elem<DT>::kBytes);
+        }
+#pragma unroll
+        for (int u = 0; u < kVecPerThread; ++u) {
+            if (f[u] >= total) continue;
+            uint32_t a = f[u] / Ln, rem = f[u] - a * Ln;
+            if (f[u] + VE <= total) {
+                uint32_t x[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                if (rem + VE <= Ln) {
+                    const float s = scale[a];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) x[q] = scaled_word<DT>(x[q], s, s);
                 } else {
-                    const uint32_t sh = 16 * (e & 1);
-                    const float y = __uint_as_float(((x[e >> 1] >> sh) & 0xFFFFu) << 16) * s;
-                    x[e >> 1] = (x[e >> 1] & ~(0xFFFFu << sh)) | (bf16_round(y) << sh);
+                    // the vector crosses into the next row (or rows, when rows are shorter than a vector)
+                    float se[VE];
+#pragma unroll
+                    for (uint32_t e = 0; e < VE; ++e) {
+                        se[e] = scale[a];
+                        if (++rem == Ln) rem = 0, ++a;
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) x[q] = DT == DNNS_F32 ? scaled_word<DT>(x[q], se[q], se[q]) : scaled_word<DT>(x[q], se[(2 * q) % VE], se[(2 * q + 1) % VE]);
                 }
-                if (++rem == Ln) {
-                    rem = 0;
-                    ++a;
-                    if (a < On) s = scale[a];
-                }
-            }
-            *reinterpret_cast<uint4*>(w + (size_t)f * Elem<DT>::kBytes) = make_uint4(x[0], x[1], x[2], x[3]);
-        } else {
-            for (uint32_t e = 0; f + e < total; ++e) {
-                if (DT == DNNS_F32) {
-                    float* p = reinterpret_cast<float*>(w) + f + e;
-                    *p = *p * s;
-                } else {
-                    uint16_t* p = reinterpret_cast<uint16_t*>(w) + f + e;
-                    *p = (uint16_t)bf16_round(__uint_as_float((uint32_t)*p << 16) * s);
-                }
-                if (++rem == Ln) {
-                    rem = 0;
-                    ++a;
-                    if (a < On) s = scale[a];
+                *reinterpret_cast<uint4*>(w + (size_t)f[u] * Elem<DT>::kBytes) = make_uint4(x[0], x[1], x[2], x[3]);
+            } else {
+                float s = scale[a];
+                for (uint32_t e = 0; f[u] + e < total; ++e) {
+                    if (DT == DNNS_F32) {
+                        float* p = reinterpret_cast<float*>(w) + f[u] + e;
+                        *p = *p * s;
+                    } else {
+                        uint16_t* p = reinterpret_cast<uint16_t*>(w) + f[u] + e;
+                        *p = (uint16_t)bf16_round(__uint_as_float((uint32_t)*p << 16) * s);
+                    }
+                    if (++rem == Ln) {
+                        rem = 0;
+                        ++a;
+                        if (a < On) s = scale[a];
+                    }
                 }
             }
         }
@@ -99,13 +143,19 @@ __global__ void __launch_bounds__(kThreads) k_fold_scale(Tables tb, FoldArgs fa)
 
 }  // namespace
 
-int launch_fold(const Tables& tb, void* arena, const uint64_t* offsets, const int32_t* shapes, cudaStream_t st) {
+int launch_fold(const Tables& tb, void* arena, const uint64_t* offsets, const int32_t* shapes, uint32_t* job_count,
+                FoldJob* jobs, int n_sm, cudaStream_t st) {
     if (tb.n_bn == 0) return 0;
     const FoldArgs fa{static_cast<char*>(arena), offsets, shapes};
-    k_fold_prepare<<<tb.n_bn, kThreads, 0, st>>>(tb, fa);
-    const dim3 grid(128, tb.n_bn);  // tensors differ a lot in size: many slices keep the large ones spread out
-    if (tb.dtype == DNNS_F32) k_fold_scale<DNNS_F32><<<grid, kThreads, 0, st>>>(tb, fa);
-    else k_fold_scale<DNNS_BF16><<<grid, kThreads, 0, st>>>(tb, fa);
+    if (cudaMemsetAsync(job_count, 0, sizeof(uint32_t), st) != cudaSuccess) return -1;
+    const int grid = (int)std::min<uint32_t>(tb.n_tiles, (uint32_t)n_sm * 8u);
+    if (tb.dtype == DNNS_F32) {
+        { ScopedKernel t("k_fold_prepare", st); k_fold_prepare<DNNS_F32><<<tb.n_bn, kThreads, 0, st>>>(tb, fa, job_count, jobs); }
+        { ScopedKernel t("k_fold_scale", st); k_fold_scale<DNNS_F32><<<grid, kTileThreads, 0, st>>>(job_count, jobs); }
+    } else {
+        { ScopedKernel t("k_fold_prepare", st); k_fold_prepare<DNNS_BF16><<<tb.n_bn, kThreads, 0, st>>>(tb, fa, job_count, jobs); }
+        { ScopedKernel t("k_fold_scale", st); k_fold_scale<DNNS_BF16><<<grid, kTileThreads, 0, st>>>(job_count, jobs); }
+    }
     return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 

@@ -65,6 +65,7 @@ struct WsMap {
     uint64_t k_dev, bitmap, sel, tie_prefix, tie_split, layouts, ebits, rowmax, colmax;
     uint64_t vec_items, extrema_bounds;
     uint64_t casc_rem0, casc_rem1, casc_lost, casc_live, casc_changed;
+    uint64_t fold_count, fold_jobs;  // the conv+BN fusion's list of tiles that hold rebuilt weights
     uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
     uint64_t any_need, need, tie_bitmap, tile_ties, hist1, hist2;
     uint64_t total;
@@ -236,6 +237,8 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.casc_lost = take(4ull * c.keep_words);
     w.casc_live = take(4ull * (c.out_words + c.in_words));
     w.casc_changed = take(4ull * (kMaxCascadePasses + 1));
+    w.fold_count = take(4);
+    w.fold_jobs = take(sizeof(FoldJob) * (uint64_t)c.tiles);
     w.clear_begin = o;
     w.any_need = take(4);
     w.need = take(4 * vs);
@@ -922,7 +925,8 @@ dnns_status dnns_fold_batchnorm(dnns_plan* p, void* dst_arena, const uint64_t* d
     if (!p || !dst_arena || !dst_offsets_dev || !dst_shapes_dev) return DNNS_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(dst_arena) & (kAlign - 1)) return DNNS_ERR_INVALID_ARG;
     ProfileScope profile_scope(p);
-    const int n = launch_fold(p->tb, dst_arena, dst_offsets_dev, dst_shapes_dev, static_cast<cudaStream_t>(stream));
+    const int n = launch_fold(p->tb, dst_arena, dst_offsets_dev, dst_shapes_dev, reinterpret_cast<uint32_t*>(p->ws + p->map.fold_count),
+                              reinterpret_cast<FoldJob*>(p->ws + p->map.fold_jobs), p->n_sm, static_cast<cudaStream_t>(stream));
     if (n < 0) return DNNS_ERR_CUDA;
     p->launches += n;
     return DNNS_OK;
