@@ -18,7 +18,8 @@
 //                     chunk's (zeroed) slot of the workspace;
 //   k_deflate_scan    exclusive scan of the chunk sizes -> chunk offsets;
 //   k_deflate_pack    moves every slot to its byte offset in the stream;
-//   k_inflate         per chunk: every lane decodes its sub-block straight into the destination.
+//   k_inflate         per group of chunks: stored chunks copied and the others zeroed by the whole block, then a
+//                     thread per sub-block (taken in order of size) decodes it and stores the non-zero bytes.
 #include "dnns_internal.cuh"
 
 namespace dnns {
@@ -283,133 +284,183 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_deflate_pack(const uint
     }
 }
 
-// One lane's output, written straight into its own 512 bytes of the destination (16-byte aligned):
-// literals are collected into words, repeats go out as words and vectors once aligned.  L2 merges
-// the partial lines.
-struct ByteOut {
-    uint8_t* dst;
-    uint32_t n = 0, acc = 0;
-    __device__ __forceinline__ explicit ByteOut(uint8_t* d) : dst(d) {}
-    __device__ __forceinline__ void push(uint32_t b) {
-        acc |= b << (8 * (n & 3));
-        if ((++n & 3) == 0) {
-            *reinterpret_cast<uint32_t*>(dst + n - 4) = acc;
-            acc = 0;
-        }
-    }
-    __device__ __forceinline__ void repeat(uint32_t b, uint32_t times) {
-        while (times && (n & 3)) push(b), --times;
-        const uint32_t s = b * 0x01010101u;
-        while (times >= 4 && (n & 15)) *reinterpret_cast<uint32_t*>(dst + n) = s, n += 4, times -= 4;
-        for (; times >= 16; times -= 16, n += 16) *reinterpret_cast<uint4*>(dst + n) = make_uint4(s, s, s, s);
-        for (; times >= 4; times -= 4, n += 4) *reinterpret_cast<uint32_t*>(dst + n) = s;
-        while (times) push(b), --times;
-    }
-    __device__ __forceinline__ void finish() {  // the data may end inside a word
-        for (uint32_t j = 0; j < (n & 3); ++j) dst[(n & ~3u) + j] = (uint8_t)(acc >> (8 * j));
-    }
-};
+// ---- the decoder
+// What the next 9 stream bits (as a code, first bit on top) say, for all 512 values: bits the code takes, whether
+// it is a literal (its value) or a length (base, number of extra bits), or something this decoder rejects.
+//   bits 0..8   literal value, or length base - 3 (0..255)
+//   bits 9..12  code bits (7, 8, 9)
+//   bits 13..15 extra bits of a length
+//   bit 16      length (a match follows); bit 17: rejected (end of block before the data is there, unassigned symbol)
+__device__ __forceinline__ uint32_t token_entry(uint32_t code9) {
+    uint32_t sym, used;
+    if ((code9 >> 2) <= 0x17) sym = 256 + (code9 >> 2), used = 7;
+    else if ((code9 >> 1) <= 0xBF) sym = (code9 >> 1) - 0x30, used = 8;
+    else if ((code9 >> 1) <= 0xC7) sym = 280 + (code9 >> 1) - 0xC0, used = 8;
+    else sym = 144 + code9 - 0x190, used = 9;
+    if (sym < 256) return sym | (used << 9);
+    const uint32_t idx = sym - 257;
+    if (sym == 256 || idx > 28) return (used << 9) | (1u << 17);
+    uint32_t base, e = 0;
+    if (idx < 8) base = idx;
+    else if (idx == 28) base = 255;
+    else e = (idx >> 2) - 1, base = (4 + (idx & 3)) << e;
+    return base | (used << 9) | (e << 13) | (1u << 16);
+}
 
-__global__ void __launch_bounds__(kWarpsPerBlock * 32) k_inflate(const uint32_t* __restrict__ stream_w, uint64_t stream_bytes,
-                                                                  const uint64_t* __restrict__ chunk_offset,
-                                                                  const uint32_t* __restrict__ sub_bits, uint64_t n_bytes,
-                                                                  uint32_t n_chunks, uint8_t* dst, uint32_t* status) {
-    const int lane = threadIdx.x & 31;
+// A block takes groups of kGroup chunks, one sub-block per thread.  First all its threads prepare the group's
+// destination together: a stored chunk is copied, a chunk of fixed Huffman codes is zeroed (whole lines).  The
+// sub-blocks differ a lot in tokens - a dense one has 512 literals, a masked one a handful of matches - and the
+// index says how many bits each one has, so the threads take them in order of size: the lanes of a warp then walk
+// about equally many tokens, in one loop that is the same for literals and matches (read 32 bits at the lane's bit
+// position, look the code up, advance).  Only non-zero bytes are stored: a match on a zero (nearly every match,
+// the masked weights) just moves the output position on.
+constexpr uint32_t kGroup = 4;
+constexpr int kInflateThreads = kGroup * kSubs;
+
+__global__ void __launch_bounds__(kInflateThreads) k_inflate(const uint32_t* __restrict__ stream_w, uint64_t stream_bytes,
+                                                             const uint64_t* __restrict__ chunk_offset,
+                                                             const uint32_t* __restrict__ sub_bits, uint64_t n_bytes,
+                                                             uint32_t n_chunks, uint8_t* dst, uint32_t* status) {
+    __shared__ uint32_t s_token[512];
+    __shared__ uint64_t s_off[kGroup + 1];
+    __shared__ uint32_t s_type[kGroup];  // 0 stored, 1 fixed Huffman, 3 nothing to decode (rejected)
+    __shared__ uint32_t s_key[kInflateThreads];
+    __shared__ uint16_t s_take[kInflateThreads];
+    for (uint32_t r = threadIdx.x; r < 512; r += kInflateThreads) s_token[r] = token_entry(r);
     const uint64_t n_words = (stream_bytes + 3) / 4;
     auto word = [&](uint64_t i) -> uint32_t { return i < n_words ? __ldg(stream_w + i) : 0u; };
     auto fail = [&]() { atomicCAS(status, 0u, (uint32_t)DNNS_ERR_UNSUPPORTED); };
-    for (uint32_t c = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); c < n_chunks; c += gridDim.x * kWarpsPerBlock) {
-        const uint64_t c0 = (uint64_t)c * kChunk;
-        const uint32_t n = (uint32_t)min((uint64_t)kChunk, n_bytes - c0);
-        const uint32_t lo = min(n, lane * kSub), n_lane = min(n - lo, kSub);
-        const uint64_t off = chunk_offset[c];
-        if (off >= stream_bytes) {
-            fail();
-            continue;
-        }
-        const uint32_t type = ((word(off >> 2) >> (8 * (off & 3))) >> 1) & 3u;
-        uint8_t* out = dst + c0 + lo;
-        if (type == 0) {
-            // stored: the lane's bytes start 5 + lo bytes into the chunk
-            const uint64_t a = off + 5 + lo;
-            const uint32_t shift = (uint32_t)(a & 3);
-            const uint64_t w0 = a >> 2;
-            for (uint32_t j = 0; j < n_lane / 4; ++j) {
-                const uint32_t x = shift ? __funnelshift_r(word(w0 + j), word(w0 + j + 1), 8 * shift) : word(w0 + j);
-                reinterpret_cast<uint32_t*>(out)[j] = x;
+    const uint32_t n_groups = (n_chunks + kGroup - 1) / kGroup;
+    for (uint32_t g = blockIdx.x; g < n_groups; g += gridDim.x) {
+        const uint32_t c_first = g * kGroup, c_count = min(kGroup, n_chunks - c_first);
+        __syncthreads();  // the previous group is done with the shared state
+        if (threadIdx.x <= c_count) {
+            const uint64_t off = chunk_offset[c_first + threadIdx.x];  // (the array has one entry past the last chunk)
+            s_off[threadIdx.x] = off;
+            if (threadIdx.x < c_count) {
+                uint32_t type = 3;
+                if (off < stream_bytes) type = ((word(off >> 2) >> (8 * (off & 3))) >> 1) & 3u;
+                if (type >= 2) {
+                    fail();
+                    type = 3;
+                }
+                s_type[threadIdx.x] = type;
             }
-            for (uint32_t j = n_lane & ~3u; j < n_lane; ++j) {
-                const uint64_t b = a + j;
-                out[j] = (uint8_t)(word(b >> 2) >> (8 * (b & 3)));
+        }
+        __syncthreads();
+        // ---- all threads: copy the stored chunks, zero the others
+        for (uint32_t k = 0; k < c_count; ++k) {
+            const uint64_t c0 = (uint64_t)(c_first + k) * kChunk;
+            const uint32_t n = (uint32_t)min((uint64_t)kChunk, n_bytes - c0);
+            uint8_t* chunk = dst + c0;
+            if (s_type[k] == 0) {
+                // the chunk's bytes start 5 bytes into its block
+                const uint64_t a = s_off[k] + 5;
+                const uint32_t shift = (uint32_t)(a & 3);
+                const uint64_t w0 = a >> 2;
+                for (uint32_t j = threadIdx.x; j < n / 4; j += kInflateThreads)
+                    reinterpret_cast<uint32_t*>(chunk)[j] = shift ? __funnelshift_r(word(w0 + j), word(w0 + j + 1), 8 * shift) : word(w0 + j);
+                for (uint32_t j = (n & ~3u) + threadIdx.x; j < n; j += kInflateThreads) {
+                    const uint64_t b = a + j;
+                    chunk[j] = (uint8_t)(word(b >> 2) >> (8 * (b & 3)));
+                }
+            } else if (s_type[k] == 1) {
+                const uint32_t n_vec = n / 16;
+                for (uint32_t j = threadIdx.x; j < n_vec; j += kInflateThreads) reinterpret_cast<uint4*>(chunk)[j] = make_uint4(0, 0, 0, 0);
+                for (uint32_t j = n_vec * 16 + threadIdx.x; j < n; j += kInflateThreads) chunk[j] = 0;
             }
-            continue;
         }
-        if (type != 1) {
-            fail();
-            continue;
+        // ---- the sub-blocks in order of their size in the stream (0 where there is nothing to decode)
+        {
+            const uint32_t k = threadIdx.x / kSubs, sb = threadIdx.x % kSubs;
+            uint32_t size = 0;
+            if (k < c_count && s_type[k] == 1) {
+                const uint32_t* bits = sub_bits + (size_t)(c_first + k) * kSubs;
+                const uint64_t end = sb + 1 < kSubs ? bits[sb + 1] : (s_off[k + 1] - s_off[k]) * 8;
+                const uint32_t start = bits[sb];
+                size = end > start ? (uint32_t)min(end - start, (uint64_t)0xFFFFFFu) : 1u;
+            }
+            s_key[threadIdx.x] = (size << 8) | threadIdx.x;  // no two alike
         }
-        // fixed Huffman codes: the lane reads tokens from its bit offset until its bytes are there
-        const uint64_t pos = off * 8 + sub_bits[(size_t)c * kSubs + lane];
-        uint64_t wi = pos >> 5;
-        uint64_t buf = (uint64_t)word(wi) >> (pos & 31);
-        uint32_t have = 32 - (uint32_t)(pos & 31);
-        // the stream words behind the bit buffer: four being used up, four more already requested
-        uint32_t a0 = word(wi + 1), a1 = word(wi + 2), a2 = word(wi + 3), a3 = word(wi + 4);
-        uint32_t b0 = word(wi + 5), b1 = word(wi + 6), b2 = word(wi + 7), b3 = word(wi + 8);
-        uint32_t left = 4;
-        wi += 9;  // the next word to request
-        ByteOut bo(out);
-        uint32_t prev = 0;
-        bool ok = true;
-        while (bo.n < n_lane) {
-            if (have <= 32) {
-                buf |= (uint64_t)a0 << have;
-                have += 32;
-                a0 = a1, a1 = a2, a2 = a3;
-                if (--left == 0) {
-                    a0 = b0, a1 = b1, a2 = b2, a3 = b3;
-                    b0 = word(wi), b1 = word(wi + 1), b2 = word(wi + 2), b3 = word(wi + 3);
-                    wi += 4;
-                    left = 4;
+        __syncthreads();  // also orders the zeroes before the bytes
+        {
+            const uint32_t mine = s_key[threadIdx.x];
+            uint32_t rank = 0;
+            for (uint32_t j = 0; j < (uint32_t)kInflateThreads; ++j) rank += s_key[j] < mine;
+            s_take[rank] = (uint16_t)threadIdx.x;
+        }
+        __syncthreads();
+        const uint32_t which = s_take[threadIdx.x], k = which / kSubs, lane_sb = which % kSubs;
+        bool busy = false;
+        const uint32_t* wp = stream_w;   // stream words from the one with the chunk's first byte
+        uint64_t w_left = 0;             // words from wp to the end of the stream
+        uint8_t* out = nullptr;
+        uint32_t n_lane = 0, pos = 0, acc = 0, prev = 0;
+        // the bits ahead: at least 33 of them in buf at every token, the stream word after them already on its way
+        uint64_t buf = 0;
+        uint32_t have = 0, nxt = 0, wi = 0;
+        auto stream_word = [&](uint32_t i) -> uint32_t { return i < w_left ? __ldg(wp + i) : 0u; };
+        if (k < c_count && s_type[k] == 1) {
+            const uint64_t c0 = (uint64_t)(c_first + k) * kChunk;
+            const uint32_t n = (uint32_t)min((uint64_t)kChunk, n_bytes - c0);
+            const uint32_t lo = min(n, lane_sb * kSub);
+            n_lane = min(n - lo, kSub);
+            const uint64_t off = s_off[k];
+            out = dst + c0 + lo;
+            wp = stream_w + (off >> 2);
+            w_left = n_words - (off >> 2);
+            const uint32_t bit = 8 * (uint32_t)(off & 3) + sub_bits[(size_t)(c_first + k) * kSubs + lane_sb];
+            wi = bit >> 5;
+            buf = (((uint64_t)stream_word(wi + 1) << 32) | stream_word(wi)) >> (bit & 31);
+            have = 64 - (bit & 31);
+            nxt = stream_word(wi + 2);
+            wi += 3;
+            busy = n_lane != 0;
+        }
+        while (__any_sync(kFull, busy)) {
+            if (busy) {
+                const uint32_t x = (uint32_t)buf;  // the next 32 stream bits
+                const uint32_t t = s_token[__brev(x) >> 23];
+                uint32_t used = (t >> 9) & 15u;
+                if (t & (3u << 16)) {
+                    // a length: extra bits, then the 5-bit distance code, which must say distance 1
+                    const uint32_t e = (t >> 13) & 7u, rest = x >> used;
+                    const uint32_t len = 3u + (t & 511u) + (rest & ((1u << e) - 1u));
+                    used += e + 5;
+                    if ((t >> 17) || ((rest >> e) & 31u) != 0 || pos == 0 || pos + len > n_lane) {
+                        busy = false;
+                        fail();
+                    } else if (prev == 0) {
+                        // zeros are there already; a word in the making is complete (the run covers its rest)
+                        if (pos & 3) *reinterpret_cast<uint32_t*>(out + (pos & ~3u)) = acc, acc = 0;
+                        pos += len;
+                    } else {
+                        for (uint32_t q = 0; q < len; ++q) {
+                            acc |= prev << (8 * (pos & 3));
+                            if ((++pos & 3) == 0) *reinterpret_cast<uint32_t*>(out + pos - 4) = acc, acc = 0;
+                        }
+                    }
+                } else {
+                    prev = t & 255u;
+                    acc |= prev << (8 * (pos & 3));
+                    if ((++pos & 3) == 0) {
+                        if (acc) *reinterpret_cast<uint32_t*>(out + pos - 4) = acc;
+                        acc = 0;
+                    }
+                }
+                buf >>= used, have -= used;
+                if (have <= 32) {
+                    buf |= (uint64_t)nxt << have;
+                    have += 32;
+                    nxt = stream_word(wi++);
+                }
+                if (busy && pos >= n_lane) {
+                    // the data may end inside a word
+                    for (uint32_t j = 0; j < (pos & 3); ++j) out[(pos & ~3u) + j] = (uint8_t)(acc >> (8 * j));
+                    busy = false;
                 }
             }
-            const uint32_t code9 = __brev((uint32_t)buf) >> 23;  // the next 9 bits as a code, first bit on top
-            uint32_t sym, used;
-            if ((code9 >> 2) <= 0x17) sym = 256 + (code9 >> 2), used = 7;
-            else if ((code9 >> 1) <= 0xBF) sym = (code9 >> 1) - 0x30, used = 8;
-            else if ((code9 >> 1) <= 0xC7) sym = 280 + (code9 >> 1) - 0xC0, used = 8;
-            else sym = 144 + code9 - 0x190, used = 9;
-            if (sym < 256) {
-                buf >>= used, have -= used;
-                bo.push(sym);
-                prev = sym;
-                continue;
-            }
-            const uint32_t idx = sym - 257;
-            if (sym == 256 || idx > 28 || bo.n == 0) {  // early end of block, unassigned symbol, nothing to repeat
-                ok = false;
-                break;
-            }
-            uint32_t len, e = 0;
-            if (idx < 8) len = 3 + idx;
-            else if (idx == 28) len = 258;
-            else {
-                e = (idx >> 2) - 1;
-                len = 3 + ((4 + (idx & 3)) << e);
-            }
-            const uint32_t rest = (uint32_t)(buf >> used);
-            len += rest & ((1u << e) - 1u);
-            const uint32_t dist_code = (rest >> e) & 31u;
-            used += e + 5;
-            if (dist_code != 0 || bo.n + len > n_lane) {  // only distance 1 is decoded here
-                ok = false;
-                break;
-            }
-            buf >>= used, have -= used;
-            bo.repeat(prev, len);
         }
-        bo.finish();
-        if (!ok) fail();
     }
 }
 
@@ -431,8 +482,8 @@ size_t deflate_workspace_bytes(uint32_t n_chunks) { return (size_t)n_chunks * kS
 
 int launch_inflate(const void* stream_in, uint64_t stream_bytes, const uint64_t* chunk_offset, const uint32_t* sub_bits,
                    uint64_t n_bytes, uint32_t n_chunks, void* dst, uint32_t* status, cudaStream_t st) {
-    const uint32_t blocks = (n_chunks + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    k_inflate<<<blocks, kWarpsPerBlock * 32, 0, st>>>(static_cast<const uint32_t*>(stream_in), stream_bytes, chunk_offset,
+    const uint32_t blocks = (n_chunks + kGroup - 1) / kGroup;
+    k_inflate<<<blocks, kInflateThreads, 0, st>>>(static_cast<const uint32_t*>(stream_in), stream_bytes, chunk_offset,
                                                       sub_bits, n_bytes, n_chunks, static_cast<uint8_t*>(dst), status);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
