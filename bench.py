@@ -588,6 +588,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph replay")
     ap.add_argument("--no-also", action="store_true", help="skip the other target configurations (resnet152 bf16, resnet50 f32)")
     ap.add_argument("--no-extras", action="store_true", help="skip fold / cascade / deflate / frozen-streams figures")
+    ap.add_argument("--extras-only", action="store_true",
+                    help="one untimed portfolio step, then only the fold / cascade / deflate figures (a short run to profile those kernels)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.stepwise:
@@ -628,8 +630,16 @@ def main():
     ms_per_variant_of = lambda ms_per_step, V: whole_job_ms_per_variant(ms_per_step, V, world)
     peak, peak_kind = load_peaks()
 
-    cfg = Config(args, args.workload, dtype, device, pinned_host=True)
+    cfg = Config(args, args.workload, dtype, device, pinned_host=not args.extras_only)
     wl, V = cfg.wl, cfg.V
+    if args.extras_only:
+        cfg.step()
+        torch.cuda.synchronize()
+        fold, cascade, deflate = extras(cfg, cfg.variant_sizes())
+        if rank == 0:
+            print(json.dumps({"extras_only": True, "config": config_of(wl, dtype), "fold_batchnorm": fold, "cascade": cascade,
+                              "deflate": deflate}))
+        return
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
