@@ -148,7 +148,7 @@ def run_reference(args, wl, dtype):
 
 FLUSH_BYTES = 512 << 20
 KERNELS = ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_ties", "k_tie_scan", "k_extrema_sweep", "k_extrema_flags",
-           "k_sweep<", "k_sweep_multi", "k_flags", "k_propagate", "k_rebuild_layout", "k_compact_gather"]
+           "k_sweep<", "k_sweep_multi", "k_flags", "k_shift_zero", "k_propagate", "k_rebuild_layout", "k_compact_gather"]
 
 
 def item_sizes(wl, keep_count, eb):

@@ -176,7 +176,7 @@ uint64_t dnns_plan_launch_count(const dnns_plan* plan);
  * on while a stream is being captured); dnns_plan_profile(plan, 0) stops recording.
  * dnns_plan_profile_read synchronises the device and returns the summed device time and the number of
  * recorded launches of the kernels whose name starts with `kernel` ("k_sweep", "k_compact_gather",
- * "k_flags", "k_propagate", "k_rebuild_layout", "k_hist1", "k_hist2", "k_ties", "k_select1", "k_select2",
+ * "k_flags", "k_shift_zero", "k_propagate", "k_rebuild_layout", "k_hist1", "k_hist2", "k_ties", "k_select1", "k_select2",
  * "k_tie_scan", "k_extrema_sweep", "k_extrema_flags").
  */
 dnns_status dnns_plan_profile(dnns_plan* plan, int32_t enable);

@@ -175,6 +175,7 @@ struct Tables {
     const uint32_t* flag_unit_tensor;  // [n_flag_units] the tensor a unit belongs to
     uint32_t* ebits;        // packed "element is non-zero" bits of the latest sweep (same packing as the mask bits)
     uint32_t* status;       // device status word (a dnns_status, 0 = ok)
+    uint32_t* shift_zero;   // per producer and channel (packed like the filter flags): a zero filter emits a structurally zero constant
     const uint32_t* extrema_bounds;  // [extrema_blocks + 1] tile ranges of the blocks of the extrema sweep (about equal cost)
     const uint32_t* vec_items;  // [n_vec_items][2] pieces of the vector items (BatchNorm vectors, biases) of the rebuild: item, piece
     uint32_t n_tensors, n_groups, n_bn, n_segs, n_items, n_tiles, n_flag_units, n_vec_items, extrema_blocks;

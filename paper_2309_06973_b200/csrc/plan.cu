@@ -65,6 +65,7 @@ struct WsMap {
     uint64_t k_dev, bitmap, sel, tie_prefix, tie_split, layouts, ebits, rowmax, colmax;
     uint64_t vec_items, extrema_bounds;
     uint64_t casc_rem0, casc_rem1, casc_lost, casc_live, casc_changed;
+    uint64_t shift_zero;             // bit words of the keep propagation's statistics
     uint64_t fold_count, fold_jobs;  // the conv+BN fusion's list of tiles that hold rebuilt weights
     uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
     uint64_t any_need, need, tie_bitmap, tile_ties, hist1, hist2;
@@ -237,6 +238,7 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.casc_lost = take(4ull * c.keep_words);
     w.casc_live = take(4ull * (c.out_words + c.in_words));
     w.casc_changed = take(4ull * (kMaxCascadePasses + 1));
+    w.shift_zero = take(4ull * (c.out_words + 1));
     w.fold_count = take(4);
     w.fold_jobs = take(sizeof(FoldJob) * (uint64_t)c.tiles);
     w.clear_begin = o;
@@ -564,6 +566,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     tb.producers = reinterpret_cast<ProducerDesc*>(w + map.producers);
     tb.consumers = reinterpret_cast<ConsumerDesc*>(w + map.consumers);
     tb.status = reinterpret_cast<uint32_t*>(w + map.status);
+    tb.shift_zero = reinterpret_cast<uint32_t*>(w + map.shift_zero);
     tb.flag_prefix = reinterpret_cast<uint32_t*>(w + map.flag_prefix);
     tb.flag_unit_tensor = reinterpret_cast<uint32_t*>(w + map.flag_unit_tensor);
     tb.ebits = reinterpret_cast<uint32_t*>(w + map.ebits);

@@ -114,7 +114,7 @@ __device__ __forceinline__ void finalize_group(const Tables& tb, const GroupDesc
                                                uint32_t removed_local, uint32_t* s_rem, const uint32_t* s_lost,
                                                uint32_t* s_pre, uint32_t* scratch, uint32_t* s_rekept,
                                                uint32_t* keep_bits, int32_t* keep_idx, int32_t* keep_count,
-                                               unsigned long long* stats) {
+                                               unsigned long long* stats, const uint32_t* __restrict__ shift_bits = nullptr) {
     const int C = gd.C;
     const int n_words = (C + 31) / 32;
     uint32_t removed;
@@ -157,9 +157,26 @@ __device__ __forceinline__ void finalize_group(const Tables& tb, const GroupDesc
         const uint32_t rem = s_rem[j >> 5], bit = 1u << (j & 31);
         if (!(rem & bit)) {
             keep_idx[gd.off_idx + s_pre[j >> 5] + __popc(~rem & (bit - 1u))] = j;
-        } else if (stats && (s_lost[j >> 5] & bit)) {
+        } else if (stats && !shift_bits && (s_lost[j >> 5] & bit)) {
             for (int p = gd.prod_begin; p < gd.prod_end; ++p)
                 if (!shift_zero(tb, p, j)) ++lost_pairs;
+        }
+    }
+    if (stats && shift_bits) {
+        // the same count word by word from the prepared bits: removed channels that somebody still reads, against
+        // every producer's "constant is zero" word (eight producers' words requested together)
+        constexpr int kProd = 8;
+        for (int w = threadIdx.x; w < n_words; w += kThreads) {
+            const uint32_t lost = s_rem[w] & s_lost[w];
+            if (!lost) continue;
+            for (int p0 = gd.prod_begin; p0 < gd.prod_end; p0 += kProd) {
+                uint32_t z[kProd];
+#pragma unroll
+                for (int t = 0; t < kProd; ++t)
+                    z[t] = p0 + t < gd.prod_end ? shift_bits[tb.producers[p0 + t].off_outnz + w] : 0xffffffffu;
+#pragma unroll
+                for (int t = 0; t < kProd; ++t) lost_pairs += __popc(lost & ~z[t]);
+            }
         }
     }
     if (threadIdx.x == 0) keep_count[g] = (int32_t)carry;
@@ -189,6 +206,22 @@ __global__ void __launch_bounds__(kThreads) k_propagate(Tables tb, const uint32_
                    keep_count, stats);
 }
 
+// For the statistics: per producer (an entry of the producer list) and channel, whether the constant a zero filter
+// still emits is structurally zero - the same for every variant of a call, so it is worked out once, a block per
+// producer, a warp per word.
+__global__ void __launch_bounds__(kThreads) k_shift_zero(Tables tb) {
+    const int p = blockIdx.x;
+    const int C = tb.tensors[tb.prod_list[p]].O;
+    const int n_words = (C + 31) / 32, lane = threadIdx.x & 31;
+    uint32_t* out = tb.shift_zero + tb.producers[p].off_outnz;
+    for (int w = threadIdx.x >> 5; w < n_words; w += kThreads / 32) {
+        const int j = w * 32 + lane;
+        const bool zero = j < C ? shift_zero(tb, p, j) : true;
+        const uint32_t word = __ballot_sync(0xffffffffu, zero);
+        if (lane == 0) out[w] = word;
+    }
+}
+
 // The same for the variants of one multi-variant sweep in one launch: blockIdx.y picks the variant's buffers.
 struct PropagateMultiArgs {
     const uint32_t* out_nz[kPortfolioMax];
@@ -210,7 +243,7 @@ __global__ void __launch_bounds__(kThreads) k_propagate_multi(Tables tb, Propaga
     const GroupDesc gd = tb.groups[g];
     const uint32_t removed_local = eval_group(tb, gd, pa.out_nz[v], pa.in_nz[v], policy, s_prod, s_cons, s_rem);
     finalize_group(tb, gd, g, min_keep, removed_local, s_rem, s_prod, s_pre, scratch, &s_rekept, pa.keep_bits[v],
-                   pa.keep_idx[v], pa.keep_count[v], stats ? stats + 4 * v : nullptr);
+                   pa.keep_idx[v], pa.keep_count[v], stats ? stats + 4 * v : nullptr, tb.shift_zero);
 }
 
 // ---- fixed point: the rule applied pass after pass on kernel maps restricted to what is still kept
@@ -364,10 +397,16 @@ int launch_propagate_multi(const Tables& tb, int n_variants, const uint32_t* con
         pa.out_nz[v] = out_nz[v], pa.in_nz[v] = in_nz[v];
         pa.keep_bits[v] = keep_bits[v], pa.keep_idx[v] = keep_idx[v], pa.keep_count[v] = keep_count[v];
     }
+    int launches = 1;
+    if (stats) {
+        ScopedKernel timed("k_shift_zero", st);
+        k_shift_zero<<<tb.n_tensors, kThreads, 0, st>>>(tb);  // the producer list has an entry per tensor
+        ++launches;
+    }
     ScopedKernel timed("k_propagate", st);
     k_propagate_multi<<<dim3(tb.n_groups, n_variants), kThreads, 0, st>>>(tb, pa, policy, min_keep,
                                                                         reinterpret_cast<unsigned long long*>(stats));
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
 int launch_propagate_cascade(const Tables& tb, const CascadeWs& cw, const uint32_t* nz_map, uint32_t policy,
