@@ -147,7 +147,7 @@ def run_reference(args, wl, dtype):
 
 
 FLUSH_BYTES = 512 << 20
-KERNELS = ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_ties", "k_tie_scan", "k_extrema_sweep", "k_extrema_flags",
+KERNELS = ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_ties", "k_tie_scan", "k_extrema_rows", "k_extrema_sweep", "k_extrema_flags",
            "k_sweep<", "k_sweep_multi", "k_flags", "k_shift_zero", "k_propagate", "k_rebuild_layout", "k_compact_gather"]
 
 
@@ -347,7 +347,11 @@ def measure(cfg, steps, warmup, barrier, max_over_ranks, ms_per_variant_of, peak
         sweeps = f"stepwise: mask sweep and structure sweep per variant; {thr_sweeps} ranking sweeps"
     stepwise_bytes = N * eb * (1 + 3 * V) + V * N / 8 + sum(rebuild)   # one read per input, one write per output of every step
 
-    kernel_alg = {"k_hist1": N * eb, "k_hist2": N * eb, "k_ties": N * eb if ties_swept else 0, "k_extrema_sweep": N * eb,
+    # the sweep for the largest keys walks tensors with long rows of whole 16-byte vectors row by row, the rest tile by tile
+    by_rows = sum(t.numel for t in wl.tensors if (t.I * t.KH * t.KW * eb) % 16 == 0 and t.I * t.KH * t.KW * eb // 16 >= 96)
+    all_weights = sum(t.numel for t in wl.tensors)
+    kernel_alg = {"k_hist1": N * eb, "k_hist2": N * eb, "k_ties": N * eb if ties_swept else 0,
+                  "k_extrema_rows": by_rows * eb, "k_extrema_sweep": (all_weights - by_rows) * eb,
                   "k_compact_gather": statistics.mean(rebuild) if (cfg.path != "sparse_free" or args.rebuild_per_variant)
                   else sum(rebuild) / ((V + 15) // 16),      # one launch rebuilds up to 16 variants
                   "k_sweep<": (3 * N * eb + N / 4) / 2 if cfg.path == "stepwise" else 2 * N * eb + N / 4}

@@ -177,7 +177,7 @@ uint64_t dnns_plan_launch_count(const dnns_plan* plan);
  * dnns_plan_profile_read synchronises the device and returns the summed device time and the number of
  * recorded launches of the kernels whose name starts with `kernel` ("k_sweep", "k_compact_gather",
  * "k_flags", "k_shift_zero", "k_propagate", "k_rebuild_layout", "k_hist1", "k_hist2", "k_ties", "k_select1", "k_select2",
- * "k_tie_scan", "k_extrema_sweep", "k_extrema_flags").
+ * "k_tie_scan", "k_extrema_rows", "k_extrema_sweep", "k_extrema_flags").
  */
 dnns_status dnns_plan_profile(dnns_plan* plan, int32_t enable);
 dnns_status dnns_plan_profile_read(dnns_plan* plan, const char* kernel, double* total_ms, uint64_t* launches);

@@ -33,6 +33,7 @@ struct TensorDesc {
     uint32_t tile0, n_tiles;
     uint32_t off_mask, off_nzmap, off_outnz, off_innz;  // word offsets into the packed bit arrays
     uint32_t off_row, off_col;  // element offsets of the tensor's filters / input columns in the per-row / per-column tables
+    uint32_t by_rows, pad;      // the sweep for the largest keys walks this tensor row by row (long rows of whole vectors)
 };
 
 struct GroupDesc {
@@ -160,6 +161,30 @@ struct SelectState {
     uint32_t pad;
 };
 
+// A piece of work of the row-walking sweep for the largest keys: a block of rows (filters) of one tensor by a chunk of
+// at most kExtremaChunkVecs 16-byte vectors of every row.
+constexpr uint32_t kExtremaChunkVecs = 128;   // four vectors per lane of a warp
+constexpr uint32_t kExtremaMinVecs = 96;      // rows shorter than this stay with the tile-walking sweep
+constexpr uint32_t kExtremaUnitBytes = 256 * 1024;
+struct ExtremaUnit {
+    uint32_t tensor, row0, n_rows;
+    uint32_t vec0, n_vec;  // the chunk: vectors [vec0, vec0 + n_vec) of a row
+    uint32_t pad[3];
+};
+// Whether the row-walking sweep takes a tensor of O rows of L elements, and how it cuts it.
+__host__ __device__ inline bool extrema_by_rows(uint64_t O, uint64_t L, uint32_t elem_bytes, uint32_t* n_chunks, uint32_t* rows_per_unit) {
+    const uint64_t row_bytes = L * elem_bytes;
+    if (row_bytes % 16 != 0 || row_bytes / 16 < kExtremaMinVecs || row_bytes >= (1ull << 31)) return false;
+    const uint32_t nv = (uint32_t)(row_bytes / 16);
+    const uint32_t chunks = (nv + kExtremaChunkVecs - 1) / kExtremaChunkVecs;
+    const uint32_t chunk_bytes = (nv < kExtremaChunkVecs ? nv : kExtremaChunkVecs) * 16;
+    uint32_t rows = kExtremaUnitBytes / chunk_bytes;
+    rows = rows < 8 ? 8 : rows;
+    if (rows > O) rows = (uint32_t)O;
+    *n_chunks = chunks, *rows_per_unit = rows;
+    return true;
+}
+
 struct Tables {
     const TensorDesc* tensors;
     const GroupDesc* groups;
@@ -177,6 +202,8 @@ struct Tables {
     uint32_t* status;       // device status word (a dnns_status, 0 = ok)
     uint32_t* shift_zero;   // per producer and channel (packed like the filter flags): a zero filter emits a structurally zero constant
     const uint32_t* extrema_bounds;  // [extrema_blocks + 1] tile ranges of the blocks of the extrema sweep (about equal cost)
+    const ExtremaUnit* extrema_units;  // [n_extrema_units] work of the row-walking extrema sweep
+    uint32_t n_extrema_units, pad_units;
     const uint32_t* vec_items;  // [n_vec_items][2] pieces of the vector items (BatchNorm vectors, biases) of the rebuild: item, piece
     uint32_t n_tensors, n_groups, n_bn, n_segs, n_items, n_tiles, n_flag_units, n_vec_items, extrema_blocks;
     uint32_t tile_elems;    // 4096 (fp32) or 8192 (bf16)
@@ -262,7 +289,7 @@ int launch_rebuild_layout(const Tables& tb, const LayoutBatch& lb, int n_layouts
 int launch_compact(const Tables& tb, const GatherBatch& gb, int n_sm, cudaStream_t st, const dnns_threshold* thr = nullptr,
                    const TieSplit* split = nullptr);
 int gather_grid(int n_sm);  // blocks of the gather kernel (the layout is cut for this many)
-int launch_extrema(const Tables& tb, uint32_t* rowmax, uint32_t* colmax, int n_sm, cudaStream_t st);
+int launch_extrema(const Tables& tb, uint32_t* rowmax, uint32_t* colmax, int n_sm, cudaStream_t st);  // (one or two launches)
 int launch_extrema_flags(const Tables& tb, const uint32_t* rowmax, const uint32_t* colmax, const dnns_threshold* thr,
                          const TieSplit* split, int first_variant, int n_variants, uint32_t* const* out_nz,
                          uint32_t* const* in_nz, cudaStream_t st);

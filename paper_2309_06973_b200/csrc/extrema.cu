@@ -15,6 +15,7 @@
 //                    row length divides the tile, a thread meets the same columns in every tile and
 //                    keeps them in registers; otherwise per-vector maxima go to a table in shared
 //                    memory.  The table is merged into global memory when the block changes tensor.
+//   k_extrema_rows   the same maxima for tensors with long rows of whole 16-byte vectors, row by row (below).
 //   k_extrema_flags  per (variant, flag word): 32 comparisons, one ballot, one store.
 #include "dnns_internal.cuh"
 
@@ -42,6 +43,10 @@ __global__ void __launch_bounds__(kTileThreads, 3) k_extrema(Tables tb, uint32_t
         // ---- per-tensor context: constant over the run of tiles [tile, span_end)
         const TensorDesc& d = tb.tensors[tb.tile_tensor[tile]];
         const uint32_t span_end = min(hi, d.tile0 + d.n_tiles);
+        if (d.by_rows) {  // the row-walking sweep's
+            tile = span_end;
+            continue;
+        }
         const uint32_t numel = d.numel, tile0 = d.tile0, KK = d.KK, I = d.I, L = I * KK;
         const char* src = static_cast<const char*>(d.src);
         uint32_t* g_row = rowmax + d.off_row;
@@ -241,6 +246,89 @@ __global__ void __launch_bounds__(kTileThreads, 3) k_extrema(Tables tb, uint32_t
     }
 }
 
+// The same maxima for tensors with long rows of whole 16-byte vectors, row by row: a block takes a unit (a block of
+// rows by a chunk of at most 128 vectors of every row), a warp takes every eighth row of it, a lane the vectors
+// lane, lane + 32, .. of the chunk.  A lane thus meets the same columns in every row and keeps their maxima in
+// registers - no index arithmetic per key - and a row's maximum is one warp reduction and one atomic per row and
+// chunk.  At the end of the unit the warps' column maxima meet in shared memory and go out, one atomic per
+// element column.
+template <int DT>
+__global__ void __launch_bounds__(kTileThreads, 3) k_extrema_rows(Tables tb, uint32_t* __restrict__ rowmax, uint32_t* __restrict__ colmax) {
+    constexpr int P = Elem<DT>::kPerVec;
+    constexpr int kV = kExtremaChunkVecs / 32;  // vectors of a row per lane
+    constexpr uint32_t kKeyMask = DT == DNNS_F32 ? 0x7FFFFFFFu : 0x7FFF7FFFu;
+    constexpr int kWarps = kTileThreads / 32;
+    __shared__ uint32_t s_col[kExtremaChunkVecs * P];  // largest key per element column of the chunk
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (uint32_t unit = blockIdx.x; unit < tb.n_extrema_units; unit += gridDim.x) {
+        const ExtremaUnit un = tb.extrema_units[unit];
+        const TensorDesc& d = tb.tensors[un.tensor];
+        const uint32_t KK = d.KK, L = (uint32_t)d.I * KK;
+        const size_t row_bytes = (size_t)L * Elem<DT>::kBytes;
+        const char* chunk = static_cast<const char*>(d.src) + (size_t)un.vec0 * 16;
+        for (uint32_t i = threadIdx.x; i < kExtremaChunkVecs * P; i += kTileThreads) s_col[i] = 0;
+        __syncthreads();
+        uint32_t acc[kV][4];
+#pragma unroll
+        for (int k = 0; k < kV; ++k)
+#pragma unroll
+            for (int w = 0; w < 4; ++w) acc[k][w] = 0;
+        uint4 nxt[kV];
+        auto issue = [&](uint32_t r) {
+            const uint4* p = reinterpret_cast<const uint4*>(chunk + (size_t)r * row_bytes);
+#pragma unroll
+            for (int k = 0; k < kV; ++k)
+                nxt[k] = (uint32_t)(lane + 32 * k) < un.n_vec ? __ldg(p + lane + 32 * k) : make_uint4(0, 0, 0, 0);
+        };
+        const uint32_t r_end = un.row0 + un.n_rows;
+        uint32_t r = un.row0 + warp;
+        if (r < r_end) issue(r);
+        for (; r < r_end; r += kWarps) {
+            uint4 v[kV];
+#pragma unroll
+            for (int k = 0; k < kV; ++k) v[k] = nxt[k];
+            if (r + kWarps < r_end) issue(r + kWarps);
+            uint32_t m = 0;
+#pragma unroll
+            for (int k = 0; k < kV; ++k) {
+                const uint32_t w[4] = {v[k].x & kKeyMask, v[k].y & kKeyMask, v[k].z & kKeyMask, v[k].w & kKeyMask};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    acc[k][q] = DT == DNNS_F32 ? max(acc[k][q], w[q]) : __vmaxu2(acc[k][q], w[q]);
+                    m = DT == DNNS_F32 ? max(m, w[q]) : __vmaxu2(m, w[q]);
+                }
+            }
+            if (DT == DNNS_BF16) m = max(m & 0xFFFFu, m >> 16);
+            m = __reduce_max_sync(kFull, m);
+            if (lane == 0 && m) atomicMax(&rowmax[d.off_row + r], m);
+        }
+        // the warps' column maxima meet in shared memory
+#pragma unroll
+        for (int k = 0; k < kV; ++k) {
+            const uint32_t vi = lane + 32 * k;
+            if (vi >= un.n_vec) continue;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (DT == DNNS_F32) {
+                    if (acc[k][q]) atomicMax(&s_col[vi * P + q], acc[k][q]);
+                } else {
+                    const uint32_t a = acc[k][q] & 0xFFFFu, b = acc[k][q] >> 16;
+                    if (a) atomicMax(&s_col[vi * P + 2 * q], a);
+                    if (b) atomicMax(&s_col[vi * P + 2 * q + 1], b);
+                }
+            }
+        }
+        __syncthreads();
+        // element columns to input columns (KK elements each)
+        const uint32_t e0 = un.vec0 * P, n_e = un.n_vec * P;
+        for (uint32_t i = threadIdx.x; i < n_e; i += kTileThreads) {
+            const uint32_t m = s_col[i];
+            if (m) atomicMax(&colmax[d.off_col + (KK == 1 ? e0 + i : (e0 + i) / KK)], m);
+        }
+        __syncthreads();
+    }
+}
+
 // Per-variant arguments of the flag kernel.
 struct ExtremaFlagArgs {
     int32_t variant[kPortfolioMax];
@@ -319,10 +407,19 @@ __global__ void __launch_bounds__(256) k_extrema_flags(Tables tb, const uint32_t
 
 int launch_extrema(const Tables& tb, uint32_t* rowmax, uint32_t* colmax, int n_sm, cudaStream_t st) {
     const dim3 grid(min((uint32_t)n_sm * 3u, tb.n_tiles));  // three resident blocks per SM
+    int launches = 1;
+    if (tb.n_extrema_units) {
+        // tensors with long rows of whole vectors, row by row (most of a CNN's weights); the rest tile by tile
+        const dim3 grid_rows(min((uint32_t)n_sm * 3u, tb.n_extrema_units));
+        ScopedKernel timed("k_extrema_rows", st);
+        if (tb.dtype == DNNS_F32) k_extrema_rows<DNNS_F32><<<grid_rows, kTileThreads, 0, st>>>(tb, rowmax, colmax);
+        else k_extrema_rows<DNNS_BF16><<<grid_rows, kTileThreads, 0, st>>>(tb, rowmax, colmax);
+        ++launches;
+    }
     ScopedKernel timed("k_extrema_sweep", st);
     if (tb.dtype == DNNS_F32) k_extrema<DNNS_F32><<<grid, kTileThreads, 0, st>>>(tb, rowmax, colmax);
     else k_extrema<DNNS_BF16><<<grid, kTileThreads, 0, st>>>(tb, rowmax, colmax);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
 int launch_extrema_flags(const Tables& tb, const uint32_t* rowmax, const uint32_t* colmax, const dnns_threshold* thr,

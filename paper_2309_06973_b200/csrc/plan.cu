@@ -63,7 +63,7 @@ struct WsMap {
     uint64_t tensors, groups, bns, segs, items, tile_tensor, prod_list, cons_list, producers, consumers, flag_prefix, flag_unit_tensor, status;
     uint64_t tables_end;  // everything before this is uploaded once at plan creation
     uint64_t k_dev, bitmap, sel, tie_prefix, tie_split, layouts, ebits, rowmax, colmax;
-    uint64_t vec_items, extrema_bounds;
+    uint64_t vec_items, extrema_bounds, extrema_units;
     uint64_t casc_rem0, casc_rem1, casc_lost, casc_live, casc_changed;
     uint64_t shift_zero;             // bit words of the keep propagation's statistics
     uint64_t fold_count, fold_jobs;  // the conv+BN fusion's list of tiles that hold rebuilt weights
@@ -76,6 +76,7 @@ struct Counts {
     uint32_t T = 0, G = 0, B = 0, S = 0, items = 0, tiles = 0, n_bias = 0;
     uint64_t mask_words = 0, keep_words = 0, out_words = 0, in_words = 0, flag_units = 0;
     uint64_t sum_O = 0, sum_I = 0;           // filters / input columns of all tensors
+    uint32_t extrema_units = 0;              // units of the row-walking sweep for the largest keys
     uint32_t n_vec = 0, element_units = 0;   // vector items of the rebuild; 16 KB units its element path can need at most
     int dtype = 0, elem_bytes = 4;
 };
@@ -155,6 +156,11 @@ dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts*
         c->in_words += ((uint64_t)t.I + 31) / 32;
         c->flag_units += flag_units_of(t);
         if (t.bias) ++c->n_bias;
+        {
+            uint32_t chunks, rows;
+            if (extrema_by_rows(t.O, (uint64_t)t.I * t.KH * t.KW, c->elem_bytes, &chunks, &rows))
+                c->extrema_units += chunks * (((uint32_t)t.O + rows - 1) / rows);
+        }
         {   // tensors the rebuild cannot stage take its element path: 16 KB units, at most the whole tensor
             ItemDesc probe{};
             probe.Cin = t.I / t.in_spatial, probe.blk = t.KH * t.KW * t.in_spatial, probe.elem_bytes = c->elem_bytes;
@@ -221,6 +227,7 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.flag_unit_tensor = take(4ull * (c.flag_units + 1));
     w.vec_items = take(8ull * (c.n_vec + 1));
     w.extrema_bounds = take(4ull * (kMaxSweepBlocks + 1));
+    w.extrema_units = take(sizeof(ExtremaUnit) * (uint64_t)(c.extrema_units + 1));
     w.status = take(4);
     w.tables_end = o;
     const uint64_t vs = (uint64_t)maxv * (c.S ? c.S : 1);
@@ -263,6 +270,7 @@ struct dnns_plan {
     char* ws;
     Tables tb;
     ThresholdWs tws;
+    uint32_t n_extrema_units = 0;
     // Layouts of the rebuild prepared for sets of keep counts: the device array a dnns_propagate_keep* call wrote
     // its counts to names the slot its layout went to; dnns_compact looks its keep_count argument up here.
     std::vector<const int32_t*> layout_owner;
@@ -491,6 +499,23 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
         producers[i] = pd;
     }
     for (int i = 0; i < nc; ++i) consumers[i] = ConsumerDesc{td[cons_list[i]].off_innz, td[cons_list[i]].S};
+    {   // the row-walking sweep for the largest keys: its tensors and their units
+        auto* units = reinterpret_cast<ExtremaUnit*>(host.data() + map.extrema_units);
+        uint32_t n_units = 0;
+        for (uint32_t i = 0; i < c.T; ++i) {
+            uint32_t chunks, rows;
+            const uint64_t L = (uint64_t)td[i].I * td[i].KK;
+            td[i].by_rows = extrema_by_rows(td[i].O, L, c.elem_bytes, &chunks, &rows) ? 1u : 0u;
+            if (!td[i].by_rows) continue;
+            const uint32_t nv = (uint32_t)(L * c.elem_bytes / 16);
+            for (uint32_t r0 = 0; r0 < (uint32_t)td[i].O; r0 += rows)
+                for (uint32_t ch = 0; ch < chunks; ++ch) {
+                    const uint32_t v0 = ch * kExtremaChunkVecs;
+                    units[n_units++] = ExtremaUnit{i, r0, std::min(rows, (uint32_t)td[i].O - r0), v0, std::min(kExtremaChunkVecs, nv - v0), {0, 0, 0}};
+                }
+        }
+        p->n_extrema_units = n_units;
+    }
     {   // tile ranges of the extrema sweep: about equal cost per block; a tile whose column maxima stay in registers
         // (rows that divide the tile) counts 2, any other tile 3
         auto* bounds = reinterpret_cast<uint32_t*>(host.data() + map.extrema_bounds);
@@ -500,7 +525,8 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
         for (uint32_t i = 0; i < c.T; ++i) {
             const uint64_t L = (uint64_t)td[i].I * td[i].KK;
             const bool cheap = L <= tile_elems && tile_elems % L == 0 && L % vec == 0 && (uint32_t)td[i].I <= 8192u;
-            for (uint32_t k = 0; k < td[i].n_tiles; ++k) cost_before[td[i].tile0 + k + 1] = cheap ? 2 : 3;
+            // (the tiles of a tensor that the row-walking sweep takes cost this one nothing)
+            for (uint32_t k = 0; k < td[i].n_tiles; ++k) cost_before[td[i].tile0 + k + 1] = td[i].by_rows ? 0 : (cheap ? 2 : 3);
         }
         for (uint32_t t = 0; t < c.tiles; ++t) cost_before[t + 1] += cost_before[t];
         uint32_t t = 0;
@@ -590,6 +616,8 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     tb.n_vec_items = c.n_vec;
     tb.extrema_bounds = reinterpret_cast<uint32_t*>(w + map.extrema_bounds);
     tb.extrema_blocks = tb_extrema_blocks;
+    tb.extrema_units = reinterpret_cast<ExtremaUnit*>(w + map.extrema_units);
+    tb.n_extrema_units = p->n_extrema_units;
     p->layout_owner.assign(layout_slots(maxv), nullptr);
     p->layout_next = 0;
     if (cudaStreamCreateWithFlags(&p->side, cudaStreamNonBlocking) != cudaSuccess ||
