@@ -228,7 +228,9 @@ struct ThresholdWs {
     uint32_t* tile_ties;    // [max_variants][n_tiles]: weights equal to tau_v in the tile
     uint32_t* tie_prefix;   // [max_variants][n_tiles]: those in earlier tiles of the segment
     TieSplit* split;        // [n_k][S]
+    uint32_t* hist_done;    // [1] blocks of the first sweep that are done (NULL: the digit selection is a launch of its own)
 };
+constexpr uint32_t kFusedSelectSegs = 4;  // up to this many segments the first sweep's last block selects the digits
 
 constexpr int kMultiMax = DNNS_MULTI_MAX;  // variants one multi-variant sweep can produce
 constexpr int kPortfolioMax = DNNS_PORTFOLIO_MAX;  // variants one portfolio-wide call (zero structures, keep sets) can take

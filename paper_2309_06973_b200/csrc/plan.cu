@@ -68,7 +68,7 @@ struct WsMap {
     uint64_t shift_zero;             // bit words of the keep propagation's statistics
     uint64_t fold_count, fold_jobs;  // the conv+BN fusion's list of tiles that hold rebuilt weights
     uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
-    uint64_t any_need, need, tie_bitmap, tile_ties, hist1, hist2;
+    uint64_t any_need, hist_done, need, tie_bitmap, tile_ties, hist1, hist2;
     uint64_t total;
 };
 
@@ -250,6 +250,7 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.fold_jobs = take(sizeof(FoldJob) * (uint64_t)c.tiles);
     w.clear_begin = o;
     w.any_need = take(4);
+    w.hist_done = take(4);
     w.need = take(4 * vs);
     w.tie_bitmap = take(4ull * kBitmapWords * (c.S ? c.S : 1));
     w.tile_ties = take(4ull * maxv * c.tiles);
@@ -609,6 +610,7 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     t.sel = reinterpret_cast<SelectState*>(w + map.sel);
     t.need = reinterpret_cast<uint32_t*>(w + map.need);
     t.any_need = reinterpret_cast<uint32_t*>(w + map.any_need);
+    t.hist_done = reinterpret_cast<uint32_t*>(w + map.hist_done);
     t.tile_ties = reinterpret_cast<uint32_t*>(w + map.tile_ties);
     t.tie_prefix = reinterpret_cast<uint32_t*>(w + map.tie_prefix);
     t.split = reinterpret_cast<TieSplit*>(w + map.tie_split);

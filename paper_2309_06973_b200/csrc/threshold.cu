@@ -104,6 +104,152 @@ __device__ __forceinline__ void for_filtered_keys(const uint4 (&v)[kVecPerThread
     }
 }
 
+// ---------------------------------------------------------------- select 1
+// One block per segment (or the last block of the first sweep, segment after segment).
+// Prune counts handed over as a kernel argument (no copy to stage, nothing to capture but the launch).
+constexpr int kInlineCounts = 64;
+struct InlineCounts {
+    uint64_t k[kInlineCounts];
+};
+
+// What select 1 keeps in shared memory.
+struct Select1Shared {
+    uint64_t scratch[33];
+    uint64_t k[kMaxVariants];
+    uint32_t digit[kMaxVariants];
+};
+
+// The selection for one segment, by all 1024 threads of a block (the block of k_select1, or the block of the first
+// sweep that finished last).
+template <int DT>
+__device__ __forceinline__ void select1_segment(const Tables& tb, const ThresholdWs& ws, uint32_t seg, int n_k,
+                                                dnns_threshold* __restrict__ thr, const InlineCounts& counts,
+                                                bool counts_inline, Select1Shared& sm) {
+    uint64_t* const scratch = sm.scratch;
+    uint64_t* const s_k = sm.k;
+    uint32_t* const s_digit = sm.digit;
+    const uint32_t S = tb.n_segs;
+    if ((int)threadIdx.x < n_k) {
+        const size_t idx = (size_t)threadIdx.x * S + seg;
+        s_k[threadIdx.x] = counts_inline ? counts.k[idx] : ws.k_dev[idx];  // one round trip for all k
+    }
+    // A warp owns 1024 consecutive bins = 256 vectors of four; a lane loads vectors lane, lane + 32, .. of them, so
+    // that every load of the warp is one contiguous 512 bytes (a thread reading its own 32 consecutive bins would
+    // touch 32 lines per load, and one SM keeps only so many requests in flight).  Bin order inside the warp: group
+    // j (32 vectors), lane, element.  (A segment holds fewer than 2^32 keys: 32-bit sums.)
+    const uint32_t* h = ws.hist1 + (size_t)seg * kHistBins;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint4* hv = reinterpret_cast<const uint4*>(h) + warp * 256;
+    uint32_t c[32], gs[8], before[8];  // the lane's bins; the sum of its vector in group j; keys of the warp before that vector
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint4 v = __ldcg(hv + j * 32 + lane);  // (written by other blocks' atomics)
+        c[4 * j] = v.x, c[4 * j + 1] = v.y, c[4 * j + 2] = v.z, c[4 * j + 3] = v.w;
+        gs[j] = v.x + v.y + v.z + v.w;
+    }
+    uint32_t warp_sum = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        uint32_t incl = gs[j];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+        }
+        before[j] = warp_sum + incl - gs[j];
+        warp_sum += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    uint64_t total;
+    const uint64_t warp_base = __shfl_sync(0xffffffffu, block_exclusive_scan<uint64_t>(lane == 0 ? warp_sum : 0u, scratch, &total), 0);
+    uint32_t* bm = ws.bitmap + (size_t)seg * kBitmapWords;
+    bm[threadIdx.x] = 0;  // 1024 words
+    for (int v = 0; v < n_k; ++v) {
+        const uint64_t k = s_k[v];  // published by the barriers of the scan above
+        SelectState* st = &ws.sel[(size_t)v * S + seg];
+        if (k == 0) {
+            if (threadIdx.x == 0) {
+                *st = SelectState{0, 0, 0xFFFFFFFFu, 0, 0, 0};
+                s_digit[v] = 0xFFFFFFFFu;
+            }
+            continue;
+        }
+        // the vector of this thread whose keys reach rank k, then the first of its four bins that does (one thread)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint64_t start = warp_base + before[j];
+            if (start < k && k <= start + gs[j]) {
+                uint64_t cum = start;
+                int b = 0;
+                uint32_t cnt = 0;
+                bool found = false;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (!found) {
+                        if (cum + c[4 * j + q] >= k) {
+                            b = q;
+                            cnt = c[4 * j + q];
+                            found = true;
+                        } else {
+                            cum += c[4 * j + q];
+                        }
+                    }
+                }
+                const uint32_t digit = (uint32_t)warp * 1024u + (uint32_t)(j * 32 + lane) * 4u + (uint32_t)b;
+                *st = SelectState{k, cum, digit, 0, cnt, 0};
+                s_digit[v] = digit;
+            }
+        }
+    }
+    __syncthreads();
+    if ((int)threadIdx.x < n_k) {
+        // variants that selected the same first digit share one second-pass histogram: its slot is
+        // the rank of the digit among the distinct selected digits of the segment
+        const uint32_t dg = s_digit[threadIdx.x];
+        if (dg != 0xFFFFFFFFu) {
+            uint32_t slot = 0;
+            for (int u = 0; u < n_k; ++u) {
+                const uint32_t du = s_digit[u];
+                bool first = du != 0xFFFFFFFFu && du < dg;  // count each smaller digit once
+                for (int t = 0; t < u && first; ++t)
+                    if (s_digit[t] == du) first = false;
+                slot += first;
+            }
+            ws.sel[(size_t)threadIdx.x * S + seg].slot = slot;
+            atomicOr(&bm[dg >> 5], 1u << (dg & 31));
+        }
+    }
+    if (DT == DNNS_BF16) {
+        // a 15-bit key is fully resolved by the first digit
+        __syncthreads();
+        if ((int)threadIdx.x < n_k) {
+            const int v = threadIdx.x;
+            const SelectState st = ws.sel[(size_t)v * S + seg];
+            dnns_threshold r{0, 0, 0, 0, 0};
+            uint32_t need = 0;
+            if (st.k) {
+                r.tau_bits = st.digit;
+                r.n_below = st.below;
+                r.n_tie = st.k - st.below;
+                r.n_equal = st.count;
+                need = r.n_tie < r.n_equal;
+            }
+            thr[(size_t)v * S + seg] = r;
+            ws.need[(size_t)v * S + seg] = need;
+            if (need) {
+                atomicOr(ws.any_need, 1u);
+                atomicOr(&ws.tie_bitmap[(size_t)seg * kBitmapWords + (r.tau_bits >> 5)], 1u << (r.tau_bits & 31));
+            }
+        }
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(1024) k_select1(Tables tb, ThresholdWs ws, int n_k, dnns_threshold* __restrict__ thr,
+                                                  InlineCounts counts, bool counts_inline) {
+    __shared__ Select1Shared sm;
+    select1_segment<DT>(tb, ws, blockIdx.x, n_k, thr, counts, counts_inline, sm);
+}
+
 // ---------------------------------------------------------------- pass 1
 // Count one stored word's key(s) by first digit; digit 0 (exact zeros, mostly) in a register.
 template <int DT>
@@ -119,7 +265,9 @@ __device__ __forceinline__ void count_word(uint32_t w, uint32_t* sh, uint32_t& z
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kHistThreads, 1) k_hist1(Tables tb, uint32_t* __restrict__ hist1) {
+__global__ void __launch_bounds__(kHistThreads, 1) k_hist1(Tables tb, ThresholdWs ws, int n_k, dnns_threshold* __restrict__ thr,
+                                                           InlineCounts counts, bool counts_inline, bool then_select) {
+    uint32_t* const hist1 = ws.hist1;
     constexpr uint32_t P = Elem<DT>::kPerVec;
     constexpr int U = 4;
     extern __shared__ uint32_t sh[];  // kHistBins counters
@@ -210,111 +358,20 @@ __global__ void __launch_bounds__(kHistThreads, 1) k_hist1(Tables tb, uint32_t* 
         tile = span_end;
     }
     flush(cur_seg);
-}
-
-// ---------------------------------------------------------------- select 1
-// One block per segment.  Thread t owns bins [32t, 32t+32).
-// Prune counts handed over as a kernel argument (no copy to stage, nothing to capture but the launch).
-constexpr int kInlineCounts = 64;
-struct InlineCounts {
-    uint64_t k[kInlineCounts];
-};
-
-template <int DT>
-__global__ void __launch_bounds__(1024) k_select1(Tables tb, ThresholdWs ws, int n_k, dnns_threshold* __restrict__ thr,
-                                                  InlineCounts counts, bool counts_inline) {
-    __shared__ uint64_t scratch[33];
-    __shared__ uint32_t s_digit[kMaxVariants];
-    __shared__ uint64_t s_k[kMaxVariants];
-    const uint32_t seg = blockIdx.x, S = tb.n_segs;
-    if ((int)threadIdx.x < n_k) {
-        const size_t idx = (size_t)threadIdx.x * S + seg;
-        s_k[threadIdx.x] = counts_inline ? counts.k[idx] : ws.k_dev[idx];  // one round trip for all k
-    }
-    const uint32_t* h = ws.hist1 + (size_t)seg * kHistBins;
-    uint32_t c[32];
-    uint64_t sum = 0;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const uint4 v = reinterpret_cast<const uint4*>(h)[threadIdx.x * 8 + j];
-        c[4 * j] = v.x, c[4 * j + 1] = v.y, c[4 * j + 2] = v.z, c[4 * j + 3] = v.w;
-        sum += (uint64_t)v.x + v.y + v.z + v.w;
-    }
-    uint64_t total;
-    const uint64_t excl = block_exclusive_scan<uint64_t>(sum, scratch, &total);
-    uint32_t* bm = ws.bitmap + (size_t)seg * kBitmapWords;
-    bm[threadIdx.x] = 0;  // 1024 words
-    for (int v = 0; v < n_k; ++v) {
-        const uint64_t k = s_k[v];  // published by the barriers of the scan above
-        SelectState* st = &ws.sel[(size_t)v * S + seg];
-        if (k == 0) {
-            if (threadIdx.x == 0) {
-                *st = SelectState{0, 0, 0xFFFFFFFFu, 0, 0, 0};
-                s_digit[v] = 0xFFFFFFFFu;
-            }
-            continue;
-        }
-        if (excl < k && k <= excl + sum) {
-            // b = the first of this thread's bins whose inclusive prefix reaches k
-            uint64_t cum = excl;
-            int b = 0;
-            uint32_t cnt = 0;
-            bool found = false;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                if (!found) {
-                    if (cum + c[j] >= k) {
-                        b = j;
-                        cnt = c[j];
-                        found = true;
-                    } else {
-                        cum += c[j];
-                    }
-                }
-            }
-            const uint32_t digit = threadIdx.x * 32 + b;
-            *st = SelectState{k, cum, digit, 0, cnt, 0};
-            s_digit[v] = digit;
-        }
-    }
-    __syncthreads();
-    if ((int)threadIdx.x < n_k) {
-        // variants that selected the same first digit share one second-pass histogram: its slot is
-        // the rank of the digit among the distinct selected digits of the segment
-        const uint32_t dg = s_digit[threadIdx.x];
-        if (dg != 0xFFFFFFFFu) {
-            uint32_t slot = 0;
-            for (int u = 0; u < n_k; ++u) {
-                const uint32_t du = s_digit[u];
-                bool first = du != 0xFFFFFFFFu && du < dg;  // count each smaller digit once
-                for (int t = 0; t < u && first; ++t)
-                    if (s_digit[t] == du) first = false;
-                slot += first;
-            }
-            ws.sel[(size_t)threadIdx.x * S + seg].slot = slot;
-            atomicOr(&bm[dg >> 5], 1u << (dg & 31));
-        }
-    }
-    if (DT == DNNS_BF16) {
-        // a 15-bit key is fully resolved by the first digit
+    if (then_select) {
+        // few segments: the block that finishes last selects the first digits at once - it is resident, while a
+        // kernel of its own would have to wait for a free SM beside whatever else is running
+        __shared__ Select1Shared sm;
+        __shared__ uint32_t s_last;
+        __threadfence();  // this thread's additions to the global histograms, before the ticket
         __syncthreads();
-        if ((int)threadIdx.x < n_k) {
-            const int v = threadIdx.x;
-            const SelectState st = ws.sel[(size_t)v * S + seg];
-            dnns_threshold r{0, 0, 0, 0, 0};
-            uint32_t need = 0;
-            if (st.k) {
-                r.tau_bits = st.digit;
-                r.n_below = st.below;
-                r.n_tie = st.k - st.below;
-                r.n_equal = st.count;
-                need = r.n_tie < r.n_equal;
-            }
-            thr[(size_t)v * S + seg] = r;
-            ws.need[(size_t)v * S + seg] = need;
-            if (need) {
-                atomicOr(ws.any_need, 1u);
-                atomicOr(&ws.tie_bitmap[(size_t)seg * kBitmapWords + (r.tau_bits >> 5)], 1u << (r.tau_bits & 31));
+        if (threadIdx.x == 0) s_last = atomicAdd(ws.hist_done, 1u) == gridDim.x - 1;
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            for (uint32_t seg = 0; seg < tb.n_segs; ++seg) {
+                select1_segment<DT>(tb, ws, seg, n_k, thr, counts, counts_inline, sm);
+                __syncthreads();
             }
         }
     }
@@ -381,7 +438,7 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_hist2(Tables tb, ThresholdW
 }
 
 // ---------------------------------------------------------------- select 2 (31-bit keys)
-// One block per (variant, segment).  Thread t owns low digits [64t, 64t+64).
+// One block per (variant, segment).
 __global__ void __launch_bounds__(1024) k_select2(Tables tb, ThresholdWs ws, int n_k, dnns_threshold* __restrict__ thr) {
     __shared__ uint64_t scratch[33];
     const uint32_t S = tb.n_segs;
@@ -395,42 +452,55 @@ __global__ void __launch_bounds__(1024) k_select2(Tables tb, ThresholdWs ws, int
         }
         return;
     }
+    // A warp owns 2048 consecutive bins = 512 vectors of four; a lane loads vectors lane, lane + 32, .. of them: every
+    // load of the warp is one contiguous 512 bytes.  Bin order inside the warp: group j (32 vectors), lane, element.
     const uint32_t* h = ws.hist2 + ((size_t)seg * n_k + st.slot) * kLowBins;
-    uint32_t part[16];  // this thread's 64 bins in groups of four
-    uint64_t sum = 0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint4* hv = reinterpret_cast<const uint4*>(h) + warp * 512;
+    uint32_t part[16], before[16];  // the sum of the lane's vector in group j; keys of the warp before that vector
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-        const uint4 q = reinterpret_cast<const uint4*>(h)[threadIdx.x * 16 + j];
+        const uint4 q = hv[j * 32 + lane];
         part[j] = q.x + q.y + q.z + q.w;
-        sum += part[j];
+    }
+    uint32_t warp_sum = 0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        uint32_t incl = part[j];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+        }
+        before[j] = warp_sum + incl - part[j];
+        warp_sum += __shfl_sync(0xffffffffu, incl, 31);
     }
     uint64_t total;
-    const uint64_t excl = st.below + block_exclusive_scan<uint64_t>(sum, scratch, &total);
-    if (excl < st.k && st.k <= excl + sum) {
-        // the group of four that holds the k-th key, then one more load for its bins
-        uint64_t cum = excl;
-        int jj = 0;
-        bool found = false;
+    const uint64_t warp_base =
+        st.below + __shfl_sync(0xffffffffu, block_exclusive_scan<uint64_t>(lane == 0 ? warp_sum : 0u, scratch, &total), 0);
+    int jj = -1;
+    uint64_t cum = 0;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            if (!found) {
-                if (cum + part[j] >= st.k) jj = j, found = true;
-                else cum += part[j];
-            }
-        }
-        const uint4 q = reinterpret_cast<const uint4*>(h)[threadIdx.x * 16 + jj];
+    for (int j = 0; j < 16; ++j) {
+        const uint64_t start = warp_base + before[j];
+        if (start < st.k && st.k <= start + part[j]) jj = j, cum = start;
+    }
+    if (jj >= 0) {
+        // this thread's vector jj holds the k-th key: one more load for its four bins
+        const uint32_t vec = (uint32_t)warp * 512u + (uint32_t)(jj * 32 + lane);
+        const uint4 q = reinterpret_cast<const uint4*>(h)[vec];
         const uint32_t c4[4] = {q.x, q.y, q.z, q.w};
+        bool found = false;
         uint32_t b = 0, cnt = 0;
-        found = false;
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
             if (!found) {
-                if (cum + c4[t] >= st.k) b = 4 * jj + t, cnt = c4[t], found = true;
+                if (cum + c4[t] >= st.k) b = (uint32_t)t, cnt = c4[t], found = true;
                 else cum += c4[t];
             }
         }
         dnns_threshold r;
-        r.tau_bits = (st.digit << 16) | (threadIdx.x * 64 + b);
+        r.tau_bits = (st.digit << 16) | (vec * 4u + b);
         r.pad = 0;
         r.n_below = cum;
         r.n_tie = st.k - cum;
@@ -639,20 +709,22 @@ int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, const uin
         return -1;
     }
     const int hist_grid = (int)min((uint32_t)n_sm, tb.n_tiles);
+    // few segments: the first sweep's last block selects the first digits itself (one launch less in the chain)
+    const bool fused = ws.hist_done != nullptr && S <= kFusedSelectSegs;
     const int sweep_grid = (int)min((uint32_t)n_sm * 4u, tb.n_tiles);
     int launches = 0;
     if (tb.dtype == DNNS_F32) {
-        { ScopedKernel t("k_hist1", st); k_hist1<DNNS_F32><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws.hist1); }
-        { ScopedKernel t("k_select1", st); k_select1<DNNS_F32><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline); }
+        { ScopedKernel t("k_hist1", st); k_hist1<DNNS_F32><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline, fused); }
+        if (!fused) { ScopedKernel t("k_select1", st); k_select1<DNNS_F32><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline); }
         { ScopedKernel t("k_hist2", st); k_hist2<<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k); }
         { ScopedKernel t("k_select2", st); k_select2<<<S * n_k, 1024, 0, st>>>(tb, ws, n_k, thr_dev); }
         { ScopedKernel t("k_ties", st); k_ties<DNNS_F32><<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k, thr_dev); }
-        launches = 5;
+        launches = fused ? 4 : 5;
     } else {
-        { ScopedKernel t("k_hist1", st); k_hist1<DNNS_BF16><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws.hist1); }
-        { ScopedKernel t("k_select1", st); k_select1<DNNS_BF16><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline); }
+        { ScopedKernel t("k_hist1", st); k_hist1<DNNS_BF16><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline, fused); }
+        if (!fused) { ScopedKernel t("k_select1", st); k_select1<DNNS_BF16><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline); }
         { ScopedKernel t("k_ties", st); k_ties<DNNS_BF16><<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k, thr_dev); }
-        launches = 3;
+        launches = fused ? 2 : 3;
     }
     {
         ScopedKernel t("k_tie_scan", st);
