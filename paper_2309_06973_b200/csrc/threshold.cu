@@ -646,23 +646,43 @@ __global__ void __launch_bounds__(1024) k_tie_scan(Tables tb, ThresholdWs ws, co
     const SegDesc sd = tb.segs[seg];
     const uint32_t* cnt = ws.tile_ties + (size_t)v * tb.n_tiles;
     uint32_t* pre = ws.tie_prefix + (size_t)v * tb.n_tiles;
-    const uint32_t n = sd.tile_end - sd.tile_begin;
-    const uint32_t run = (n + 1023) / 1024;
-    const uint32_t t0 = min(sd.tile_end, sd.tile_begin + threadIdx.x * run), t1 = min(sd.tile_end, t0 + run);
-    uint32_t sum = 0;
-    for (uint32_t t = t0; t < t1; ++t) sum += cnt[t];
-    uint32_t total;
-    const uint32_t ex0 = block_exclusive_scan<uint32_t>(sum, scratch, &total);
+    // a warp owns a contiguous run of tiles and reads them 32 at a time (coalesced); two passes: the warps' sums, then
+    // the prefixes in order
     const dnns_threshold r = thr[idx];
     const uint32_t n_tie = (uint32_t)r.n_tie;  // below n_equal, which fits 32 bits
-    // the tile that holds the tie of rank n_tie lies in the run of exactly one thread
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t n = sd.tile_end - sd.tile_begin, per_warp = (n + 31) / 32;
+    const uint32_t w0 = min(sd.tile_end, sd.tile_begin + warp * per_warp), w1 = min(sd.tile_end, w0 + per_warp);
+    constexpr int kScanBatch = 4;
+    uint32_t warp_sum = 0;
+    for (uint32_t base = w0; base < w1; base += 32 * kScanBatch) {
+        uint32_t c[kScanBatch];
+#pragma unroll
+        for (int i = 0; i < kScanBatch; ++i) c[i] = base + i * 32 + lane < w1 ? cnt[base + i * 32 + lane] : 0u;
+#pragma unroll
+        for (int i = 0; i < kScanBatch; ++i) warp_sum += c[i];
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) warp_sum += __shfl_xor_sync(0xffffffffu, warp_sum, d);
+    uint32_t total;
+    uint32_t before = __shfl_sync(0xffffffffu, block_exclusive_scan<uint32_t>(lane == 0 ? warp_sum : 0u, scratch, &total), 0);
+    // the tile that holds the tie of rank n_tie is found by exactly one thread
     __shared__ uint32_t s_tile, s_want;
-    uint32_t ex = ex0;
-    for (uint32_t t = t0; t < t1; ++t) {
-        pre[t] = ex;
-        const uint32_t c = cnt[t];
-        if (ex <= n_tie && n_tie < ex + c) s_tile = t, s_want = n_tie - ex;
-        ex += c;
+    for (uint32_t base = w0; base < w1; base += 32) {
+        const uint32_t t = base + lane;
+        const uint32_t c = t < w1 ? cnt[t] : 0u;
+        uint32_t incl = c;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+        }
+        const uint32_t ex = before + incl - c;
+        if (t < w1) {
+            pre[t] = ex;
+            if (ex <= n_tie && n_tie < ex + c) s_tile = t, s_want = n_tie - ex;
+        }
+        before += __shfl_sync(0xffffffffu, incl, 31);
     }
     __syncthreads();
     const uint32_t tile = s_tile, want = s_want;  // rank, inside the tile, of the tie that stays
