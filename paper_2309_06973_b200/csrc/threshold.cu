@@ -132,6 +132,7 @@ __device__ __forceinline__ void select1_segment(const Tables& tb, const Threshol
     if ((int)threadIdx.x < n_k) {
         const size_t idx = (size_t)threadIdx.x * S + seg;
         s_k[threadIdx.x] = counts_inline ? counts.k[idx] : ws.k_dev[idx];  // one round trip for all k
+        s_digit[threadIdx.x] = 0xFFFFFFFFu;  // stays so if no bin reaches rank k (weights rewritten under the sweep): nothing selected
     }
     // A warp owns 1024 consecutive bins = 256 vectors of four; a lane loads vectors lane, lane + 32, .. of them, so
     // that every load of the warp is one contiguous 512 bytes (a thread reading its own 32 consecutive bins would
@@ -666,8 +667,11 @@ __global__ void __launch_bounds__(1024) k_tie_scan(Tables tb, ThresholdWs ws, co
     for (int d = 16; d > 0; d >>= 1) warp_sum += __shfl_xor_sync(0xffffffffu, warp_sum, d);
     uint32_t total;
     uint32_t before = __shfl_sync(0xffffffffu, block_exclusive_scan<uint32_t>(lane == 0 ? warp_sum : 0u, scratch, &total), 0);
-    // the tile that holds the tie of rank n_tie is found by exactly one thread
+    // the tile that holds the tie of rank n_tie is found by exactly one thread (the defaults stand only if the counts
+    // do not add up to the record, i.e. the weights were rewritten under the sweeps: a valid tile, a rank nobody has)
     __shared__ uint32_t s_tile, s_want;
+    if (threadIdx.x == 0) s_tile = sd.tile_begin, s_want = 0xFFFFFFFFu;
+    __syncthreads();
     for (uint32_t base = w0; base < w1; base += 32) {
         const uint32_t t = base + lane;
         const uint32_t c = t < w1 ? cnt[t] : 0u;
