@@ -843,7 +843,7 @@ dnns_status dnns_propagate_keep_multi(dnns_plan* p, int32_t n_variants, const ui
                 return DNNS_ERR_INVALID_ARG;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (stats && cudaMemsetAsync(stats, 0, 32 * (size_t)n_variants, st) != cudaSuccess) return DNNS_ERR_CUDA;
+    // (the statistics are cleared by the kernel that prepares their bit words, ahead of the propagation)
     ProfileScope profile_scope(p);
     const int n = launch_propagate_multi(p->tb, n_variants, out_nz, in_nz, policy, min_keep, keep_bits, keep_idx, keep_count,
                                          stats, st);

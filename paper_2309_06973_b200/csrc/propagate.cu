@@ -209,8 +209,10 @@ __global__ void __launch_bounds__(kThreads) k_propagate(Tables tb, const uint32_
 // For the statistics: per producer (an entry of the producer list) and channel, whether the constant a zero filter
 // still emits is structurally zero - the same for every variant of a call, so it is worked out once, a block per
 // producer, a warp per word.
-__global__ void __launch_bounds__(kThreads) k_shift_zero(Tables tb) {
+__global__ void __launch_bounds__(kThreads) k_shift_zero(Tables tb, unsigned long long* __restrict__ stats, int n_stats) {
     const int p = blockIdx.x;
+    if (p == 0)  // the statistics of the propagation that follows start at zero
+        for (int i = threadIdx.x; i < n_stats; i += kThreads) stats[i] = 0;
     const int C = tb.tensors[tb.prod_list[p]].O;
     const int n_words = (C + 31) / 32, lane = threadIdx.x & 31;
     uint32_t* out = tb.shift_zero + tb.producers[p].off_outnz;
@@ -400,7 +402,7 @@ int launch_propagate_multi(const Tables& tb, int n_variants, const uint32_t* con
     int launches = 1;
     if (stats) {
         ScopedKernel timed("k_shift_zero", st);
-        k_shift_zero<<<tb.n_tensors, kThreads, 0, st>>>(tb);  // the producer list has an entry per tensor
+        k_shift_zero<<<tb.n_tensors, kThreads, 0, st>>>(tb, reinterpret_cast<unsigned long long*>(stats), 4 * n_variants);  // the producer list has an entry per tensor
         ++launches;
     }
     ScopedKernel timed("k_propagate", st);
