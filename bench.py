@@ -147,7 +147,7 @@ def run_reference(args, wl, dtype):
 
 
 FLUSH_BYTES = 512 << 20
-KERNELS = ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_ties", "k_tie_scan", "k_extrema_rows", "k_extrema_sweep", "k_extrema_flags",
+KERNELS = ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_tie_find", "k_tie_pick", "k_ties", "k_tie_scan", "k_extrema_rows", "k_extrema_sweep", "k_extrema_flags",
            "k_sweep<", "k_sweep_multi", "k_flags", "k_shift_zero", "k_propagate", "k_rebuild_layout", "k_compact_gather"]
 
 
@@ -290,7 +290,7 @@ def measure(cfg, steps, warmup, barrier, max_over_ranks, ms_per_variant_of, peak
     assert ses.device_status() == B.DNNS_OK
     sizes = cfg.variant_sizes()
     rec = ses.records()
-    ties_swept = bool((rec["n_tie"] < rec["n_equal"]).any())     # the tie sweep only reads the weights when some variant splits its ties
+    ties_swept = ses.tie_sweep_ran()     # the tie sweep reads the weights only when some variant splits its ties and the lists of the second sweep cannot say where
 
     graph, launches_per_step = None, None
     if not args.no_graph:

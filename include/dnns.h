@@ -177,10 +177,23 @@ uint64_t dnns_plan_launch_count(const dnns_plan* plan);
  * dnns_plan_profile_read synchronises the device and returns the summed device time and the number of
  * recorded launches of the kernels whose name starts with `kernel` ("k_sweep", "k_compact_gather",
  * "k_flags", "k_shift_zero", "k_propagate", "k_rebuild_layout", "k_hist1", "k_hist2", "k_ties", "k_select1", "k_select2",
- * "k_tie_scan", "k_extrema_rows", "k_extrema_sweep", "k_extrema_flags").
+ * "k_tie_scan", "k_tie_find", "k_tie_pick", "k_extrema_rows", "k_extrema_sweep", "k_extrema_flags").
  */
 dnns_status dnns_plan_profile(dnns_plan* plan, int32_t enable);
 dnns_status dnns_plan_profile_read(dnns_plan* plan, const char* kernel, double* total_ms, uint64_t* launches);
+
+/*
+ * For reports: whether the latest dnns_magnitude_threshold call read the weights once more to count, tile by tile,
+ * the weights equal to tau (*swept = 1) or not (*swept = 0).  With 32-bit weights the second ranking sweep lists the
+ * keys it counts together with their positions, and the place where a variant stops masking the weights equal to
+ * tau is then found in that list; the extra sweep runs only when no list is kept (16-bit weights; plans with more
+ * than 255 segments or more than 1024 (variant, segment) pairs), when a list cannot answer (it ran over, tau is
+ * zero, or more than 1024 weights equal tau), or later, on demand, when a sweep that masks tile by tile
+ * (dnns_apply_mask, dnns_mask_and_structures, dnns_mask_and_structures_multi) needs the per-tile tables.  Never when
+ * no variant masks only part of the weights equal to tau.  Synchronises the device.
+ * Errors: INVALID_ARG (null), CUDA.
+ */
+dnns_status dnns_plan_tie_sweep(dnns_plan* plan, int32_t* swept);
 
 /*
  * Step 1 - exact k-th-magnitude threshold by radix select over the magnitude keys.

@@ -25,7 +25,7 @@ DNNS_PORTFOLIO_MAX = 16
 EXPORTS = ["dnns_status_string", "dnns_workspace_bytes", "dnns_plan_create", "dnns_plan_destroy", "dnns_plan_layout",
            "dnns_plan_launch_count", "dnns_magnitude_threshold", "dnns_apply_mask", "dnns_zero_structures",
            "dnns_propagate_keep", "dnns_compact", "dnns_last_device_status", "dnns_magnitude_threshold_static", "dnns_mask_and_structures", "dnns_fold_batchnorm", "dnns_propagate_keep_cascade",
-           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_mask_and_structures_multi", "dnns_propagate_keep_multi", "dnns_compact_masked", "dnns_zero_structures_portfolio", "dnns_compact_masked_multi", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
+           "dnns_plan_profile", "dnns_plan_profile_read", "dnns_plan_tie_sweep", "dnns_mask_and_structures_multi", "dnns_propagate_keep_multi", "dnns_compact_masked", "dnns_zero_structures_portfolio", "dnns_compact_masked_multi", "dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes", "dnns_deflate", "dnns_inflate"]
 
 
 class dnns_tensor(C.Structure):
@@ -110,6 +110,7 @@ def lib() -> C.CDLL:
         L.dnns_zero_structures_portfolio.argtypes = [vp, vp, i32, i32, vp, vp, vp]
         L.dnns_compact_masked_multi.argtypes = [vp, vp, i32, i32, vp, vp, vp, C.c_size_t, vp, vp, vp]
         L.dnns_plan_profile.argtypes = [vp, i32]
+        L.dnns_plan_tie_sweep.argtypes = [vp, C.POINTER(i32)]
         L.dnns_plan_profile_read.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(u64)]
         for name in ("dnns_deflate_chunks", "dnns_deflate_bound", "dnns_deflate_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
@@ -235,6 +236,13 @@ def dnns_inflate(stream_dev: int, stream_bytes: int, chunk_offset_dev: int, sub_
 
 def dnns_plan_profile(plan, enable: bool) -> None:
     _check(lib().dnns_plan_profile(plan, int(enable)), "dnns_plan_profile")
+
+
+def dnns_plan_tie_sweep(plan) -> bool:
+    """Whether the latest threshold call (or a masking sweep after it) read the weights once more for the tie tables."""
+    flag = C.c_int32(0)
+    _check(lib().dnns_plan_tie_sweep(plan, C.byref(flag)), "dnns_plan_tie_sweep")
+    return bool(flag.value)
 
 
 def dnns_plan_profile_read(plan, kernel: str):

@@ -229,7 +229,18 @@ struct ThresholdWs {
     uint32_t* tie_prefix;   // [max_variants][n_tiles]: those in earlier tiles of the segment
     TieSplit* split;        // [n_k][S]
     uint32_t* hist_done;    // [1] blocks of the first sweep that are done (NULL: the digit selection is a launch of its own)
+    // 31-bit keys: the second sweep lists the keys it counts with their positions, so that the place where the weights
+    // equal to tau split is found without another sweep (tie_list NULL: no lists, the tie sweep always runs)
+    unsigned long long* tie_list;  // entries: position | low 16 key bits << 32 | histogram slot << 48 | segment << 56
+    uint32_t tie_list_cap;
+    uint32_t* tie_list_n;     // [1] entries appended (may exceed the capacity: then the list is not used)
+    uint32_t* tie_match;      // [n_k][S][kTieMatchCap] positions of the weights equal to tau
+    uint32_t* tie_match_n;    // [n_k][S]
+    uint32_t* tie_fallback;   // [1] set when the lists cannot answer: the tie sweep and its scan run after all
+    const uint32_t* ties_if;  // non-null: the tie sweep and its scan return at once while this word is zero
 };
+constexpr uint32_t kTieMatchCap = 1024;   // weights equal to tau per (variant, segment) that the lists handle
+constexpr uint32_t kTieListMaxSegs = 255, kTieListMaxPairs = 1024;  // segment and slot fit a byte; (variant, segment) pairs in shared memory
 constexpr uint32_t kFusedSelectSegs = 4;  // up to this many segments the first sweep's last block selects the digits
 
 constexpr int kMultiMax = DNNS_MULTI_MAX;  // variants one multi-variant sweep can produce
@@ -270,6 +281,8 @@ struct ScopedKernel {
 // ---- launch wrappers (each returns the number of kernels it launched, or -1 on a CUDA error) ----
 int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, const uint64_t* k_host, dnns_threshold* thr_dev,
                      int n_sm, cudaStream_t st);
+int launch_tie_tables(const Tables& tb, const ThresholdWs& ws, int n_k, const dnns_threshold* thr_dev, int n_sm,
+                      cudaStream_t st);  // per-tile counts of the weights equal to tau and their prefix sums, on their own
 int launch_tile_sweep(const Tables& tb, const ThresholdWs& ws, bool do_mask, bool do_struct,
                       const dnns_threshold* thr_dev, int variant, const void* src_arena, void* dst_arena,
                       uint32_t* mask_bits, uint32_t* nz_map, uint32_t* out_nz, uint32_t* in_nz, uint32_t n_out_words,

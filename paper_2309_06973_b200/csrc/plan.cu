@@ -68,7 +68,8 @@ struct WsMap {
     uint64_t shift_zero;             // bit words of the keep propagation's statistics
     uint64_t fold_count, fold_jobs;  // the conv+BN fusion's list of tiles that hold rebuilt weights
     uint64_t clear_begin;  // [clear_begin, hist2 + used part) is zeroed by every threshold call
-    uint64_t any_need, hist_done, need, tie_bitmap, tile_ties, hist1, hist2;
+    uint64_t any_need, hist_done, tie_list_n, tie_fallback, tie_match_n, need, tie_bitmap, tile_ties, hist1, hist2;
+    uint64_t tie_list, tie_match;  // (outside the cleared region)
     uint64_t total;
 };
 
@@ -76,6 +77,7 @@ struct Counts {
     uint32_t T = 0, G = 0, B = 0, S = 0, items = 0, tiles = 0, n_bias = 0;
     uint64_t mask_words = 0, keep_words = 0, out_words = 0, in_words = 0, flag_units = 0;
     uint64_t sum_O = 0, sum_I = 0;           // filters / input columns of all tensors
+    uint64_t tie_list_entries = 0;           // entries of the second ranking sweep's list (0: the plan keeps none)
     uint32_t extrema_units = 0;              // units of the row-walking sweep for the largest keys
     uint32_t n_vec = 0, element_units = 0;   // vector items of the rebuild; 16 KB units its element path can need at most
     int dtype = 0, elem_bytes = 4;
@@ -178,6 +180,11 @@ dnns_status inspect(const dnns_model* m, dnns_scope scope, int32_t maxv, Counts*
     } else {
         c->S = (uint32_t)seg_count;
     }
+    // 31-bit keys: the second ranking sweep keeps a list of the keys it counts (the tie split then needs no sweep of
+    // its own) where segment and slot fit its entries and the (variant, segment) pairs fit shared memory
+    if (c->dtype == DNNS_F32 && c->S >= 1 && c->S <= kTieListMaxSegs && (uint64_t)maxv * c->S <= kTieListMaxPairs &&
+        c->tiles < (1u << 20))
+        c->tie_list_entries = std::max<uint64_t>(65536, n_prunable / 16);
     std::vector<char> has_bn(m->n_tensors, 0);
     for (int b = 0; b < m->n_bn; ++b) {
         const dnns_bn& bn = m->bns[b];
@@ -248,9 +255,14 @@ WsMap map_workspace(const Counts& c, int32_t maxv) {
     w.shift_zero = take(4ull * (c.out_words + 1));
     w.fold_count = take(4);
     w.fold_jobs = take(sizeof(FoldJob) * (uint64_t)c.tiles);
+    w.tie_list = take(8ull * c.tie_list_entries);
+    w.tie_match = take(c.tie_list_entries ? 4ull * kTieMatchCap * vs : 0);
     w.clear_begin = o;
     w.any_need = take(4);
     w.hist_done = take(4);
+    w.tie_list_n = take(4);
+    w.tie_fallback = take(4);
+    w.tie_match_n = take(4 * vs);
     w.need = take(4 * vs);
     w.tie_bitmap = take(4ull * kBitmapWords * (c.S ? c.S : 1));
     w.tile_ties = take(4ull * maxv * c.tiles);
@@ -271,6 +283,7 @@ struct dnns_plan {
     char* ws;
     Tables tb;
     ThresholdWs tws;
+    bool tie_tables_valid = false;  // the per-tile tables of the weights equal to tau belong to the latest threshold call
     uint32_t n_extrema_units = 0;
     // Layouts of the rebuild prepared for sets of keep counts: the device array a dnns_propagate_keep* call wrote
     // its counts to names the slot its layout went to; dnns_compact looks its keep_count argument up here.
@@ -349,6 +362,18 @@ int prepare_layouts(dnns_plan* p, const int32_t* const* keep_count, int n, cudaS
         ++launches;
     }
     return launches;
+}
+
+// The sweeps that mask tile by tile read per-tile tables of the weights equal to tau.  A threshold call that finds the
+// tie split in the lists of its second sweep does not make them: the first such sweep after it enqueues them (one
+// more read of the weights).
+bool ensure_tie_tables(dnns_plan* p, const dnns_threshold* thr_dev, cudaStream_t st) {
+    if (p->tie_tables_valid) return true;
+    const int n = launch_tie_tables(p->tb, p->tws, p->last_n_k, thr_dev, p->n_sm, st);
+    if (n < 0) return false;
+    p->launches += n;
+    p->tie_tables_valid = true;
+    return true;
 }
 
 }  // namespace
@@ -611,6 +636,13 @@ dnns_status dnns_plan_create(const dnns_model* m, dnns_scope scope, int32_t maxv
     t.need = reinterpret_cast<uint32_t*>(w + map.need);
     t.any_need = reinterpret_cast<uint32_t*>(w + map.any_need);
     t.hist_done = reinterpret_cast<uint32_t*>(w + map.hist_done);
+    t.tie_list = c.tie_list_entries ? reinterpret_cast<unsigned long long*>(w + map.tie_list) : nullptr;
+    t.tie_list_cap = (uint32_t)c.tie_list_entries;
+    t.tie_list_n = reinterpret_cast<uint32_t*>(w + map.tie_list_n);
+    t.tie_match = reinterpret_cast<uint32_t*>(w + map.tie_match);
+    t.tie_match_n = reinterpret_cast<uint32_t*>(w + map.tie_match_n);
+    t.tie_fallback = reinterpret_cast<uint32_t*>(w + map.tie_fallback);
+    t.ties_if = nullptr;
     t.tile_ties = reinterpret_cast<uint32_t*>(w + map.tile_ties);
     t.tie_prefix = reinterpret_cast<uint32_t*>(w + map.tie_prefix);
     t.split = reinterpret_cast<TieSplit*>(w + map.tie_split);
@@ -696,6 +728,7 @@ dnns_status dnns_magnitude_threshold(dnns_plan* p, const uint64_t* k, int32_t n_
     if (!joined || cudaStreamWaitEvent(st, p->ev_join, 0) != cudaSuccess || n < 0 || n_side < 0) return DNNS_ERR_CUDA;
     p->launches += n + n_side;
     p->last_n_k = n_k;
+    p->tie_tables_valid = p->tws.tie_list == nullptr;  // (a call that found the tie split in its lists may have left them out)
     return DNNS_OK;
 }
 
@@ -705,6 +738,7 @@ dnns_status dnns_apply_mask(dnns_plan* p, const dnns_threshold* thr_dev, int32_t
     if (!p || !thr_dev || variant < 0 || variant >= p->last_n_k) return DNNS_ERR_INVALID_ARG;  // a variant of the latest threshold call
     if (masked_arena && (reinterpret_cast<uintptr_t>(masked_arena) & 15)) return DNNS_ERR_INVALID_ARG;
     ProfileScope profile_scope(p);
+    if (!ensure_tie_tables(p, thr_dev, static_cast<cudaStream_t>(stream))) return DNNS_ERR_CUDA;
     const int n = launch_tile_sweep(p->tb, p->tws, true, false, thr_dev, variant, nullptr, masked_arena, mask_bits,
                                     nullptr, nullptr, nullptr, 0, 0, p->n_sm, static_cast<cudaStream_t>(stream));
     if (n < 0) return DNNS_ERR_CUDA;
@@ -738,6 +772,7 @@ dnns_status dnns_mask_and_structures(dnns_plan* p, const dnns_threshold* thr_dev
     const dnns_layout& L = p->layout;
     // the flag words are OR-ed into; the kernel map is stored word by word and needs no clearing
     ProfileScope profile_scope(p);
+    if (!ensure_tie_tables(p, thr_dev, st)) return DNNS_ERR_CUDA;
     const int n = launch_tile_sweep(p->tb, p->tws, true, true, thr_dev, variant, nullptr, masked_arena, mask_bits,
                                     nz_map, out_nz, in_nz, (uint32_t)L.out_nz_words, (uint32_t)L.in_nz_words, p->n_sm, st);
     if (n < 0) return DNNS_ERR_CUDA;
@@ -780,6 +815,7 @@ dnns_status dnns_mask_and_structures_multi(dnns_plan* p, const dnns_threshold* t
     }
     const dnns_layout& L = p->layout;
     ProfileScope profile_scope(p);
+    if (!ensure_tie_tables(p, thr_dev, static_cast<cudaStream_t>(stream))) return DNNS_ERR_CUDA;
     const int n = launch_multi_sweep(p->tb, p->tws, thr_dev, ma, n_variants, nz_map, (uint32_t)L.out_nz_words,
                                      (uint32_t)L.in_nz_words, p->n_sm, static_cast<cudaStream_t>(stream));
     if (n < 0) return DNNS_ERR_CUDA;
@@ -972,6 +1008,18 @@ dnns_status dnns_plan_profile(dnns_plan* p, int32_t enable) {
         p->timer.clear();
     }
     p->timer.on = enable != 0;
+    return DNNS_OK;
+}
+
+dnns_status dnns_plan_tie_sweep(dnns_plan* p, int32_t* swept) {
+    if (!p || !swept) return DNNS_ERR_INVALID_ARG;
+    uint32_t any_need = 0, fallback = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess ||
+        cudaMemcpy(&any_need, p->tws.any_need, sizeof(any_need), cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemcpy(&fallback, p->tws.tie_fallback, sizeof(fallback), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return DNNS_ERR_CUDA;
+    const bool lists = p->tws.tie_list != nullptr;
+    *swept = any_need && (!lists || fallback || p->tie_tables_valid) ? 1 : 0;
     return DNNS_OK;
 }
 

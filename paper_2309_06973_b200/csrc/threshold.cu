@@ -72,7 +72,7 @@ __device__ __forceinline__ void walk_prunable_tiles(const Tables& tb, SpanFn on_
     }
 }
 
-// The keys of a tile that pass a bitmap filter: f(key) is called by the thread holding the key.
+// The keys of a tile that pass a bitmap filter: f(key, element offset in the tile) is called by the thread holding the key.
 // SHIFT32 / the two 16-bit halves select which 15 bits of a stored word index the bitmap.
 template <int DT, int SHIFT32, typename F>
 __device__ __forceinline__ void for_filtered_keys(const uint4 (&v)[kVecPerThread], uint32_t n_e, const uint32_t* bm, F f) {
@@ -99,7 +99,7 @@ __device__ __forceinline__ void for_filtered_keys(const uint4 (&v)[kVecPerThread
             hits &= hits - 1;
             uint32_t x = DT == DNNS_F32 ? j : j >> 1;
             x = x == 0 ? w[0] : (x == 1 ? w[1] : (x == 2 ? w[2] : w[3]));
-            f(DT == DNNS_F32 ? (x & 0x7FFFFFFFu) : ((x >> (16 * (j & 1))) & 0x7FFFu));
+            f(DT == DNNS_F32 ? (x & 0x7FFFFFFFu) : ((x >> (16 * (j & 1))) & 0x7FFFu), (uint32_t)((u * kTileThreads + threadIdx.x) * P + j));
         }
     }
 }
@@ -401,17 +401,35 @@ __device__ __forceinline__ void load_bitmap_with_ranks(const uint32_t* g_bm, uin
     __syncthreads();
 }
 
+constexpr uint32_t kTieStage = 1024;  // listed keys a block of the second sweep holds before it writes them out
+
 __global__ void __launch_bounds__(kTileThreads, 4) k_hist2(Tables tb, ThresholdWs ws, int n_k) {
     __shared__ uint32_t s_bm[kBitmapWords], s_rank[kBitmapWords];
     __shared__ uint32_t scratch[33];
+    __shared__ unsigned long long s_ent[kTieStage];
+    __shared__ uint32_t s_n, s_base;
+    const bool listing = ws.tie_list != nullptr;
+    uint32_t tiles_done = 0;
     int cur_seg = -1;
     uint32_t* h2 = nullptr;
     uint32_t zeros = 0;  // exact zeros among the selected keys: counted in a register, added once
+    if (threadIdx.x == 0) s_n = 0;
     auto flush_zeros = [&]() {
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) zeros += __shfl_xor_sync(0xffffffffu, zeros, d);
         if ((threadIdx.x & 31) == 0 && zeros) atomicAdd(&h2[0], zeros);  // digit 0 has rank 0, low digit 0
         zeros = 0;
+    };
+    // the staged entries go to the list: one reservation for the block (block-uniform; s_n is settled)
+    auto flush_list = [&]() {
+        const uint32_t n = min(s_n, kTieStage);
+        if (threadIdx.x == 0) s_base = atomicAdd(ws.tie_list_n, n);
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < n; i += kTileThreads)
+            if (s_base + i < ws.tie_list_cap) ws.tie_list[s_base + i] = s_ent[i];
+        __syncthreads();
+        if (threadIdx.x == 0) s_n = 0;
+        __syncthreads();
     };
     walk_prunable_tiles<DNNS_F32>(
         tb,
@@ -424,18 +442,81 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_hist2(Tables tb, ThresholdW
             }
             return true;
         },
-        [&](uint32_t, uint32_t n_e, const uint4(&v)[kVecPerThread]) {
-            for_filtered_keys<DNNS_F32, 16>(v, n_e, s_bm, [&](uint32_t key) {
-                if (key == 0) {
-                    ++zeros;
-                    return;
+        [&](uint32_t tile, uint32_t n_e, const uint4(&v)[kVecPerThread]) {
+            // which of the thread's 16 keys have a selected first digit (bit 4 * u + j), and how many of those are not zero
+            uint32_t hits = 0;
+#pragma unroll
+            for (int u = 0; u < kVecPerThread; ++u) {
+                const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                uint32_t h = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) h |= bitmap_test<16>(s_bm, w[q]) << q;
+                if (n_e != kTileBytes / 4) {  // ragged tile: drop the slots past the end of the tensor
+                    const uint32_t first = (u * kTileThreads + threadIdx.x) * 4;
+                    h &= first >= n_e ? 0u : (n_e - first >= 4u ? 0xFu : ((1u << (n_e - first)) - 1u));
                 }
+                hits |= h << (4 * u);
+            }
+            auto key_of = [&](int b) {
+                const int u = b >> 2, q = b & 3;
+                const uint4 x = u == 0 ? v[0] : (u == 1 ? v[1] : (u == 2 ? v[2] : v[3]));
+                return (q == 0 ? x.x : (q == 1 ? x.y : (q == 2 ? x.z : x.w))) & 0x7FFFFFFFu;
+            };
+            uint32_t mine = __popc(hits);  // non-zero selected keys of this thread: they are listed
+            if (s_bm[0] & 1u) {  // digit 0 is selected (a tau below 2^16): exact zeros are counted, not listed
+                mine = 0;
+                for (uint32_t m = hits; m; m &= m - 1) {
+                    const uint32_t key = key_of(__ffs(m) - 1);
+                    if (key == 0) ++zeros, hits &= ~(1u << (__ffs(m) - 1));
+                    else ++mine;
+                }
+            }
+            // the warp reserves its places in the block's stage with one addition
+            uint32_t at = 0;
+            if (listing) {
+                const int lane = threadIdx.x & 31;
+                uint32_t incl = mine;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, d);
+                    if (lane >= d) incl += y;
+                }
+                const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+                uint32_t base = 0;
+                if (total) {
+                    if (lane == 31) base = atomicAdd(&s_n, total);
+                    base = __shfl_sync(0xffffffffu, base, 31);
+                }
+                at = base + incl - mine;
+            }
+            for (uint32_t m = hits; m; m &= m - 1) {
+                const int b = __ffs(m) - 1;
+                const uint32_t key = key_of(b);
                 const uint32_t dg = key >> 16;
                 const uint32_t slot = s_rank[dg >> 5] + __popc(s_bm[dg >> 5] & ((1u << (dg & 31)) - 1u));
                 atomicAdd(&h2[(size_t)slot * kLowBins + (key & 0xFFFFu)], 1u);
-            });
+                if (listing) {
+                    const uint32_t off = ((b >> 2) * kTileThreads + threadIdx.x) * 4 + (b & 3);
+                    const unsigned long long e = (unsigned long long)(tile * (kTileBytes / 4) + off) | ((unsigned long long)(key & 0xFFFFu) << 32) |
+                                                 ((unsigned long long)slot << 48) | ((unsigned long long)cur_seg << 56);
+                    if (at < kTieStage) {
+                        s_ent[at] = e;
+                    } else {  // the stage is full (a tile dense with selected keys): straight to the list
+                        const uint32_t g = atomicAdd(ws.tie_list_n, 1u);
+                        if (g < ws.tie_list_cap) ws.tie_list[g] = e;
+                    }
+                    ++at;
+                }
+            }
+            // every fourth tile the block looks whether the stage is half full (every thread looks at the counter after
+            // its warp's reservation, the last warp to reserve sees them all)
+            if (listing && (++tiles_done & 3) == 0 && __syncthreads_or(s_n >= kTieStage / 2)) flush_list();
         });
     if (cur_seg >= 0) flush_zeros();
+    if (listing) {
+        __syncthreads();
+        if (s_n) flush_list();
+    }
 }
 
 // ---------------------------------------------------------------- select 2 (31-bit keys)
@@ -524,7 +605,7 @@ __global__ void __launch_bounds__(1024) k_select2(Tables tb, ThresholdWs ws, int
 template <int DT>
 __global__ void __launch_bounds__(kTileThreads, 4) k_ties(Tables tb, ThresholdWs ws, int n_k,
                                                           const dnns_threshold* __restrict__ thr) {
-    if (*ws.any_need == 0) return;
+    if (*ws.any_need == 0 || (ws.ties_if && *ws.ties_if == 0)) return;
     // 31-bit keys: a bitmap of the low 15 bits of the thresholds filters the keys, survivors are compared with
     // every threshold.  15-bit keys: a key is its own index into a byte table that names the first variant
     // whose threshold it equals (0: none) - one lookup per key and one counter update per hit, because keys
@@ -573,7 +654,7 @@ __global__ void __launch_bounds__(kTileThreads, 4) k_ties(Tables tb, ThresholdWs
         [&](uint32_t tile, uint32_t n_e, const uint4(&v)[kVecPerThread]) {
             uint32_t zeros = 0;
             if (DT == DNNS_F32) {
-                for_filtered_keys<DT, 0>(v, n_e, s_bm, [&](uint32_t key) {
+                for_filtered_keys<DT, 0>(v, n_e, s_bm, [&](uint32_t key, uint32_t) {
                     if (key == 0) {
                         ++zeros;
                         return;
@@ -640,6 +721,7 @@ __global__ void __launch_bounds__(1024) k_tie_scan(Tables tb, ThresholdWs ws, co
     const uint32_t S = tb.n_segs;
     const uint32_t v = blockIdx.x / S, seg = blockIdx.x % S;
     const size_t idx = (size_t)v * S + seg;
+    if (ws.ties_if && *ws.ties_if == 0) return;  // the lists gave the split
     if (*ws.any_need == 0 || !ws.need[idx]) {
         if (threadIdx.x == 0) ws.split[idx] = TieSplit{0xFFFFFFFFu, 0u};  // no weight equal to tau stays
         return;
@@ -712,6 +794,64 @@ __global__ void __launch_bounds__(1024) k_tie_scan(Tables tb, ThresholdWs ws, co
     }
 }
 
+// ---------------------------------------------------------------- the tie split from the lists (31-bit keys)
+// One pass over the list of the second sweep: the entries whose segment, histogram slot and low key bits are those of a
+// variant's tau are the weights equal to tau; their positions go to the variant's short list.
+__global__ void __launch_bounds__(256) k_tie_find(Tables tb, ThresholdWs ws, int n_k, const dnns_threshold* __restrict__ thr) {
+    __shared__ uint32_t s_code[kTieListMaxPairs];  // segment << 24 | slot << 16 | low 16 bits of tau; 0xFFFFFFFF: not wanted
+    if (*ws.any_need == 0) return;
+    const uint32_t S = tb.n_segs, n_pairs = (uint32_t)n_k * S;
+    for (uint32_t i = threadIdx.x; i < n_pairs; i += blockDim.x) {
+        const uint32_t seg = i % S;
+        const dnns_threshold r = thr[i];
+        s_code[i] = ws.need[i] && r.tau_bits != 0 ? (seg << 24) | (ws.sel[i].slot << 16) | (r.tau_bits & 0xFFFFu) : 0xFFFFFFFFu;
+    }
+    __syncthreads();
+    const uint32_t n = min(*ws.tie_list_n, ws.tie_list_cap);
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const unsigned long long e = ws.tie_list[i];
+        const uint32_t code = (uint32_t)(e >> 32);
+        for (uint32_t q = 0; q < n_pairs; ++q) {
+            if (s_code[q] == code) {
+                const uint32_t at = atomicAdd(&ws.tie_match_n[q], 1u);
+                if (at < kTieMatchCap) ws.tie_match[(size_t)q * kTieMatchCap + at] = (uint32_t)e;
+            }
+        }
+    }
+}
+
+// Per (variant, segment): the weights equal to tau are masked in index order, so the first one that stays is the one
+// with n_tie of them before it.  Where the lists cannot say (they ran over, tau is zero - zeros are not listed -, or
+// there are more equal weights than a short list holds), a flag sends the call to the tie sweep.
+template <int DT>
+__global__ void __launch_bounds__(256) k_tie_pick(Tables tb, ThresholdWs ws, const dnns_threshold* __restrict__ thr) {
+    constexpr uint32_t kTileElems = kTileBytes / Elem<DT>::kBytes;
+    __shared__ uint32_t s_pos[kTieMatchCap];
+    const uint32_t idx = blockIdx.x;
+    if (*ws.any_need == 0 || !ws.need[idx]) {
+        if (threadIdx.x == 0) ws.split[idx] = TieSplit{0xFFFFFFFFu, 0u};  // no weight equal to tau stays
+        return;
+    }
+    const dnns_threshold r = thr[idx];
+    const uint32_t m = ws.tie_match_n[idx];
+    if (*ws.tie_list_n > ws.tie_list_cap || r.tau_bits == 0 || (uint64_t)m != r.n_equal || m > kTieMatchCap) {
+        if (threadIdx.x == 0) atomicOr(ws.tie_fallback, 1u);
+        return;
+    }
+    for (uint32_t i = threadIdx.x; i < m; i += blockDim.x) s_pos[i] = ws.tie_match[(size_t)idx * kTieMatchCap + i];
+    __syncthreads();
+    const uint32_t n_tie = (uint32_t)r.n_tie;
+    for (uint32_t i = threadIdx.x; i < m; i += blockDim.x) {
+        const uint32_t mine = s_pos[i];
+        uint32_t before = 0;
+        for (uint32_t q = 0; q < m; ++q) before += s_pos[q] < mine;
+        if (before == n_tie) {
+            const uint32_t tile = mine / kTileElems, t = tb.tile_tensor[tile];
+            ws.split[idx] = TieSplit{t, (tile - tb.tensors[t].tile0) * kTileElems + mine % kTileElems};
+        }
+    }
+}
+
 }  // namespace
 
 cudaError_t init_kernel_attributes() {
@@ -742,21 +882,47 @@ int launch_threshold(const Tables& tb, const ThresholdWs& ws, int n_k, const uin
         if (!fused) { ScopedKernel t("k_select1", st); k_select1<DNNS_F32><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline); }
         { ScopedKernel t("k_hist2", st); k_hist2<<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k); }
         { ScopedKernel t("k_select2", st); k_select2<<<S * n_k, 1024, 0, st>>>(tb, ws, n_k, thr_dev); }
-        { ScopedKernel t("k_ties", st); k_ties<DNNS_F32><<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k, thr_dev); }
-        launches = fused ? 4 : 5;
+        launches = fused ? 3 : 4;
+        if (ws.tie_list) {
+            // the place where the weights equal to tau split, from the lists of the second sweep; the tie sweep and its
+            // scan stand by behind a flag (huge blocks of equal weights, tau = 0)
+            const int find_grid = (int)min((uint32_t)n_sm * 4u, (ws.tie_list_cap + 255u) / 256u);
+            { ScopedKernel t("k_tie_find", st); k_tie_find<<<find_grid, 256, 0, st>>>(tb, ws, n_k, thr_dev); }
+            { ScopedKernel t("k_tie_pick", st); k_tie_pick<DNNS_F32><<<S * n_k, 256, 0, st>>>(tb, ws, thr_dev); }
+            launches += 2;
+        }
+        ThresholdWs tw = ws;
+        tw.ties_if = ws.tie_list ? ws.tie_fallback : nullptr;
+        { ScopedKernel t("k_ties", st); k_ties<DNNS_F32><<<sweep_grid, kTileThreads, 0, st>>>(tb, tw, n_k, thr_dev); }
+        { ScopedKernel t("k_tie_scan", st); k_tie_scan<DNNS_F32><<<S * n_k, 1024, 0, st>>>(tb, tw, thr_dev); }
+        launches += 2;
     } else {
         { ScopedKernel t("k_hist1", st); k_hist1<DNNS_BF16><<<hist_grid, kHistThreads, kHistBins * 4, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline, fused); }
         if (!fused) { ScopedKernel t("k_select1", st); k_select1<DNNS_BF16><<<S, 1024, 0, st>>>(tb, ws, n_k, thr_dev, counts, counts_inline); }
         { ScopedKernel t("k_ties", st); k_ties<DNNS_BF16><<<sweep_grid, kTileThreads, 0, st>>>(tb, ws, n_k, thr_dev); }
-        launches = fused ? 2 : 3;
+        { ScopedKernel t("k_tie_scan", st); k_tie_scan<DNNS_BF16><<<S * n_k, 1024, 0, st>>>(tb, ws, thr_dev); }
+        launches = fused ? 3 : 4;
     }
-    {
-        ScopedKernel t("k_tie_scan", st);
-        if (tb.dtype == DNNS_F32) k_tie_scan<DNNS_F32><<<S * n_k, 1024, 0, st>>>(tb, ws, thr_dev);
-        else k_tie_scan<DNNS_BF16><<<S * n_k, 1024, 0, st>>>(tb, ws, thr_dev);
-    }
-    ++launches;
     return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+// The per-tile tables of the weights equal to tau on their own (the sweeps that mask tile by tile read them; a
+// threshold call that found the tie split in its lists leaves them out).
+int launch_tie_tables(const Tables& tb, const ThresholdWs& ws, int n_k, const dnns_threshold* thr_dev, int n_sm,
+                      cudaStream_t st) {
+    const uint32_t S = tb.n_segs;
+    const int sweep_grid = (int)min((uint32_t)n_sm * 4u, tb.n_tiles);
+    if (cudaMemsetAsync(ws.tile_ties, 0, 4ull * n_k * tb.n_tiles, st) != cudaSuccess) return -1;
+    ThresholdWs tw = ws;
+    tw.ties_if = nullptr;
+    if (tb.dtype == DNNS_F32) {
+        { ScopedKernel t("k_ties", st); k_ties<DNNS_F32><<<sweep_grid, kTileThreads, 0, st>>>(tb, tw, n_k, thr_dev); }
+        { ScopedKernel t("k_tie_scan", st); k_tie_scan<DNNS_F32><<<S * n_k, 1024, 0, st>>>(tb, tw, thr_dev); }
+    } else {
+        { ScopedKernel t("k_ties", st); k_ties<DNNS_BF16><<<sweep_grid, kTileThreads, 0, st>>>(tb, tw, n_k, thr_dev); }
+        { ScopedKernel t("k_tie_scan", st); k_tie_scan<DNNS_BF16><<<S * n_k, 1024, 0, st>>>(tb, tw, thr_dev); }
+    }
+    return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
 }  // namespace dnns

@@ -265,6 +265,9 @@ class Session:
     def launch_count(self) -> int:
         return B.dnns_plan_launch_count(self.plan)
 
+    def tie_sweep_ran(self) -> bool:
+        return B.dnns_plan_tie_sweep(self.plan)
+
     def profile(self, enable: bool):
         B.dnns_plan_profile(self.plan, enable)
 

@@ -26,7 +26,7 @@ def test_profile_counts_kernels_only_while_on():
     ses.profile(False)
     launched = ses.launch_count() - before
     ses.variant(3, fused=True)                       # off again
-    per_kernel = {k: ses.kernel_time(k) for k in ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_ties", "k_tie_scan", "k_extrema_rows", "k_extrema_sweep",
+    per_kernel = {k: ses.kernel_time(k) for k in ["k_hist1", "k_select1", "k_hist2", "k_select2", "k_tie_find", "k_tie_pick", "k_ties", "k_tie_scan", "k_extrema_rows", "k_extrema_sweep",
                                                   "k_sweep", "k_flags", "k_propagate", "k_rebuild_layout", "k_compact"]}
     assert per_kernel["k_sweep"][1] == 3 and per_kernel["k_flags"][1] == 3 and per_kernel["k_propagate"][1] == 3
     assert per_kernel["k_hist1"][1] == 1 and per_kernel["k_compact"][1] >= 3 and per_kernel["k_rebuild_layout"][1] == 3
