@@ -200,10 +200,11 @@ dnns_status dnns_plan_tie_sweep(dnns_plan* plan, int32_t* swept);
  * k (host): k[v*n_segments + s] = how many weights of segment s variant v masks, 0 <= k <= the
  * segment's size, 1 <= n_k <= max_variants.  thr_dev (device, n_k*n_segments records, same
  * indexing) receives the records.  One call serves the whole portfolio: the sweeps over the
- * weights are shared by all n_k counts.  The call also leaves, in the workspace, the per-tile
- * tie tables that dnns_apply_mask needs to mask exactly k weights when several weights equal
- * tau, the place (tensor, element) where each variant stops masking them, which
- * dnns_compact_masked reads, and the largest key of every filter and every input column of every
+ * weights are shared by all n_k counts.  The call also leaves, in the workspace, the place
+ * (tensor, element) where each variant stops masking the weights equal to tau, which
+ * dnns_compact_masked reads (the per-tile tables of those weights, which dnns_apply_mask needs to
+ * mask exactly k weights tile by tile, are made by the call itself or, see dnns_plan_tie_sweep,
+ * by the first such sweep after it), and the largest key of every filter and every input column of every
  * tensor, which dnns_zero_structures_portfolio reads (one more sweep over the weights, enqueued on a
  * stream of the plan's own that forks from `stream` at the start of the call and joins it again at
  * the end, so that it runs beside the ranking kernels; a call inside a stream capture records that
